@@ -1,0 +1,200 @@
+/*
+ * diffpro.h — C ABI of libdiffpro: the quantized linear layer of a deployed DiffPro plan
+ * (arxiv 2511.11446) as hand-written CUDA for NVIDIA B200 (sm_100a).
+ *
+ * One call of the hot path =
+ *   DAQ (Step 3, Eq. "daq": symmetric INT8, zero-point 0, scale tau/(2^(b-1)-1) with b = 8; here
+ *        tau = per-token absmax over K, i.e. the p = 100, one-group case of the equation)
+ *   -> unpack of the GPTQ-style packed b-bit weights (Step 1/Step 3: "pack int8/int4 weights";
+ *        Algorithm 1 names W3/W4/W8)
+ *   -> INT8 x INT8 -> INT32 GEMM with per-output-channel weight scales (Step 5; Implementation)
+ *   -> dequantisation y = acc * s_a[m] * s_w[n] + bias[n], stored as bf16.
+ * dp_plan_run is Phase B of Algorithm 2: for t in reverse(K*), run every wrapped linear per the
+ * bit plan.
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller unless the name says `host`.
+ *   - Nothing on the hot path (dp_daq_quantize, dp_wq_linear, dp_plan_run) allocates, frees or
+ *     synchronises: work is enqueued on `stream` and the call returns.
+ *   - Return value is a dp_status (0 = DP_OK). Argument errors are found on the host before any
+ *     launch; nothing is enqueued in that case. dp_last_error() gives a thread-local detail string.
+ *   - Data pointers must be 16-byte aligned and leading dimensions (in elements) must make every
+ *     row start 16-byte aligned, else DP_ERR_ALIGN.
+ *   - Only compute-capability 10.x devices are accepted (DP_ERR_ARCH). There is no CPU fallback.
+ *   - Device-side waits are bounded; if one expires the kernel records DP_ERR_TIMEOUT in the
+ *     `device_status` word (when given) and exits without trapping.
+ */
+#ifndef DIFFPRO_H_
+#define DIFFPRO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum dp_status {
+  DP_OK = 0,
+  DP_ERR_INVALID_ARG = 1, /* NULL where a pointer is required, negative size, bad flag        */
+  DP_ERR_SHAPE = 2,       /* K not a multiple of 128, N not a multiple of 16, ld < row length  */
+  DP_ERR_ALIGN = 3,       /* pointer or row pitch not 16-byte aligned                          */
+  DP_ERR_BITS = 4,        /* weight bit-width not in {3,4,8}                                   */
+  DP_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than dp_*_workspace() says              */
+  DP_ERR_ARCH = 6,        /* current device is not sm_100                                      */
+  DP_ERR_CUDA = 7,        /* a CUDA runtime/driver call failed (see dp_last_error)             */
+  DP_ERR_TIMEOUT = 8      /* written by a kernel into device_status when a bounded wait expired */
+} dp_status;
+
+/* A CUDA stream handle (cudaStream_t), passed as an opaque pointer so this header needs no CUDA. */
+typedef void* dp_stream;
+
+/*
+ * Constant data of one quantized linear (device pointers, caller-owned, read-only).
+ * Weights are symmetric per-output-channel b-bit integers w[n][k] in [-2^(b-1), 2^(b-1)-1]:
+ *   bits == 8 : qweight is int8 [N][K], two's complement, row-major.
+ *   bits == 4 : qweight is uint32 [N][K/8];  field k of row n = bits [4k, 4k+4) of the row's
+ *               little-endian bit stream (8 values per 32-bit word), code u = w + 8.
+ *   bits == 3 : qweight is uint32 [N][3K/32]; field k = bits [3k, 3k+3) of the row's bit stream
+ *               (32 values per 3 words; fields 10 and 21 of each group straddle words), u = w + 4.
+ * s_w  : fp32 [N] per-output-channel scale (Step 5: "per output channel weight scales").
+ * bias : bf16 [N] or NULL.
+ * Requirements: K % 128 == 0, N % 16 == 0, N,K >= 128.
+ */
+typedef struct dp_weight {
+  int32_t N;
+  int32_t K;
+  int32_t bits;
+  int32_t reserved; /* must be 0 */
+  const void* qweight;
+  const float* s_w;
+  const void* bias;
+} dp_weight;
+
+/* Optional taps for tests: any member may be NULL. */
+typedef struct dp_debug {
+  int8_t* q;      /* [M][ldq] receives the DAQ codes                     */
+  int64_t ldq;
+  float* s_a;     /* [M] receives the activation scales                  */
+  int32_t* acc;   /* [M][ldacc] receives the raw int32 accumulators      */
+  int64_t ldacc;
+} dp_debug;
+
+/* flags for dp_wq_linear / dp_plan_create */
+#define DP_FLAG_NONE 0u
+#define DP_FLAG_FORCE_SIMT 1u   /* route through the CUDA-core weight-streaming kernel (any M)   */
+#define DP_FLAG_FORCE_MMA 2u    /* route through the tcgen05 kernel even for small M              */
+#define DP_FLAG_NO_PDL 4u       /* do not use programmatic dependent launch between the kernels  */
+
+/* flags for dp_plan_run */
+#define DP_PLAN_SAME_X 1u       /* x_ptrs has n_layers entries reused by every step              */
+#define DP_PLAN_SAME_Y 2u       /* y_ptrs has n_layers entries reused (overwritten) every step   */
+
+/*
+ * Dynamic activation quantization of a bf16 matrix, one scale per row (token).
+ *   Step 3, Eq. "daq" with b = 8, zero-point 0, tau = max_k |x[m,k]|:
+ *     a      = max_k |x[m,k]|
+ *     s_a[m] = a / 127                       (fp32, round to nearest)
+ *     q[m,k] = clamp(RNE(x[m,k] * (127/a)), -127, 127)   (127/a is one fp32 division; the product
+ *              is rounded once, half to even, to an integer)
+ *     a < 2^-100 (incl. 0): s_a[m] = 0 and q[m,:] = 0.
+ *   x      : bf16 [M][ldx], ldx >= K, ldx % 8 == 0
+ *   q      : int8 [M][ldq], ldq >= K, ldq % 16 == 0
+ *   s_a    : fp32 [M]
+ *   rowsum : int32 [M] receives sum_k q[m,k], or NULL
+ * K % 8 == 0, 8 <= K <= 65536. M == 0 is a no-op returning DP_OK. Non-finite inputs are outside
+ * the contract.
+ */
+int dp_daq_quantize(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq,
+                    float* s_a, int32_t* rowsum, dp_stream stream);
+
+/* Bytes of device scratch dp_wq_linear needs for this problem (holds the int8 activations and
+ * their scales between the two kernels of the large-M path). Never 0; multiple of 256. */
+size_t dp_wq_linear_workspace(int64_t M, int32_t N, int32_t K, int32_t bits, uint32_t flags);
+
+/*
+ * One quantized linear: y[M][N] = dequant( DAQ(x)[M][K] . unpack(w)[N][K]^T ) + bias.
+ *   Step 5 / Implementation: INT8 x INT8 -> INT32, per-output-channel weight scale; epilogue
+ *     t = (float)acc; sc = s_a[m] * s_w[n]; y = bf16_rne(fma(t, sc, bias[n]))     (all fp32).
+ *   w        : host pointer to a dp_weight whose members are device pointers
+ *   x, ldx   : s_a_in == NULL -> bf16 [M][ldx] (DAQ runs inside the call);
+ *              s_a_in != NULL -> int8 [M][ldx] already quantized, with scales s_a_in fp32 [M]
+ *   y, ldy   : bf16 [M][ldy], ldy >= N, ldy % 8 == 0
+ *   workspace: >= dp_wq_linear_workspace(...) bytes, 256-byte aligned; contents undefined after
+ *   dbg      : NULL or taps (slower path when dbg->acc is set)
+ *   device_status : int32 device word or NULL; set to DP_ERR_TIMEOUT by a kernel whose wait expired
+ * M == 0 is a no-op. Calls on the same stream are ordered; the workspace may be reused by the
+ * next call on that stream.
+ */
+int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_a_in, int64_t M,
+                 void* y_bf16, int64_t ldy, void* workspace, size_t workspace_bytes,
+                 const dp_debug* dbg, int32_t* device_status, uint32_t flags, dp_stream stream);
+
+/*
+ * A deployed plan (Algorithm 2, Phase B: "wrap layers per the bit plan"): n_layers quantized
+ * linears with their row counts. Creation validates every layer, chooses kernel variants, encodes
+ * TMA descriptors and may allocate/synchronise; it is not on the timed path. The dp_weight array is
+ * copied; the device buffers it points to must outlive the plan.
+ */
+typedef struct dp_plan dp_plan;
+int dp_plan_create(const dp_weight* layers, int32_t n_layers, const int64_t* M_per_layer,
+                   uint32_t flags, dp_plan** out);
+size_t dp_plan_workspace(const dp_plan* plan);
+void dp_plan_destroy(dp_plan* plan);
+
+/*
+ * Algorithm 2, Phase B: for i = n_steps-1 down to start_index... the retained timesteps are visited
+ * in REVERSE order of the `steps` array (the sampler walks reverse(K*)); for each visited step
+ * every layer l = 0..n_layers-1 is run in order:
+ *     y_ptrs[i*n_layers + l] = wq_linear(layers[l], x_ptrs[i*n_layers + l])
+ * (index i drops out under DP_PLAN_SAME_X / DP_PLAN_SAME_Y). x is bf16 [M_l][K_l] contiguous,
+ * y is bf16 [M_l][N_l] contiguous. `steps` holds the timestep labels (host array; only its order
+ * and length matter to the linears). Visits i = n_steps-1-start_index, ..., 0, so a caller can
+ * resume an interrupted schedule by passing the number of steps already done as start_index.
+ * x_ptrs / y_ptrs are HOST arrays of device pointers. Enqueues only; capturable in a CUDA graph.
+ */
+int dp_plan_run(const dp_plan* plan, const int32_t* steps, int32_t n_steps, int32_t start_index,
+                const void* const* x_ptrs, void* const* y_ptrs, void* workspace,
+                size_t workspace_bytes, int32_t* device_status, uint32_t flags, dp_stream stream);
+
+/*
+ * Same as dp_plan_run but the activations live in HOST memory (pinned for speed): for every
+ * visited step the inputs of all layers are copied host->device into `x_stage` (two alternating
+ * halves so the copy of one step overlaps the compute of the previous one, on an internal copy
+ * stream), the layers run, and the outputs named by d2h_layers are copied back to y_host.
+ *   x_host  : host array [n_steps*n_layers] of host pointers (or [n_layers] with DP_PLAN_SAME_X)
+ *   x_stage : device buffer of 2 * dp_plan_x_bytes(plan) bytes
+ *   y_dev   : host array [n_layers] of device output buffers (overwritten every step)
+ *   y_host  : host array [n_steps] of host pointers receiving layer `d2h_layer`'s output per step
+ * Returns after enqueueing; the caller synchronises `stream`.
+ */
+size_t dp_plan_x_bytes(const dp_plan* plan);
+int dp_plan_run_host(const dp_plan* plan, const int32_t* steps, int32_t n_steps,
+                     const void* const* x_host, void* x_stage, size_t x_stage_bytes,
+                     void* const* y_dev, int32_t d2h_layer, void* const* y_host, void* workspace,
+                     size_t workspace_bytes, int32_t* device_status, uint32_t flags,
+                     dp_stream stream);
+
+/*
+ * Host helper: pack int8 weights w[N][K] (values in [-2^(b-1), 2^(b-1)-1]) into the layout
+ * dp_weight documents. `out` is a host buffer of N*K*bits/8 bytes. Values out of range give
+ * DP_ERR_INVALID_ARG.
+ */
+int dp_pack_weights_host(const int8_t* w, int32_t N, int32_t K, int32_t bits, void* out);
+
+/*
+ * Measurement helper: runs `iters` back-to-back tcgen05 kind::i8 MMAs (128 x 256 x 32 each) per
+ * SM on operands resident in shared memory, no global loads; used to establish the measured INT8
+ * tensor ceiling of the device. Enqueues one kernel on `stream`; ops = 2*128*256*32*iters*ctas.
+ */
+int dp_bench_mma_i8(int32_t ctas, int32_t iters, int32_t* device_status, dp_stream stream);
+
+const char* dp_status_string(int status);
+const char* dp_last_error(void);
+/* Library ABI version: (major << 16) | minor. */
+int dp_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DIFFPRO_H_ */
