@@ -1,0 +1,181 @@
+"""ctypes binding of libdiffpro.so — argument marshalling only.
+
+Every function has the name and argument order of its C entry point in ``include/diffpro.h``.
+torch tensors supply device memory and the current CUDA stream; every step of the quantized
+linear runs in the library's kernels. If the shared object is missing this module raises: there is
+no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdiffpro.so")
+
+DP_OK = 0
+(DP_ERR_INVALID_ARG, DP_ERR_SHAPE, DP_ERR_ALIGN, DP_ERR_BITS, DP_ERR_WORKSPACE, DP_ERR_ARCH,
+ DP_ERR_CUDA, DP_ERR_TIMEOUT) = range(1, 9)
+DP_FLAG_NONE, DP_FLAG_FORCE_SIMT, DP_FLAG_FORCE_MMA, DP_FLAG_NO_PDL = 0, 1, 2, 4
+DP_PLAN_SAME_X, DP_PLAN_SAME_Y = 1, 2
+
+EXPORTS = ["dp_daq_quantize", "dp_wq_linear_workspace", "dp_wq_linear", "dp_plan_create",
+           "dp_plan_workspace", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
+           "dp_plan_run_host", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_status_string",
+           "dp_last_error", "dp_version"]
+
+
+class dp_weight(C.Structure):
+    _fields_ = [("N", C.c_int32), ("K", C.c_int32), ("bits", C.c_int32), ("reserved", C.c_int32),
+                ("qweight", C.c_void_p), ("s_w", C.c_void_p), ("bias", C.c_void_p)]
+
+
+class dp_debug(C.Structure):
+    _fields_ = [("q", C.c_void_p), ("ldq", C.c_int64), ("s_a", C.c_void_p), ("acc", C.c_void_p),
+                ("ldacc", C.c_int64)]
+
+
+class DiffproError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        msg = lib().dp_last_error().decode()
+        super().__init__(f"{where}: {lib().dp_status_string(status).decode()} ({msg})")
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                               "`python -m paper_2511_11446_b200.build` (no fallback exists)")
+        L = C.CDLL(LIB_PATH)
+        L.dp_wq_linear_workspace.restype = C.c_size_t
+        L.dp_wq_linear_workspace.argtypes = [C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_uint32]
+        L.dp_plan_workspace.restype = C.c_size_t
+        L.dp_plan_workspace.argtypes = [C.c_void_p]
+        L.dp_plan_x_bytes.restype = C.c_size_t
+        L.dp_plan_x_bytes.argtypes = [C.c_void_p]
+        L.dp_plan_destroy.restype = None
+        L.dp_plan_destroy.argtypes = [C.c_void_p]
+        L.dp_status_string.restype = C.c_char_p
+        L.dp_last_error.restype = C.c_char_p
+        L.dp_daq_quantize.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
+                                      C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.dp_wq_linear.argtypes = [C.POINTER(dp_weight), C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
+                                   C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t,
+                                   C.POINTER(dp_debug), C.c_void_p, C.c_uint32, C.c_void_p]
+        L.dp_plan_create.argtypes = [C.POINTER(dp_weight), C.c_int32, C.POINTER(C.c_int64), C.c_uint32,
+                                     C.POINTER(C.c_void_p)]
+        L.dp_plan_run.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.c_int32, C.c_int32,
+                                  C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.c_void_p, C.c_size_t,
+                                  C.c_void_p, C.c_uint32, C.c_void_p]
+        L.dp_plan_run_host.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.c_int32,
+                                       C.POINTER(C.c_void_p), C.c_void_p, C.c_size_t,
+                                       C.POINTER(C.c_void_p), C.c_int32, C.POINTER(C.c_void_p),
+                                       C.c_void_p, C.c_size_t, C.c_void_p, C.c_uint32, C.c_void_p]
+        L.dp_pack_weights_host.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
+        L.dp_bench_mma_i8.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _check(st, where):
+    if st != DP_OK:
+        raise DiffproError(st, where)
+
+
+def make_weight(qweight: torch.Tensor, s_w: torch.Tensor, bias, N: int, K: int, bits: int) -> dp_weight:
+    return dp_weight(N, K, bits, 0, qweight.data_ptr(), s_w.data_ptr(),
+                     None if bias is None else bias.data_ptr())
+
+
+def dp_daq_quantize(x, M, K, ldx, q, ldq, s_a, rowsum=None, stream=None):
+    _check(lib().dp_daq_quantize(_ptr(x), M, K, ldx, _ptr(q), ldq, _ptr(s_a), _ptr(rowsum),
+                                 _stream(stream)), "dp_daq_quantize")
+
+
+def dp_wq_linear_workspace(M, N, K, bits, flags=0) -> int:
+    return int(lib().dp_wq_linear_workspace(M, N, K, bits, flags))
+
+
+def dp_wq_linear(w: dp_weight, x, ldx, s_a_in, M, y, ldy, workspace, dbg: dp_debug | None = None,
+                 device_status=None, flags=0, stream=None):
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().dp_wq_linear(C.byref(w), _ptr(x), ldx, _ptr(s_a_in), M, _ptr(y), ldy, _ptr(workspace),
+                              ws_bytes, None if dbg is None else C.byref(dbg), _ptr(device_status),
+                              flags, _stream(stream)), "dp_wq_linear")
+
+
+def dp_plan_create(weights: list[dp_weight], Ms: list[int], flags=0) -> C.c_void_p:
+    arr = (dp_weight * len(weights))(*weights)
+    ms = (C.c_int64 * len(Ms))(*Ms)
+    out = C.c_void_p()
+    _check(lib().dp_plan_create(arr, len(weights), ms, flags, C.byref(out)), "dp_plan_create")
+    return out
+
+
+def dp_plan_workspace(plan) -> int:
+    return int(lib().dp_plan_workspace(plan))
+
+
+def dp_plan_x_bytes(plan) -> int:
+    return int(lib().dp_plan_x_bytes(plan))
+
+
+def dp_plan_destroy(plan):
+    lib().dp_plan_destroy(plan)
+
+
+def ptr_array(ptrs):
+    return (C.c_void_p * len(ptrs))(*ptrs)
+
+
+def dp_plan_run(plan, steps, start_index, x_ptrs, y_ptrs, workspace, device_status=None, flags=0,
+                stream=None):
+    """x_ptrs / y_ptrs: ctypes arrays of device addresses (see ptr_array)."""
+    st = (C.c_int32 * len(steps))(*steps)
+    _check(lib().dp_plan_run(plan, st, len(steps), start_index, x_ptrs, y_ptrs, _ptr(workspace),
+                             workspace.numel() * workspace.element_size(), _ptr(device_status), flags,
+                             _stream(stream)), "dp_plan_run")
+
+
+def dp_plan_run_host(plan, steps, x_host, x_stage, y_dev, d2h_layer, y_host, workspace,
+                     device_status=None, flags=0, stream=None):
+    st = (C.c_int32 * len(steps))(*steps)
+    _check(lib().dp_plan_run_host(plan, st, len(steps), x_host, _ptr(x_stage),
+                                  x_stage.numel() * x_stage.element_size(), y_dev, d2h_layer, y_host,
+                                  _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                  _ptr(device_status), flags, _stream(stream)), "dp_plan_run_host")
+
+
+def dp_pack_weights_host(w, bits: int):
+    """w: numpy int8 [N,K] -> numpy packed array (int8 [N,K] or uint32 [N, K*bits/32])."""
+    import numpy as np
+    assert w.dtype == np.int8 and w.flags.c_contiguous
+    N, K = w.shape
+    out = np.empty((N, K), np.int8) if bits == 8 else np.empty((N, K * bits // 32), np.uint32)
+    _check(lib().dp_pack_weights_host(w.ctypes.data_as(C.c_void_p), N, K, bits,
+                                      out.ctypes.data_as(C.c_void_p)), "dp_pack_weights_host")
+    return out
+
+
+def dp_bench_mma_i8(ctas, iters, device_status=None, stream=None):
+    _check(lib().dp_bench_mma_i8(ctas, iters, _ptr(device_status), _stream(stream)), "dp_bench_mma_i8")
+
+
+def dp_version() -> int:
+    return int(lib().dp_version())

@@ -1,0 +1,469 @@
+// C-ABI entry points of libdiffpro: argument checks, kernel-variant dispatch, plan objects.
+#include <stdarg.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "dp_common.cuh"
+#include "dp_internal.h"
+
+namespace dp {
+
+// ---- error reporting ---------------------------------------------------------------------------
+static thread_local char g_err[512] = "";
+
+void set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+}
+int fail(int status, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return status;
+}
+
+int check_device() {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail(DP_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  static int cached_dev = -1, cached_status = DP_OK;
+  if (dev == cached_dev) {
+    if (cached_status != DP_OK) set_error("device %d is not compute capability 10.x", dev);
+    return cached_status;
+  }
+  int major = 0;
+  e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (e != cudaSuccess) return fail(DP_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
+  cached_dev = dev;
+  cached_status = (major == 10) ? DP_OK : DP_ERR_ARCH;
+  if (cached_status != DP_OK)
+    return fail(DP_ERR_ARCH, "device %d has compute capability %d.x; sm_100 required", dev, major);
+  return gemm_init();
+}
+
+static size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
+
+constexpr int64_t kSimtMaxRows = 32;  // at or below this the CUDA-core streaming kernel is used
+
+static bool use_simt(int64_t M, int32_t N, int32_t K, uint32_t flags) {
+  if (flags & DP_FLAG_FORCE_SIMT) return true;
+  if (N % 64 != 0) return true;  // tensor path tiles N by 64/128/192/256
+  if (flags & DP_FLAG_FORCE_MMA) return false;
+  (void)K;
+  return M <= kSimtMaxRows;
+}
+
+static int check_weight(const dp_weight* w) {
+  if (!w) return fail(DP_ERR_INVALID_ARG, "dp_weight is NULL");
+  if (w->bits != 3 && w->bits != 4 && w->bits != 8)
+    return fail(DP_ERR_BITS, "bits=%d not in {3,4,8}", w->bits);
+  if (w->N < 16 || w->K < 128 || (w->K % 128) || (w->N % 16))
+    return fail(DP_ERR_SHAPE, "N=%d K=%d: need K %% 128 == 0, N %% 16 == 0", w->N, w->K);
+  if (w->reserved != 0) return fail(DP_ERR_INVALID_ARG, "dp_weight.reserved must be 0");
+  if (!w->qweight || !w->s_w) return fail(DP_ERR_INVALID_ARG, "dp_weight has a NULL member");
+  if (!aligned16(w->qweight) || (reinterpret_cast<uintptr_t>(w->s_w) & 3u) ||
+      (w->bias && (reinterpret_cast<uintptr_t>(w->bias) & 1u)))
+    return fail(DP_ERR_ALIGN, "dp_weight pointers misaligned");
+  return DP_OK;
+}
+
+// One layer, all checks done. tmap_w may be a pre-encoded descriptor (plan) or nullptr.
+static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_a_in, int64_t M,
+                      void* y, int64_t ldy, void* workspace, const dp_debug* dbg, int32_t* status,
+                      uint32_t flags, cudaStream_t stream, const CUtensorMap* tmap_w, int bn,
+                      const CUtensorMap* tmap_a_cached) {
+  const bool pdl = !(flags & DP_FLAG_NO_PDL);
+  if (use_simt(M, w->N, w->K, flags)) {
+    if (static_cast<size_t>(w->K) > simt_max_k())
+      return fail(DP_ERR_SHAPE, "K=%d too large for the small-M kernel", w->K);
+    SimtArgs a;
+    a.x = x;
+    a.ldx = ldx;
+    a.s_a_in = s_a_in;
+    a.M = M;
+    a.N = w->N;
+    a.K = w->K;
+    a.bits = w->bits;
+    a.qweight = w->qweight;
+    a.s_w = w->s_w;
+    a.bias = static_cast<const uint16_t*>(w->bias);
+    a.y = static_cast<uint16_t*>(y);
+    a.ldy = ldy;
+    a.dbg_q = dbg ? dbg->q : nullptr;
+    a.dbg_ldq = dbg ? dbg->ldq : 0;
+    a.dbg_sa = dbg ? dbg->s_a : nullptr;
+    a.dbg_acc = dbg ? dbg->acc : nullptr;
+    a.dbg_ldacc = dbg ? dbg->ldacc : 0;
+    return launch_simt_linear(a, stream, pdl);
+  }
+  const int8_t* q;
+  const float* s_a;
+  int64_t ldq;
+  if (s_a_in == nullptr) {
+    int8_t* wq = static_cast<int8_t*>(workspace);
+    float* wsa = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align256(static_cast<size_t>(M) * w->K));
+    int st = launch_daq(x, M, w->K, ldx, wq, w->K, wsa, nullptr, stream, pdl);
+    if (st != DP_OK) return st;
+    q = wq;
+    s_a = wsa;
+    ldq = w->K;
+  } else {
+    q = static_cast<const int8_t*>(x);
+    s_a = s_a_in;
+    ldq = ldx;
+  }
+  GemmProblem g;
+  if (tmap_a_cached != nullptr) {
+    g.tmap_a = *tmap_a_cached;
+  } else {
+    int st = gemm_encode_a(&g.tmap_a, q, M, w->K, ldq);
+    if (st != DP_OK) return st;
+  }
+  if (bn == 0) bn = gemm_pick_bn(M, w->N, w->K, w->bits);
+  if (tmap_w != nullptr) {
+    g.tmap_w = *tmap_w;
+  } else {
+    int st = gemm_encode_w(&g.tmap_w, w->qweight, w->N, w->K, w->bits, bn);
+    if (st != DP_OK) return st;
+  }
+  g.s_a = s_a;
+  g.s_w = w->s_w;
+  g.bias = static_cast<const uint16_t*>(w->bias);
+  g.y = static_cast<uint16_t*>(y);
+  g.ldy = ldy;
+  g.dbg_acc = dbg ? dbg->acc : nullptr;
+  g.dbg_ldacc = dbg ? dbg->ldacc : 0;
+  g.M = M;
+  g.N = w->N;
+  g.K = w->K;
+  g.bits = w->bits;
+  g.bn = bn;
+  g.status = status;
+  int st = launch_gemm(g, stream, pdl);
+  if (st != DP_OK) return st;
+  if (dbg != nullptr) {
+    if (dbg->q != nullptr)
+      DP_CUDA_OK(cudaMemcpy2DAsync(dbg->q, dbg->ldq, q, ldq, w->K, M, cudaMemcpyDeviceToDevice, stream));
+    if (dbg->s_a != nullptr)
+      DP_CUDA_OK(cudaMemcpyAsync(dbg->s_a, s_a, sizeof(float) * M, cudaMemcpyDeviceToDevice, stream));
+  }
+  return DP_OK;
+}
+
+static int check_linear_args(const dp_weight* w, const void* x, int64_t ldx, const float* s_a_in,
+                             int64_t M, void* y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                             const dp_debug* dbg, uint32_t flags) {
+  int st = check_weight(w);
+  if (st != DP_OK) return st;
+  if (M < 0) return fail(DP_ERR_SHAPE, "M=%lld is negative", (long long)M);
+  if (flags & ~(DP_FLAG_FORCE_SIMT | DP_FLAG_FORCE_MMA | DP_FLAG_NO_PDL))
+    return fail(DP_ERR_INVALID_ARG, "unknown flag bits 0x%x", flags);
+  if ((flags & DP_FLAG_FORCE_SIMT) && (flags & DP_FLAG_FORCE_MMA))
+    return fail(DP_ERR_INVALID_ARG, "FORCE_SIMT and FORCE_MMA are exclusive");
+  if (M == 0) return DP_OK;
+  if (!x || !y) return fail(DP_ERR_INVALID_ARG, "x or y is NULL");
+  if (ldx < w->K || ldy < w->N) return fail(DP_ERR_SHAPE, "leading dimension smaller than the row");
+  const int64_t xa = s_a_in ? 16 : 8;  // elements per 16 bytes
+  if (!aligned16(x) || !aligned16(y) || (ldx % xa) || (ldy % 8))
+    return fail(DP_ERR_ALIGN, "x/y pointers and pitches must be 16-byte aligned");
+  if (dbg) {
+    if (dbg->q && (!aligned16(dbg->q) || dbg->ldq < w->K || (dbg->ldq % 16)))
+      return fail(DP_ERR_ALIGN, "dbg.q misaligned or too narrow");
+    if (dbg->acc && (dbg->ldacc < w->N || (reinterpret_cast<uintptr_t>(dbg->acc) & 3u)))
+      return fail(DP_ERR_ALIGN, "dbg.acc misaligned or too narrow");
+  }
+  if (!use_simt(M, w->N, w->K, flags) && s_a_in == nullptr) {
+    const size_t need = dp_wq_linear_workspace(M, w->N, w->K, w->bits, flags);
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+      return fail(DP_ERR_WORKSPACE, "workspace needs %zu bytes, 256-byte aligned (got %zu)", need,
+                  workspace_bytes);
+  }
+  return DP_OK;
+}
+
+}  // namespace dp
+
+// ================================================================================================
+using namespace dp;
+
+extern "C" size_t dp_wq_linear_workspace(int64_t M, int32_t N, int32_t K, int32_t bits, uint32_t flags) {
+  (void)bits;
+  if (M <= 0 || K <= 0) return 256;
+  if (use_simt(M, N, K, flags)) return 256;
+  return align256(static_cast<size_t>(M) * K) + align256(sizeof(float) * static_cast<size_t>(M));
+}
+
+extern "C" int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_a_in,
+                            int64_t M, void* y_bf16, int64_t ldy, void* workspace,
+                            size_t workspace_bytes, const dp_debug* dbg, int32_t* device_status,
+                            uint32_t flags, dp_stream stream) {
+  int st = check_linear_args(w, x, ldx, s_a_in, M, y_bf16, ldy, workspace, workspace_bytes, dbg, flags);
+  if (st != DP_OK || M == 0) return st;
+  st = check_device();
+  if (st != DP_OK) return st;
+  return run_linear(w, x, ldx, s_a_in, M, y_bf16, ldy, workspace, dbg, device_status, flags,
+                    static_cast<cudaStream_t>(stream), nullptr, 0, nullptr);
+}
+
+// ---- plans ---------------------------------------------------------------------------------------
+struct PlanLayer {
+  dp_weight w;
+  int64_t M;
+  bool simt;
+  int bn;
+  CUtensorMap tmap_w;
+  size_t x_offset;  // byte offset of this layer's input inside one staged step (host-input path)
+};
+struct TmapACache {
+  const void* ptr;
+  int64_t M, K;
+  CUtensorMap map;
+};
+struct dp_plan {
+  std::vector<PlanLayer> layers;
+  uint32_t flags;
+  size_t workspace_bytes;
+  size_t x_bytes;
+  std::vector<TmapACache> a_cache;
+  cudaStream_t copy_stream;
+  cudaEvent_t ev_copied[2], ev_consumed[2];
+};
+
+extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const int64_t* M_per_layer,
+                              uint32_t flags, dp_plan** out) {
+  if (!out) return fail(DP_ERR_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  if (!layers || !M_per_layer || n_layers <= 0)
+    return fail(DP_ERR_INVALID_ARG, "layers/M_per_layer NULL or n_layers <= 0");
+  if (flags & ~(DP_FLAG_FORCE_SIMT | DP_FLAG_FORCE_MMA | DP_FLAG_NO_PDL))
+    return fail(DP_ERR_INVALID_ARG, "unknown flag bits 0x%x", flags);
+  int st = check_device();
+  if (st != DP_OK) return st;
+  dp_plan* p = new (std::nothrow) dp_plan();
+  if (!p) return fail(DP_ERR_CUDA, "out of host memory");
+  p->flags = flags;
+  p->workspace_bytes = 256;
+  p->x_bytes = 0;
+  p->copy_stream = nullptr;
+  for (int i = 0; i < 2; ++i) p->ev_copied[i] = p->ev_consumed[i] = nullptr;
+  for (int32_t l = 0; l < n_layers; ++l) {
+    st = check_weight(&layers[l]);
+    if (st == DP_OK && M_per_layer[l] < 0) st = fail(DP_ERR_SHAPE, "layer %d: negative M", l);
+    if (st != DP_OK) {
+      delete p;
+      return st;
+    }
+    PlanLayer L;
+    L.w = layers[l];
+    L.M = M_per_layer[l];
+    L.simt = use_simt(L.M, L.w.N, L.w.K, flags);
+    L.bn = 0;
+    memset(&L.tmap_w, 0, sizeof(L.tmap_w));
+    if (L.simt && static_cast<size_t>(L.w.K) > simt_max_k()) {
+      delete p;
+      return fail(DP_ERR_SHAPE, "layer %d: K too large for the small-M kernel", l);
+    }
+    if (!L.simt && L.M > 0) {
+      L.bn = gemm_pick_bn(L.M, L.w.N, L.w.K, L.w.bits);
+      st = gemm_encode_w(&L.tmap_w, L.w.qweight, L.w.N, L.w.K, L.w.bits, L.bn);
+      if (st != DP_OK) {
+        delete p;
+        return st;
+      }
+    }
+    const size_t ws = dp_wq_linear_workspace(L.M, L.w.N, L.w.K, L.w.bits, flags);
+    if (ws > p->workspace_bytes) p->workspace_bytes = ws;
+    L.x_offset = p->x_bytes;
+    p->x_bytes += align256(static_cast<size_t>(L.M) * L.w.K * 2);
+    p->layers.push_back(L);
+  }
+  cudaError_t e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
+  for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+    e = cudaEventCreateWithFlags(&p->ev_copied[i], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_consumed[i], cudaEventDisableTiming);
+  }
+  if (e != cudaSuccess) {
+    dp_plan_destroy(p);
+    return fail(DP_ERR_CUDA, "plan stream/event creation: %s", cudaGetErrorString(e));
+  }
+  *out = p;
+  return DP_OK;
+}
+
+extern "C" size_t dp_plan_workspace(const dp_plan* plan) { return plan ? plan->workspace_bytes : 0; }
+extern "C" size_t dp_plan_x_bytes(const dp_plan* plan) { return plan ? plan->x_bytes : 0; }
+
+extern "C" void dp_plan_destroy(dp_plan* plan) {
+  if (!plan) return;
+  for (int i = 0; i < 2; ++i) {
+    if (plan->ev_copied[i]) cudaEventDestroy(plan->ev_copied[i]);
+    if (plan->ev_consumed[i]) cudaEventDestroy(plan->ev_consumed[i]);
+  }
+  if (plan->copy_stream) cudaStreamDestroy(plan->copy_stream);
+  delete plan;
+}
+
+// The int8 activations of every tensor-path layer live at the start of the workspace, so their TMA
+// descriptor depends only on (workspace, M, K): encoded once and reused across layers and steps.
+static const CUtensorMap* cached_tmap_a(dp_plan* plan, const void* ws, int64_t M, int64_t K, int* st) {
+  for (const TmapACache& c : plan->a_cache)
+    if (c.ptr == ws && c.M == M && c.K == K) return &c.map;
+  TmapACache c;
+  c.ptr = ws;
+  c.M = M;
+  c.K = K;
+  *st = gemm_encode_a(&c.map, static_cast<const int8_t*>(ws), M, K, K);
+  if (*st != DP_OK) return nullptr;
+  if (plan->a_cache.size() > 64) plan->a_cache.clear();
+  plan->a_cache.push_back(c);
+  return &plan->a_cache.back().map;
+}
+
+static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, void* workspace,
+                         int32_t* status, cudaStream_t stream) {
+  const int n = static_cast<int>(plan->layers.size());
+  for (int l = 0; l < n; ++l) {
+    const PlanLayer& L = plan->layers[l];
+    if (L.M == 0) continue;
+    if (!xs[l] || !ys[l]) return fail(DP_ERR_INVALID_ARG, "layer %d: NULL x or y", l);
+    if (!aligned16(xs[l]) || !aligned16(ys[l])) return fail(DP_ERR_ALIGN, "layer %d: x/y misaligned", l);
+    const CUtensorMap* ta = nullptr;
+    if (!L.simt) {
+      int st = DP_OK;
+      ta = cached_tmap_a(plan, workspace, L.M, L.w.K, &st);
+      if (st != DP_OK) return st;
+    }
+    int st = run_linear(&L.w, xs[l], L.w.K, nullptr, L.M, ys[l], L.w.N, workspace, nullptr, status,
+                        plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, ta);
+    if (st != DP_OK) return st;
+  }
+  return DP_OK;
+}
+
+static int check_plan_run(const dp_plan* plan, const int32_t* steps, int32_t n_steps,
+                          int32_t start_index, const void* xp, const void* yp, void* workspace,
+                          size_t workspace_bytes, uint32_t flags) {
+  if (!plan || !xp || !yp) return fail(DP_ERR_INVALID_ARG, "plan, x_ptrs or y_ptrs is NULL");
+  if (n_steps < 0 || start_index < 0 || start_index > n_steps || (n_steps > 0 && !steps))
+    return fail(DP_ERR_INVALID_ARG, "bad steps/n_steps/start_index");
+  if (flags & ~(DP_PLAN_SAME_X | DP_PLAN_SAME_Y)) return fail(DP_ERR_INVALID_ARG, "unknown plan-run flags");
+  if (!workspace || workspace_bytes < plan->workspace_bytes || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return fail(DP_ERR_WORKSPACE, "plan workspace needs %zu bytes, 256-byte aligned", plan->workspace_bytes);
+  return DP_OK;
+}
+
+extern "C" int dp_plan_run(const dp_plan* plan_c, const int32_t* steps, int32_t n_steps,
+                           int32_t start_index, const void* const* x_ptrs, void* const* y_ptrs,
+                           void* workspace, size_t workspace_bytes, int32_t* device_status,
+                           uint32_t flags, dp_stream stream) {
+  int st = check_plan_run(plan_c, steps, n_steps, start_index, x_ptrs, y_ptrs, workspace,
+                          workspace_bytes, flags);
+  if (st != DP_OK) return st;
+  dp_plan* plan = const_cast<dp_plan*>(plan_c);
+  const int64_t n = static_cast<int64_t>(plan->layers.size());
+  for (int32_t i = n_steps - 1 - start_index; i >= 0; --i) {  // reverse(K*)
+    const void* const* xs = x_ptrs + ((flags & DP_PLAN_SAME_X) ? 0 : i * n);
+    void* const* ys = y_ptrs + ((flags & DP_PLAN_SAME_Y) ? 0 : i * n);
+    st = plan_run_step(plan, xs, ys, workspace, device_status, static_cast<cudaStream_t>(stream));
+    if (st != DP_OK) return st;
+  }
+  return DP_OK;
+}
+
+extern "C" int dp_plan_run_host(const dp_plan* plan_c, const int32_t* steps, int32_t n_steps,
+                                const void* const* x_host, void* x_stage, size_t x_stage_bytes,
+                                void* const* y_dev, int32_t d2h_layer, void* const* y_host,
+                                void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                uint32_t flags, dp_stream stream_) {
+  int st = check_plan_run(plan_c, steps, n_steps, 0, x_host, y_dev, workspace, workspace_bytes,
+                          flags & DP_PLAN_SAME_X);
+  if (st != DP_OK) return st;
+  if (flags & ~DP_PLAN_SAME_X) return fail(DP_ERR_INVALID_ARG, "unknown plan-run flags");
+  dp_plan* plan = const_cast<dp_plan*>(plan_c);
+  const int64_t n = static_cast<int64_t>(plan->layers.size());
+  if (!x_stage || x_stage_bytes < 2 * plan->x_bytes || (reinterpret_cast<uintptr_t>(x_stage) & 255u))
+    return fail(DP_ERR_WORKSPACE, "x_stage needs %zu bytes, 256-byte aligned", 2 * plan->x_bytes);
+  if (d2h_layer >= n || (d2h_layer >= 0 && !y_host))
+    return fail(DP_ERR_INVALID_ARG, "bad d2h_layer / y_host");
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  std::vector<const void*> xs(n);
+  int j = 0;
+  for (int32_t i = n_steps - 1; i >= 0; --i, ++j) {
+    const int h = j & 1;
+    uint8_t* stage = static_cast<uint8_t*>(x_stage) + h * plan->x_bytes;
+    if (j >= 2) DP_CUDA_OK(cudaStreamWaitEvent(plan->copy_stream, plan->ev_consumed[h], 0));
+    const void* const* src = x_host + ((flags & DP_PLAN_SAME_X) ? 0 : i * n);
+    for (int64_t l = 0; l < n; ++l) {
+      const PlanLayer& L = plan->layers[l];
+      xs[l] = stage + L.x_offset;
+      if (L.M == 0) continue;
+      if (!src[l]) return fail(DP_ERR_INVALID_ARG, "layer %lld: NULL host input", (long long)l);
+      DP_CUDA_OK(cudaMemcpyAsync(stage + L.x_offset, src[l], static_cast<size_t>(L.M) * L.w.K * 2,
+                                 cudaMemcpyHostToDevice, plan->copy_stream));
+    }
+    DP_CUDA_OK(cudaEventRecord(plan->ev_copied[h], plan->copy_stream));
+    DP_CUDA_OK(cudaStreamWaitEvent(stream, plan->ev_copied[h], 0));
+    st = plan_run_step(plan, xs.data(), y_dev, workspace, device_status, stream);
+    if (st != DP_OK) return st;
+    DP_CUDA_OK(cudaEventRecord(plan->ev_consumed[h], stream));
+    if (d2h_layer >= 0) {
+      const PlanLayer& L = plan->layers[d2h_layer];
+      DP_CUDA_OK(cudaMemcpyAsync(y_host[i], y_dev[d2h_layer], static_cast<size_t>(L.M) * L.w.N * 2,
+                                 cudaMemcpyDeviceToHost, stream));
+    }
+  }
+  return DP_OK;
+}
+
+// ---- host helpers ----------------------------------------------------------------------------------
+extern "C" int dp_pack_weights_host(const int8_t* w, int32_t N, int32_t K, int32_t bits, void* out) {
+  if (!w || !out || N <= 0 || K <= 0) return fail(DP_ERR_INVALID_ARG, "dp_pack_weights_host: bad arguments");
+  if (bits == 8) {
+    memcpy(out, w, static_cast<size_t>(N) * K);
+    return DP_OK;
+  }
+  if (bits != 3 && bits != 4) return fail(DP_ERR_BITS, "bits=%d not in {3,4,8}", bits);
+  if (K % 32) return fail(DP_ERR_SHAPE, "K=%d not a multiple of 32", K);
+  const int half = 1 << (bits - 1);
+  uint32_t* o = static_cast<uint32_t*>(out);
+  for (int64_t n = 0; n < N; ++n) {
+    uint64_t buf = 0;
+    int nb = 0;
+    for (int64_t k = 0; k < K; ++k) {
+      const int v = w[n * K + k];
+      if (v < -half || v >= half)
+        return fail(DP_ERR_INVALID_ARG, "weight %d at [%lld,%lld] outside the %d-bit range", v,
+                    (long long)n, (long long)k, bits);
+      buf |= static_cast<uint64_t>(v + half) << nb;
+      nb += bits;
+      if (nb >= 32) {
+        *o++ = static_cast<uint32_t>(buf);
+        buf >>= 32;
+        nb -= 32;
+      }
+    }
+  }
+  return DP_OK;
+}
+
+extern "C" const char* dp_status_string(int s) {
+  switch (s) {
+    case DP_OK: return "DP_OK";
+    case DP_ERR_INVALID_ARG: return "DP_ERR_INVALID_ARG";
+    case DP_ERR_SHAPE: return "DP_ERR_SHAPE";
+    case DP_ERR_ALIGN: return "DP_ERR_ALIGN";
+    case DP_ERR_BITS: return "DP_ERR_BITS";
+    case DP_ERR_WORKSPACE: return "DP_ERR_WORKSPACE";
+    case DP_ERR_ARCH: return "DP_ERR_ARCH";
+    case DP_ERR_CUDA: return "DP_ERR_CUDA";
+    case DP_ERR_TIMEOUT: return "DP_ERR_TIMEOUT";
+    default: return "DP_ERR_UNKNOWN";
+  }
+}
+extern "C" const char* dp_last_error(void) { return dp::g_err; }
+extern "C" int dp_version(void) { return (0 << 16) | 1; }

@@ -1,0 +1,64 @@
+// Internal interfaces between the translation units of libdiffpro (host side).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/diffpro.h"
+
+namespace dp {
+
+// daq.cu
+int launch_daq(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq,
+               float* s_a, int32_t* rowsum, cudaStream_t stream, bool pdl);
+
+// simt.cu — CUDA-core weight-streaming linear for small M (DAQ fused in the CTA prologue).
+struct SimtArgs {
+  const void* x;        // bf16 [M][ldx] or int8 [M][ldx] when s_a_in != nullptr
+  int64_t ldx;
+  const float* s_a_in;  // nullptr -> DAQ inside the kernel
+  int64_t M;
+  int32_t N, K, bits;
+  const void* qweight;
+  const float* s_w;
+  const uint16_t* bias;
+  uint16_t* y;
+  int64_t ldy;
+  int8_t* dbg_q;
+  int64_t dbg_ldq;
+  float* dbg_sa;
+  int32_t* dbg_acc;
+  int64_t dbg_ldacc;
+};
+int launch_simt_linear(const SimtArgs& a, cudaStream_t stream, bool pdl);
+size_t simt_max_k();
+
+// gemm_tc.cu — tcgen05 kind::i8 GEMM with in-smem weight unpack and fused dequant epilogue.
+struct GemmTile {  // kernel variant
+  int bn;          // tile width in output channels: 64, 128, 192 or 256
+};
+struct GemmProblem {
+  CUtensorMap tmap_a;  // int8 activations [M][K]
+  CUtensorMap tmap_w;  // packed weights, byte view [N][K*bits/8]
+  const float* s_a;    // [M]
+  const float* s_w;    // [N]
+  const uint16_t* bias;
+  uint16_t* y;
+  int64_t ldy;
+  int32_t* dbg_acc;
+  int64_t dbg_ldacc;
+  int64_t M;
+  int32_t N, K, bits, bn;
+  int32_t* status;
+};
+int gemm_pick_bn(int64_t M, int32_t N, int32_t K, int32_t bits);
+int gemm_encode_a(CUtensorMap* out, const int8_t* q, int64_t M, int64_t K, int64_t ldq);
+int gemm_encode_w(CUtensorMap* out, const void* qweight, int32_t N, int32_t K, int32_t bits,
+                  int32_t bn);
+int launch_gemm(const GemmProblem& p, cudaStream_t stream, bool pdl);
+int gemm_init();  // sets kernel attributes, resolves the tensor-map encoder; idempotent
+
+int num_sms();
+
+}  // namespace dp

@@ -1,0 +1,114 @@
+"""GPU parity of dp_wq_linear against the CPU oracle.
+
+int8 codes, fp32 scales and int32 accumulators must be bit-exact; bf16 outputs within 1 bf16 ulp
+(the kernels mirror the oracle's fp32 operation sequence, so 0 ulp is expected and asserted for
+the vast majority)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_11446_b200 import binding as B, synth
+from gpu_util import DevLayer, run_linear
+from helpers import bf16_ulp_dist
+
+pytestmark = pytest.mark.gpu
+SEED = synth.BASE_SEED
+
+
+def _case(M, K, N, bits, layer=0, n_out=None, bias=True, full_range=False):
+    x = synth.activations(SEED, layer, 0, M, K, 1.0, n_out=K // 100 if n_out is None else n_out)
+    if full_range:  # every code incl. -2^(b-1)
+        rng = np.random.default_rng(bits * 1000 + N)
+        w = rng.integers(-(1 << (bits - 1)), 1 << (bits - 1), size=(N, K)).astype(np.int8)
+        s_w = (np.abs(rng.standard_normal(N)) * 1e-3 + 1e-4).astype(np.float32)
+    else:
+        w, s_w = synth.weights(SEED, layer, N, K, bits)
+    b = synth.bias(SEED, layer, N) if bias else None
+    return x, w, s_w, b
+
+
+def _check(out, x, w, s_w, b, bits, exact_y=True):
+    y, q, s_a, acc = oracle.wq_linear(x, oracle.pack(w, bits), s_w, b, bits, taps=True)
+    assert out["status"] == 0
+    assert np.array_equal(out["s_a"].view(np.uint32), s_a.view(np.uint32)), "scales differ"
+    assert np.array_equal(out["q"], q), "int8 codes differ"
+    bad = np.argwhere(out["acc"] != acc)
+    assert bad.size == 0, f"{len(bad)} accumulators differ, first at {bad[:5].tolist()}"
+    d = bf16_ulp_dist(out["y"], y)
+    assert d.max() <= 1, f"max bf16 distance {d.max()}"
+    if exact_y:
+        assert (d != 0).mean() < 1e-4
+
+
+@pytest.mark.parametrize("bits", [3, 4, 8])
+@pytest.mark.parametrize("M,K,N", [(1, 128, 32), (8, 1152, 96), (16, 1152, 6912), (21, 256, 48),
+                                   (32, 4608, 64)])
+def test_simt_path(bits, M, K, N):
+    x, w, s_w, b = _case(M, K, N, bits, full_range=(N == 48))
+    L = DevLayer(w, s_w, b, bits)
+    _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_SIMT), x, w, s_w, b, bits)
+
+
+@pytest.mark.parametrize("bits", [8, 4, 3])
+@pytest.mark.parametrize("M,K,N", [(128, 128, 64), (128, 256, 128), (256, 1152, 1152),
+                                   (300, 1152, 384), (1000, 4608, 1152), (77, 384, 192),
+                                   (2048, 1152, 4608)])
+def test_mma_path(bits, M, K, N):
+    x, w, s_w, b = _case(M, K, N, bits, full_range=(N in (64, 192)), bias=(N != 384))
+    L = DevLayer(w, s_w, b, bits)
+    _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA), x, w, s_w, b, bits)
+
+
+@pytest.mark.parametrize("bits", [8, 4, 3])
+def test_mma_one_hot_and_constant_inputs(bits):
+    """One-hot tokens expose any permutation of k or n inside the tiles: acc[m,n] = 127*w[n,k_m]."""
+    M, K, N = 128, 384, 128
+    f = np.zeros((M, K), np.float32)
+    for m in range(M):
+        f[m, (m * 7) % K] = 1.0 if m % 2 == 0 else -2.0
+    x = synth.f32_to_bf16_bits(f)
+    rng = np.random.default_rng(bits)
+    w = rng.integers(-(1 << (bits - 1)), 1 << (bits - 1), size=(N, K)).astype(np.int8)
+    s_w = np.ones(N, np.float32)
+    L = DevLayer(w, s_w, None, bits)
+    out = run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA)
+    _check(out, x, w, s_w, None, bits)
+    km = (np.arange(M) * 7) % K
+    sign = np.where(np.arange(M) % 2 == 0, 127, -127)
+    assert np.array_equal(out["acc"], sign[:, None] * w[:, km].T.astype(np.int32))
+    xc = synth.f32_to_bf16_bits(np.full((M, K), 0.75, np.float32))
+    _check(run_linear(L, xc, flags=B.DP_FLAG_FORCE_MMA), xc, w, s_w, None, bits)
+
+
+@pytest.mark.parametrize("flags", [B.DP_FLAG_FORCE_SIMT, B.DP_FLAG_FORCE_MMA])
+def test_prequantized_input(flags):
+    M, K, N, bits = 130, 256, 128, 4
+    x, w, s_w, b = _case(M, K, N, bits)
+    q, s_a, _ = oracle.daq(x)
+    L = DevLayer(w, s_w, b, bits)
+    out = run_linear(L, x, flags=flags, prequant=(q, s_a), taps=False)
+    y = oracle.wq_linear(x, oracle.pack(w, bits), s_w, b, bits)
+    assert out["status"] == 0 and bf16_ulp_dist(out["y"], y).max() <= 1
+
+
+def test_default_dispatch_and_argument_errors():
+    x, w, s_w, b = _case(16, 1152, 128, 8)
+    L = DevLayer(w, s_w, b, 8)
+    _check(run_linear(L, x), x, w, s_w, b, 8)            # small M -> streaming kernel
+    x, w, s_w, b = _case(200, 1152, 128, 8)
+    _check(run_linear(DevLayer(w, s_w, b, 8), x), x, w, s_w, b, 8)   # large M -> tensor cores
+    y = torch.empty((16, 128), dtype=torch.bfloat16, device="cuda")
+    xt = torch.empty((16, 1152), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    bad = B.make_weight(L.qweight, L.s_w, None, 128, 1152, 5)
+    with pytest.raises(B.DiffproError) as e:
+        B.dp_wq_linear(bad, xt, 1152, None, 16, y, 128, ws)
+    assert e.value.status == B.DP_ERR_BITS
+    with pytest.raises(B.DiffproError) as e:
+        B.dp_wq_linear(L.w, xt, 1152, None, 16, y, 64, ws)
+    assert e.value.status == B.DP_ERR_SHAPE
+    with pytest.raises(B.DiffproError) as e:
+        B.dp_wq_linear(L.w, xt, 1152, None, 200, y, 128, None, flags=B.DP_FLAG_FORCE_MMA)
+    assert e.value.status == B.DP_ERR_WORKSPACE
+    B.dp_wq_linear(L.w, xt, 1152, None, 0, y, 128, ws)   # M = 0: no-op
