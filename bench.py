@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark of the DiffPro quantized-linear hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Workload (config.workload = "c4"): the whole DiT-XL/2 linear stack (28 blocks x {qkv, proj, fc1, fc2,
+adaLN} = 140 quantized linears, mixed {3,4,8}-bit plan) executed by dp_plan_run over 25 retained of 50
+timesteps at batch 8, 256 px (M = 2048 tokens; adaLN M = 8). One bench "step" = one dp_plan_run over
+the full retained schedule = 3500 quantized linears (DAQ -> unpack -> INT8 GEMM -> dequant each).
+`value` = int8 TOPS = 2*M*N*K summed over all calls / time; `us_per_dit_step` = time per denoising
+timestep (140 linears). With N > 1 GPUs every rank runs the same-size workload on its own batch
+(rows shard with no collective; weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "fused DAQ+WbA8 linear int8 TOPS (dp_plan_run, DiT-XL/2 linear stack)"
+UNIT = "TOPS"
+NOMINAL_INT8_TOPS = 4500.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16=d["bf16_tflops"], bf16_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons, pw = [], [], set(), []
+        for line in out.splitlines():
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); pw.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "power_w_max": max(pw), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------------
+def oracle_sample(seconds_target=15.0):
+    """The CPU oracle, as it stands, on a bounded sample of the workload: the first layers of the
+    stack (in plan order, their planned bit-widths) at the last retained timestep, as many as fit
+    the time target. Returns (tops, seconds, description, cores)."""
+    import oracle
+    from paper_2511_11446_b200 import synth
+    seed = synth.BASE_SEED + 4
+    table = synth.dit_layers(8, 256)
+    bits = synth.bit_plan(seed, len(table))
+    t = synth.kept_timesteps(seed)[-1]
+
+    def make(l, rows=None):
+        _, M, K, N = table[l]
+        M = M if rows is None else min(M, rows)
+        w, s_w = synth.weights(seed, l, N, K, bits[l])
+        x = synth.activations(seed, l, t, M, K, synth.sigma_t(t, 50), n_out=max(1, K // 100))
+        return x, oracle.pack(w, bits[l]), s_w, synth.bias(seed, l, N), bits[l], 2.0 * M * N * K
+
+    x, pw, s_w, b, bt, ops = make(0, rows=128)
+    t0 = time.perf_counter(); oracle.wq_linear(x, pw, s_w, b, bt); rate = ops / (time.perf_counter() - t0)
+    budget, chosen, tot = rate * seconds_target, [], 0.0
+    for l in range(len(table)):
+        o = 2.0 * table[l][1] * table[l][2] * table[l][3]
+        if chosen and tot + o > budget:
+            break
+        chosen.append(l); tot += o
+    secs = 0.0
+    for l in chosen:
+        x, pw, s_w, b, bt, ops = make(l)
+        t0 = time.perf_counter(); oracle.wq_linear(x, pw, s_w, b, bt); secs += time.perf_counter() - t0
+    desc = (f"layers 0..{chosen[-1]} of 140 (plan order, planned bits) of timestep {t}: "
+            f"{tot / 1e9:.1f} of {sum(2.0 * M * N * K for _, M, K, N in table) * 25 / 1e9:.0f} GOP per plan run")
+    return tot / secs / 1e12, secs, desc, oracle.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", 0))
+    if rank != 0:
+        return
+    vals, secs, desc, cores = [], [], "", 1
+    for i in range(args.warmup + args.steps):
+        tops, dt, desc, cores = oracle_sample(seconds_target=max(2.0, min(15.0, 120.0 / (args.warmup + args.steps))))
+        if i >= args.warmup:
+            vals.append(tops); secs.append(dt)
+    v = sum(vals) / len(vals)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs) / len(secs), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": "c4", "note": "CPU oracle on a bounded sample per step: " + desc},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# --------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    from paper_2511_11446_b200 import binding as B, dist as D
+    from paper_2511_11446_b200.workloads import DitStack
+    from paper_2511_11446_b200 import synth
+
+    rank, local_rank, world = D.init()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    peaks = measured_peaks()
+
+    seed = D.rank_seed(synth.BASE_SEED + 4, rank)
+    stack = DitStack(seed=seed)
+    nL, nS = len(stack.table), len(stack.kept)
+    ops_step = stack.ops_per_timestep() * nS
+    graph = stack.capture()
+    torch.cuda.synchronize()
+
+    # ---- device-resident timing: K plan runs (graph replays), CUDA events on the launch stream ----
+    for _ in range(args.warmup):
+        graph.replay()
+    torch.cuda.synchronize()
+    D.barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    D.barrier()
+    ms_total = D.max_over_ranks(e0.elapsed_time(e1), dev)
+    clocks = sampler.stop()
+    assert int(stack.status.item()) == 0, "a kernel reported DP_ERR_TIMEOUT"
+    ms_per_step = ms_total / args.steps
+    value = world * ops_step / (ms_per_step * 1e-3) / 1e12
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int8", "data": "synthetic",
+        "config": {"workload": "c4", "layers": nL, "retained_timesteps": nS, "of_timesteps": stack.T,
+                   "M": 2048, "M_adaln": 8, "bit_plan_counts": {str(b): stack.bits.count(b) for b in (3, 4, 8)},
+                   "parallelism": f"rows x{world} (no collective)", "l2": "inputs+weights per timestep (>1.1 GB) exceed L2",
+                   "launch": "one CUDA graph per plan run"},
+        "us_per_dit_step": 1e3 * ms_per_step / nS,
+        "roofline_step": {"ideal_us_per_dit_step_nominal": None},
+        "gpu_launches": stack.launches_per_timestep() * nS * args.steps,
+        "clocks": clocks,
+    }
+
+    if rank == 0:
+        # ---- roofline of the dominant kernel (tcgen05 GEMM), timed alone with CUDA events ----
+        out["roofline"] = gemm_roofline(stack, peaks)
+        # ideal time of a timestep: per layer max(ops / int8 peak, bytes / HBM)
+        int8_peak = 2.0 * peaks["bf16_sustained"]
+        ideal = 0.0
+        for L, (_, M, K, N) in zip(stack.layers, stack.table):
+            by = 2 * M * K + L.packed_bytes() + 6 * N + 2 * M * N
+            ideal += max(2.0 * M * N * K / (int8_peak * 1e12), by / (peaks["hbm_gbs"] * 1e9))
+        out["roofline_step"] = {"ideal_us_per_dit_step": ideal * 1e6, "frac": ideal * 1e6 / out["us_per_dit_step"],
+                                "int8_peak_tops_used": int8_peak, "hbm_gbs_used": peaks["hbm_gbs"],
+                                "peaks": peaks["source"]}
+        out["mma_i8_peak_tops_measured"] = measure_mma_peak()
+        out["e2e"] = e2e(stack, ops_step, world)
+        tops, dt, desc, cores = oracle_sample()
+        out["cpu_baseline"] = {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
+                               "seconds": dt}
+        print(json.dumps(out))
+    stack.close()
+    D.barrier()
+
+
+def gemm_roofline(stack, peaks):
+    """Times the GEMM launches of one timestep alone (pre-quantized activations, so no DAQ launch
+    in between), CUDA events on the launch stream; cold: 0.9 GB of other traffic between passes."""
+    import torch
+    from paper_2511_11446_b200 import binding as B
+    x0 = stack.x[0]
+    idx = [l for l, (_, M, K, N) in enumerate(stack.table) if M > 32]
+    qs, sas = {}, {}
+    for l in idx:
+        _, M, K, N = stack.table[l]
+        qs[l] = torch.empty((M, K), dtype=torch.int8, device="cuda")
+        sas[l] = torch.empty(M, dtype=torch.float32, device="cuda")
+        B.dp_daq_quantize(x0[l], M, K, K, qs[l], K, sas[l])
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    times = []
+    for it in range(5):
+        flush.fill_(it)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for l in idx:
+            _, M, K, N = stack.table[l]
+            B.dp_wq_linear(stack.layers[l].w, qs[l], K, sas[l], M, stack.y[l], N, None, None, stack.status)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    ms = statistics.median(times[1:])
+    ops = sum(2.0 * stack.table[l][1] * stack.table[l][2] * stack.table[l][3] for l in idx)
+    achieved = ops / (ms * 1e-3) / 1e12
+    peak = 2.0 * peaks["bf16_sustained"]
+    return {"kernel": "gemm_i8_kernel (tcgen05 kind::i8)", "bound": "tensor", "achieved": achieved, "peak": peak,
+            "unit": "TOPS", "frac": achieved / peak,
+            "peak_note": f"{peaks['source']} bf16 sustained x2 (nominal int8:bf16 ratio); nominal dense int8 is {NOMINAL_INT8_TOPS}",
+            "frac_of_nominal": achieved / NOMINAL_INT8_TOPS, "launches": len(idx),
+            "avg_launch_us": 1e3 * ms / len(idx), "traffic": None}
+
+
+def measure_mma_peak():
+    import torch
+    from paper_2511_11446_b200 import binding as B
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    iters = 20000
+    B.dp_bench_mma_i8(sms, 2000, st)
+    torch.cuda.synchronize()
+    best = 0.0
+    for _ in range(3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.dp_bench_mma_i8(sms, iters, st)
+        e1.record()
+        torch.cuda.synchronize()
+        best = max(best, 2.0 * 128 * 256 * 128 * iters * sms / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+    return best if int(st.item()) == 0 else None
+
+
+def e2e(stack, ops_step, world):
+    """Same plan run through dp_plan_run_host: every timestep's inputs are copied from pinned host
+    memory inside the timed region and the last block's fc2 output is read back per timestep."""
+    import psutil
+    import torch
+    from paper_2511_11446_b200 import binding as B
+    nL, nS = len(stack.table), len(stack.kept)
+    xbytes = sum(t.numel() * 2 for t in stack.x[0])
+    distinct = psutil.virtual_memory().available > 3 * xbytes * nS
+    n_host = nS if distinct else 1
+    xh = [[torch.empty(t.shape, dtype=torch.bfloat16, pin_memory=True) for t in stack.x[0]] for _ in range(n_host)]
+    for i in range(n_host):
+        for l in range(nL):
+            xh[i][l].copy_(stack.x[i][l])
+    last = nL - 2
+    M, N = stack.table[last][1], stack.table[last][3]
+    yh = [torch.empty((M, N), dtype=torch.bfloat16, pin_memory=True) for _ in range(nS)]
+    stage = torch.empty(2 * B.dp_plan_x_bytes(stack.plan), dtype=torch.uint8, device="cuda")
+    xp = B.ptr_array([xh[i][l].data_ptr() for i in range(n_host) for l in range(nL)])
+    yp = B.ptr_array([t.data_ptr() for t in stack.y])
+    yhp = B.ptr_array([t.data_ptr() for t in yh])
+    flags = 0 if distinct else B.DP_PLAN_SAME_X
+    times = []
+    for it in range(3):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.dp_plan_run_host(stack.plan, stack.kept, xp, stage, yp, last, yhp, stack.workspace, stack.status, flags)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    ms = min(times[1:])
+    return {"value": world * ops_step / (ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms,
+            "h2d_bytes_per_step": xbytes * nS, "d2h_bytes_per_step": M * N * 2 * nS,
+            "host_inputs": "distinct per timestep" if distinct else "one timestep's buffers re-copied every timestep"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

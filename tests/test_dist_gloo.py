@@ -1,0 +1,66 @@
+"""Multi-rank plumbing on CPU (gloo, world_size 2): the row sharding partitions the batch, the
+sharded oracle results concatenate to the unsharded result (no exchange step exists on this path),
+and the timing reduction takes the max over ranks."""
+import os
+import socket
+import sys
+
+import numpy as np
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    p = s.getsockname()[1]
+    s.close()
+    return p
+
+
+def _worker(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    import oracle
+    from paper_2511_11446_b200 import dist as D, synth
+    r, lr, w = D.init("gloo")
+    assert (r, w) == (rank, world)
+    M, K, N, bits = 300, 256, 64, 4
+    lo, hi = D.shard_rows(M, r, w, multiple=128)
+    x = synth.activations(3, 0, 0, M, K, 1.0, n_out=2)
+    wq, s_w = synth.weights(3, 0, N, K, bits)
+    y = oracle.wq_linear(np.ascontiguousarray(x[lo:hi]), oracle.pack(wq, bits), s_w, None, bits)
+    np.save(os.path.join(out_dir, f"y{rank}.npy"), y)
+    np.save(os.path.join(out_dir, f"r{rank}.npy"), np.array([lo, hi]))
+    D.barrier()
+    mx = D.max_over_ranks(10.0 + rank)
+    sm = D.sum_over_ranks(1.0 + rank)
+    assert mx == 10.0 + world - 1 and sm == sum(range(1, world + 1))
+    assert D.rank_seed(5, 0) != D.rank_seed(5, 1)
+
+
+def test_two_ranks_shard_rows_without_collective(tmp_path):
+    world = 2
+    mp.spawn(_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    sys.path.insert(0, ROOT)
+    import oracle
+    from paper_2511_11446_b200 import synth
+    M, K, N, bits = 300, 256, 64, 4
+    x = synth.activations(3, 0, 0, M, K, 1.0, n_out=2)
+    wq, s_w = synth.weights(3, 0, N, K, bits)
+    full = oracle.wq_linear(x, oracle.pack(wq, bits), s_w, None, bits)
+    rs = [np.load(tmp_path / f"r{r}.npy") for r in range(world)]
+    assert rs[0][0] == 0 and rs[0][1] == rs[1][0] and rs[1][1] == M
+    assert np.array_equal(np.concatenate([np.load(tmp_path / f"y{r}.npy") for r in range(world)]), full)
+
+
+def test_shard_rows_partitions():
+    from paper_2511_11446_b200.dist import shard_rows
+    for M in (0, 1, 127, 128, 300, 2048, 32768):
+        for world in (1, 2, 3, 8):
+            for mult in (1, 128):
+                spans = [shard_rows(M, r, world, mult) for r in range(world)]
+                assert spans[0][0] == 0 and spans[-1][1] == M
+                assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))

@@ -1,0 +1,130 @@
+"""GPU parity of dp_plan_run (Algorithm 2, Phase B over the linears) against the oracle."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_11446_b200 import binding as B, synth
+from gpu_util import DevLayer, to_dev_bf16, bf16_to_np
+from helpers import bf16_ulp_dist
+
+pytestmark = pytest.mark.gpu
+SEED = synth.BASE_SEED + 4
+
+
+def _mini_plan(tokens=256, batch=2, blocks=2):
+    """A scaled-down DiT stack: same five linears per block, mixed {3,4,8} plan."""
+    table = synth.dit_layers(batch, tokens, blocks)
+    bits = synth.bit_plan(SEED, len(table))
+    layers, dev = [], []
+    for l, (name, M, K, N) in enumerate(table):
+        w, s_w = synth.weights(SEED, l, N, K, bits[l])
+        b = synth.bias(SEED, l, N)
+        dev.append(DevLayer(w, s_w, b, bits[l]))
+        layers.append(dict(M=M, N=N, K=K, bits=bits[l], qweight=oracle.pack(w, bits[l]), s_w=s_w, bias=b))
+    return table, layers, dev
+
+
+def test_plan_run_matches_oracle_every_step_and_layer():
+    table, layers, dev = _mini_plan()
+    T = 10
+    kept = synth.kept_timesteps(SEED, T, 4, 0.2)
+    nL, nS = len(layers), len(kept)
+    xs = [[synth.activations(SEED, l, t, L["M"], L["K"], synth.sigma_t(t, T), n_out=max(1, L["K"] // 100))
+           for l, L in enumerate(layers)] for t in kept]
+    ref = oracle.plan_run(layers, kept, xs)
+    plan = B.dp_plan_create([d.w for d in dev], [L["M"] for L in layers])
+    try:
+        ws = torch.empty(B.dp_plan_workspace(plan), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        xd = [[to_dev_bf16(xs[i][l]) for l in range(nL)] for i in range(nS)]
+        yd = [[torch.full((L["M"], L["N"]), float("nan"), dtype=torch.bfloat16, device="cuda")
+               for L in layers] for _ in range(nS)]
+        xp = B.ptr_array([xd[i][l].data_ptr() for i in range(nS) for l in range(nL)])
+        yp = B.ptr_array([yd[i][l].data_ptr() for i in range(nS) for l in range(nL)])
+        B.dp_plan_run(plan, kept, 0, xp, yp, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for i in range(nS):
+            for l in range(nL):
+                d = bf16_ulp_dist(bf16_to_np(yd[i][l]), ref[i][l])
+                assert d.max() <= 1, (i, l, table[l], int(d.max()))
+        # resume: with start_index = 1 the last kept step (visited first) is skipped
+        for i in range(nS):
+            for l in range(nL):
+                yd[i][l].fill_(float("nan"))
+        B.dp_plan_run(plan, kept, 1, xp, yp, ws, status)
+        torch.cuda.synchronize()
+        assert torch.isnan(yd[nS - 1][0].float()).all()
+        assert bf16_ulp_dist(bf16_to_np(yd[0][1]), ref[0][1]).max() <= 1
+        # SAME_Y: every step overwrites one output set; the last write is kept[0]'s (reverse order)
+        ys = [torch.empty((L["M"], L["N"]), dtype=torch.bfloat16, device="cuda") for L in layers]
+        B.dp_plan_run(plan, kept, 0, xp, B.ptr_array([t.data_ptr() for t in ys]), ws, status,
+                      flags=B.DP_PLAN_SAME_Y)
+        torch.cuda.synchronize()
+        for l in range(nL):
+            assert bf16_ulp_dist(bf16_to_np(ys[l]), ref[0][l]).max() <= 1
+        # the same run captured in a CUDA graph and replayed
+        g = torch.cuda.CUDAGraph()
+        for t in ys:
+            t.zero_()
+        side = torch.cuda.Stream()
+        with torch.cuda.graph(g, stream=side):
+            B.dp_plan_run(plan, kept, 0, xp, B.ptr_array([t.data_ptr() for t in ys]), ws, status,
+                          flags=B.DP_PLAN_SAME_Y)
+        g.replay()
+        torch.cuda.synchronize()
+        for l in range(nL):
+            assert bf16_ulp_dist(bf16_to_np(ys[l]), ref[0][l]).max() <= 1
+        assert int(status.item()) == 0
+    finally:
+        B.dp_plan_destroy(plan)
+
+
+def test_plan_run_host_inputs():
+    table, layers, dev = _mini_plan(tokens=128, batch=2, blocks=1)
+    kept = [1, 3, 4]
+    nL, nS = len(layers), len(kept)
+    xs = [[synth.activations(SEED, l, t, L["M"], L["K"], 1.0, n_out=3) for l, L in enumerate(layers)]
+          for t in kept]
+    ref = oracle.plan_run(layers, kept, xs)
+    plan = B.dp_plan_create([d.w for d in dev], [L["M"] for L in layers])
+    try:
+        ws = torch.empty(B.dp_plan_workspace(plan), dtype=torch.uint8, device="cuda")
+        stage = torch.empty(2 * B.dp_plan_x_bytes(plan), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        xh = [[torch.from_numpy(xs[i][l].view(np.int16).copy()).pin_memory() for l in range(nL)] for i in range(nS)]
+        yd = [torch.empty((L["M"], L["N"]), dtype=torch.bfloat16, device="cuda") for L in layers]
+        last = nL - 2  # fc2 of the block
+        yh = [torch.empty((layers[last]["M"], layers[last]["N"]), dtype=torch.bfloat16).pin_memory()
+              for _ in range(nS)]
+        B.dp_plan_run_host(plan, kept, B.ptr_array([xh[i][l].data_ptr() for i in range(nS) for l in range(nL)]),
+                           stage, B.ptr_array([t.data_ptr() for t in yd]), last,
+                           B.ptr_array([t.data_ptr() for t in yh]), ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for i in range(nS):
+            got = yh[i].view(torch.int16).numpy().view(np.uint16)
+            assert bf16_ulp_dist(got, ref[i][last]).max() <= 1
+    finally:
+        B.dp_plan_destroy(plan)
+
+
+def test_plan_errors():
+    table, layers, dev = _mini_plan(tokens=128, batch=1, blocks=1)
+    bad = B.make_weight(dev[0].qweight, dev[0].s_w, None, dev[0].N, dev[0].K, 7)
+    with pytest.raises(B.DiffproError) as e:
+        B.dp_plan_create([bad], [128])
+    assert e.value.status == B.DP_ERR_BITS
+    plan = B.dp_plan_create([dev[0].w], [128])
+    try:
+        small = torch.empty(256, dtype=torch.uint8, device="cuda")
+        x = torch.zeros((128, dev[0].K), dtype=torch.bfloat16, device="cuda")
+        y = torch.zeros((128, dev[0].N), dtype=torch.bfloat16, device="cuda")
+        with pytest.raises(B.DiffproError) as e:
+            B.dp_plan_run(plan, [0], 0, B.ptr_array([x.data_ptr()]), B.ptr_array([y.data_ptr()]), small)
+        assert e.value.status == B.DP_ERR_WORKSPACE
+    finally:
+        B.dp_plan_destroy(plan)
