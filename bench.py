@@ -257,13 +257,13 @@ def measure_mma_peak():
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
     iters = 20000
-    B.dp_bench_mma_i8(sms, 2000, st)
+    B.dp_bench_mma_i8(sms, 2000, 256, st)
     torch.cuda.synchronize()
     best = 0.0
     for _ in range(3):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        B.dp_bench_mma_i8(sms, iters, st)
+        B.dp_bench_mma_i8(sms, iters, 256, st)
         e1.record()
         torch.cuda.synchronize()
         best = max(best, 2.0 * 128 * 256 * 128 * iters * sms / (e0.elapsed_time(e1) * 1e-3) / 1e12)
@@ -313,7 +313,20 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sweep", default=None, choices=["c1", "c2", "c3", "c4", "c5"],
+                    help="per-shape timing table (one JSON line per layer shape and bit-width) instead of the plan run")
+    ap.add_argument("--bits", default="3,4,8")
+    ap.add_argument("--layers", default=None, help="comma list out of qkv,proj,fc1,fc2,adaln")
+    ap.add_argument("--only", default=None, choices=["layer", "gemm", "daq"])
+    ap.add_argument("--iters", type=int, default=None)
     args = ap.parse_args()
+    if args.sweep:
+        import torch
+        from paper_2511_11446_b200 import sweep
+        torch.cuda.set_device(0)
+        sweep.run(args.sweep, [int(b) for b in args.bits.split(",")], measured_peaks(), only=args.only,
+                  layers=args.layers.split(",") if args.layers else None, iters=args.iters)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)

@@ -85,6 +85,10 @@ typedef struct dp_debug {
 #define DP_FLAG_FORCE_SIMT 1u   /* route through the CUDA-core weight-streaming kernel (any M)   */
 #define DP_FLAG_FORCE_MMA 2u    /* route through the tcgen05 kernel even for small M              */
 #define DP_FLAG_NO_PDL 4u       /* do not use programmatic dependent launch between the kernels  */
+/* Tuning/testing: force the tensor-core kernel's tile width in output channels (64, 128, 192 or
+ * 256; must divide N) instead of letting the library choose. */
+#define DP_FLAG_TILE_N(bn) ((uint32_t)((bn) / 64) << 8)
+#define DP_FLAG_TILE_N_MASK 0x700u
 
 /* flags for dp_plan_run */
 #define DP_PLAN_SAME_X 1u       /* x_ptrs has n_layers entries reused by every step              */
@@ -183,11 +187,13 @@ int dp_plan_run_host(const dp_plan* plan, const int32_t* steps, int32_t n_steps,
 int dp_pack_weights_host(const int8_t* w, int32_t N, int32_t K, int32_t bits, void* out);
 
 /*
- * Measurement helper: runs `iters` back-to-back tcgen05 kind::i8 MMAs (128 x 256 x 32 each) per
- * SM on operands resident in shared memory, no global loads; used to establish the measured INT8
- * tensor ceiling of the device. Enqueues one kernel on `stream`; ops = 2*128*256*32*iters*ctas.
+ * Measurement helper: each of `ctas` CTAs issues `iters` groups of four back-to-back tcgen05
+ * kind::i8 MMAs (128 x tile_n x 32 each; tile_n a multiple of 16 up to 256) on operands resident in
+ * shared memory, no global loads; used to establish the measured INT8 tensor ceiling of the device.
+ * Enqueues one kernel on `stream`; ops = 2*128*tile_n*128*iters*ctas.
  */
-int dp_bench_mma_i8(int32_t ctas, int32_t iters, int32_t* device_status, dp_stream stream);
+int dp_bench_mma_i8(int32_t ctas, int32_t iters, int32_t tile_n, int32_t* device_status,
+                    dp_stream stream);
 
 const char* dp_status_string(int status);
 const char* dp_last_error(void);

@@ -21,6 +21,10 @@ DP_OK = 0
 DP_FLAG_NONE, DP_FLAG_FORCE_SIMT, DP_FLAG_FORCE_MMA, DP_FLAG_NO_PDL = 0, 1, 2, 4
 DP_PLAN_SAME_X, DP_PLAN_SAME_Y = 1, 2
 
+
+def DP_FLAG_TILE_N(bn: int) -> int:
+    return (bn // 64) << 8
+
 EXPORTS = ["dp_daq_quantize", "dp_wq_linear_workspace", "dp_wq_linear", "dp_plan_create",
            "dp_plan_workspace", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
            "dp_plan_run_host", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_status_string",
@@ -79,7 +83,7 @@ def lib():
                                        C.POINTER(C.c_void_p), C.c_int32, C.POINTER(C.c_void_p),
                                        C.c_void_p, C.c_size_t, C.c_void_p, C.c_uint32, C.c_void_p]
         L.dp_pack_weights_host.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
-        L.dp_bench_mma_i8.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.dp_bench_mma_i8.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -173,8 +177,9 @@ def dp_pack_weights_host(w, bits: int):
     return out
 
 
-def dp_bench_mma_i8(ctas, iters, device_status=None, stream=None):
-    _check(lib().dp_bench_mma_i8(ctas, iters, _ptr(device_status), _stream(stream)), "dp_bench_mma_i8")
+def dp_bench_mma_i8(ctas, iters, tile_n=256, device_status=None, stream=None):
+    _check(lib().dp_bench_mma_i8(ctas, iters, tile_n, _ptr(device_status), _stream(stream)),
+           "dp_bench_mma_i8")
 
 
 def dp_version() -> int:

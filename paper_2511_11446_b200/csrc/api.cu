@@ -48,6 +48,10 @@ int check_device() {
 
 static size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
 
+constexpr uint32_t kLinearFlags =
+    DP_FLAG_FORCE_SIMT | DP_FLAG_FORCE_MMA | DP_FLAG_NO_PDL | DP_FLAG_TILE_N_MASK;
+static int forced_bn(uint32_t flags) { return static_cast<int>((flags & DP_FLAG_TILE_N_MASK) >> 8) * 64; }
+
 constexpr int64_t kSimtMaxRows = 32;  // at or below this the CUDA-core streaming kernel is used
 
 static bool use_simt(int64_t M, int32_t N, int32_t K, uint32_t flags) {
@@ -73,10 +77,13 @@ static int check_weight(const dp_weight* w) {
 }
 
 // One layer, all checks done. tmap_w may be a pre-encoded descriptor (plan) or nullptr.
+// `chained`: the kernel preceding this layer's first launch on the stream is a launch of the same
+// dp_plan_run call, so it cannot be a producer of this layer's weights and they may be prefetched
+// while it drains.
 static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_a_in, int64_t M,
                       void* y, int64_t ldy, void* workspace, const dp_debug* dbg, int32_t* status,
                       uint32_t flags, cudaStream_t stream, const CUtensorMap* tmap_w, int bn,
-                      const CUtensorMap* tmap_a_cached) {
+                      const CUtensorMap* tmap_a_cached, const CUtensorMap* tmap_y_cached, bool chained) {
   const bool pdl = !(flags & DP_FLAG_NO_PDL);
   if (use_simt(M, w->N, w->K, flags)) {
     if (static_cast<size_t>(w->K) > simt_max_k())
@@ -99,15 +106,18 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
     a.dbg_sa = dbg ? dbg->s_a : nullptr;
     a.dbg_acc = dbg ? dbg->acc : nullptr;
     a.dbg_ldacc = dbg ? dbg->ldacc : 0;
+    a.early_w = chained ? 1 : 0;
     return launch_simt_linear(a, stream, pdl);
   }
   const int8_t* q;
   const float* s_a;
   int64_t ldq;
+  int korder = KORDER_NATURAL;
   if (s_a_in == nullptr) {
     int8_t* wq = static_cast<int8_t*>(workspace);
     float* wsa = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align256(static_cast<size_t>(M) * w->K));
-    int st = launch_daq(x, M, w->K, ldx, wq, w->K, wsa, nullptr, stream, pdl);
+    korder = gemm_korder(w->bits);
+    int st = launch_daq(x, M, w->K, ldx, wq, w->K, wsa, nullptr, korder, stream, pdl);
     if (st != DP_OK) return st;
     q = wq;
     s_a = wsa;
@@ -118,17 +128,25 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
     ldq = ldx;
   }
   GemmProblem g;
+  g.korder = korder;
+  g.early_w = (s_a_in == nullptr) ? 1 : 0;
   if (tmap_a_cached != nullptr) {
     g.tmap_a = *tmap_a_cached;
   } else {
     int st = gemm_encode_a(&g.tmap_a, q, M, w->K, ldq);
     if (st != DP_OK) return st;
   }
-  if (bn == 0) bn = gemm_pick_bn(M, w->N, w->K, w->bits);
+  if (bn == 0) bn = forced_bn(flags) ? forced_bn(flags) : gemm_pick_bn(M, w->N, w->K, w->bits);
   if (tmap_w != nullptr) {
     g.tmap_w = *tmap_w;
   } else {
     int st = gemm_encode_w(&g.tmap_w, w->qweight, w->N, w->K, w->bits, bn);
+    if (st != DP_OK) return st;
+  }
+  if (tmap_y_cached != nullptr) {
+    g.tmap_y = *tmap_y_cached;
+  } else {
+    int st = gemm_encode_y(&g.tmap_y, y, M, w->N, ldy);
     if (st != DP_OK) return st;
   }
   g.s_a = s_a;
@@ -147,8 +165,15 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
   int st = launch_gemm(g, stream, pdl);
   if (st != DP_OK) return st;
   if (dbg != nullptr) {
-    if (dbg->q != nullptr)
-      DP_CUDA_OK(cudaMemcpy2DAsync(dbg->q, dbg->ldq, q, ldq, w->K, M, cudaMemcpyDeviceToDevice, stream));
+    if (dbg->q != nullptr) {
+      if (korder != KORDER_NATURAL) {  // the scratch holds a permuted copy: quantize again, in order
+        st = launch_daq(x, M, w->K, ldx, dbg->q, dbg->ldq, const_cast<float*>(s_a), nullptr, KORDER_NATURAL,
+                        stream, false);
+        if (st != DP_OK) return st;
+      } else {
+        DP_CUDA_OK(cudaMemcpy2DAsync(dbg->q, dbg->ldq, q, ldq, w->K, M, cudaMemcpyDeviceToDevice, stream));
+      }
+    }
     if (dbg->s_a != nullptr)
       DP_CUDA_OK(cudaMemcpyAsync(dbg->s_a, s_a, sizeof(float) * M, cudaMemcpyDeviceToDevice, stream));
   }
@@ -161,8 +186,9 @@ static int check_linear_args(const dp_weight* w, const void* x, int64_t ldx, con
   int st = check_weight(w);
   if (st != DP_OK) return st;
   if (M < 0) return fail(DP_ERR_SHAPE, "M=%lld is negative", (long long)M);
-  if (flags & ~(DP_FLAG_FORCE_SIMT | DP_FLAG_FORCE_MMA | DP_FLAG_NO_PDL))
-    return fail(DP_ERR_INVALID_ARG, "unknown flag bits 0x%x", flags);
+  if (flags & ~kLinearFlags) return fail(DP_ERR_INVALID_ARG, "unknown flag bits 0x%x", flags);
+  if (forced_bn(flags) != 0 && (forced_bn(flags) > 256 || w->N % forced_bn(flags)))
+    return fail(DP_ERR_SHAPE, "forced tile width %d does not divide N=%d", forced_bn(flags), w->N);
   if ((flags & DP_FLAG_FORCE_SIMT) && (flags & DP_FLAG_FORCE_MMA))
     return fail(DP_ERR_INVALID_ARG, "FORCE_SIMT and FORCE_MMA are exclusive");
   if (M == 0) return DP_OK;
@@ -207,7 +233,7 @@ extern "C" int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, cons
   st = check_device();
   if (st != DP_OK) return st;
   return run_linear(w, x, ldx, s_a_in, M, y_bf16, ldy, workspace, dbg, device_status, flags,
-                    static_cast<cudaStream_t>(stream), nullptr, 0, nullptr);
+                    static_cast<cudaStream_t>(stream), nullptr, 0, nullptr, nullptr, false);
 }
 
 // ---- plans ---------------------------------------------------------------------------------------
@@ -224,12 +250,17 @@ struct TmapACache {
   int64_t M, K;
   CUtensorMap map;
 };
+struct TmapYCache {  // one entry per layer: the descriptor of the output buffer last used
+  const void* ptr = nullptr;
+  CUtensorMap map;
+};
 struct dp_plan {
   std::vector<PlanLayer> layers;
   uint32_t flags;
   size_t workspace_bytes;
   size_t x_bytes;
   std::vector<TmapACache> a_cache;
+  std::vector<TmapYCache> y_cache;
   cudaStream_t copy_stream;
   cudaEvent_t ev_copied[2], ev_consumed[2];
 };
@@ -240,8 +271,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
   *out = nullptr;
   if (!layers || !M_per_layer || n_layers <= 0)
     return fail(DP_ERR_INVALID_ARG, "layers/M_per_layer NULL or n_layers <= 0");
-  if (flags & ~(DP_FLAG_FORCE_SIMT | DP_FLAG_FORCE_MMA | DP_FLAG_NO_PDL))
-    return fail(DP_ERR_INVALID_ARG, "unknown flag bits 0x%x", flags);
+  if (flags & ~kLinearFlags) return fail(DP_ERR_INVALID_ARG, "unknown flag bits 0x%x", flags);
   int st = check_device();
   if (st != DP_OK) return st;
   dp_plan* p = new (std::nothrow) dp_plan();
@@ -269,7 +299,8 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
       return fail(DP_ERR_SHAPE, "layer %d: K too large for the small-M kernel", l);
     }
     if (!L.simt && L.M > 0) {
-      L.bn = gemm_pick_bn(L.M, L.w.N, L.w.K, L.w.bits);
+      L.bn = (forced_bn(flags) && L.w.N % forced_bn(flags) == 0) ? forced_bn(flags)
+                                                                 : gemm_pick_bn(L.M, L.w.N, L.w.K, L.w.bits);
       st = gemm_encode_w(&L.tmap_w, L.w.qweight, L.w.N, L.w.K, L.w.bits, L.bn);
       if (st != DP_OK) {
         delete p;
@@ -282,6 +313,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
     p->x_bytes += align256(static_cast<size_t>(L.M) * L.w.K * 2);
     p->layers.push_back(L);
   }
+  p->y_cache.resize(p->layers.size());
   cudaError_t e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
   for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
     e = cudaEventCreateWithFlags(&p->ev_copied[i], cudaEventDisableTiming);
@@ -325,7 +357,7 @@ static const CUtensorMap* cached_tmap_a(dp_plan* plan, const void* ws, int64_t M
 }
 
 static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, void* workspace,
-                         int32_t* status, cudaStream_t stream) {
+                         int32_t* status, cudaStream_t stream, bool* chained) {
   const int n = static_cast<int>(plan->layers.size());
   for (int l = 0; l < n; ++l) {
     const PlanLayer& L = plan->layers[l];
@@ -333,14 +365,23 @@ static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, 
     if (!xs[l] || !ys[l]) return fail(DP_ERR_INVALID_ARG, "layer %d: NULL x or y", l);
     if (!aligned16(xs[l]) || !aligned16(ys[l])) return fail(DP_ERR_ALIGN, "layer %d: x/y misaligned", l);
     const CUtensorMap* ta = nullptr;
+    const CUtensorMap* ty = nullptr;
     if (!L.simt) {
       int st = DP_OK;
       ta = cached_tmap_a(plan, workspace, L.M, L.w.K, &st);
       if (st != DP_OK) return st;
+      TmapYCache& yc = plan->y_cache[l];
+      if (yc.ptr != ys[l]) {
+        st = gemm_encode_y(&yc.map, ys[l], L.M, L.w.N, L.w.N);
+        if (st != DP_OK) return st;
+        yc.ptr = ys[l];
+      }
+      ty = &yc.map;
     }
     int st = run_linear(&L.w, xs[l], L.w.K, nullptr, L.M, ys[l], L.w.N, workspace, nullptr, status,
-                        plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, ta);
+                        plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, ta, ty, *chained);
     if (st != DP_OK) return st;
+    *chained = true;
   }
   return DP_OK;
 }
@@ -366,10 +407,11 @@ extern "C" int dp_plan_run(const dp_plan* plan_c, const int32_t* steps, int32_t 
   if (st != DP_OK) return st;
   dp_plan* plan = const_cast<dp_plan*>(plan_c);
   const int64_t n = static_cast<int64_t>(plan->layers.size());
+  bool chained = false;
   for (int32_t i = n_steps - 1 - start_index; i >= 0; --i) {  // reverse(K*)
     const void* const* xs = x_ptrs + ((flags & DP_PLAN_SAME_X) ? 0 : i * n);
     void* const* ys = y_ptrs + ((flags & DP_PLAN_SAME_Y) ? 0 : i * n);
-    st = plan_run_step(plan, xs, ys, workspace, device_status, static_cast<cudaStream_t>(stream));
+    st = plan_run_step(plan, xs, ys, workspace, device_status, static_cast<cudaStream_t>(stream), &chained);
     if (st != DP_OK) return st;
   }
   return DP_OK;
@@ -408,7 +450,8 @@ extern "C" int dp_plan_run_host(const dp_plan* plan_c, const int32_t* steps, int
     }
     DP_CUDA_OK(cudaEventRecord(plan->ev_copied[h], plan->copy_stream));
     DP_CUDA_OK(cudaStreamWaitEvent(stream, plan->ev_copied[h], 0));
-    st = plan_run_step(plan, xs.data(), y_dev, workspace, device_status, stream);
+    bool chained = false;  // an event wait precedes every step's first launch
+    st = plan_run_step(plan, xs.data(), y_dev, workspace, device_status, stream, &chained);
     if (st != DP_OK) return st;
     DP_CUDA_OK(cudaEventRecord(plan->ev_consumed[h], stream));
     if (d2h_layer >= 0) {

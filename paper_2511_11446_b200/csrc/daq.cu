@@ -33,10 +33,18 @@ __device__ __forceinline__ uint32_t quant_pair(uint32_t w, float inv) {
   return __byte_perm(a, b, 0x0040);  // byte0 = a.byte0, byte1 = b.byte0
 }
 
+// Eight consecutive codes. EO = false: stored in order; EO = true: stored as k = 0,2,4,6,1,3,5,7.
+template <bool EO>
 __device__ __forceinline__ uint2 quant_vec(const uint4& v, float inv) {
   uint32_t p0 = quant_pair(v.x, inv), p1 = quant_pair(v.y, inv);
   uint32_t p2 = quant_pair(v.z, inv), p3 = quant_pair(v.w, inv);
-  return make_uint2(__byte_perm(p0, p1, 0x5410), __byte_perm(p2, p3, 0x5410));
+  if constexpr (EO) {
+    const uint32_t t0 = __byte_perm(p0, p1, 0x5140);  // k0 k2 k1 k3
+    const uint32_t t1 = __byte_perm(p2, p3, 0x5140);  // k4 k6 k5 k7
+    return make_uint2(__byte_perm(t0, t1, 0x5410), __byte_perm(t0, t1, 0x7632));
+  } else {
+    return make_uint2(__byte_perm(p0, p1, 0x5410), __byte_perm(p2, p3, 0x5410));
+  }
 }
 
 // Scale and reciprocal of one token from its absmax magnitude bits (a bf16 pattern, sign cleared).
@@ -65,7 +73,7 @@ __device__ __forceinline__ int warp_sum_i32(int s) {
 constexpr int kDaqWarps = 8;
 
 // MAXV = 16-byte vectors held per lane (row of up to 256*MAXV elements in registers).
-template <int MAXV>
+template <int MAXV, bool EO>
 __global__ void __launch_bounds__(kDaqWarps * 32)
 daq_rows_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t ldx,
                 int8_t* __restrict__ q, int64_t ldq, float* __restrict__ s_a,
@@ -101,7 +109,7 @@ daq_rows_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t ldx,
   for (int i = 0; i < MAXV; ++i) {
     const int idx = lane + 32 * i;
     if (idx < nvec) {
-      uint2 o = quant_vec(v[i], inv);
+      uint2 o = quant_vec<EO>(v[i], inv);
       qr[idx] = o;
       sum = __dp4a(static_cast<int>(o.x), 0x01010101, sum);
       sum = __dp4a(static_cast<int>(o.y), 0x01010101, sum);
@@ -115,6 +123,7 @@ daq_rows_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t ldx,
 }
 
 // Any K (multiple of 8): two passes over the row, the second served by L1/L2.
+template <bool EO>
 __global__ void __launch_bounds__(kDaqWarps * 32)
 daq_rows_2pass_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t ldx,
                       int8_t* __restrict__ q, int64_t ldq, float* __restrict__ s_a,
@@ -137,7 +146,7 @@ daq_rows_2pass_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t 
   uint2* qr = reinterpret_cast<uint2*>(q + row * ldq);
   int sum = 0;
   for (int idx = lane; idx < nvec; idx += 32) {
-    uint2 o = quant_vec(xr[idx], inv);
+    uint2 o = quant_vec<EO>(xr[idx], inv);
     qr[idx] = o;
     sum = __dp4a(static_cast<int>(o.x), 0x01010101, sum);
     sum = __dp4a(static_cast<int>(o.y), 0x01010101, sum);
@@ -149,24 +158,28 @@ daq_rows_2pass_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t 
   }
 }
 
-int launch_daq(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq,
-               float* s_a, int32_t* rowsum, cudaStream_t stream, bool pdl) {
-  if (M == 0) return DP_OK;
+template <bool EO>
+static cudaError_t launch_daq_t(const uint16_t* xp, int64_t M, int k, int64_t ldx, int8_t* q, int64_t ldq,
+                                float* s_a, int32_t* rowsum, cudaStream_t stream, bool pdl) {
   const dim3 grid(static_cast<unsigned>((M + kDaqWarps - 1) / kDaqWarps));
   const dim3 block(kDaqWarps * 32);
+  if (k <= 256 * 5)
+    return launch(daq_rows_kernel<5, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum);
+  if (k <= 256 * 9)
+    return launch(daq_rows_kernel<9, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum);
+  if (k <= 256 * 18)
+    return launch(daq_rows_kernel<18, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum);
+  return launch(daq_rows_2pass_kernel<EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum);
+}
+
+int launch_daq(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq,
+               float* s_a, int32_t* rowsum, int korder, cudaStream_t stream, bool pdl) {
+  if (M == 0) return DP_OK;
   const uint16_t* xp = static_cast<const uint16_t*>(x);
   const int k = static_cast<int>(K);
-  cudaError_t e;
-  if (K <= 256 * 5)
-    e = launch(daq_rows_kernel<5>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum);
-  else if (K <= 256 * 9)
-    e = launch(daq_rows_kernel<9>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum);
-  else if (K <= 256 * 18)
-    e = launch(daq_rows_kernel<18>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a,
-               rowsum);
-  else
-    e = launch(daq_rows_2pass_kernel, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a,
-               rowsum);
+  const cudaError_t e = korder == KORDER_EVEN_ODD
+                            ? launch_daq_t<true>(xp, M, k, ldx, q, ldq, s_a, rowsum, stream, pdl)
+                            : launch_daq_t<false>(xp, M, k, ldx, q, ldq, s_a, rowsum, stream, pdl);
   if (e != cudaSuccess) return fail(DP_ERR_CUDA, "DAQ launch failed: %s", cudaGetErrorString(e));
   return DP_OK;
 }
@@ -187,6 +200,6 @@ extern "C" int dp_daq_quantize(const void* x_bf16, int64_t M, int64_t K, int64_t
     return fail(DP_ERR_ALIGN, "dp_daq_quantize: pointers/pitches must be 16-byte aligned");
   int st = check_device();
   if (st != DP_OK) return st;
-  return launch_daq(x_bf16, M, K, ldx, q, ldq, s_a, rowsum, static_cast<cudaStream_t>(stream),
-                    false);
+  return launch_daq(x_bf16, M, K, ldx, q, ldq, s_a, rowsum, KORDER_NATURAL,
+                    static_cast<cudaStream_t>(stream), false);
 }

@@ -9,9 +9,17 @@
 
 namespace dp {
 
+// Order in which the int8 codes of a token are stored along K in the activation scratch.
+enum KOrder {
+  KORDER_NATURAL = 0,   // q[k] at byte k
+  KORDER_EVEN_ODD = 1   // every group of 8 codes stored as k = 0,2,4,6,1,3,5,7 (4-bit weight path)
+};
+// The order the tensor-core path wants for weights of this width when it runs DAQ itself.
+int gemm_korder(int32_t bits);
+
 // daq.cu
 int launch_daq(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq,
-               float* s_a, int32_t* rowsum, cudaStream_t stream, bool pdl);
+               float* s_a, int32_t* rowsum, int korder, cudaStream_t stream, bool pdl);
 
 // simt.cu — CUDA-core weight-streaming linear for small M (DAQ fused in the CTA prologue).
 struct SimtArgs {
@@ -30,6 +38,7 @@ struct SimtArgs {
   float* dbg_sa;
   int32_t* dbg_acc;
   int64_t dbg_ldacc;
+  int32_t early_w;  // weights may be fetched before the preceding kernel on the stream has finished
 };
 int launch_simt_linear(const SimtArgs& a, cudaStream_t stream, bool pdl);
 size_t simt_max_k();
@@ -41,6 +50,7 @@ struct GemmTile {  // kernel variant
 struct GemmProblem {
   CUtensorMap tmap_a;  // int8 activations [M][K]
   CUtensorMap tmap_w;  // packed weights, byte view [N][K*bits/8]
+  CUtensorMap tmap_y;  // bf16 outputs [M][N]
   const float* s_a;    // [M]
   const float* s_w;    // [N]
   const uint16_t* bias;
@@ -50,12 +60,16 @@ struct GemmProblem {
   int64_t dbg_ldacc;
   int64_t M;
   int32_t N, K, bits, bn;
+  int32_t korder;   // KOrder of the activations behind tmap_a
+  int32_t early_w;  // the preceding kernel on the stream is this call's own DAQ: weights may be
+                    // fetched before it has finished
   int32_t* status;
 };
 int gemm_pick_bn(int64_t M, int32_t N, int32_t K, int32_t bits);
 int gemm_encode_a(CUtensorMap* out, const int8_t* q, int64_t M, int64_t K, int64_t ldq);
 int gemm_encode_w(CUtensorMap* out, const void* qweight, int32_t N, int32_t K, int32_t bits,
                   int32_t bn);
+int gemm_encode_y(CUtensorMap* out, const void* y, int64_t M, int32_t N, int64_t ldy);
 int launch_gemm(const GemmProblem& p, cudaStream_t stream, bool pdl);
 int gemm_init();  // sets kernel attributes, resolves the tensor-map encoder; idempotent
 

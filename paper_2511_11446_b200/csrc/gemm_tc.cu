@@ -8,8 +8,14 @@
 //   warp 1      MMA issuer: tcgen05.mma kind::i8, int32 accumulators in tensor memory (two
 //               accumulator buffers, so a tile's epilogue overlaps the next tile's mainloop)
 //   warps 2-5   epilogue: tcgen05.ld -> (float)acc * s_a[m]*s_w[n] + bias -> bf16 -> global
-//   warps 6-9   unpack (3/4-bit only): packed tile in smem -> int8 operand tile in smem, written in
+//   warps 6-13  unpack (3/4-bit only): packed tile in smem -> int8 operand tile in smem, written in
 //               the swizzled layout the MMA descriptor expects, then fence.proxy.async
+//
+// K order. The contraction over k does not care in which order the k's of a 128-wide block sit in
+// the two operand tiles as long as both agree. With PERM the activations arrive (from the DAQ
+// kernel of the same call) with every group of 8 codes stored as k = 0,2,4,6,1,3,5,7, which is the
+// order two mask operations leave the nibbles of a 4-bit word in, so the expansion needs no byte
+// shuffles.
 //
 // Low-bit codes are expanded as w * 2^(8-b) (the two's-complement field moved to the top of the
 // byte: two logic ops per word instead of a sign-extension); the accumulator is then an exact
@@ -24,9 +30,13 @@ namespace dp {
 
 constexpr int BM = 128;
 constexpr int BK = 128;  // int8 elements = bytes = one 128-byte swizzle row
-constexpr int kGemmThreads = 320;
-constexpr int kEpiWarp0 = 2, kUnpackWarp0 = 6;
-constexpr int kSmemBudget = 200 * 1024;
+constexpr int kEpiWarp0 = 2, kUnpackWarp0 = 6, kUnpackWarps = 8;
+constexpr int kUnpackThreads = kUnpackWarps * 32;
+__host__ __device__ constexpr int gemm_threads(int bits) {
+  return (kUnpackWarp0 + (bits == 8 ? 0 : kUnpackWarps)) * 32;
+}
+constexpr int kYStageBytes = 32 * 128;  // per epilogue warp: 32 tokens x 64 bf16
+constexpr int kSmemBudget = 196 * 1024;
 constexpr int kPStages = 3;
 
 __host__ __device__ constexpr int p_stage_bytes(int bn, int bits) {
@@ -50,6 +60,7 @@ struct GemmParams {
   int64_t M;
   int32_t N, K;
   int32_t m_tiles, n_tiles;
+  int32_t early_w;  // weights may be fetched before the preceding kernel on the stream has finished
   int32_t* status;
 };
 
@@ -67,24 +78,25 @@ struct Ring {  // stage index + phase bit of a circular buffer
 // ---- in-smem weight expansion ------------------------------------------------------------------
 // 4-bit: tile P is [BN][64 bytes]; each thread expands 8 bytes (16 codes) into one 16-byte chunk of
 // the operand tile B = [BN][128 bytes], chunk position XOR-swizzled by (row & 7).
-template <int BN>
+template <int BN, bool PERM>
 __device__ __forceinline__ void unpack4_tile(const uint8_t* P, uint8_t* B, int tid) {
-#pragma unroll 4
-  for (int idx = tid; idx < BN * 8; idx += 128) {
+#pragma unroll
+  for (int i = 0; i < BN * 8 / kUnpackThreads; ++i) {
+    const int idx = tid + i * kUnpackThreads;
     const int row = idx >> 3, kc = idx & 7;
     const uint2 in = *reinterpret_cast<const uint2*>(P + row * 64 + kc * 8);
     uint4 o;
-    {
-      const uint32_t lo = ((in.x << 4) & 0xF0F0F0F0u) ^ 0x80808080u;  // even fields
-      const uint32_t hi = (in.x & 0xF0F0F0F0u) ^ 0x80808080u;         // odd fields
-      o.x = __byte_perm(lo, hi, 0x5140);
-      o.y = __byte_perm(lo, hi, 0x7362);
-    }
-    {
-      const uint32_t lo = ((in.y << 4) & 0xF0F0F0F0u) ^ 0x80808080u;
-      const uint32_t hi = (in.y & 0xF0F0F0F0u) ^ 0x80808080u;
-      o.z = __byte_perm(lo, hi, 0x5140);
-      o.w = __byte_perm(lo, hi, 0x7362);
+    const uint32_t lo0 = ((in.x << 4) & 0xF0F0F0F0u) ^ 0x80808080u;  // even fields
+    const uint32_t hi0 = (in.x & 0xF0F0F0F0u) ^ 0x80808080u;         // odd fields
+    const uint32_t lo1 = ((in.y << 4) & 0xF0F0F0F0u) ^ 0x80808080u;
+    const uint32_t hi1 = (in.y & 0xF0F0F0F0u) ^ 0x80808080u;
+    if constexpr (PERM) {
+      o = make_uint4(lo0, hi0, lo1, hi1);
+    } else {
+      o.x = __byte_perm(lo0, hi0, 0x5140);
+      o.y = __byte_perm(lo0, hi0, 0x7362);
+      o.z = __byte_perm(lo1, hi1, 0x5140);
+      o.w = __byte_perm(lo1, hi1, 0x7362);
     }
     *reinterpret_cast<uint4*>(B + row * 128 + ((kc ^ (row & 7)) << 4)) = o;
   }
@@ -97,8 +109,9 @@ __device__ __forceinline__ uint32_t spread3(uint32_t v) {  // 4 fields of 3 bits
 }
 template <int BN>
 __device__ __forceinline__ void unpack3_tile(const uint8_t* P, uint8_t* B, int tid) {
-#pragma unroll 2
-  for (int idx = tid; idx < BN * 4; idx += 128) {
+#pragma unroll
+  for (int i = 0; i < BN * 4 / kUnpackThreads; ++i) {
+    const int idx = tid + i * kUnpackThreads;
     const int row = idx >> 2, g = idx & 3;
     const uint32_t* src = reinterpret_cast<const uint32_t*>(P + row * 48 + g * 12);
     const uint32_t s0 = src[0], s1 = src[1], s2 = src[2];
@@ -118,23 +131,70 @@ __device__ __forceinline__ void unpack3_tile(const uint8_t* P, uint8_t* B, int t
   }
 }
 
+// ---- epilogue arithmetic -----------------------------------------------------------------------------
+// 32 accumulators of one token (half of a 64-column slab) -> bf16 into the warp's staging tile
+// [32 tokens][128 bytes], 16-byte chunks XOR-swizzled by (token & 7) as the 128-byte-swizzle TMA
+// store expects. Per element, in this order: t = (float)acc (times 2^-SHIFT, exact),
+// sc = s_a * s_w[n], y = fma(t, sc, bias[n]), bf16 round-to-nearest-even.
+template <int SHIFT>
+__device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], float sa, const float* ts,
+                                               const float* tb, uint8_t* stage_row, int half, int sw,
+                                               int32_t* acc_dst) {
+  const float4* s4 = reinterpret_cast<const float4*>(ts);
+  const float4* b4 = reinterpret_cast<const float4*>(tb);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {  // 16-byte chunk = 8 outputs
+    uint32_t o[4];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const float4 sw4 = s4[2 * j + h], bb = b4[2 * j + h];
+      float t0 = __int2float_rn(static_cast<int>(r[8 * j + 4 * h + 0]));
+      float t1 = __int2float_rn(static_cast<int>(r[8 * j + 4 * h + 1]));
+      float t2 = __int2float_rn(static_cast<int>(r[8 * j + 4 * h + 2]));
+      float t3 = __int2float_rn(static_cast<int>(r[8 * j + 4 * h + 3]));
+      if constexpr (SHIFT != 0) {
+        constexpr float kInv = 1.0f / (1 << SHIFT);
+        t0 = __fmul_rn(t0, kInv);
+        t1 = __fmul_rn(t1, kInv);
+        t2 = __fmul_rn(t2, kInv);
+        t3 = __fmul_rn(t3, kInv);
+      }
+      const float y0 = __fmaf_rn(t0, __fmul_rn(sa, sw4.x), bb.x);
+      const float y1 = __fmaf_rn(t1, __fmul_rn(sa, sw4.y), bb.y);
+      const float y2 = __fmaf_rn(t2, __fmul_rn(sa, sw4.z), bb.z);
+      const float y3 = __fmaf_rn(t3, __fmul_rn(sa, sw4.w), bb.w);
+      const __nv_bfloat162 h0 = __floats2bfloat162_rn(y0, y1);
+      const __nv_bfloat162 h1 = __floats2bfloat162_rn(y2, y3);
+      o[2 * h] = *reinterpret_cast<const uint32_t*>(&h0);
+      o[2 * h + 1] = *reinterpret_cast<const uint32_t*>(&h1);
+    }
+    *reinterpret_cast<uint4*>(stage_row + (((half * 4 + j) ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+  if (acc_dst != nullptr) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) acc_dst[j] = static_cast<int>(r[j]) >> SHIFT;
+  }
+}
+
 // ---- the kernel ----------------------------------------------------------------------------------
-template <int BN, int BITS>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+template <int BN, int BITS, bool PERM>
+__global__ void __launch_bounds__(gemm_threads(BITS), 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
-               const GemmParams p) {
+               const __grid_constant__ CUtensorMap tmap_y, const GemmParams p) {
   constexpr int NS = num_stages(BN, BITS);
   constexpr int NP = kPStages;
   constexpr int A_BYTES = BM * BK, B_BYTES = BN * BK, P_BYTES = p_stage_bytes(BN, BITS);
   constexpr int TCOLS = tmem_cols(BN);
   constexpr int SHIFT = 8 - BITS;  // accumulator carries a factor 2^SHIFT
+  constexpr int NCH = BN / 32;     // 32-column chunks per tile (even)
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem;
   uint8_t* sB = sA + NS * A_BYTES;
   uint8_t* sP = sB + NS * B_BYTES;
-  uint8_t* tail = sP + NP * P_BYTES;
+  uint8_t* sY = sP + NP * P_BYTES;  // [4 epilogue warps][32 tokens][128 bytes] output staging
+  uint8_t* tail = sY + 4 * kYStageBytes;
   uint64_t* full_a = reinterpret_cast<uint64_t*>(tail);
   uint64_t* bready = full_a + NS;
   uint64_t* empty = bready + NS;
@@ -144,7 +204,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint64_t* acc_empty = acc_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* s_scale = reinterpret_cast<float*>(tmem_slot + 4);  // [4 warps][BN] weight scales of the tile
+  float* s_scale = reinterpret_cast<float*>(                 // [4 warps][BN] weight scales of the tile
+      (reinterpret_cast<uintptr_t>(tmem_slot + 4) + 15) & ~uintptr_t(15));
   float* s_bias = s_scale + 4 * BN;                           // [4 warps][BN]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -154,12 +215,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   if (threadIdx.x == 0) {
     for (int i = 0; i < NS; ++i) {
       mbar_init(&full_a[i], 1);
-      mbar_init(&bready[i], 128);
+      mbar_init(&bready[i], kUnpackThreads);
       mbar_init(&empty[i], 1);
     }
     for (int i = 0; i < NP; ++i) {
       mbar_init(&pfull[i], 1);
-      mbar_init(&pempty[i], 128);
+      mbar_init(&pempty[i], kUnpackThreads);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&acc_full[i], 1);
@@ -169,6 +230,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     fence_barrier_init();
     tma_prefetch_desc(&tmap_a);
     tma_prefetch_desc(&tmap_w);
+    tma_prefetch_desc(&tmap_y);
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, TCOLS);
@@ -180,33 +242,55 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   const uint32_t tmem_base = *tmem_slot;
 
   pdl_launch_dependents();
-  pdl_wait();  // everything below reads what the previous kernel on the stream produced
+  // Activations and their scales come from the preceding kernel on the stream: the roles that read
+  // them wait for it (griddepcontrol.wait) right before their first such read. Weights are
+  // constants; unless early_w is set, everything waits here.
+  if (!p.early_w) pdl_wait();
 
   if (warp == 0) {
     // ================= TMA producer =================
     if (lane == 0) {
       Ring st, ps;
-      int issued = 0;
       bool ok = true;
+      bool a_open = !p.early_w;  // false until griddepcontrol.wait has been executed
+      int deferred = 0;          // stages whose weight tile is in flight but whose A tile is not
+      int def_kb[NS], def_m[NS], def_s[NS];
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int m_blk = tile % p.m_tiles, n_blk = tile / p.m_tiles;
+        const int n_blk = tile % p.n_tiles, m_blk = tile / p.n_tiles;  // column tiles of one row strip run together
         for (int kb = 0; kb < KB; ++kb) {
+          if (!a_open && deferred == NS) {  // ring full of weight tiles: now wait for the activations
+            pdl_wait();
+            a_open = true;
+            for (int d = 0; d < deferred; ++d)
+              tma_load_2d(sA + def_s[d] * A_BYTES, &tmap_a, def_kb[d] * BK, def_m[d] * BM, &full_a[def_s[d]]);
+            deferred = 0;
+          }
           if (!(ok = mbar_wait(&empty[st.s], st.ph ^ 1u, abort_flag))) break;
           if constexpr (BITS == 8) {
             mbar_arrive_expect_tx(&full_a[st.s], A_BYTES + B_BYTES);
-            tma_load_2d(sA + st.s * A_BYTES, &tmap_a, kb * BK, m_blk * BM, &full_a[st.s]);
             tma_load_2d(sB + st.s * B_BYTES, &tmap_w, kb * BK, n_blk * BN, &full_a[st.s]);
           } else {
             if (!(ok = mbar_wait(&pempty[ps.s], ps.ph ^ 1u, abort_flag))) break;
             mbar_arrive_expect_tx(&pfull[ps.s], P_BYTES);
             tma_load_2d(sP + ps.s * P_BYTES, &tmap_w, kb * (BK * BITS / 8), n_blk * BN, &pfull[ps.s]);
             mbar_arrive_expect_tx(&full_a[st.s], A_BYTES);
-            tma_load_2d(sA + st.s * A_BYTES, &tmap_a, kb * BK, m_blk * BM, &full_a[st.s]);
             ps.next(NP);
           }
+          if (a_open) {
+            tma_load_2d(sA + st.s * A_BYTES, &tmap_a, kb * BK, m_blk * BM, &full_a[st.s]);
+          } else {
+            def_kb[deferred] = kb;
+            def_m[deferred] = m_blk;
+            def_s[deferred] = st.s;
+            ++deferred;
+          }
           st.next(NS);
-          ++issued;
         }
+      }
+      if (!a_open) {  // fewer k-blocks than stages in the whole CTA
+        pdl_wait();
+        for (int d = 0; d < deferred; ++d)
+          tma_load_2d(sA + def_s[d] * A_BYTES, &tmap_a, def_kb[d] * BK, def_m[d] * BM, &full_a[def_s[d]]);
       }
       if (!ok) {
         // drain: give copies still in flight a bounded time to land before the CTA exits
@@ -250,63 +334,73 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     const int qd = warp & 3;  // TMEM lane quadrant this warp may read
     float* ts = s_scale + (warp - kEpiWarp0) * BN;  // this warp's private copy: no CTA-wide sync
     float* tb = s_bias + (warp - kEpiWarp0) * BN;
+    uint8_t* stage = sY + (warp - kEpiWarp0) * kYStageBytes;
+    uint8_t* stage_row = stage + lane * 128;
     bool ok = true;
-    int tcount = 0;
+    int tcount = 0, staged_n = -1;
+    if (p.early_w) pdl_wait();  // s_a below is written by the preceding kernel
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-      const int m_blk = tile % p.m_tiles, n_blk = tile / p.m_tiles;
+      const int n_blk = tile % p.n_tiles, m_blk = tile / p.n_tiles;  // column tiles of one row strip run together
       const int buf = tcount & 1;
       const uint32_t aph = (tcount >> 1) & 1;
       const int n0 = n_blk * BN;
-      __syncwarp();
-      for (int i = lane; i < BN; i += 32) {
-        ts[i] = p.s_w[n0 + i];
-        tb[i] = p.bias != nullptr ? __uint_as_float(static_cast<uint32_t>(p.bias[n0 + i]) << 16) : 0.0f;
-      }
-      __syncwarp();
       const int64_t row = static_cast<int64_t>(m_blk) * BM + qd * 32 + lane;
       const bool row_ok = row < p.M;
-      const float sa = row_ok ? p.s_a[row] : 0.0f;
+      // independent loads first, their latency overlaps the wait for the accumulator
+      const float sa = row_ok ? __ldg(p.s_a + row) : 0.0f;
+      if (n_blk != staged_n) {
+        float sv[NCH], bv[NCH];
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) sv[j] = __ldg(p.s_w + n0 + lane + 32 * j);
+#pragma unroll
+        for (int j = 0; j < NCH; ++j)
+          bv[j] = p.bias != nullptr
+                      ? __uint_as_float(static_cast<uint32_t>(__ldg(p.bias + n0 + lane + 32 * j)) << 16)
+                      : 0.0f;
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) {
+          ts[lane + 32 * j] = sv[j];
+          tb[lane + 32 * j] = bv[j];
+        }
+        __syncwarp();
+        staged_n = n_blk;
+      }
       ok = mbar_wait(&acc_full[buf], aph, abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + buf * (TCOLS / 2);
-      uint16_t* yrow = p.y + row * p.ldy + n0;
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld_32x32(t_addr + c * 32, r);
+      const int row0 = m_blk * BM + qd * 32;  // first token of this warp's slab
+      int32_t* arow = (p.dbg_acc != nullptr && row_ok) ? p.dbg_acc + row * p.dbg_ldacc + n0 : nullptr;
+      uint32_t ra[32], rb[32];
+      tmem_ld_32x32(t_addr, ra);
+#pragma unroll
+      for (int c = 0; c < NCH; c += 2) {  // one 64-column slab per iteration
         tmem_ld_wait();
-        if (row_ok) {
-          uint32_t o[16];
-#pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            float t0 = __int2float_rn(static_cast<int>(r[j]));
-            float t1 = __int2float_rn(static_cast<int>(r[j + 1]));
-            if constexpr (SHIFT != 0) {
-              t0 = __fmul_rn(t0, 1.0f / (1 << SHIFT));
-              t1 = __fmul_rn(t1, 1.0f / (1 << SHIFT));
-            }
-            const float y0 = __fmaf_rn(t0, __fmul_rn(sa, ts[c * 32 + j]), tb[c * 32 + j]);
-            const float y1 = __fmaf_rn(t1, __fmul_rn(sa, ts[c * 32 + j + 1]), tb[c * 32 + j + 1]);
-            const __nv_bfloat162 h = __floats2bfloat162_rn(y0, y1);
-            o[j >> 1] = *reinterpret_cast<const uint32_t*>(&h);
-          }
-          uint4* dst = reinterpret_cast<uint4*>(yrow + c * 32);
-          dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-          dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
-          dst[2] = make_uint4(o[8], o[9], o[10], o[11]);
-          dst[3] = make_uint4(o[12], o[13], o[14], o[15]);
-          if (p.dbg_acc != nullptr) {
-            int32_t* arow = p.dbg_acc + row * p.dbg_ldacc + n0 + c * 32;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) arow[j] = static_cast<int>(r[j]) >> SHIFT;
-          }
+        tmem_ld_32x32(t_addr + (c + 1) * 32, rb);
+        if (lane == 0) tma_store_wait_read<0>();  // the previous slab's store has read the staging tile
+        __syncwarp();
+        epilogue_chunk<SHIFT>(ra, sa, ts + c * 32, tb + c * 32, stage_row, 0, lane & 7,
+                              arow ? arow + c * 32 : nullptr);
+        tmem_ld_wait();
+        if (c + 2 < NCH) {
+          tmem_ld_32x32(t_addr + (c + 2) * 32, ra);
+        } else {  // every accumulator of the tile is in registers: hand the buffer back
+          tc_fence_before();
+          mbar_arrive(&acc_empty[buf]);
+        }
+        epilogue_chunk<SHIFT>(rb, sa, ts + (c + 1) * 32, tb + (c + 1) * 32, stage_row, 1, lane & 7,
+                              arow ? arow + (c + 1) * 32 : nullptr);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0 && row0 < p.M) {  // rows past M are clipped by the copy engine
+          tma_store_2d(&tmap_y, n0 + c * 32, row0, stage);
+          tma_store_commit();
         }
       }
-      tc_fence_before();
-      mbar_arrive(&acc_empty[buf]);
     }
+    if (lane == 0) tma_store_wait_all<0>();
   } else {
     // ================= unpack (3/4-bit weights) =================
     if constexpr (BITS != 8) {
@@ -319,7 +413,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                mbar_wait(&empty[st.s], st.ph ^ 1u, abort_flag);
           ok = __all_sync(0xFFFFFFFFu, ok);
           if (!ok) break;
-          if constexpr (BITS == 4) unpack4_tile<BN>(sP + ps.s * P_BYTES, sB + st.s * B_BYTES, ut);
+          if constexpr (BITS == 4) unpack4_tile<BN, PERM>(sP + ps.s * P_BYTES, sB + st.s * B_BYTES, ut);
           else unpack3_tile<BN>(sP + ps.s * P_BYTES, sB + st.s * B_BYTES, ut);
           fence_proxy_async_smem();
           mbar_arrive(&bready[st.s]);
@@ -345,7 +439,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 template <int BN, int BITS>
 constexpr size_t gemm_smem_bytes() {
   return 1024 + static_cast<size_t>(num_stages(BN, BITS)) * ab_stage_bytes(BN) +
-         kPStages * p_stage_bytes(BN, BITS) + (3 * 8 + 2 * kPStages + 4) * 8 + 16 + 8 * BN * 4 + 64;
+         kPStages * p_stage_bytes(BN, BITS) + 4 * kYStageBytes + (3 * 8 + 2 * kPStages + 4) * 8 + 32 +
+         8 * BN * 4 + 64;
 }
 
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -355,13 +450,15 @@ using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, voi
 static EncodeFn g_encode = nullptr;
 static int g_num_sms = 0;
 
-template <int BN, int BITS>
+template <int BN, int BITS, bool PERM>
 static cudaError_t set_attr() {
-  return cudaFuncSetAttribute(gemm_i8_kernel<BN, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  return cudaFuncSetAttribute(gemm_i8_kernel<BN, BITS, PERM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               static_cast<int>(gemm_smem_bytes<BN, BITS>()));
 }
 
 int num_sms() { return g_num_sms; }
+
+int gemm_korder(int32_t bits) { return bits == 4 ? KORDER_EVEN_ODD : KORDER_NATURAL; }
 
 int gemm_init() {
   static int state = -1;  // -1 not tried, else status
@@ -376,9 +473,10 @@ int gemm_init() {
   DP_CUDA_OK(cudaGetDevice(&dev));
   DP_CUDA_OK(cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev));
 #define DP_SET(BN)                               \
-  DP_CUDA_OK((set_attr<BN, 8>()));               \
-  DP_CUDA_OK((set_attr<BN, 4>()));               \
-  DP_CUDA_OK((set_attr<BN, 3>()));
+  DP_CUDA_OK((set_attr<BN, 8, false>()));        \
+  DP_CUDA_OK((set_attr<BN, 4, false>()));        \
+  DP_CUDA_OK((set_attr<BN, 4, true>()));         \
+  DP_CUDA_OK((set_attr<BN, 3, false>()));
   DP_SET(64) DP_SET(128) DP_SET(192) DP_SET(256)
 #undef DP_SET
   state = DP_OK;
@@ -386,12 +484,14 @@ int gemm_init() {
 }
 
 static int encode_2d(CUtensorMap* out, const void* base, uint64_t inner_bytes, uint64_t rows,
-                     uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows, bool swizzle128) {
-  const cuuint64_t dims[2] = {inner_bytes, rows};
+                     uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows, bool swizzle128,
+                     int elem_bytes = 1) {
+  const cuuint64_t dims[2] = {inner_bytes / elem_bytes, rows};
   const cuuint64_t strides[1] = {pitch_bytes};
-  const cuuint32_t box[2] = {box_inner, box_rows};
+  const cuuint32_t box[2] = {box_inner / elem_bytes, box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  CUresult r = g_encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides,
+  CUresult r = g_encode(out, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8,
+                        2, const_cast<void*>(base), dims, strides,
                         box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                         swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -407,6 +507,11 @@ int gemm_encode_w(CUtensorMap* out, const void* qweight, int32_t N, int32_t K, i
                   int32_t bn) {
   const uint64_t row_bytes = static_cast<uint64_t>(K) * bits / 8;
   return encode_2d(out, qweight, row_bytes, N, row_bytes, BK * bits / 8, bn, bits == 8);
+}
+
+// Output tensor: bf16 [M][N] with pitch ldy elements; stored in boxes of 64 columns x 32 tokens.
+int gemm_encode_y(CUtensorMap* out, const void* y, int64_t M, int32_t N, int64_t ldy) {
+  return encode_2d(out, y, static_cast<uint64_t>(N) * 2, M, static_cast<uint64_t>(ldy) * 2, 128, 32, true, 2);
 }
 
 // Tile width: the widest of {256, 192, 128, 64} dividing N whose tile count keeps the last wave
@@ -437,17 +542,20 @@ int gemm_pick_bn(int64_t M, int32_t N, int32_t K, int32_t bits) {
 template <int BN>
 static cudaError_t launch_bn(const GemmProblem& g, const GemmParams& p, dim3 grid, cudaStream_t stream,
                              bool pdl) {
-  const dim3 block(kGemmThreads);
+  const dim3 block(gemm_threads(g.bits));
   switch (g.bits) {
     case 8:
-      return launch(gemm_i8_kernel<BN, 8>, grid, block, gemm_smem_bytes<BN, 8>(), stream, pdl, g.tmap_a,
-                    g.tmap_w, p);
+      return launch(gemm_i8_kernel<BN, 8, false>, grid, block, gemm_smem_bytes<BN, 8>(), stream, pdl,
+                    g.tmap_a, g.tmap_w, g.tmap_y, p);
     case 4:
-      return launch(gemm_i8_kernel<BN, 4>, grid, block, gemm_smem_bytes<BN, 4>(), stream, pdl, g.tmap_a,
-                    g.tmap_w, p);
+      if (g.korder == KORDER_EVEN_ODD)
+        return launch(gemm_i8_kernel<BN, 4, true>, grid, block, gemm_smem_bytes<BN, 4>(), stream, pdl,
+                      g.tmap_a, g.tmap_w, g.tmap_y, p);
+      return launch(gemm_i8_kernel<BN, 4, false>, grid, block, gemm_smem_bytes<BN, 4>(), stream, pdl,
+                    g.tmap_a, g.tmap_w, g.tmap_y, p);
     default:
-      return launch(gemm_i8_kernel<BN, 3>, grid, block, gemm_smem_bytes<BN, 3>(), stream, pdl, g.tmap_a,
-                    g.tmap_w, p);
+      return launch(gemm_i8_kernel<BN, 3, false>, grid, block, gemm_smem_bytes<BN, 3>(), stream, pdl,
+                    g.tmap_a, g.tmap_w, g.tmap_y, p);
   }
 }
 
@@ -466,6 +574,7 @@ int launch_gemm(const GemmProblem& g, cudaStream_t stream, bool pdl) {
   p.K = g.K;
   p.m_tiles = static_cast<int32_t>((g.M + BM - 1) / BM);
   p.n_tiles = g.N / g.bn;
+  p.early_w = (pdl && g.early_w) ? 1 : 0;
   p.status = g.status;
   const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
   const dim3 grid(static_cast<unsigned>(tiles < g_num_sms ? tiles : g_num_sms));

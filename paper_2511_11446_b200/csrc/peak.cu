@@ -1,13 +1,13 @@
 // Measurement helper: the INT8 tensor-core ceiling of the device as seen by this library's own
 // instruction stream. Each CTA fills one 128 x 128 (A) and one 256 x 128 (B) int8 operand tile in
 // shared memory with pseudo-random bytes and issues `iters` k-blocks of four tcgen05.mma kind::i8
-// (128 x 256 x 32) each, alternating between two accumulator buffers; no global traffic.
+// (128 x tile_n x 32) each, alternating between two accumulator buffers; no global traffic.
 #include "dp_common.cuh"
 #include "dp_internal.h"
 
 namespace dp {
 
-__global__ void __launch_bounds__(128, 1) mma_i8_peak_kernel(int iters, int32_t* status) {
+__global__ void __launch_bounds__(128, 1) mma_i8_peak_kernel(int iters, int tile_n, int32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem;                 // 16 KB
@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(128, 1) mma_i8_peak_kernel(int iters, int32_t*
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   if (threadIdx.x == 0) {
-    constexpr uint32_t idesc = idesc_i8(128, 256);
+    const uint32_t idesc = idesc_i8(128, tile_n);
     const uint64_t adesc = smem_desc_sw128(smem_u32(sA));
     const uint64_t bdesc = smem_desc_sw128(smem_u32(sB));
     for (int it = 0; it < iters; ++it) {
@@ -67,17 +67,18 @@ __global__ void __launch_bounds__(128, 1) mma_i8_peak_kernel(int iters, int32_t*
 
 }  // namespace dp
 
-extern "C" int dp_bench_mma_i8(int32_t ctas, int32_t iters, int32_t* device_status, dp_stream stream) {
+extern "C" int dp_bench_mma_i8(int32_t ctas, int32_t iters, int32_t tile_n, int32_t* device_status,
+                               dp_stream stream) {
   using namespace dp;
-  if (ctas <= 0 || iters <= 0 || iters > (1 << 22))
-    return fail(DP_ERR_INVALID_ARG, "dp_bench_mma_i8: bad ctas/iters");
+  if (ctas <= 0 || iters <= 0 || iters > (1 << 22) || tile_n < 16 || tile_n > 256 || (tile_n % 16))
+    return fail(DP_ERR_INVALID_ARG, "dp_bench_mma_i8: bad ctas/iters/tile_n");
   int st = check_device();
   if (st != DP_OK) return st;
   const size_t smem = 128 * 1024;  // more than half an SM: one CTA (and one TMEM allocation) per SM
   DP_CUDA_OK(cudaFuncSetAttribute(mma_i8_peak_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   static_cast<int>(smem)));
   cudaError_t e = launch(mma_i8_peak_kernel, dim3(ctas), dim3(128), smem,
-                         static_cast<cudaStream_t>(stream), false, iters, device_status);
+                         static_cast<cudaStream_t>(stream), false, iters, tile_n, device_status);
   if (e != cudaSuccess) return fail(DP_ERR_CUDA, "peak kernel launch: %s", cudaGetErrorString(e));
   return DP_OK;
 }

@@ -1,9 +1,13 @@
 // CUDA-core path of the quantized linear for small row counts (adaLN modulation: M = batch).
 //
-// The whole layer in one launch: each CTA quantizes its (up to 8) tokens into shared memory
-// (DAQ, Step 3 Eq. "daq"), then its warps stream packed weight rows from HBM, expand them to int8
-// in registers, take dp4a dot products against the shared int8 tokens, and apply the dequant
-// epilogue. The shape is bound by the weight bytes (M <= 32: 2..144 int8 ops per weight byte).
+// The whole layer in one launch, bound by the weight bytes (M <= 32: 2..144 int8 ops per weight
+// byte). A CTA owns 32 output channels and up to 8 tokens. Eight lanes share one channel: each
+// lane fetches its 32-code units of the packed weight row straight into registers, all loads of a
+// pass issued back to back and BEFORE the CTA quantizes its tokens (DAQ, Step 3 Eq. "daq", one
+// warp per token, codes to shared memory), so the HBM latency of the weights overlaps the
+// prologue. The units are then expanded to int8 in registers, contracted against the shared int8
+// tokens with dp4a, reduced over the eight lanes by a transpose-reduction (7 shuffles leave lane j
+// with token j's sum) and sent through the dequant epilogue.
 #include <cuda_bf16.h>
 
 #include "dp_common.cuh"
@@ -11,39 +15,57 @@
 
 namespace dp {
 
-constexpr int kSimtRows = 8;     // tokens per CTA
+constexpr int kSimtRows = 8;        // tokens per CTA
 constexpr int kSimtWarps = 8;
-constexpr int kSimtChPerCta = 32;  // output channels per CTA
+constexpr int kSimtLanesPerCh = 8;  // lanes sharing one output channel
+constexpr int kSimtChPerCta = kSimtWarps * (32 / kSimtLanesPerCh);
+constexpr int kSimtSlots = 5;       // units a lane holds per pass (K = 1152: 36 units / 8 lanes)
 
-// 32 consecutive k of one weight row -> 8 words of 4 int8 (true values).
+// Packed form of one unit (32 consecutive k of one weight row): BITS words.
 template <int BITS>
-__device__ __forceinline__ void load_unit(const uint32_t* __restrict__ row, int unit,
-                                          uint32_t (&w)[8]) {
+__device__ __forceinline__ void fetch_unit(const uint32_t* __restrict__ row, int unit, uint32_t (&pk)[BITS]) {
   if constexpr (BITS == 8) {
     const uint4* p = reinterpret_cast<const uint4*>(row) + unit * 2;
-    uint4 a = __ldg(p), b = __ldg(p + 1);
-    w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w;
-    w[4] = b.x; w[5] = b.y; w[6] = b.z; w[7] = b.w;
+    uint4 a, b;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w) : "l"(p));
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "l"(p + 1));
+    pk[0] = a.x; pk[1] = a.y; pk[2] = a.z; pk[3] = a.w;
+    pk[4] = b.x; pk[5] = b.y; pk[6] = b.z; pk[7] = b.w;
   } else if constexpr (BITS == 4) {
-    uint4 a = __ldg(reinterpret_cast<const uint4*>(row) + unit);
-    const uint32_t in[4] = {a.x, a.y, a.z, a.w};
+    const uint4* p = reinterpret_cast<const uint4*>(row) + unit;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(pk[0]), "=r"(pk[1]), "=r"(pk[2]), "=r"(pk[3]) : "l"(p));
+  } else {
+    const uint32_t* p = row + unit * 3;
+#pragma unroll
+    for (int i = 0; i < 3; ++i)
+      asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(pk[i]) : "l"(p + i));
+  }
+}
+
+// Packed unit -> 8 words of 4 int8 (true values, k ascending).
+template <int BITS>
+__device__ __forceinline__ void expand_unit(const uint32_t (&pk)[BITS], uint32_t (&w)[8]) {
+  if constexpr (BITS == 8) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) w[i] = pk[i];
+  } else if constexpr (BITS == 4) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      uint32_t lo = in[i] & 0x0F0F0F0Fu, hi = (in[i] >> 4) & 0x0F0F0F0Fu;
+      const uint32_t lo = pk[i] & 0x0F0F0F0Fu, hi = (pk[i] >> 4) & 0x0F0F0F0Fu;
       w[2 * i] = __vsub4(__byte_perm(lo, hi, 0x5140), 0x08080808u);
       w[2 * i + 1] = __vsub4(__byte_perm(lo, hi, 0x7362), 0x08080808u);
     }
   } else {
-    const uint32_t* p = row + unit * 3;
-    const uint32_t s0 = __ldg(p), s1 = __ldg(p + 1), s2 = __ldg(p + 2);
-    const uint64_t lo64 = (static_cast<uint64_t>(s1) << 32) | s0;
-    const uint64_t hi64 = (static_cast<uint64_t>(s2) << 32) | s1;
+    const uint64_t lo64 = (static_cast<uint64_t>(pk[1]) << 32) | pk[0];
+    const uint64_t hi64 = (static_cast<uint64_t>(pk[2]) << 32) | pk[1];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const int bit = 12 * j;
-      const uint32_t x = static_cast<uint32_t>(bit < 32 ? (lo64 >> bit) : (hi64 >> (bit - 32))) &
-                         0xFFFu;
-      uint32_t o = (x & 7u) | ((x & 0x38u) << 5) | ((x & 0x1C0u) << 10) | ((x & 0xE00u) << 15);
+      const uint32_t x = static_cast<uint32_t>(bit < 32 ? (lo64 >> bit) : (hi64 >> (bit - 32))) & 0xFFFu;
+      const uint32_t o = (x & 7u) | ((x & 0x38u) << 5) | ((x & 0x1C0u) << 10) | ((x & 0xE00u) << 15);
       w[j] = __vsub4(o, 0x04040404u);
     }
   }
@@ -56,10 +78,25 @@ simt_linear_kernel(SimtArgs a) {
   int8_t* sq = reinterpret_cast<int8_t*>(smem);                       // [kSimtRows][K]
   float* ssa = reinterpret_cast<float*>(smem + kSimtRows * a.K);      // [kSimtRows]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int sub = lane & (kSimtLanesPerCh - 1);
   const int64_t m0 = static_cast<int64_t>(blockIdx.y) * kSimtRows;
   const int K = a.K;
+  const int units = K >> 5;
+  const int n = blockIdx.x * kSimtChPerCta + warp * (32 / kSimtLanesPerCh) + (lane >> 3);
+  const bool n_ok = n < a.N;
+  const uint32_t* wrow = static_cast<const uint32_t*>(a.qweight) +
+                         static_cast<int64_t>(n_ok ? n : 0) * ((K * BITS) >> 5);
   pdl_launch_dependents();
-  pdl_wait();
+  if (!a.early_w) pdl_wait();
+
+  // ---- first pass of this lane's weight units: in flight across the prologue ----
+  uint32_t pk[kSimtSlots][BITS];
+#pragma unroll
+  for (int i = 0; i < kSimtSlots; ++i) {
+    const int u = sub + kSimtLanesPerCh * i;
+    if (n_ok && u < units) fetch_unit<BITS>(wrow, u, pk[i]);
+  }
+  if (a.early_w) pdl_wait();  // the tokens come from the preceding kernel on the stream
 
   // ---- prologue: this CTA's tokens -> int8 in shared memory (one warp per token) ----
   {
@@ -76,6 +113,7 @@ simt_linear_kernel(SimtArgs a) {
     } else {
       const uint4* xr = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(a.x) + row * a.ldx);
       uint32_t mx = 0;
+#pragma unroll 5
       for (int i = lane; i < nvec; i += 32) {
         uint4 v = xr[i];
         mx = __vmaxu2(mx, v.x & 0x7FFF7FFFu);
@@ -93,6 +131,7 @@ simt_linear_kernel(SimtArgs a) {
         inv = __fdiv_rn(127.0f, amax);
       }
       const float magic = 12582912.0f;
+#pragma unroll 5
       for (int i = lane; i < nvec; i += 32) {
         uint4 v = xr[i];
         const uint32_t in[4] = {v.x, v.y, v.z, v.w};
@@ -119,53 +158,73 @@ simt_linear_kernel(SimtArgs a) {
   }
   __syncthreads();
 
-  // ---- weight streaming: warp w takes channels n0 + w, n0 + w + 8, ... ----
-  const int units = K >> 5;
-  const int row_words = (K * BITS) >> 5;
-  const int n0 = blockIdx.x * kSimtChPerCta;
-  for (int c = warp; c < kSimtChPerCta; c += kSimtWarps) {
-    const int n = n0 + c;
-    if (n >= a.N) break;
-    const uint32_t* wrow = static_cast<const uint32_t*>(a.qweight) + static_cast<int64_t>(n) * row_words;
-    int acc[kSimtRows];
+  // ---- contraction: passes of kSimtSlots units per lane ----
+  int acc[kSimtRows];
 #pragma unroll
-    for (int m = 0; m < kSimtRows; ++m) acc[m] = 0;
-    for (int u = lane; u < units; u += 32) {
-      uint32_t w[8];
-      load_unit<BITS>(wrow, u, w);
+  for (int m = 0; m < kSimtRows; ++m) acc[m] = 0;
+  for (int base = 0; base < units; base += kSimtLanesPerCh * kSimtSlots) {
+    if (base != 0) {
 #pragma unroll
-      for (int m = 0; m < kSimtRows; ++m) {
-        const uint4* qp = reinterpret_cast<const uint4*>(sq + m * K + u * 32);
-        const uint4 q0 = qp[0], q1 = qp[1];
-        int s = acc[m];
-        s = __dp4a(static_cast<int>(q0.x), static_cast<int>(w[0]), s);
-        s = __dp4a(static_cast<int>(q0.y), static_cast<int>(w[1]), s);
-        s = __dp4a(static_cast<int>(q0.z), static_cast<int>(w[2]), s);
-        s = __dp4a(static_cast<int>(q0.w), static_cast<int>(w[3]), s);
-        s = __dp4a(static_cast<int>(q1.x), static_cast<int>(w[4]), s);
-        s = __dp4a(static_cast<int>(q1.y), static_cast<int>(w[5]), s);
-        s = __dp4a(static_cast<int>(q1.z), static_cast<int>(w[6]), s);
-        s = __dp4a(static_cast<int>(q1.w), static_cast<int>(w[7]), s);
-        acc[m] = s;
+      for (int i = 0; i < kSimtSlots; ++i) {
+        const int u = base + sub + kSimtLanesPerCh * i;
+        if (n_ok && u < units) fetch_unit<BITS>(wrow, u, pk[i]);
       }
     }
-    int mine = 0;
 #pragma unroll
-    for (int m = 0; m < kSimtRows; ++m) {
-      int s = acc[m];
+    for (int i = 0; i < kSimtSlots; ++i) {
+      const int u = base + sub + kSimtLanesPerCh * i;
+      if (n_ok && u < units) {
+        uint32_t w[8];
+        expand_unit<BITS>(pk[i], w);
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
-      if (lane == m) mine = s;
+        for (int m = 0; m < kSimtRows; ++m) {
+          const uint4* qp = reinterpret_cast<const uint4*>(sq + m * K + u * 32);
+          const uint4 q0 = qp[0], q1 = qp[1];
+          int s = acc[m];
+          s = __dp4a(static_cast<int>(q0.x), static_cast<int>(w[0]), s);
+          s = __dp4a(static_cast<int>(q0.y), static_cast<int>(w[1]), s);
+          s = __dp4a(static_cast<int>(q0.z), static_cast<int>(w[2]), s);
+          s = __dp4a(static_cast<int>(q0.w), static_cast<int>(w[3]), s);
+          s = __dp4a(static_cast<int>(q1.x), static_cast<int>(w[4]), s);
+          s = __dp4a(static_cast<int>(q1.y), static_cast<int>(w[5]), s);
+          s = __dp4a(static_cast<int>(q1.z), static_cast<int>(w[6]), s);
+          s = __dp4a(static_cast<int>(q1.w), static_cast<int>(w[7]), s);
+          acc[m] = s;
+        }
+      }
     }
-    if (lane < kSimtRows && m0 + lane < a.M) {
-      const int64_t row = m0 + lane;
-      const float t = static_cast<float>(mine);
-      const float sc = __fmul_rn(ssa[lane], a.s_w[n]);
-      const float b = a.bias != nullptr ? __uint_as_float(static_cast<uint32_t>(a.bias[n]) << 16) : 0.0f;
-      const float y = __fmaf_rn(t, sc, b);
-      a.y[row * a.ldy + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
-      if (a.dbg_acc != nullptr) a.dbg_acc[row * a.dbg_ldacc + n] = mine;
+  }
+
+  // ---- transpose-reduction over the 8 lanes of a channel: lane j ends with token j's sum ----
+  {
+    const bool hi4 = (sub & 4) != 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int send = hi4 ? acc[i] : acc[i + 4];
+      const int keep = hi4 ? acc[i + 4] : acc[i];
+      acc[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 4);
     }
+    const bool hi2 = (sub & 2) != 0;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int send = hi2 ? acc[i] : acc[i + 2];
+      const int keep = hi2 ? acc[i + 2] : acc[i];
+      acc[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 2);
+    }
+    const bool hi1 = (sub & 1) != 0;
+    const int send = hi1 ? acc[0] : acc[1];
+    const int keep = hi1 ? acc[1] : acc[0];
+    acc[0] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 1);
+  }
+  const int64_t row = m0 + sub;
+  if (n_ok && row < a.M) {
+    const int mine = acc[0];
+    const float t = static_cast<float>(mine);
+    const float sc = __fmul_rn(ssa[sub], a.s_w[n]);
+    const float b = a.bias != nullptr ? __uint_as_float(static_cast<uint32_t>(a.bias[n]) << 16) : 0.0f;
+    const float y = __fmaf_rn(t, sc, b);
+    a.y[row * a.ldy + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
+    if (a.dbg_acc != nullptr) a.dbg_acc[row * a.dbg_ldacc + n] = mine;
   }
 }
 
@@ -184,7 +243,9 @@ int launch_simt_linear(const SimtArgs& a, cudaStream_t stream, bool pdl) {
                                          static_cast<int>(smem));
     if (e != cudaSuccess) return fail(DP_ERR_CUDA, "simt smem attribute: %s", cudaGetErrorString(e));
   }
-  cudaError_t e = launch(kern, grid, block, smem, stream, pdl, a);
+  SimtArgs args = a;
+  if (!pdl) args.early_w = 0;
+  cudaError_t e = launch(kern, grid, block, smem, stream, pdl, args);
   if (e != cudaSuccess) return fail(DP_ERR_CUDA, "simt launch failed: %s", cudaGetErrorString(e));
   return DP_OK;
 }

@@ -1,0 +1,108 @@
+"""Per-shape timing of the quantized linear on one GPU (used by ``bench.py --sweep``).
+
+For every (layer shape, weight bit-width) of a workload this times, with CUDA events on the launch
+stream, (a) the whole layer through dp_wq_linear (DAQ inside the call), (b) the GEMM alone on
+pre-quantized activations and (c) dp_daq_quantize alone. Buffers rotate over enough copies to exceed
+the L2 cache, so every launch streams its operands from HBM as it does inside a plan run.
+Only input preparation and bookkeeping live here; the arithmetic is in the CUDA library.
+"""
+from __future__ import annotations
+
+import json
+
+import torch
+
+from . import binding as B
+from . import synth, synth_cuda
+from .workloads import DevWeights
+
+L2_BYTES = 126 << 20
+SHAPES = (("qkv", synth.HIDDEN, 3 * synth.HIDDEN), ("proj", synth.HIDDEN, synth.HIDDEN),
+          ("fc1", synth.HIDDEN, synth.MLP), ("fc2", synth.MLP, synth.HIDDEN))
+WORKLOADS = {"c1": (256, 1), "c2": (2048, 8), "c3": (4096, 16), "c4": (2048, 8), "c5": (32768, 32)}
+
+
+def alg_bytes(M, K, N, bits):
+    """Bytes the method itself must move for one layer: X bf16, packed W, s_w, bias, Y bf16."""
+    return 2 * M * K + N * K * bits // 8 + 6 * N + 2 * M * N
+
+
+def _time(fn, n_sets, iters, warmup=3):
+    """us per launch of fn(set_index): `iters` launches captured in one CUDA graph (so the host's
+    launch cost is not in the number), replayed after a warm-up replay."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for i in range(min(warmup, n_sets)):
+            fn(i % n_sets)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        for i in range(iters):
+            fn(i % n_sets)
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / iters
+
+
+def time_shape(name, M, K, N, bits, peaks, seed=synth.BASE_SEED + 5, iters=None, only=None, flags=0):
+    per_set = 2 * M * K + M * K + 2 * M * N + N * K * bits // 8
+    n_sets = max(2, min(24, -(-2 * L2_BYTES // per_set)))
+    iters = iters or max(10, min(200, int(2e9 // per_set)))
+    iters = -(-iters // n_sets) * n_sets
+    Ws = [DevWeights(seed, s, N, K, bits) for s in range(n_sets)]
+    xs = [synth_cuda.activations(seed, s, 0, M, K, 1.0, n_out=max(1, K // 100)) for s in range(n_sets)]
+    qs = [torch.empty((M, K), dtype=torch.int8, device="cuda") for _ in range(n_sets)]
+    sas = [torch.empty(M, dtype=torch.float32, device="cuda") for _ in range(n_sets)]
+    ys = [torch.empty((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(n_sets)]
+    ws = torch.empty(B.dp_wq_linear_workspace(M, N, K, bits, flags), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for s in range(n_sets):
+        B.dp_daq_quantize(xs[s], M, K, K, qs[s], K, sas[s])
+    out = {"layer": name, "M": M, "K": K, "N": N, "bits": bits, "buffer_sets": n_sets, "iters": iters}
+    ops, by = 2.0 * M * N * K, alg_bytes(M, K, N, bits)
+    int8_peak = 2.0 * peaks["bf16"]
+    t_ideal = max(ops / (int8_peak * 1e12), by / (peaks["hbm_gbs"] * 1e9)) * 1e6
+    out["ideal_us"] = t_ideal
+    out["bound"] = "tensor" if ops / (int8_peak * 1e12) > by / (peaks["hbm_gbs"] * 1e9) else "hbm"
+    if only in (None, "layer"):
+        t = _time(lambda s: B.dp_wq_linear(Ws[s].w, xs[s], K, None, M, ys[s], N, ws, None, status, flags),
+                  n_sets, iters)
+        out.update(layer_us=t, layer_tops=ops / t / 1e6, layer_gbs=by / t / 1e3, layer_frac=t_ideal / t)
+    if only in (None, "gemm"):
+        t = _time(lambda s: B.dp_wq_linear(Ws[s].w, qs[s], K, sas[s], M, ys[s], N, None, None, status, flags),
+                  n_sets, iters)
+        out.update(gemm_us=t, gemm_tops=ops / t / 1e6, gemm_frac_int8_peak=ops / t / 1e6 / int8_peak)
+    if only in (None, "daq"):
+        t = _time(lambda s: B.dp_daq_quantize(xs[s], M, K, K, qs[s], K, sas[s]), n_sets, iters)
+        out.update(daq_us=t, daq_gbs=(3 * M * K + 4 * M) / t / 1e3,
+                   daq_frac_hbm=(3 * M * K + 4 * M) / t / 1e3 / peaks["hbm_gbs"])
+    assert int(status.item()) == 0, "a kernel reported DP_ERR_TIMEOUT"
+    return out
+
+
+def run(workload, bits_list, peaks, only=None, layers=None, iters=None, flags=0, emit=print):
+    M, batch = WORKLOADS[workload]
+    rows = []
+    for name, K, N in SHAPES:
+        if layers and name not in layers:
+            continue
+        for bits in bits_list:
+            r = time_shape(name, M, K, N, bits, peaks, iters=iters, only=only, flags=flags)
+            r["workload"] = workload
+            rows.append(r)
+            emit(json.dumps(r))
+            torch.cuda.empty_cache()
+    if not layers or "adaln" in layers:
+        for bits in bits_list:
+            r = time_shape("adaln", batch, synth.HIDDEN, synth.ADALN, bits, peaks, iters=iters, only="layer",
+                           flags=flags)
+            r["workload"] = workload
+            rows.append(r)
+            emit(json.dumps(r))
+    return rows

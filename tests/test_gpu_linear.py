@@ -61,6 +61,27 @@ def test_mma_path(bits, M, K, N):
 
 
 @pytest.mark.parametrize("bits", [8, 4, 3])
+@pytest.mark.parametrize("bn", [64, 128, 192, 256])
+def test_mma_every_tile_width(bits, bn):
+    """Each tile-width variant of the tensor-core kernel, several tiles per CTA is not needed for
+    coverage of the variant itself: ragged M, two column tiles, K of three k-blocks."""
+    M, K, N = 200, 384, 2 * bn
+    x, w, s_w, b = _case(M, K, N, bits, full_range=True)
+    L = DevLayer(w, s_w, b, bits)
+    _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | B.DP_FLAG_TILE_N(bn)), x, w, s_w, b, bits)
+
+
+def test_mma_many_tiles_per_cta():
+    """More tiles than SMs, so the persistent loop, both accumulator buffers and the stage ring
+    wrap-around are exercised (M = 1300 -> 11 row tiles x 18 column tiles of 64)."""
+    M, K, N = 1300, 256, 1152
+    for bits in (8, 4, 3):
+        x, w, s_w, b = _case(M, K, N, bits)
+        L = DevLayer(w, s_w, b, bits)
+        _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | B.DP_FLAG_TILE_N(64)), x, w, s_w, b, bits)
+
+
+@pytest.mark.parametrize("bits", [8, 4, 3])
 def test_mma_one_hot_and_constant_inputs(bits):
     """One-hot tokens expose any permutation of k or n inside the tiles: acc[m,n] = 127*w[n,k_m]."""
     M, K, N = 128, 384, 128
