@@ -83,7 +83,7 @@ static int check_weight(const dp_weight* w) {
 static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_a_in, int64_t M,
                       void* y, int64_t ldy, void* workspace, const dp_debug* dbg, int32_t* status,
                       uint32_t flags, cudaStream_t stream, const CUtensorMap* tmap_w, int bn,
-                      const CUtensorMap* tmap_a_cached, const CUtensorMap* tmap_y_cached, bool chained) {
+                      const CUtensorMap* tmap_a_cached, bool chained) {
   const bool pdl = !(flags & DP_FLAG_NO_PDL);
   if (use_simt(M, w->N, w->K, flags)) {
     if (static_cast<size_t>(w->K) > simt_max_k())
@@ -141,12 +141,6 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
     g.tmap_w = *tmap_w;
   } else {
     int st = gemm_encode_w(&g.tmap_w, w->qweight, w->N, w->K, w->bits, bn);
-    if (st != DP_OK) return st;
-  }
-  if (tmap_y_cached != nullptr) {
-    g.tmap_y = *tmap_y_cached;
-  } else {
-    int st = gemm_encode_y(&g.tmap_y, y, M, w->N, ldy);
     if (st != DP_OK) return st;
   }
   g.s_a = s_a;
@@ -233,7 +227,7 @@ extern "C" int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, cons
   st = check_device();
   if (st != DP_OK) return st;
   return run_linear(w, x, ldx, s_a_in, M, y_bf16, ldy, workspace, dbg, device_status, flags,
-                    static_cast<cudaStream_t>(stream), nullptr, 0, nullptr, nullptr, false);
+                    static_cast<cudaStream_t>(stream), nullptr, 0, nullptr, false);
 }
 
 // ---- plans ---------------------------------------------------------------------------------------
@@ -250,17 +244,12 @@ struct TmapACache {
   int64_t M, K;
   CUtensorMap map;
 };
-struct TmapYCache {  // one entry per layer: the descriptor of the output buffer last used
-  const void* ptr = nullptr;
-  CUtensorMap map;
-};
 struct dp_plan {
   std::vector<PlanLayer> layers;
   uint32_t flags;
   size_t workspace_bytes;
   size_t x_bytes;
   std::vector<TmapACache> a_cache;
-  std::vector<TmapYCache> y_cache;
   cudaStream_t copy_stream;
   cudaEvent_t ev_copied[2], ev_consumed[2];
 };
@@ -313,7 +302,6 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
     p->x_bytes += align256(static_cast<size_t>(L.M) * L.w.K * 2);
     p->layers.push_back(L);
   }
-  p->y_cache.resize(p->layers.size());
   cudaError_t e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
   for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
     e = cudaEventCreateWithFlags(&p->ev_copied[i], cudaEventDisableTiming);
@@ -365,21 +353,13 @@ static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, 
     if (!xs[l] || !ys[l]) return fail(DP_ERR_INVALID_ARG, "layer %d: NULL x or y", l);
     if (!aligned16(xs[l]) || !aligned16(ys[l])) return fail(DP_ERR_ALIGN, "layer %d: x/y misaligned", l);
     const CUtensorMap* ta = nullptr;
-    const CUtensorMap* ty = nullptr;
     if (!L.simt) {
       int st = DP_OK;
       ta = cached_tmap_a(plan, workspace, L.M, L.w.K, &st);
       if (st != DP_OK) return st;
-      TmapYCache& yc = plan->y_cache[l];
-      if (yc.ptr != ys[l]) {
-        st = gemm_encode_y(&yc.map, ys[l], L.M, L.w.N, L.w.N);
-        if (st != DP_OK) return st;
-        yc.ptr = ys[l];
-      }
-      ty = &yc.map;
     }
     int st = run_linear(&L.w, xs[l], L.w.K, nullptr, L.M, ys[l], L.w.N, workspace, nullptr, status,
-                        plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, ta, ty, *chained);
+                        plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, ta, *chained);
     if (st != DP_OK) return st;
     *chained = true;
   }

@@ -50,7 +50,6 @@ struct GemmTile {  // kernel variant
 struct GemmProblem {
   CUtensorMap tmap_a;  // int8 activations [M][K]
   CUtensorMap tmap_w;  // packed weights, byte view [N][K*bits/8]
-  CUtensorMap tmap_y;  // bf16 outputs [M][N]
   const float* s_a;    // [M]
   const float* s_w;    // [N]
   const uint16_t* bias;
@@ -69,7 +68,6 @@ int gemm_pick_bn(int64_t M, int32_t N, int32_t K, int32_t bits);
 int gemm_encode_a(CUtensorMap* out, const int8_t* q, int64_t M, int64_t K, int64_t ldq);
 int gemm_encode_w(CUtensorMap* out, const void* qweight, int32_t N, int32_t K, int32_t bits,
                   int32_t bn);
-int gemm_encode_y(CUtensorMap* out, const void* y, int64_t M, int32_t N, int64_t ldy);
 int launch_gemm(const GemmProblem& p, cudaStream_t stream, bool pdl);
 int gemm_init();  // sets kernel attributes, resolves the tensor-map encoder; idempotent
 

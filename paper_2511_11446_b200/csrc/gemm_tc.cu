@@ -7,8 +7,10 @@
 //   warp 0      TMA producer: int8 activation tiles (128-byte-swizzled) and packed weight tiles
 //   warp 1      MMA issuer: tcgen05.mma kind::i8, int32 accumulators in tensor memory (two
 //               accumulator buffers, so a tile's epilogue overlaps the next tile's mainloop)
-//   warps 2-5   epilogue: tcgen05.ld -> (float)acc * s_a[m]*s_w[n] + bias -> bf16 -> global
-//   warps 6-13  unpack (3/4-bit only): packed tile in smem -> int8 operand tile in smem, written in
+//   warps 2-9   epilogue: tcgen05.ld -> (float)acc * s_a[m]*s_w[n] + bias -> bf16 -> global; two warps
+//               per 32-token TMEM quadrant, each taking half of the tile's 64-column slabs, so one
+//               warp's conversion burst overlaps the other's shared-memory and store phases
+//   warps 10-17 unpack (3/4-bit only): packed tile in smem -> int8 operand tile in smem, written in
 //               the swizzled layout the MMA descriptor expects, then fence.proxy.async
 //
 // K order. The contraction over k does not care in which order the k's of a 128-wide block sit in
@@ -30,13 +32,13 @@ namespace dp {
 
 constexpr int BM = 128;
 constexpr int BK = 128;  // int8 elements = bytes = one 128-byte swizzle row
-constexpr int kEpiWarp0 = 2, kUnpackWarp0 = 6, kUnpackWarps = 8;
+constexpr int kEpiWarp0 = 2, kEpiWarps = 8, kUnpackWarp0 = kEpiWarp0 + kEpiWarps, kUnpackWarps = 8;
 constexpr int kUnpackThreads = kUnpackWarps * 32;
 __host__ __device__ constexpr int gemm_threads(int bits) {
   return (kUnpackWarp0 + (bits == 8 ? 0 : kUnpackWarps)) * 32;
 }
-constexpr int kYStageBytes = 32 * 128;  // per epilogue warp: 32 tokens x 64 bf16
-constexpr int kSmemBudget = 196 * 1024;
+constexpr int kYStageBytes = 32 * 64;  // per epilogue warp: 32 tokens x 32 bf16
+constexpr int kSmemBudget = 200 * 1024;
 constexpr int kPStages = 3;
 
 __host__ __device__ constexpr int p_stage_bytes(int bn, int bits) {
@@ -132,44 +134,45 @@ __device__ __forceinline__ void unpack3_tile(const uint8_t* P, uint8_t* B, int t
 }
 
 // ---- epilogue arithmetic -----------------------------------------------------------------------------
-// 32 accumulators of one token (half of a 64-column slab) -> bf16 into the warp's staging tile
-// [32 tokens][128 bytes], 16-byte chunks XOR-swizzled by (token & 7) as the 128-byte-swizzle TMA
-// store expects. Per element, in this order: t = (float)acc (times 2^-SHIFT, exact),
+// 32 accumulators of one token -> bf16 into the warp's staging tile [32 tokens][64 bytes], 16-byte
+// chunks XOR-swizzled by ((token >> 1) & 3) so that both the per-token writes and the row-wise
+// read-back are free of bank conflicts. Per element, in this order: t = (float)(acc / 2^SHIFT),
 // sc = s_a * s_w[n], y = fma(t, sc, bias[n]), bf16 round-to-nearest-even.
 template <int SHIFT>
-__device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], float sa, const float* ts,
-                                               const float* tb, uint8_t* stage_row, int half, int sw,
+__device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], float sa,
+                                               const float4* __restrict__ s4,
+                                               const float4* __restrict__ b4,
+                                               uint4* __restrict__ stage_row, int sw,
                                                int32_t* acc_dst) {
-  const float4* s4 = reinterpret_cast<const float4*>(ts);
-  const float4* b4 = reinterpret_cast<const float4*>(tb);
+  // all shared-memory reads and all arithmetic first, the four 16-byte stores last: nothing in the
+  // arithmetic then has to wait behind a store the compiler cannot reorder
+  uint32_t o[16];
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {  // 16-byte chunk = 8 outputs
-    uint32_t o[4];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const float4 sw4 = s4[2 * j + h], bb = b4[2 * j + h];
-      float t0 = __int2float_rn(static_cast<int>(r[8 * j + 4 * h + 0]));
-      float t1 = __int2float_rn(static_cast<int>(r[8 * j + 4 * h + 1]));
-      float t2 = __int2float_rn(static_cast<int>(r[8 * j + 4 * h + 2]));
-      float t3 = __int2float_rn(static_cast<int>(r[8 * j + 4 * h + 3]));
-      if constexpr (SHIFT != 0) {
-        constexpr float kInv = 1.0f / (1 << SHIFT);
-        t0 = __fmul_rn(t0, kInv);
-        t1 = __fmul_rn(t1, kInv);
-        t2 = __fmul_rn(t2, kInv);
-        t3 = __fmul_rn(t3, kInv);
-      }
-      const float y0 = __fmaf_rn(t0, __fmul_rn(sa, sw4.x), bb.x);
-      const float y1 = __fmaf_rn(t1, __fmul_rn(sa, sw4.y), bb.y);
-      const float y2 = __fmaf_rn(t2, __fmul_rn(sa, sw4.z), bb.z);
-      const float y3 = __fmaf_rn(t3, __fmul_rn(sa, sw4.w), bb.w);
-      const __nv_bfloat162 h0 = __floats2bfloat162_rn(y0, y1);
-      const __nv_bfloat162 h1 = __floats2bfloat162_rn(y2, y3);
-      o[2 * h] = *reinterpret_cast<const uint32_t*>(&h0);
-      o[2 * h + 1] = *reinterpret_cast<const uint32_t*>(&h1);
+  for (int j = 0; j < 8; ++j) {
+    const float4 sw4 = s4[j], bb = b4[j];
+    float t0 = __int2float_rn(static_cast<int>(r[4 * j + 0]));
+    float t1 = __int2float_rn(static_cast<int>(r[4 * j + 1]));
+    float t2 = __int2float_rn(static_cast<int>(r[4 * j + 2]));
+    float t3 = __int2float_rn(static_cast<int>(r[4 * j + 3]));
+    if constexpr (SHIFT != 0) {  // exact: the accumulator is a multiple of 2^SHIFT
+      constexpr float kInv = 1.0f / (1 << SHIFT);
+      t0 = __fmul_rn(t0, kInv);
+      t1 = __fmul_rn(t1, kInv);
+      t2 = __fmul_rn(t2, kInv);
+      t3 = __fmul_rn(t3, kInv);
     }
-    *reinterpret_cast<uint4*>(stage_row + (((half * 4 + j) ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+    const float y0 = __fmaf_rn(t0, __fmul_rn(sa, sw4.x), bb.x);
+    const float y1 = __fmaf_rn(t1, __fmul_rn(sa, sw4.y), bb.y);
+    const float y2 = __fmaf_rn(t2, __fmul_rn(sa, sw4.z), bb.z);
+    const float y3 = __fmaf_rn(t3, __fmul_rn(sa, sw4.w), bb.w);
+    const __nv_bfloat162 h0 = __floats2bfloat162_rn(y0, y1);
+    const __nv_bfloat162 h1 = __floats2bfloat162_rn(y2, y3);
+    o[2 * j] = *reinterpret_cast<const uint32_t*>(&h0);
+    o[2 * j + 1] = *reinterpret_cast<const uint32_t*>(&h1);
   }
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+    stage_row[j ^ sw] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
   if (acc_dst != nullptr) {
 #pragma unroll
     for (int j = 0; j < 32; ++j) acc_dst[j] = static_cast<int>(r[j]) >> SHIFT;
@@ -180,7 +183,7 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], float sa
 template <int BN, int BITS, bool PERM>
 __global__ void __launch_bounds__(gemm_threads(BITS), 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
-               const __grid_constant__ CUtensorMap tmap_y, const GemmParams p) {
+               const GemmParams p) {
   constexpr int NS = num_stages(BN, BITS);
   constexpr int NP = kPStages;
   constexpr int A_BYTES = BM * BK, B_BYTES = BN * BK, P_BYTES = p_stage_bytes(BN, BITS);
@@ -193,8 +196,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint8_t* sA = smem;
   uint8_t* sB = sA + NS * A_BYTES;
   uint8_t* sP = sB + NS * B_BYTES;
-  uint8_t* sY = sP + NP * P_BYTES;  // [4 epilogue warps][32 tokens][128 bytes] output staging
-  uint8_t* tail = sY + 4 * kYStageBytes;
+  uint8_t* sY = sP + NP * P_BYTES;  // [epilogue warps][32 tokens][128 bytes] output staging
+  uint8_t* tail = sY + kEpiWarps * kYStageBytes;
   uint64_t* full_a = reinterpret_cast<uint64_t*>(tail);
   uint64_t* bready = full_a + NS;
   uint64_t* empty = bready + NS;
@@ -204,9 +207,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint64_t* acc_empty = acc_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* s_scale = reinterpret_cast<float*>(                 // [4 warps][BN] weight scales of the tile
+  constexpr int SLABS = BN / 64;            // 64-column slabs per tile
+  constexpr int SLABS_LO = (SLABS + 1) / 2;  // slabs of the first warp of a quadrant; the rest go to the second
+  constexpr int EPI_ACTIVE = SLABS > 1 ? kEpiWarps : kEpiWarps / 2;  // BN = 64: one warp per quadrant
+  float* s_scale = reinterpret_cast<float*>(                 // [warps][64 * SLABS_LO] weight scales
       (reinterpret_cast<uintptr_t>(tmem_slot + 4) + 15) & ~uintptr_t(15));
-  float* s_bias = s_scale + 4 * BN;                           // [4 warps][BN]
+  float* s_bias = s_scale + kEpiWarps * 64 * SLABS_LO;        // [warps][64 * SLABS_LO]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int KB = p.K / BK;
@@ -224,13 +230,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&acc_full[i], 1);
-      mbar_init(&acc_empty[i], 128);
+      mbar_init(&acc_empty[i], EPI_ACTIVE * 32);
     }
     *abort_flag = 0;
     fence_barrier_init();
     tma_prefetch_desc(&tmap_a);
     tma_prefetch_desc(&tmap_w);
-    tma_prefetch_desc(&tmap_y);
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, TCOLS);
@@ -331,14 +336,18 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
   } else if (warp < kUnpackWarp0) {
     // ================= epilogue =================
-    const int qd = warp & 3;  // TMEM lane quadrant this warp may read
-    float* ts = s_scale + (warp - kEpiWarp0) * BN;  // this warp's private copy: no CTA-wide sync
-    float* tb = s_bias + (warp - kEpiWarp0) * BN;
-    uint8_t* stage = sY + (warp - kEpiWarp0) * kYStageBytes;
-    uint8_t* stage_row = stage + lane * 128;
-    bool ok = true;
+    const int ew = warp - kEpiWarp0;
+    const int qd = warp & 3;                  // TMEM lane quadrant this warp may read
+    const int slab0 = ew < 4 ? 0 : SLABS_LO;  // this warp's slabs: [slab0, slab1)
+    const int slab1 = ew < 4 ? SLABS_LO : SLABS;
+    float* ts = s_scale + ew * 64 * SLABS_LO;  // this warp's private copy: no CTA-wide sync
+    float* tb = s_bias + ew * 64 * SLABS_LO;
+    uint8_t* stage = sY + ew * kYStageBytes;
+    const uint4* stage4 = reinterpret_cast<const uint4*>(stage);
+    uint4* stage_row = reinterpret_cast<uint4*>(stage + lane * 64);
+    bool ok = slab0 < slab1;
     int tcount = 0, staged_n = -1;
-    if (p.early_w) pdl_wait();  // s_a below is written by the preceding kernel
+    if (ok && p.early_w) pdl_wait();  // s_a below is written by the preceding kernel
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
       const int n_blk = tile % p.n_tiles, m_blk = tile / p.n_tiles;  // column tiles of one row strip run together
       const int buf = tcount & 1;
@@ -349,17 +358,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       // independent loads first, their latency overlaps the wait for the accumulator
       const float sa = row_ok ? __ldg(p.s_a + row) : 0.0f;
       if (n_blk != staged_n) {
-        float sv[NCH], bv[NCH];
+        constexpr int NV = 2 * SLABS_LO;  // 32-column groups this warp may need
+        float sv[NV], bv[NV];
 #pragma unroll
-        for (int j = 0; j < NCH; ++j) sv[j] = __ldg(p.s_w + n0 + lane + 32 * j);
-#pragma unroll
-        for (int j = 0; j < NCH; ++j)
-          bv[j] = p.bias != nullptr
-                      ? __uint_as_float(static_cast<uint32_t>(__ldg(p.bias + n0 + lane + 32 * j)) << 16)
+        for (int j = 0; j < NV; ++j) {
+          const int col = slab0 * 64 + lane + 32 * j;
+          sv[j] = col < slab1 * 64 ? __ldg(p.s_w + n0 + col) : 0.0f;
+          bv[j] = (col < slab1 * 64 && p.bias != nullptr)
+                      ? __uint_as_float(static_cast<uint32_t>(__ldg(p.bias + n0 + col)) << 16)
                       : 0.0f;
+        }
         __syncwarp();
 #pragma unroll
-        for (int j = 0; j < NCH; ++j) {
+        for (int j = 0; j < NV; ++j) {
           ts[lane + 32 * j] = sv[j];
           tb[lane + 32 * j] = bv[j];
         }
@@ -371,36 +382,36 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       if (!ok) break;
       tc_fence_after();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + buf * (TCOLS / 2);
-      const int row0 = m_blk * BM + qd * 32;  // first token of this warp's slab
+      const int row0 = m_blk * BM + qd * 32;  // first token of this warp's slabs
       int32_t* arow = (p.dbg_acc != nullptr && row_ok) ? p.dbg_acc + row * p.dbg_ldacc + n0 : nullptr;
-      uint32_t ra[32], rb[32];
-      tmem_ld_32x32(t_addr, ra);
-#pragma unroll
-      for (int c = 0; c < NCH; c += 2) {  // one 64-column slab per iteration
+      for (int c = 2 * slab0; c < 2 * slab1; ++c) {  // 32-column chunks of this warp
+        uint32_t r[32];
+        tmem_ld_32x32(t_addr + c * 32, r);
         tmem_ld_wait();
-        tmem_ld_32x32(t_addr + (c + 1) * 32, rb);
-        if (lane == 0) tma_store_wait_read<0>();  // the previous slab's store has read the staging tile
-        __syncwarp();
-        epilogue_chunk<SHIFT>(ra, sa, ts + c * 32, tb + c * 32, stage_row, 0, lane & 7,
-                              arow ? arow + c * 32 : nullptr);
-        tmem_ld_wait();
-        if (c + 2 < NCH) {
-          tmem_ld_32x32(t_addr + (c + 2) * 32, ra);
-        } else {  // every accumulator of the tile is in registers: hand the buffer back
+        if (c + 1 == 2 * slab1) {  // this warp's last accumulators are in registers
           tc_fence_before();
           mbar_arrive(&acc_empty[buf]);
         }
-        epilogue_chunk<SHIFT>(rb, sa, ts + (c + 1) * 32, tb + (c + 1) * 32, stage_row, 1, lane & 7,
-                              arow ? arow + (c + 1) * 32 : nullptr);
-        fence_proxy_async_smem();
+        const int lc = (c - 2 * slab0) * 32;  // column inside this warp's staged scales
+        epilogue_chunk<SHIFT>(r, sa, reinterpret_cast<const float4*>(ts + lc),
+                              reinterpret_cast<const float4*>(tb + lc), stage_row, (lane >> 1) & 3,
+                              arow ? arow + c * 32 : nullptr);
         __syncwarp();
-        if (lane == 0 && row0 < p.M) {  // rows past M are clipped by the copy engine
-          tma_store_2d(&tmap_y, n0 + c * 32, row0, stage);
-          tma_store_commit();
+        // staged chunk -> global: every store instruction covers eight 64-byte row segments
+        {
+          const int ch = lane & 3;
+          uint16_t* ycol = p.y + n0 + c * 32 + ch * 8;
+#pragma unroll
+          for (int it = 0; it < 4; ++it) {
+            const int rr = 8 * it + (lane >> 2);
+            const uint4 v = stage4[rr * 4 + (ch ^ ((rr >> 1) & 3))];
+            const int64_t grow = static_cast<int64_t>(row0) + rr;
+            if (grow < p.M) *reinterpret_cast<uint4*>(ycol + grow * p.ldy) = v;
+          }
         }
+        __syncwarp();  // the staging tile is rewritten by the next chunk
       }
     }
-    if (lane == 0) tma_store_wait_all<0>();
   } else {
     // ================= unpack (3/4-bit weights) =================
     if constexpr (BITS != 8) {
@@ -439,8 +450,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 template <int BN, int BITS>
 constexpr size_t gemm_smem_bytes() {
   return 1024 + static_cast<size_t>(num_stages(BN, BITS)) * ab_stage_bytes(BN) +
-         kPStages * p_stage_bytes(BN, BITS) + 4 * kYStageBytes + (3 * 8 + 2 * kPStages + 4) * 8 + 32 +
-         8 * BN * 4 + 64;
+         kPStages * p_stage_bytes(BN, BITS) + kEpiWarps * kYStageBytes +
+         (3 * 8 + 2 * kPStages + 4) * 8 + 32 + 2 * kEpiWarps * 64 * ((BN / 64 + 1) / 2) * 4 + 64;
 }
 
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -509,11 +520,6 @@ int gemm_encode_w(CUtensorMap* out, const void* qweight, int32_t N, int32_t K, i
   return encode_2d(out, qweight, row_bytes, N, row_bytes, BK * bits / 8, bn, bits == 8);
 }
 
-// Output tensor: bf16 [M][N] with pitch ldy elements; stored in boxes of 64 columns x 32 tokens.
-int gemm_encode_y(CUtensorMap* out, const void* y, int64_t M, int32_t N, int64_t ldy) {
-  return encode_2d(out, y, static_cast<uint64_t>(N) * 2, M, static_cast<uint64_t>(ldy) * 2, 128, 32, true, 2);
-}
-
 // Tile width: the widest of {256, 192, 128, 64} dividing N whose tile count keeps the last wave
 // reasonably full; small problems take narrower tiles to spread over the SMs.
 int gemm_pick_bn(int64_t M, int32_t N, int32_t K, int32_t bits) {
@@ -546,16 +552,16 @@ static cudaError_t launch_bn(const GemmProblem& g, const GemmParams& p, dim3 gri
   switch (g.bits) {
     case 8:
       return launch(gemm_i8_kernel<BN, 8, false>, grid, block, gemm_smem_bytes<BN, 8>(), stream, pdl,
-                    g.tmap_a, g.tmap_w, g.tmap_y, p);
+                    g.tmap_a, g.tmap_w, p);
     case 4:
       if (g.korder == KORDER_EVEN_ODD)
         return launch(gemm_i8_kernel<BN, 4, true>, grid, block, gemm_smem_bytes<BN, 4>(), stream, pdl,
-                      g.tmap_a, g.tmap_w, g.tmap_y, p);
+                      g.tmap_a, g.tmap_w, p);
       return launch(gemm_i8_kernel<BN, 4, false>, grid, block, gemm_smem_bytes<BN, 4>(), stream, pdl,
-                    g.tmap_a, g.tmap_w, g.tmap_y, p);
+                    g.tmap_a, g.tmap_w, p);
     default:
       return launch(gemm_i8_kernel<BN, 3, false>, grid, block, gemm_smem_bytes<BN, 3>(), stream, pdl,
-                    g.tmap_a, g.tmap_w, g.tmap_y, p);
+                    g.tmap_a, g.tmap_w, p);
   }
 }
 

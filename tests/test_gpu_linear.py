@@ -102,6 +102,30 @@ def test_mma_one_hot_and_constant_inputs(bits):
     _check(run_linear(L, xc, flags=B.DP_FLAG_FORCE_MMA), xc, w, s_w, None, bits)
 
 
+@pytest.mark.parametrize("bits", [8, 4, 3])
+def test_mma_extreme_accumulators(bits):
+    """Saturated tokens against saturated weight rows at K = 4608: |acc| reaches 4608*127*2^(b-1)
+    (7.5e7 at 8 bits, beyond 2^24), so the int32 -> fp32 step of the epilogue has to round; mixed
+    with random rows and signs so every magnitude in between occurs too."""
+    M, K, N = 128, 4608, 128
+    rng = np.random.default_rng(bits + 100)
+    f = rng.standard_normal((M, K)).astype(np.float32)
+    f[0::4] = 3.0
+    f[1::4] = -3.0
+    f[2::4, ::2] = 1.0
+    x = synth.f32_to_bf16_bits(f)
+    lo, hi = -(1 << (bits - 1)), (1 << (bits - 1)) - 1
+    w = rng.integers(lo, hi + 1, size=(N, K)).astype(np.int8)
+    w[0::4] = lo
+    w[1::4] = hi
+    w[2::4, : K // 2] = lo
+    s_w = np.full(N, 2.0 ** -10, np.float32)
+    L = DevLayer(w, s_w, None, bits)
+    out = run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA)
+    assert np.abs(out["acc"]).max() == 4608 * 127 * (1 << (bits - 1))
+    _check(out, x, w, s_w, None, bits)
+
+
 @pytest.mark.parametrize("flags", [B.DP_FLAG_FORCE_SIMT, B.DP_FLAG_FORCE_MMA])
 def test_prequantized_input(flags):
     M, K, N, bits = 130, 256, 128, 4
