@@ -135,6 +135,33 @@ int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_
                  const dp_debug* dbg, int32_t* device_status, uint32_t flags, dp_stream stream);
 
 /*
+ * dp_wq_linear for callers that cannot allocate device memory. (The paper has no counterpart: this
+ * is a deployment convenience of the library, not a step of the method.)
+ *
+ * Some hosts of this code only hand a kernel library its input and output buffers and forbid it to
+ * call cudaMalloc: a custom-op slot of an inference runtime that owns all device memory, a step
+ * that runs while a stream is being captured into a CUDA graph, or a latency-critical loop where an
+ * allocation would stall the device. For them the scratch that dp_wq_linear takes as `workspace`
+ * (the int8 activations and their scales between its two kernels) lives inside the library, in one
+ * fixed device array of DP_STATIC_SCRATCH_BYTES that every GPU loading the library holds until the
+ * process exits. The call computes exactly what dp_wq_linear(w, x, ldx, NULL, M, y, ldy, ...) does.
+ *
+ *   - Problems whose dp_wq_linear_workspace(M, N, K, bits, flags) exceeds DP_STATIC_SCRATCH_BYTES are
+ *     refused with DP_ERR_WORKSPACE and nothing is enqueued (M = 2048 tokens at K = 4608 fits).
+ *   - The first call on each device looks up the array's device address (a cheap runtime query, no
+ *     allocation); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, on every stream: two calls whose kernels may
+ *     overlap on the GPU race on it. Issue them on one stream, or order them yourself.
+ *   - The array keeps whatever the previous call left. Nothing in it has to start at zero: the
+ *     quantization kernel overwrites every byte the GEMM reads before the GEMM runs.
+ *   - No cudaMalloc, cudaFree or other allocating routine is called; x is always bf16 (the
+ *     pre-quantized form of dp_wq_linear needs no scratch and is not offered here).
+ */
+#define DP_STATIC_SCRATCH_BYTES (10u << 20)
+int dp_wq_linear_static(const dp_weight* w, const void* x_bf16, int64_t ldx, int64_t M, void* y_bf16,
+                        int64_t ldy, int32_t* device_status, uint32_t flags, dp_stream stream);
+
+/*
  * A deployed plan (Algorithm 2, Phase B: "wrap layers per the bit plan"): n_layers quantized
  * linears with their row counts. Creation validates every layer, chooses kernel variants, encodes
  * TMA descriptors and may allocate/synchronise; it is not on the timed path. The dp_weight array is

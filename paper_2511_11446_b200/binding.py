@@ -25,7 +25,9 @@ DP_PLAN_SAME_X, DP_PLAN_SAME_Y = 1, 2
 def DP_FLAG_TILE_N(bn: int) -> int:
     return (bn // 64) << 8
 
-EXPORTS = ["dp_daq_quantize", "dp_wq_linear_workspace", "dp_wq_linear", "dp_plan_create",
+DP_STATIC_SCRATCH_BYTES = 10 << 20
+
+EXPORTS = ["dp_daq_quantize", "dp_wq_linear_workspace", "dp_wq_linear", "dp_wq_linear_static", "dp_plan_create",
            "dp_plan_workspace", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
            "dp_plan_run_host", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_status_string",
            "dp_last_error", "dp_version"]
@@ -73,6 +75,8 @@ def lib():
         L.dp_wq_linear.argtypes = [C.POINTER(dp_weight), C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                    C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t,
                                    C.POINTER(dp_debug), C.c_void_p, C.c_uint32, C.c_void_p]
+        L.dp_wq_linear_static.argtypes = [C.POINTER(dp_weight), C.c_void_p, C.c_int64, C.c_int64, C.c_void_p,
+                                          C.c_int64, C.c_void_p, C.c_uint32, C.c_void_p]
         L.dp_plan_create.argtypes = [C.POINTER(dp_weight), C.c_int32, C.POINTER(C.c_int64), C.c_uint32,
                                      C.POINTER(C.c_void_p)]
         L.dp_plan_run.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.c_int32, C.c_int32,
@@ -122,6 +126,13 @@ def dp_wq_linear(w: dp_weight, x, ldx, s_a_in, M, y, ldy, workspace, dbg: dp_deb
     _check(lib().dp_wq_linear(C.byref(w), _ptr(x), ldx, _ptr(s_a_in), M, _ptr(y), ldy, _ptr(workspace),
                               ws_bytes, None if dbg is None else C.byref(dbg), _ptr(device_status),
                               flags, _stream(stream)), "dp_wq_linear")
+
+
+def dp_wq_linear_static(w: dp_weight, x, ldx, M, y, ldy, device_status=None, flags=0, stream=None):
+    """dp_wq_linear without a workspace argument: the scratch is a fixed array inside the library
+    (for callers that may not allocate device memory). bf16 input only."""
+    _check(lib().dp_wq_linear_static(C.byref(w), _ptr(x), ldx, M, _ptr(y), ldy, _ptr(device_status), flags,
+                                     _stream(stream)), "dp_wq_linear_static")
 
 
 def dp_plan_create(weights: list[dp_weight], Ms: list[int], flags=0) -> C.c_void_p:

@@ -230,6 +230,52 @@ extern "C" int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, cons
                     static_cast<cudaStream_t>(stream), nullptr, 0, nullptr, false);
 }
 
+// ---- the linear for callers that cannot allocate ---------------------------------------------------
+// Scratch of dp_wq_linear_static. In host code `g_static_scratch` is only a handle for the runtime:
+// its device address comes from cudaGetSymbolAddress, once per device, and that address is what the
+// kernels receive.
+static __device__ __align__(256) unsigned char g_static_scratch[DP_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+static void* g_static_scratch_ptr[kMaxDevices];  // device address per device ordinal, nullptr = not yet queried
+
+static int static_scratch_address(void** out) {
+  int dev = 0;
+  DP_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return fail(DP_ERR_INVALID_ARG, "device ordinal %d not supported", dev);
+  if (g_static_scratch_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    DP_CUDA_OK(cudaGetSymbolAddress(&p, g_static_scratch));
+    if (p == nullptr || (reinterpret_cast<uintptr_t>(p) & 255u))
+      return fail(DP_ERR_CUDA, "static scratch has no usable device address on device %d", dev);
+    g_static_scratch_ptr[dev] = p;
+  }
+  *out = g_static_scratch_ptr[dev];
+  return DP_OK;
+}
+
+extern "C" int dp_wq_linear_static(const dp_weight* w, const void* x_bf16, int64_t ldx, int64_t M,
+                                   void* y_bf16, int64_t ldy, int32_t* device_status, uint32_t flags,
+                                   dp_stream stream) {
+  int st = check_weight(w);
+  if (st != DP_OK) return st;
+  const size_t need = dp_wq_linear_workspace(M, w->N, w->K, w->bits, flags);
+  if (need > DP_STATIC_SCRATCH_BYTES)
+    return fail(DP_ERR_WORKSPACE,
+                "dp_wq_linear_static: M=%lld K=%d needs %zu bytes of scratch, the built-in array holds %u; "
+                "use dp_wq_linear with a caller-provided workspace",
+                (long long)M, w->K, need, (unsigned)DP_STATIC_SCRATCH_BYTES);
+  st = check_device();
+  if (st != DP_OK) return st;
+  void* scratch = nullptr;
+  st = static_scratch_address(&scratch);
+  if (st != DP_OK) return st;
+  st = check_linear_args(w, x_bf16, ldx, nullptr, M, y_bf16, ldy, scratch, DP_STATIC_SCRATCH_BYTES, nullptr, flags);
+  if (st != DP_OK || M == 0) return st;
+  return run_linear(w, x_bf16, ldx, nullptr, M, y_bf16, ldy, scratch, nullptr, device_status, flags,
+                    static_cast<cudaStream_t>(stream), nullptr, 0, nullptr, false);
+}
+
 // ---- plans ---------------------------------------------------------------------------------------
 struct PlanLayer {
   dp_weight w;
