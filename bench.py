@@ -319,13 +319,14 @@ def main():
     ap.add_argument("--layers", default=None, help="comma list out of qkv,proj,fc1,fc2,adaln")
     ap.add_argument("--only", default=None, choices=["layer", "gemm", "daq"])
     ap.add_argument("--iters", type=int, default=None)
+    ap.add_argument("--flags", type=lambda v: int(v, 0), default=0, help="dp_wq_linear tuning flags for --sweep")
     args = ap.parse_args()
     if args.sweep:
         import torch
         from paper_2511_11446_b200 import sweep
         torch.cuda.set_device(0)
         sweep.run(args.sweep, [int(b) for b in args.bits.split(",")], measured_peaks(), only=args.only,
-                  layers=args.layers.split(",") if args.layers else None, iters=args.iters)
+                  layers=args.layers.split(",") if args.layers else None, iters=args.iters, flags=args.flags)
         return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

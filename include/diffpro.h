@@ -89,6 +89,10 @@ typedef struct dp_debug {
  * 256; must divide N) instead of letting the library choose. */
 #define DP_FLAG_TILE_N(bn) ((uint32_t)((bn) / 64) << 8)
 #define DP_FLAG_TILE_N_MASK 0x700u
+/* Tuning/testing: force (or forbid) the tensor-core kernel variant in which the two CTAs of a
+ * thread-block cluster share a 256-row tile (tile width 128, 192 or 256 only). */
+#define DP_FLAG_CTA_PAIR 0x800u
+#define DP_FLAG_NO_CTA_PAIR 0x1000u
 
 /* flags for dp_plan_run */
 #define DP_PLAN_SAME_X 1u       /* x_ptrs has n_layers entries reused by every step              */

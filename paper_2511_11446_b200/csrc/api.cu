@@ -49,8 +49,34 @@ int check_device() {
 static size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
 
 constexpr uint32_t kLinearFlags =
-    DP_FLAG_FORCE_SIMT | DP_FLAG_FORCE_MMA | DP_FLAG_NO_PDL | DP_FLAG_TILE_N_MASK;
+    DP_FLAG_FORCE_SIMT | DP_FLAG_FORCE_MMA | DP_FLAG_NO_PDL | DP_FLAG_TILE_N_MASK | DP_FLAG_CTA_PAIR |
+    DP_FLAG_NO_CTA_PAIR;
 static int forced_bn(uint32_t flags) { return static_cast<int>((flags & DP_FLAG_TILE_N_MASK) >> 8) * 64; }
+
+// Tile width and CTA-group size of the tensor-core kernel for this problem, honouring the tuning
+// flags (validated by check_tile_flags).
+static void choose_tile(uint32_t flags, int64_t M, int32_t N, int32_t K, int32_t bits, int* bn, int* cg) {
+  uint32_t allow = 0x6;
+  if (flags & DP_FLAG_CTA_PAIR) allow = 0x4;
+  if (flags & DP_FLAG_NO_CTA_PAIR) allow = 0x2;
+  gemm_pick_tile(M, N, K, bits, allow, bn, cg);
+  const int fb = forced_bn(flags);
+  if (fb != 0 && N % fb == 0) {
+    *bn = fb;
+    if (fb < 128) *cg = 1;
+    else if (allow == 0x4) *cg = 2;
+    else if (allow == 0x2) *cg = 1;
+  }
+}
+static int check_tile_flags(uint32_t flags, int32_t N) {
+  const int fb = forced_bn(flags);
+  if (fb != 0 && (fb > 256 || N % fb)) return fail(DP_ERR_SHAPE, "forced tile width %d does not divide N=%d", fb, N);
+  if ((flags & DP_FLAG_CTA_PAIR) && (flags & DP_FLAG_NO_CTA_PAIR))
+    return fail(DP_ERR_INVALID_ARG, "CTA_PAIR and NO_CTA_PAIR are exclusive");
+  if ((flags & DP_FLAG_CTA_PAIR) && ((fb != 0 && fb < 128) || N % 128))
+    return fail(DP_ERR_SHAPE, "CTA-pair tiles need a tile width of 128, 192 or 256 dividing N=%d", N);
+  return DP_OK;
+}
 
 constexpr int64_t kSimtMaxRows = 32;  // at or below this the CUDA-core streaming kernel is used
 
@@ -82,7 +108,7 @@ static int check_weight(const dp_weight* w) {
 // while it drains.
 static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_a_in, int64_t M,
                       void* y, int64_t ldy, void* workspace, const dp_debug* dbg, int32_t* status,
-                      uint32_t flags, cudaStream_t stream, const CUtensorMap* tmap_w, int bn,
+                      uint32_t flags, cudaStream_t stream, const CUtensorMap* tmap_w, int bn, int cg,
                       const CUtensorMap* tmap_a_cached, bool chained) {
   const bool pdl = !(flags & DP_FLAG_NO_PDL);
   if (use_simt(M, w->N, w->K, flags)) {
@@ -136,11 +162,12 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
     int st = gemm_encode_a(&g.tmap_a, q, M, w->K, ldq);
     if (st != DP_OK) return st;
   }
-  if (bn == 0) bn = forced_bn(flags) ? forced_bn(flags) : gemm_pick_bn(M, w->N, w->K, w->bits);
+  if (bn == 0) choose_tile(flags, M, w->N, w->K, w->bits, &bn, &cg);
+  g.cg = cg;
   if (tmap_w != nullptr) {
     g.tmap_w = *tmap_w;
   } else {
-    int st = gemm_encode_w(&g.tmap_w, w->qweight, w->N, w->K, w->bits, bn);
+    int st = gemm_encode_w(&g.tmap_w, w->qweight, w->N, w->K, w->bits, bn, cg);
     if (st != DP_OK) return st;
   }
   g.s_a = s_a;
@@ -181,8 +208,7 @@ static int check_linear_args(const dp_weight* w, const void* x, int64_t ldx, con
   if (st != DP_OK) return st;
   if (M < 0) return fail(DP_ERR_SHAPE, "M=%lld is negative", (long long)M);
   if (flags & ~kLinearFlags) return fail(DP_ERR_INVALID_ARG, "unknown flag bits 0x%x", flags);
-  if (forced_bn(flags) != 0 && (forced_bn(flags) > 256 || w->N % forced_bn(flags)))
-    return fail(DP_ERR_SHAPE, "forced tile width %d does not divide N=%d", forced_bn(flags), w->N);
+  if (int tst = check_tile_flags(flags, w->N)) return tst;
   if ((flags & DP_FLAG_FORCE_SIMT) && (flags & DP_FLAG_FORCE_MMA))
     return fail(DP_ERR_INVALID_ARG, "FORCE_SIMT and FORCE_MMA are exclusive");
   if (M == 0) return DP_OK;
@@ -227,7 +253,7 @@ extern "C" int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, cons
   st = check_device();
   if (st != DP_OK) return st;
   return run_linear(w, x, ldx, s_a_in, M, y_bf16, ldy, workspace, dbg, device_status, flags,
-                    static_cast<cudaStream_t>(stream), nullptr, 0, nullptr, false);
+                    static_cast<cudaStream_t>(stream), nullptr, 0, 0, nullptr, false);
 }
 
 // ---- the linear for callers that cannot allocate ---------------------------------------------------
@@ -273,7 +299,7 @@ extern "C" int dp_wq_linear_static(const dp_weight* w, const void* x_bf16, int64
   st = check_linear_args(w, x_bf16, ldx, nullptr, M, y_bf16, ldy, scratch, DP_STATIC_SCRATCH_BYTES, nullptr, flags);
   if (st != DP_OK || M == 0) return st;
   return run_linear(w, x_bf16, ldx, nullptr, M, y_bf16, ldy, scratch, nullptr, device_status, flags,
-                    static_cast<cudaStream_t>(stream), nullptr, 0, nullptr, false);
+                    static_cast<cudaStream_t>(stream), nullptr, 0, 0, nullptr, false);
 }
 
 // ---- plans ---------------------------------------------------------------------------------------
@@ -281,7 +307,7 @@ struct PlanLayer {
   dp_weight w;
   int64_t M;
   bool simt;
-  int bn;
+  int bn, cg;
   CUtensorMap tmap_w;
   size_t x_offset;  // byte offset of this layer's input inside one staged step (host-input path)
 };
@@ -328,15 +354,17 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
     L.M = M_per_layer[l];
     L.simt = use_simt(L.M, L.w.N, L.w.K, flags);
     L.bn = 0;
+    L.cg = 1;
     memset(&L.tmap_w, 0, sizeof(L.tmap_w));
     if (L.simt && static_cast<size_t>(L.w.K) > simt_max_k()) {
       delete p;
       return fail(DP_ERR_SHAPE, "layer %d: K too large for the small-M kernel", l);
     }
     if (!L.simt && L.M > 0) {
-      L.bn = (forced_bn(flags) && L.w.N % forced_bn(flags) == 0) ? forced_bn(flags)
-                                                                 : gemm_pick_bn(L.M, L.w.N, L.w.K, L.w.bits);
-      st = gemm_encode_w(&L.tmap_w, L.w.qweight, L.w.N, L.w.K, L.w.bits, L.bn);
+      uint32_t lf = flags;  // a pair request that this layer's N cannot honour falls back to the default
+      if ((lf & DP_FLAG_CTA_PAIR) && L.w.N % 128) lf &= ~DP_FLAG_CTA_PAIR;
+      choose_tile(lf, L.M, L.w.N, L.w.K, L.w.bits, &L.bn, &L.cg);
+      st = gemm_encode_w(&L.tmap_w, L.w.qweight, L.w.N, L.w.K, L.w.bits, L.bn, L.cg);
       if (st != DP_OK) {
         delete p;
         return st;
@@ -405,7 +433,7 @@ static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, 
       if (st != DP_OK) return st;
     }
     int st = run_linear(&L.w, xs[l], L.w.K, nullptr, L.M, ys[l], L.w.N, workspace, nullptr, status,
-                        plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, ta, *chained);
+                        plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, L.cg, ta, *chained);
     if (st != DP_OK) return st;
     *chained = true;
   }

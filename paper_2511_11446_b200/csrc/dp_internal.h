@@ -59,15 +59,18 @@ struct GemmProblem {
   int64_t dbg_ldacc;
   int64_t M;
   int32_t N, K, bits, bn;
+  int32_t cg;       // 1: one CTA per 128-row tile; 2: a CTA pair per 256-row tile
   int32_t korder;   // KOrder of the activations behind tmap_a
   int32_t early_w;  // the preceding kernel on the stream is this call's own DAQ: weights may be
                     // fetched before it has finished
   int32_t* status;
 };
-int gemm_pick_bn(int64_t M, int32_t N, int32_t K, int32_t bits);
+// allow: bit 1 = single-CTA tiles permitted, bit 2 = CTA-pair tiles permitted
+void gemm_pick_tile(int64_t M, int32_t N, int32_t K, int32_t bits, uint32_t allow, int* bn_out, int* cg_out);
+int gemm_max_pairs();
 int gemm_encode_a(CUtensorMap* out, const int8_t* q, int64_t M, int64_t K, int64_t ldq);
 int gemm_encode_w(CUtensorMap* out, const void* qweight, int32_t N, int32_t K, int32_t bits,
-                  int32_t bn);
+                  int32_t bn, int32_t cg);
 int launch_gemm(const GemmProblem& p, cudaStream_t stream, bool pdl);
 int gemm_init();  // sets kernel attributes, resolves the tensor-map encoder; idempotent
 

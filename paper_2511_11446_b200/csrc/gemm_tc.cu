@@ -3,7 +3,13 @@
 //   Step 5 / Implementation of the paper: INT8 x INT8 -> INT32 GEMM with per-output-channel weight
 //   scales; Step 3: weights are GPTQ-style packed low-bit integers, expanded on the fly.
 //
-// One persistent CTA per SM walks a static list of 128 x BN output tiles. Warp roles:
+// One persistent CTA per SM walks a static list of output tiles. CG = 1: a CTA owns 128 x BN tiles.
+// CG = 2: the two CTAs of a thread-block cluster own a 256 x BN tile together (tcgen05 cta_group::2):
+// each loads its own 128 token rows and only ITS half of the BN weight rows (plain TMA loads, no
+// multicast), the pair's leader issues one MMA per 32 bytes of K that reads both CTAs' shared
+// memory, and each CTA ends up with its 128 x BN accumulator in its own tensor memory. Per CTA this
+// halves the weight bytes fetched, expanded and read by the tensor core for the same MACs.
+// Warp roles:
 //   warp 0      TMA producer: int8 activation tiles (128-byte-swizzled) and packed weight tiles
 //   warp 1      MMA issuer: tcgen05.mma kind::i8, int32 accumulators in tensor memory (two
 //               accumulator buffers, so a tile's epilogue overlaps the next tile's mainloop)
@@ -41,6 +47,7 @@ constexpr int kYStageBytes = 32 * 64;  // per epilogue warp: 32 tokens x 32 bf16
 constexpr int kSmemBudget = 200 * 1024;
 constexpr int kPStages = 3;
 
+// bn below is the number of weight rows ONE CTA holds (BN for CG = 1, BN / 2 for a pair).
 __host__ __device__ constexpr int p_stage_bytes(int bn, int bits) {
   return bits == 8 ? 0 : bn * (BK * bits / 8);
 }
@@ -61,7 +68,7 @@ struct GemmParams {
   int64_t dbg_ldacc;
   int64_t M;
   int32_t N, K;
-  int32_t m_tiles, n_tiles;
+  int32_t m_tiles, n_tiles;  // m_tiles counts row tiles of 128 * CG tokens
   int32_t early_w;  // weights may be fetched before the preceding kernel on the stream has finished
   int32_t* status;
 };
@@ -83,8 +90,9 @@ struct Ring {  // stage index + phase bit of a circular buffer
 template <int BN, bool PERM>
 __device__ __forceinline__ void unpack4_tile(const uint8_t* P, uint8_t* B, int tid) {
 #pragma unroll
-  for (int i = 0; i < BN * 8 / kUnpackThreads; ++i) {
+  for (int i = 0; i < (BN * 8 + kUnpackThreads - 1) / kUnpackThreads; ++i) {
     const int idx = tid + i * kUnpackThreads;
+    if (BN * 8 % kUnpackThreads != 0 && idx >= BN * 8) break;
     const int row = idx >> 3, kc = idx & 7;
     const uint2 in = *reinterpret_cast<const uint2*>(P + row * 64 + kc * 8);
     uint4 o;
@@ -112,8 +120,9 @@ __device__ __forceinline__ uint32_t spread3(uint32_t v) {  // 4 fields of 3 bits
 template <int BN>
 __device__ __forceinline__ void unpack3_tile(const uint8_t* P, uint8_t* B, int tid) {
 #pragma unroll
-  for (int i = 0; i < BN * 4 / kUnpackThreads; ++i) {
+  for (int i = 0; i < (BN * 4 + kUnpackThreads - 1) / kUnpackThreads; ++i) {
     const int idx = tid + i * kUnpackThreads;
+    if (BN * 4 % kUnpackThreads != 0 && idx >= BN * 4) break;
     const int row = idx >> 2, g = idx & 3;
     const uint32_t* src = reinterpret_cast<const uint32_t*>(P + row * 48 + g * 12);
     const uint32_t s0 = src[0], s1 = src[1], s2 = src[2];
@@ -180,31 +189,32 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], float sa
 }
 
 // ---- the kernel ----------------------------------------------------------------------------------
-template <int BN, int BITS, bool PERM>
+template <int BN, int BITS, bool PERM, int CG>
 __global__ void __launch_bounds__(gemm_threads(BITS), 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                const GemmParams p) {
-  constexpr int NS = num_stages(BN, BITS);
+  constexpr int BNL = BN / CG;  // weight rows held by this CTA
+  constexpr int NS = num_stages(BNL, BITS);
   constexpr int NP = kPStages;
-  constexpr int A_BYTES = BM * BK, B_BYTES = BN * BK, P_BYTES = p_stage_bytes(BN, BITS);
+  constexpr int A_BYTES = BM * BK, B_BYTES = BNL * BK, P_BYTES = p_stage_bytes(BNL, BITS);
   constexpr int TCOLS = tmem_cols(BN);
   constexpr int SHIFT = 8 - BITS;  // accumulator carries a factor 2^SHIFT
-  constexpr int NCH = BN / 32;     // 32-column chunks per tile (even)
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem;
   uint8_t* sB = sA + NS * A_BYTES;
   uint8_t* sP = sB + NS * B_BYTES;
-  uint8_t* sY = sP + NP * P_BYTES;  // [epilogue warps][32 tokens][128 bytes] output staging
+  uint8_t* sY = sP + NP * P_BYTES;  // [epilogue warps][32 tokens][64 bytes] output staging
   uint8_t* tail = sY + kEpiWarps * kYStageBytes;
   uint64_t* full_a = reinterpret_cast<uint64_t*>(tail);
   uint64_t* bready = full_a + NS;
   uint64_t* empty = bready + NS;
-  uint64_t* pfull = empty + NS;
+  uint64_t* peer_ready = empty + NS;  // pair leader only: the other CTA's stage is loaded (and expanded)
+  uint64_t* pfull = peer_ready + NS;
   uint64_t* pempty = pfull + NP;
   uint64_t* acc_full = pempty + NP;
-  uint64_t* acc_empty = acc_full + 2;
+  uint64_t* acc_empty = acc_full + 2;  // CG = 2: the leader's copy collects both CTAs' epilogue warps
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   constexpr int SLABS = BN / 64;            // 64-column slabs per tile
@@ -217,12 +227,15 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int KB = p.K / BK;
   const int total_tiles = p.m_tiles * p.n_tiles;
+  const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;  // 0 = leader of the pair
+  const int first_tile = blockIdx.x / CG, tile_stride = gridDim.x / CG;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NS; ++i) {
       mbar_init(&full_a[i], 1);
       mbar_init(&bready[i], kUnpackThreads);
       mbar_init(&empty[i], 1);
+      mbar_init(&peer_ready[i], 1);
     }
     for (int i = 0; i < NP; ++i) {
       mbar_init(&pfull[i], 1);
@@ -230,7 +243,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&acc_full[i], 1);
-      mbar_init(&acc_empty[i], EPI_ACTIVE * 32);
+      mbar_init(&acc_empty[i], CG * EPI_ACTIVE);  // one arrival per epilogue warp
     }
     *abort_flag = 0;
     fence_barrier_init();
@@ -238,11 +251,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     tma_prefetch_desc(&tmap_w);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, TCOLS);
-    tmem_relinquish();
+    if constexpr (CG == 2) {
+      tmem_alloc_pair(tmem_slot, TCOLS);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(tmem_slot, TCOLS);
+      tmem_relinquish();
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if constexpr (CG == 2) cluster_sync();  // both CTAs' barriers exist before either signals the other
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -260,32 +279,34 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       bool a_open = !p.early_w;  // false until griddepcontrol.wait has been executed
       int deferred = 0;          // stages whose weight tile is in flight but whose A tile is not
       int def_kb[NS], def_m[NS], def_s[NS];
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int n_blk = tile % p.n_tiles, m_blk = tile / p.n_tiles;  // column tiles of one row strip run together
+      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_stride) {
+        const int n_blk = tile % p.n_tiles;  // column tiles of one row strip run together
+        const int m_row = (tile / p.n_tiles) * (BM * CG) + static_cast<int>(rank) * BM;
+        const int w_row = n_blk * BN + static_cast<int>(rank) * BNL;
         for (int kb = 0; kb < KB; ++kb) {
           if (!a_open && deferred == NS) {  // ring full of weight tiles: now wait for the activations
             pdl_wait();
             a_open = true;
             for (int d = 0; d < deferred; ++d)
-              tma_load_2d(sA + def_s[d] * A_BYTES, &tmap_a, def_kb[d] * BK, def_m[d] * BM, &full_a[def_s[d]]);
+              tma_load_2d(sA + def_s[d] * A_BYTES, &tmap_a, def_kb[d] * BK, def_m[d], &full_a[def_s[d]]);
             deferred = 0;
           }
           if (!(ok = mbar_wait(&empty[st.s], st.ph ^ 1u, abort_flag))) break;
           if constexpr (BITS == 8) {
             mbar_arrive_expect_tx(&full_a[st.s], A_BYTES + B_BYTES);
-            tma_load_2d(sB + st.s * B_BYTES, &tmap_w, kb * BK, n_blk * BN, &full_a[st.s]);
+            tma_load_2d(sB + st.s * B_BYTES, &tmap_w, kb * BK, w_row, &full_a[st.s]);
           } else {
             if (!(ok = mbar_wait(&pempty[ps.s], ps.ph ^ 1u, abort_flag))) break;
             mbar_arrive_expect_tx(&pfull[ps.s], P_BYTES);
-            tma_load_2d(sP + ps.s * P_BYTES, &tmap_w, kb * (BK * BITS / 8), n_blk * BN, &pfull[ps.s]);
+            tma_load_2d(sP + ps.s * P_BYTES, &tmap_w, kb * (BK * BITS / 8), w_row, &pfull[ps.s]);
             mbar_arrive_expect_tx(&full_a[st.s], A_BYTES);
             ps.next(NP);
           }
           if (a_open) {
-            tma_load_2d(sA + st.s * A_BYTES, &tmap_a, kb * BK, m_blk * BM, &full_a[st.s]);
+            tma_load_2d(sA + st.s * A_BYTES, &tmap_a, kb * BK, m_row, &full_a[st.s]);
           } else {
             def_kb[deferred] = kb;
-            def_m[deferred] = m_blk;
+            def_m[deferred] = m_row;
             def_s[deferred] = st.s;
             ++deferred;
           }
@@ -295,7 +316,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       if (!a_open) {  // fewer k-blocks than stages in the whole CTA
         pdl_wait();
         for (int d = 0; d < deferred; ++d)
-          tma_load_2d(sA + def_s[d] * A_BYTES, &tmap_a, def_kb[d] * BK, def_m[d] * BM, &full_a[def_s[d]]);
+          tma_load_2d(sA + def_s[d] * A_BYTES, &tmap_a, def_kb[d] * BK, def_m[d], &full_a[def_s[d]]);
       }
       if (!ok) {
         // drain: give copies still in flight a bounded time to land before the CTA exits
@@ -305,33 +326,62 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       }
     }
   } else if (warp == 1) {
-    // ================= MMA issuer =================
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_i8(BM, BN);
-      Ring st;
-      bool ok = true;
-      int tcount = 0;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-        const int buf = tcount & 1;
-        const uint32_t aph = (tcount >> 1) & 1;
-        if (!(ok = mbar_wait(&acc_empty[buf], aph ^ 1u, abort_flag))) break;
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * (TCOLS / 2);
-        for (int kb = 0; kb < KB; ++kb) {
-          if (!(ok = mbar_wait(&full_a[st.s], st.ph, abort_flag))) break;
-          if constexpr (BITS != 8) {
-            if (!(ok = mbar_wait(&bready[st.s], st.ph, abort_flag))) break;
+      if (CG == 2 && rank != 0) {
+        // ================= pair follower: report each loaded stage to the leader =================
+        Ring st;
+        bool ok = true;
+        for (int tile = first_tile; tile < total_tiles && ok; tile += tile_stride) {
+          for (int kb = 0; kb < KB; ++kb) {
+            if (!(ok = mbar_wait(&full_a[st.s], st.ph, abort_flag))) break;
+            if constexpr (BITS != 8) {
+              if (!(ok = mbar_wait(&bready[st.s], st.ph, abort_flag))) break;
+            }
+            mbar_arrive_cluster(map_to_cta(&peer_ready[st.s], 0));
+            st.next(NS);
           }
-          tc_fence_after();
-          const uint64_t adesc = smem_desc_sw128(smem_u32(sA + st.s * A_BYTES));
-          const uint64_t bdesc = smem_desc_sw128(smem_u32(sB + st.s * B_BYTES));
-#pragma unroll
-          for (int k4 = 0; k4 < BK / 32; ++k4)  // 32 bytes of K per instruction: +2 in 16-byte units
-            mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
-          mma_commit(&empty[st.s]);
-          st.next(NS);
         }
-        if (ok) mma_commit(&acc_full[buf]);
+      } else {
+        // ================= MMA issuer =================
+        constexpr uint32_t idesc = idesc_i8(BM * CG, BN);
+        Ring st;
+        bool ok = true;
+        int tcount = 0;
+        for (int tile = first_tile; tile < total_tiles && ok; tile += tile_stride, ++tcount) {
+          const int buf = tcount & 1;
+          const uint32_t aph = (tcount >> 1) & 1;
+          if (!(ok = CG == 2 ? mbar_wait_cluster(&acc_empty[buf], aph ^ 1u, abort_flag)
+                             : mbar_wait(&acc_empty[buf], aph ^ 1u, abort_flag)))
+            break;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + buf * (TCOLS / 2);
+          for (int kb = 0; kb < KB; ++kb) {
+            if (!(ok = mbar_wait(&full_a[st.s], st.ph, abort_flag))) break;
+            if constexpr (BITS != 8) {
+              if (!(ok = mbar_wait(&bready[st.s], st.ph, abort_flag))) break;
+            }
+            if constexpr (CG == 2) {
+              if (!(ok = mbar_wait_cluster(&peer_ready[st.s], st.ph, abort_flag))) break;
+            }
+            tc_fence_after();
+            const uint64_t adesc = smem_desc_sw128(smem_u32(sA + st.s * A_BYTES));
+            const uint64_t bdesc = smem_desc_sw128(smem_u32(sB + st.s * B_BYTES));
+#pragma unroll
+            for (int k4 = 0; k4 < BK / 32; ++k4) {  // 32 bytes of K per instruction: +2 in 16-byte units
+              if constexpr (CG == 2)
+                mma_i8_ss_pair(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+              else
+                mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+            }
+            if constexpr (CG == 2) mma_commit_pair(&empty[st.s]);
+            else mma_commit(&empty[st.s]);
+            st.next(NS);
+          }
+          if (ok) {
+            if constexpr (CG == 2) mma_commit_pair(&acc_full[buf]);
+            else mma_commit(&acc_full[buf]);
+          }
+        }
       }
     }
   } else if (warp < kUnpackWarp0) {
@@ -345,15 +395,20 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     uint8_t* stage = sY + ew * kYStageBytes;
     const uint4* stage4 = reinterpret_cast<const uint4*>(stage);
     uint4* stage_row = reinterpret_cast<uint4*>(stage + lane * 64);
+    uint32_t acc_empty_addr[2];  // where this warp reports a drained accumulator buffer
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+      acc_empty_addr[i] = CG == 2 ? map_to_cta(&acc_empty[i], 0) : smem_u32(&acc_empty[i]);
     bool ok = slab0 < slab1;
     int tcount = 0, staged_n = -1;
     if (ok && p.early_w) pdl_wait();  // s_a below is written by the preceding kernel
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-      const int n_blk = tile % p.n_tiles, m_blk = tile / p.n_tiles;  // column tiles of one row strip run together
+    for (int tile = first_tile; tile < total_tiles && ok; tile += tile_stride, ++tcount) {
+      const int n_blk = tile % p.n_tiles;  // column tiles of one row strip run together
       const int buf = tcount & 1;
       const uint32_t aph = (tcount >> 1) & 1;
       const int n0 = n_blk * BN;
-      const int64_t row = static_cast<int64_t>(m_blk) * BM + qd * 32 + lane;
+      const int row0 = (tile / p.n_tiles) * (BM * CG) + static_cast<int>(rank) * BM + qd * 32;
+      const int64_t row = static_cast<int64_t>(row0) + lane;
       const bool row_ok = row < p.M;
       // independent loads first, their latency overlaps the wait for the accumulator
       const float sa = row_ok ? __ldg(p.s_a + row) : 0.0f;
@@ -382,7 +437,6 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       if (!ok) break;
       tc_fence_after();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + buf * (TCOLS / 2);
-      const int row0 = m_blk * BM + qd * 32;  // first token of this warp's slabs
       int32_t* arow = (p.dbg_acc != nullptr && row_ok) ? p.dbg_acc + row * p.dbg_ldacc + n0 : nullptr;
       for (int c = 2 * slab0; c < 2 * slab1; ++c) {  // 32-column chunks of this warp
         uint32_t r[32];
@@ -390,7 +444,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         tmem_ld_wait();
         if (c + 1 == 2 * slab1) {  // this warp's last accumulators are in registers
           tc_fence_before();
-          mbar_arrive(&acc_empty[buf]);
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(acc_empty_addr[buf]);
         }
         const int lc = (c - 2 * slab0) * 32;  // column inside this warp's staged scales
         epilogue_chunk<SHIFT>(r, sa, reinterpret_cast<const float4*>(ts + lc),
@@ -418,14 +473,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const int ut = threadIdx.x - kUnpackWarp0 * 32;
       Ring st, ps;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_stride) {
         for (int kb = 0; kb < KB; ++kb) {
           ok = mbar_wait(&pfull[ps.s], ps.ph, abort_flag) &&
                mbar_wait(&empty[st.s], st.ph ^ 1u, abort_flag);
           ok = __all_sync(0xFFFFFFFFu, ok);
           if (!ok) break;
-          if constexpr (BITS == 4) unpack4_tile<BN, PERM>(sP + ps.s * P_BYTES, sB + st.s * B_BYTES, ut);
-          else unpack3_tile<BN>(sP + ps.s * P_BYTES, sB + st.s * B_BYTES, ut);
+          if constexpr (BITS == 4) unpack4_tile<BNL, PERM>(sP + ps.s * P_BYTES, sB + st.s * B_BYTES, ut);
+          else unpack3_tile<BNL>(sP + ps.s * P_BYTES, sB + st.s * B_BYTES, ut);
           fence_proxy_async_smem();
           mbar_arrive(&bready[st.s]);
           mbar_arrive(&pempty[ps.s]);
@@ -439,19 +494,21 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   // ---- teardown ----
   tc_fence_before();
   __syncthreads();
+  if constexpr (CG == 2) cluster_sync();  // neither CTA frees tensor memory or exits while the other may still touch it
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, TCOLS);
+    if constexpr (CG == 2) tmem_dealloc_pair(tmem_base, TCOLS);
+    else tmem_dealloc(tmem_base, TCOLS);
   }
   if (threadIdx.x == 0 && *abort_flag && p.status != nullptr) atomicExch(p.status, DP_ERR_TIMEOUT);
 }
 
 // ---- host side -------------------------------------------------------------------------------------
-template <int BN, int BITS>
+template <int BN, int BITS, int CG>
 constexpr size_t gemm_smem_bytes() {
-  return 1024 + static_cast<size_t>(num_stages(BN, BITS)) * ab_stage_bytes(BN) +
-         kPStages * p_stage_bytes(BN, BITS) + kEpiWarps * kYStageBytes +
-         (3 * 8 + 2 * kPStages + 4) * 8 + 32 + 2 * kEpiWarps * 64 * ((BN / 64 + 1) / 2) * 4 + 64;
+  return 1024 + static_cast<size_t>(num_stages(BN / CG, BITS)) * ab_stage_bytes(BN / CG) +
+         kPStages * p_stage_bytes(BN / CG, BITS) + kEpiWarps * kYStageBytes +
+         (4 * 8 + 2 * kPStages + 4) * 8 + 32 + 2 * kEpiWarps * 64 * ((BN / 64 + 1) / 2) * 4 + 64;
 }
 
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -460,11 +517,12 @@ using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, voi
                               CUtensorMapFloatOOBfill);
 static EncodeFn g_encode = nullptr;
 static int g_num_sms = 0;
+static int g_max_pairs = 0;  // CTA pairs of the widest pair kernel that can be resident at once
 
-template <int BN, int BITS, bool PERM>
+template <int BN, int BITS, bool PERM, int CG>
 static cudaError_t set_attr() {
-  return cudaFuncSetAttribute(gemm_i8_kernel<BN, BITS, PERM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              static_cast<int>(gemm_smem_bytes<BN, BITS>()));
+  return cudaFuncSetAttribute(gemm_i8_kernel<BN, BITS, PERM, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              static_cast<int>(gemm_smem_bytes<BN, BITS, CG>()));
 }
 
 int num_sms() { return g_num_sms; }
@@ -483,26 +541,44 @@ int gemm_init() {
   int dev = 0;
   DP_CUDA_OK(cudaGetDevice(&dev));
   DP_CUDA_OK(cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev));
-#define DP_SET(BN)                               \
-  DP_CUDA_OK((set_attr<BN, 8, false>()));        \
-  DP_CUDA_OK((set_attr<BN, 4, false>()));        \
-  DP_CUDA_OK((set_attr<BN, 4, true>()));         \
-  DP_CUDA_OK((set_attr<BN, 3, false>()));
-  DP_SET(64) DP_SET(128) DP_SET(192) DP_SET(256)
+#define DP_SET(BN, CG)                               \
+  DP_CUDA_OK((set_attr<BN, 8, false, CG>()));        \
+  DP_CUDA_OK((set_attr<BN, 4, false, CG>()));        \
+  DP_CUDA_OK((set_attr<BN, 4, true, CG>()));         \
+  DP_CUDA_OK((set_attr<BN, 3, false, CG>()));
+  DP_SET(64, 1) DP_SET(128, 1) DP_SET(192, 1) DP_SET(256, 1)
+  DP_SET(128, 2) DP_SET(192, 2) DP_SET(256, 2)
 #undef DP_SET
+  {  // how many CTA pairs fit on the device at once (one CTA per SM)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(g_num_sms & ~1));
+    cfg.blockDim = dim3(gemm_threads(4));
+    cfg.dynamicSmemBytes = gemm_smem_bytes<256, 4, 2>();
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    e = cudaOccupancyMaxActiveClusters(&n, gemm_i8_kernel<256, 4, true, 2>, &cfg);
+    if (e != cudaSuccess) return fail(DP_ERR_CUDA, "cudaOccupancyMaxActiveClusters: %s", cudaGetErrorString(e));
+    g_max_pairs = n;
+  }
   state = DP_OK;
   return state;
 }
 
+int gemm_max_pairs() { return g_max_pairs; }
+
 static int encode_2d(CUtensorMap* out, const void* base, uint64_t inner_bytes, uint64_t rows,
-                     uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows, bool swizzle128,
-                     int elem_bytes = 1) {
-  const cuuint64_t dims[2] = {inner_bytes / elem_bytes, rows};
+                     uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows, bool swizzle128) {
+  const cuuint64_t dims[2] = {inner_bytes, rows};
   const cuuint64_t strides[1] = {pitch_bytes};
-  const cuuint32_t box[2] = {box_inner / elem_bytes, box_rows};
+  const cuuint32_t box[2] = {box_inner, box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  CUresult r = g_encode(out, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8,
-                        2, const_cast<void*>(base), dims, strides,
+  CUresult r = g_encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides,
                         box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                         swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -514,59 +590,67 @@ int gemm_encode_a(CUtensorMap* out, const int8_t* q, int64_t M, int64_t K, int64
   return encode_2d(out, q, K, M, ldq, BK, BM, true);
 }
 
+// The box of the weight descriptor is what ONE CTA fetches per k-block: bn / cg rows.
 int gemm_encode_w(CUtensorMap* out, const void* qweight, int32_t N, int32_t K, int32_t bits,
-                  int32_t bn) {
+                  int32_t bn, int32_t cg) {
   const uint64_t row_bytes = static_cast<uint64_t>(K) * bits / 8;
-  return encode_2d(out, qweight, row_bytes, N, row_bytes, BK * bits / 8, bn, bits == 8);
+  return encode_2d(out, qweight, row_bytes, N, row_bytes, BK * bits / 8, bn / cg, bits == 8);
 }
 
-// Tile width: the widest of {256, 192, 128, 64} dividing N whose tile count keeps the last wave
-// reasonably full; small problems take narrower tiles to spread over the SMs.
-int gemm_pick_bn(int64_t M, int32_t N, int32_t K, int32_t bits) {
+// Tile shape: width from {256, 192, 128, 64} dividing N, rows 128 (one CTA) or 256 (a CTA pair),
+// by a small time model: waves of tiles over the SMs (or pairs) times the tile's mainloop time plus
+// a fixed per-tile cost; pairs move half the weight bytes per MAC and are preferred on ties.
+void gemm_pick_tile(int64_t M, int32_t N, int32_t K, int32_t bits, uint32_t allow, int* bn_out, int* cg_out) {
   (void)K;
   (void)bits;
-  const int64_t m_tiles = (M + BM - 1) / BM;
   const int sms = g_num_sms > 0 ? g_num_sms : 148;
+  const int pairs = g_max_pairs > 0 ? g_max_pairs : sms / 2;
   const int cand[4] = {256, 192, 128, 64};
-  int best = 0;
+  int best_bn = 0, best_cg = 1;
   double best_cost = 1e30;
-  for (int i = 0; i < 4; ++i) {
-    const int bn = cand[i];
-    if (N % bn) continue;
-    const int64_t tiles = m_tiles * (N / bn);
-    const int64_t waves = (tiles + sms - 1) / sms;
-    // time model: waves * (tile MMA time + fixed per-tile overhead), MMA time ~ bn
-    const double cost = static_cast<double>(waves) * (bn + 24.0);
-    if (cost < best_cost) {
-      best_cost = cost;
-      best = bn;
+  for (int cg = 2; cg >= 1; --cg) {
+    if (!(allow & (1u << cg))) continue;
+    for (int i = 0; i < 4; ++i) {
+      const int bn = cand[i];
+      if (N % bn || (cg == 2 && bn < 128)) continue;
+      const int64_t tiles = ((M + BM * cg - 1) / (BM * cg)) * (N / bn);
+      const int64_t slots = cg == 2 ? pairs : sms;
+      const int64_t waves = (tiles + slots - 1) / slots;
+      const double cost = static_cast<double>(waves) * (bn + 24.0) * (cg == 2 ? 0.98 : 1.0);
+      if (cost < best_cost) {
+        best_cost = cost;
+        best_bn = bn;
+        best_cg = cg;
+      }
     }
   }
-  return best;
+  *bn_out = best_bn;
+  *cg_out = best_cg;
 }
 
-template <int BN>
+template <int BN, int CG>
 static cudaError_t launch_bn(const GemmProblem& g, const GemmParams& p, dim3 grid, cudaStream_t stream,
                              bool pdl) {
   const dim3 block(gemm_threads(g.bits));
   switch (g.bits) {
     case 8:
-      return launch(gemm_i8_kernel<BN, 8, false>, grid, block, gemm_smem_bytes<BN, 8>(), stream, pdl,
-                    g.tmap_a, g.tmap_w, p);
+      return launch_cluster(gemm_i8_kernel<BN, 8, false, CG>, grid, block, gemm_smem_bytes<BN, 8, CG>(), stream,
+                            pdl, CG, g.tmap_a, g.tmap_w, p);
     case 4:
       if (g.korder == KORDER_EVEN_ODD)
-        return launch(gemm_i8_kernel<BN, 4, true>, grid, block, gemm_smem_bytes<BN, 4>(), stream, pdl,
-                      g.tmap_a, g.tmap_w, p);
-      return launch(gemm_i8_kernel<BN, 4, false>, grid, block, gemm_smem_bytes<BN, 4>(), stream, pdl,
-                    g.tmap_a, g.tmap_w, p);
+        return launch_cluster(gemm_i8_kernel<BN, 4, true, CG>, grid, block, gemm_smem_bytes<BN, 4, CG>(), stream,
+                              pdl, CG, g.tmap_a, g.tmap_w, p);
+      return launch_cluster(gemm_i8_kernel<BN, 4, false, CG>, grid, block, gemm_smem_bytes<BN, 4, CG>(), stream,
+                            pdl, CG, g.tmap_a, g.tmap_w, p);
     default:
-      return launch(gemm_i8_kernel<BN, 3, false>, grid, block, gemm_smem_bytes<BN, 3>(), stream, pdl,
-                    g.tmap_a, g.tmap_w, p);
+      return launch_cluster(gemm_i8_kernel<BN, 3, false, CG>, grid, block, gemm_smem_bytes<BN, 3, CG>(), stream,
+                            pdl, CG, g.tmap_a, g.tmap_w, p);
   }
 }
 
 int launch_gemm(const GemmProblem& g, cudaStream_t stream, bool pdl) {
   if (g.M == 0) return DP_OK;
+  const int cg = g.cg == 2 ? 2 : 1;
   GemmParams p;
   p.s_a = g.s_a;
   p.s_w = g.s_w;
@@ -578,19 +662,29 @@ int launch_gemm(const GemmProblem& g, cudaStream_t stream, bool pdl) {
   p.M = g.M;
   p.N = g.N;
   p.K = g.K;
-  p.m_tiles = static_cast<int32_t>((g.M + BM - 1) / BM);
+  p.m_tiles = static_cast<int32_t>((g.M + BM * cg - 1) / (BM * cg));
   p.n_tiles = g.N / g.bn;
   p.early_w = (pdl && g.early_w) ? 1 : 0;
   p.status = g.status;
   const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
-  const dim3 grid(static_cast<unsigned>(tiles < g_num_sms ? tiles : g_num_sms));
+  const int64_t slots = cg == 2 ? (g_max_pairs > 0 ? g_max_pairs : g_num_sms / 2) : g_num_sms;
+  const dim3 grid(static_cast<unsigned>((tiles < slots ? tiles : slots) * cg));
   cudaError_t e;
-  switch (g.bn) {
-    case 64: e = launch_bn<64>(g, p, grid, stream, pdl); break;
-    case 128: e = launch_bn<128>(g, p, grid, stream, pdl); break;
-    case 192: e = launch_bn<192>(g, p, grid, stream, pdl); break;
-    case 256: e = launch_bn<256>(g, p, grid, stream, pdl); break;
-    default: return fail(DP_ERR_INVALID_ARG, "unsupported tile width %d", g.bn);
+  if (cg == 2) {
+    switch (g.bn) {
+      case 128: e = launch_bn<128, 2>(g, p, grid, stream, pdl); break;
+      case 192: e = launch_bn<192, 2>(g, p, grid, stream, pdl); break;
+      case 256: e = launch_bn<256, 2>(g, p, grid, stream, pdl); break;
+      default: return fail(DP_ERR_INVALID_ARG, "unsupported pair tile width %d", g.bn);
+    }
+  } else {
+    switch (g.bn) {
+      case 64: e = launch_bn<64, 1>(g, p, grid, stream, pdl); break;
+      case 128: e = launch_bn<128, 1>(g, p, grid, stream, pdl); break;
+      case 192: e = launch_bn<192, 1>(g, p, grid, stream, pdl); break;
+      case 256: e = launch_bn<256, 1>(g, p, grid, stream, pdl); break;
+      default: return fail(DP_ERR_INVALID_ARG, "unsupported tile width %d", g.bn);
+    }
   }
   if (e != cudaSuccess) return fail(DP_ERR_CUDA, "GEMM launch failed: %s", cudaGetErrorString(e));
   return DP_OK;

@@ -71,6 +71,30 @@ def test_mma_every_tile_width(bits, bn):
     _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | B.DP_FLAG_TILE_N(bn)), x, w, s_w, b, bits)
 
 
+@pytest.mark.parametrize("bits", [8, 4, 3])
+@pytest.mark.parametrize("bn", [128, 192, 256])
+def test_mma_cta_pair_tiles(bits, bn):
+    """The variant in which the two CTAs of a cluster share a 256-row tile (each holding half of
+    the weight rows): ragged M (the second CTA's rows partly / wholly past M), two column tiles."""
+    for M in (200, 100):
+        K, N = 384, 2 * bn
+        x, w, s_w, b = _case(M, K, N, bits, full_range=True)
+        L = DevLayer(w, s_w, b, bits)
+        _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | B.DP_FLAG_CTA_PAIR | B.DP_FLAG_TILE_N(bn)),
+               x, w, s_w, b, bits)
+
+
+def test_mma_cta_pair_many_tiles():
+    """More pair tiles than CTA pairs on the device: persistent loop, both accumulator buffers, ring
+    wrap-around and the cross-CTA barriers over several rounds (M = 2100 -> 9 row tiles x 18)."""
+    M, K, N = 2100, 256, 2304
+    for bits in (8, 4, 3):
+        x, w, s_w, b = _case(M, K, N, bits)
+        L = DevLayer(w, s_w, b, bits)
+        _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | B.DP_FLAG_CTA_PAIR | B.DP_FLAG_TILE_N(128)),
+               x, w, s_w, b, bits)
+
+
 def test_mma_many_tiles_per_cta():
     """More tiles than SMs, so the persistent loop, both accumulator buffers and the stage ring
     wrap-around are exercised (M = 1300 -> 11 row tiles x 18 column tiles of 64)."""
