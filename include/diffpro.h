@@ -93,6 +93,10 @@ typedef struct dp_debug {
  * thread-block cluster share a 256-row tile (tile width 128, 192 or 256 only). */
 #define DP_FLAG_CTA_PAIR 0x800u
 #define DP_FLAG_NO_CTA_PAIR 0x1000u
+/* Tuning/testing: force (or forbid) the weight-stationary CTA-pair kernel, which keeps a strip of
+ * output channels resident in shared memory for the whole K (K <= 1152, N a multiple of 192). */
+#define DP_FLAG_WEIGHT_STATIONARY 0x2000u
+#define DP_FLAG_NO_WEIGHT_STATIONARY 0x4000u
 
 /* flags for dp_plan_run */
 #define DP_PLAN_SAME_X 1u       /* x_ptrs has n_layers entries reused by every step              */

@@ -47,15 +47,28 @@ int check_device() {
 }
 
 static size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
+// Bytes of the int8 activation scratch: whole 128-token tiles.
+static size_t scratch_q_bytes(int64_t M, int32_t K) { return static_cast<size_t>((M + 127) / 128 * 128) * K; }
 
 constexpr uint32_t kLinearFlags =
     DP_FLAG_FORCE_SIMT | DP_FLAG_FORCE_MMA | DP_FLAG_NO_PDL | DP_FLAG_TILE_N_MASK | DP_FLAG_CTA_PAIR |
-    DP_FLAG_NO_CTA_PAIR;
+    DP_FLAG_NO_CTA_PAIR | DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_NO_WEIGHT_STATIONARY;
+constexpr int64_t kWsMinRows = 4096;  // from here on a resident weight strip is reused often enough to pay
 static int forced_bn(uint32_t flags) { return static_cast<int>((flags & DP_FLAG_TILE_N_MASK) >> 8) * 64; }
 
 // Tile width and CTA-group size of the tensor-core kernel for this problem, honouring the tuning
 // flags (validated by check_tile_flags).
-static void choose_tile(uint32_t flags, int64_t M, int32_t N, int32_t K, int32_t bits, int* bn, int* cg) {
+static void choose_tile(uint32_t flags, int64_t M, int32_t N, int32_t K, int32_t bits, int* bn, int* cg,
+                        int* ws) {
+  *ws = 0;
+  const bool ws_ok = gemm_ws_supported(N, K) && !(flags & (DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_NO_CTA_PAIR));
+  if (ws_ok && ((flags & DP_FLAG_WEIGHT_STATIONARY) || M >= kWsMinRows)) {
+    const int fb = forced_bn(flags);
+    *bn = ((fb == 192 || fb == 256) && N % fb == 0) ? fb : gemm_ws_pick_bn(N);
+    *cg = 2;
+    *ws = 1;
+    return;
+  }
   uint32_t allow = 0x6;
   if (flags & DP_FLAG_CTA_PAIR) allow = 0x4;
   if (flags & DP_FLAG_NO_CTA_PAIR) allow = 0x2;
@@ -75,6 +88,8 @@ static int check_tile_flags(uint32_t flags, int32_t N) {
     return fail(DP_ERR_INVALID_ARG, "CTA_PAIR and NO_CTA_PAIR are exclusive");
   if ((flags & DP_FLAG_CTA_PAIR) && ((fb != 0 && fb < 128) || N % 128))
     return fail(DP_ERR_SHAPE, "CTA-pair tiles need a tile width of 128, 192 or 256 dividing N=%d", N);
+  if ((flags & DP_FLAG_WEIGHT_STATIONARY) && (flags & (DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_NO_CTA_PAIR)))
+    return fail(DP_ERR_INVALID_ARG, "WEIGHT_STATIONARY contradicts another flag");
   return DP_OK;
 }
 
@@ -108,7 +123,7 @@ static int check_weight(const dp_weight* w) {
 // while it drains.
 static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_a_in, int64_t M,
                       void* y, int64_t ldy, void* workspace, const dp_debug* dbg, int32_t* status,
-                      uint32_t flags, cudaStream_t stream, const CUtensorMap* tmap_w, int bn, int cg,
+                      uint32_t flags, cudaStream_t stream, const CUtensorMap* tmap_w, int bn, int cg, int ws,
                       const CUtensorMap* tmap_a_cached, bool chained) {
   const bool pdl = !(flags & DP_FLAG_NO_PDL);
   if (use_simt(M, w->N, w->K, flags)) {
@@ -139,11 +154,12 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
   const float* s_a;
   int64_t ldq;
   int korder = KORDER_NATURAL;
+  const bool tiled = s_a_in == nullptr;  // the library's own scratch: stored as contiguous 128 x 128 tiles
   if (s_a_in == nullptr) {
     int8_t* wq = static_cast<int8_t*>(workspace);
-    float* wsa = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align256(static_cast<size_t>(M) * w->K));
+    float* wsa = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align256(scratch_q_bytes(M, w->K)));
     korder = gemm_korder(w->bits);
-    int st = launch_daq(x, M, w->K, ldx, wq, w->K, wsa, nullptr, korder, stream, pdl);
+    int st = launch_daq(x, M, w->K, ldx, wq, w->K, wsa, nullptr, korder, true, stream, pdl);
     if (st != DP_OK) return st;
     q = wq;
     s_a = wsa;
@@ -155,15 +171,17 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
   }
   GemmProblem g;
   g.korder = korder;
+  g.a_tiled = tiled ? 1 : 0;
   g.early_w = (s_a_in == nullptr) ? 1 : 0;
   if (tmap_a_cached != nullptr) {
     g.tmap_a = *tmap_a_cached;
   } else {
-    int st = gemm_encode_a(&g.tmap_a, q, M, w->K, ldq);
+    int st = tiled ? gemm_encode_a_tiled(&g.tmap_a, q, M, w->K) : gemm_encode_a(&g.tmap_a, q, M, w->K, ldq);
     if (st != DP_OK) return st;
   }
-  if (bn == 0) choose_tile(flags, M, w->N, w->K, w->bits, &bn, &cg);
+  if (bn == 0) choose_tile(flags, M, w->N, w->K, w->bits, &bn, &cg, &ws);
   g.cg = cg;
+  g.ws = ws;
   if (tmap_w != nullptr) {
     g.tmap_w = *tmap_w;
   } else {
@@ -183,13 +201,13 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
   g.bits = w->bits;
   g.bn = bn;
   g.status = status;
-  int st = launch_gemm(g, stream, pdl);
+  int st = ws ? launch_gemm_ws(g, stream, pdl) : launch_gemm(g, stream, pdl);
   if (st != DP_OK) return st;
   if (dbg != nullptr) {
     if (dbg->q != nullptr) {
-      if (korder != KORDER_NATURAL) {  // the scratch holds a permuted copy: quantize again, in order
+      if (tiled || korder != KORDER_NATURAL) {  // the scratch holds a tiled / permuted copy: quantize again
         st = launch_daq(x, M, w->K, ldx, dbg->q, dbg->ldq, const_cast<float*>(s_a), nullptr, KORDER_NATURAL,
-                        stream, false);
+                        false, stream, false);
         if (st != DP_OK) return st;
       } else {
         DP_CUDA_OK(cudaMemcpy2DAsync(dbg->q, dbg->ldq, q, ldq, w->K, M, cudaMemcpyDeviceToDevice, stream));
@@ -241,7 +259,7 @@ extern "C" size_t dp_wq_linear_workspace(int64_t M, int32_t N, int32_t K, int32_
   (void)bits;
   if (M <= 0 || K <= 0) return 256;
   if (use_simt(M, N, K, flags)) return 256;
-  return align256(static_cast<size_t>(M) * K) + align256(sizeof(float) * static_cast<size_t>(M));
+  return align256(scratch_q_bytes(M, K)) + align256(sizeof(float) * static_cast<size_t>(M));
 }
 
 extern "C" int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_a_in,
@@ -253,7 +271,7 @@ extern "C" int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, cons
   st = check_device();
   if (st != DP_OK) return st;
   return run_linear(w, x, ldx, s_a_in, M, y_bf16, ldy, workspace, dbg, device_status, flags,
-                    static_cast<cudaStream_t>(stream), nullptr, 0, 0, nullptr, false);
+                    static_cast<cudaStream_t>(stream), nullptr, 0, 0, 0, nullptr, false);
 }
 
 // ---- the linear for callers that cannot allocate ---------------------------------------------------
@@ -299,7 +317,7 @@ extern "C" int dp_wq_linear_static(const dp_weight* w, const void* x_bf16, int64
   st = check_linear_args(w, x_bf16, ldx, nullptr, M, y_bf16, ldy, scratch, DP_STATIC_SCRATCH_BYTES, nullptr, flags);
   if (st != DP_OK || M == 0) return st;
   return run_linear(w, x_bf16, ldx, nullptr, M, y_bf16, ldy, scratch, nullptr, device_status, flags,
-                    static_cast<cudaStream_t>(stream), nullptr, 0, 0, nullptr, false);
+                    static_cast<cudaStream_t>(stream), nullptr, 0, 0, 0, nullptr, false);
 }
 
 // ---- plans ---------------------------------------------------------------------------------------
@@ -307,7 +325,7 @@ struct PlanLayer {
   dp_weight w;
   int64_t M;
   bool simt;
-  int bn, cg;
+  int bn, cg, ws;
   CUtensorMap tmap_w;
   size_t x_offset;  // byte offset of this layer's input inside one staged step (host-input path)
 };
@@ -355,6 +373,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
     L.simt = use_simt(L.M, L.w.N, L.w.K, flags);
     L.bn = 0;
     L.cg = 1;
+    L.ws = 0;
     memset(&L.tmap_w, 0, sizeof(L.tmap_w));
     if (L.simt && static_cast<size_t>(L.w.K) > simt_max_k()) {
       delete p;
@@ -363,7 +382,8 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
     if (!L.simt && L.M > 0) {
       uint32_t lf = flags;  // a pair request that this layer's N cannot honour falls back to the default
       if ((lf & DP_FLAG_CTA_PAIR) && L.w.N % 128) lf &= ~DP_FLAG_CTA_PAIR;
-      choose_tile(lf, L.M, L.w.N, L.w.K, L.w.bits, &L.bn, &L.cg);
+      if ((lf & DP_FLAG_WEIGHT_STATIONARY) && !gemm_ws_supported(L.w.N, L.w.K)) lf &= ~DP_FLAG_WEIGHT_STATIONARY;
+      choose_tile(lf, L.M, L.w.N, L.w.K, L.w.bits, &L.bn, &L.cg, &L.ws);
       st = gemm_encode_w(&L.tmap_w, L.w.qweight, L.w.N, L.w.K, L.w.bits, L.bn, L.cg);
       if (st != DP_OK) {
         delete p;
@@ -411,7 +431,7 @@ static const CUtensorMap* cached_tmap_a(dp_plan* plan, const void* ws, int64_t M
   c.ptr = ws;
   c.M = M;
   c.K = K;
-  *st = gemm_encode_a(&c.map, static_cast<const int8_t*>(ws), M, K, K);
+  *st = gemm_encode_a_tiled(&c.map, static_cast<const int8_t*>(ws), M, K);
   if (*st != DP_OK) return nullptr;
   if (plan->a_cache.size() > 64) plan->a_cache.clear();
   plan->a_cache.push_back(c);
@@ -433,7 +453,7 @@ static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, 
       if (st != DP_OK) return st;
     }
     int st = run_linear(&L.w, xs[l], L.w.K, nullptr, L.M, ys[l], L.w.N, workspace, nullptr, status,
-                        plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, L.cg, ta, *chained);
+                        plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, L.cg, L.ws, ta, *chained);
     if (st != DP_OK) return st;
     *chained = true;
   }

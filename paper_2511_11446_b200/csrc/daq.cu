@@ -70,6 +70,23 @@ __device__ __forceinline__ int warp_sum_i32(int s) {
   return s;
 }
 
+// Where the 8 codes of vector `idx` (k = 8 idx ..) of one token go. Row-major: q[row][k]. Tiled
+// (tiled_kb = K / 128 > 0): the matrix is cut into 128-token x 128-code tiles of 16 KB, stored one
+// after the other ([row tile][k block][128][128]), so that the GEMM's TMA loads of an activation tile
+// read one contiguous 16 KB range instead of 128 rows a whole row pitch apart.
+struct QRow {
+  uint2* base;
+  int tiled;
+  __device__ __forceinline__ QRow(int8_t* q, int64_t row, int64_t ldq, int tiled_kb) : tiled(tiled_kb) {
+    base = tiled_kb ? reinterpret_cast<uint2*>(q + ((row >> 7) * tiled_kb) * 16384 + (row & 127) * 128)
+                    : reinterpret_cast<uint2*>(q + row * ldq);
+  }
+  __device__ __forceinline__ void store(int idx, uint2 v) const {
+    if (tiled) base[(idx >> 4) * 2048 + (idx & 15)] = v;  // next k block: + 16384 bytes
+    else base[idx] = v;
+  }
+};
+
 constexpr int kDaqWarps = 8;
 
 // MAXV = 16-byte vectors held per lane (row of up to 256*MAXV elements in registers).
@@ -77,7 +94,7 @@ template <int MAXV, bool EO>
 __global__ void __launch_bounds__(kDaqWarps * 32)
 daq_rows_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t ldx,
                 int8_t* __restrict__ q, int64_t ldq, float* __restrict__ s_a,
-                int32_t* __restrict__ rowsum) {
+                int32_t* __restrict__ rowsum, int tiled_kb) {
   pdl_launch_dependents();
   const int64_t row = static_cast<int64_t>(blockIdx.x) * kDaqWarps + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -103,14 +120,14 @@ daq_rows_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t ldx,
   m = warp_max_u32(max(m & 0xFFFFu, m >> 16));
   float sc, inv;
   token_scale(m, sc, inv);
-  uint2* qr = reinterpret_cast<uint2*>(q + row * ldq);
+  const QRow qr(q, row, ldq, tiled_kb);
   int sum = 0;
 #pragma unroll
   for (int i = 0; i < MAXV; ++i) {
     const int idx = lane + 32 * i;
     if (idx < nvec) {
       uint2 o = quant_vec<EO>(v[i], inv);
-      qr[idx] = o;
+      qr.store(idx, o);
       sum = __dp4a(static_cast<int>(o.x), 0x01010101, sum);
       sum = __dp4a(static_cast<int>(o.y), 0x01010101, sum);
     }
@@ -127,7 +144,7 @@ template <bool EO>
 __global__ void __launch_bounds__(kDaqWarps * 32)
 daq_rows_2pass_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t ldx,
                       int8_t* __restrict__ q, int64_t ldq, float* __restrict__ s_a,
-                      int32_t* __restrict__ rowsum) {
+                      int32_t* __restrict__ rowsum, int tiled_kb) {
   pdl_launch_dependents();
   const int64_t row = static_cast<int64_t>(blockIdx.x) * kDaqWarps + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -143,11 +160,11 @@ daq_rows_2pass_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t 
   m = warp_max_u32(max(m & 0xFFFFu, m >> 16));
   float sc, inv;
   token_scale(m, sc, inv);
-  uint2* qr = reinterpret_cast<uint2*>(q + row * ldq);
+  const QRow qr(q, row, ldq, tiled_kb);
   int sum = 0;
   for (int idx = lane; idx < nvec; idx += 32) {
     uint2 o = quant_vec<EO>(xr[idx], inv);
-    qr[idx] = o;
+    qr.store(idx, o);
     sum = __dp4a(static_cast<int>(o.x), 0x01010101, sum);
     sum = __dp4a(static_cast<int>(o.y), 0x01010101, sum);
   }
@@ -160,26 +177,27 @@ daq_rows_2pass_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t 
 
 template <bool EO>
 static cudaError_t launch_daq_t(const uint16_t* xp, int64_t M, int k, int64_t ldx, int8_t* q, int64_t ldq,
-                                float* s_a, int32_t* rowsum, cudaStream_t stream, bool pdl) {
+                                float* s_a, int32_t* rowsum, int tiled_kb, cudaStream_t stream, bool pdl) {
   const dim3 grid(static_cast<unsigned>((M + kDaqWarps - 1) / kDaqWarps));
   const dim3 block(kDaqWarps * 32);
   if (k <= 256 * 5)
-    return launch(daq_rows_kernel<5, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum);
+    return launch(daq_rows_kernel<5, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb);
   if (k <= 256 * 9)
-    return launch(daq_rows_kernel<9, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum);
+    return launch(daq_rows_kernel<9, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb);
   if (k <= 256 * 18)
-    return launch(daq_rows_kernel<18, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum);
-  return launch(daq_rows_2pass_kernel<EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum);
+    return launch(daq_rows_kernel<18, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb);
+  return launch(daq_rows_2pass_kernel<EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb);
 }
 
 int launch_daq(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq,
-               float* s_a, int32_t* rowsum, int korder, cudaStream_t stream, bool pdl) {
+               float* s_a, int32_t* rowsum, int korder, bool tiled, cudaStream_t stream, bool pdl) {
   if (M == 0) return DP_OK;
   const uint16_t* xp = static_cast<const uint16_t*>(x);
   const int k = static_cast<int>(K);
+  const int tiled_kb = tiled ? k / 128 : 0;
   const cudaError_t e = korder == KORDER_EVEN_ODD
-                            ? launch_daq_t<true>(xp, M, k, ldx, q, ldq, s_a, rowsum, stream, pdl)
-                            : launch_daq_t<false>(xp, M, k, ldx, q, ldq, s_a, rowsum, stream, pdl);
+                            ? launch_daq_t<true>(xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb, stream, pdl)
+                            : launch_daq_t<false>(xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb, stream, pdl);
   if (e != cudaSuccess) return fail(DP_ERR_CUDA, "DAQ launch failed: %s", cudaGetErrorString(e));
   return DP_OK;
 }
@@ -200,6 +218,6 @@ extern "C" int dp_daq_quantize(const void* x_bf16, int64_t M, int64_t K, int64_t
     return fail(DP_ERR_ALIGN, "dp_daq_quantize: pointers/pitches must be 16-byte aligned");
   int st = check_device();
   if (st != DP_OK) return st;
-  return launch_daq(x_bf16, M, K, ldx, q, ldq, s_a, rowsum, KORDER_NATURAL,
+  return launch_daq(x_bf16, M, K, ldx, q, ldq, s_a, rowsum, KORDER_NATURAL, false,
                     static_cast<cudaStream_t>(stream), false);
 }

@@ -19,7 +19,7 @@ int gemm_korder(int32_t bits);
 
 // daq.cu
 int launch_daq(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq,
-               float* s_a, int32_t* rowsum, int korder, cudaStream_t stream, bool pdl);
+               float* s_a, int32_t* rowsum, int korder, bool tiled, cudaStream_t stream, bool pdl);
 
 // simt.cu — CUDA-core weight-streaming linear for small M (DAQ fused in the CTA prologue).
 struct SimtArgs {
@@ -60,7 +60,9 @@ struct GemmProblem {
   int64_t M;
   int32_t N, K, bits, bn;
   int32_t cg;       // 1: one CTA per 128-row tile; 2: a CTA pair per 256-row tile
+  int32_t ws;       // weight-stationary pair kernel (cg == 2, bn in {192, 256})
   int32_t korder;   // KOrder of the activations behind tmap_a
+  int32_t a_tiled;  // the activations behind tmap_a are stored as 128 x 128 tiles (see gemm_encode_a_tiled)
   int32_t early_w;  // the preceding kernel on the stream is this call's own DAQ: weights may be
                     // fetched before it has finished
   int32_t* status;
@@ -69,9 +71,16 @@ struct GemmProblem {
 void gemm_pick_tile(int64_t M, int32_t N, int32_t K, int32_t bits, uint32_t allow, int* bn_out, int* cg_out);
 int gemm_max_pairs();
 int gemm_encode_a(CUtensorMap* out, const int8_t* q, int64_t M, int64_t K, int64_t ldq);
+// int8 activations stored as [ceil(M/128)][K/128] tiles of 128 tokens x 128 codes (16 KB each).
+int gemm_encode_a_tiled(CUtensorMap* out, const int8_t* q, int64_t M, int64_t K);
 int gemm_encode_w(CUtensorMap* out, const void* qweight, int32_t N, int32_t K, int32_t bits,
                   int32_t bn, int32_t cg);
 int launch_gemm(const GemmProblem& p, cudaStream_t stream, bool pdl);
+
+// gemm_ws.cu -- weight-stationary CTA-pair kernel (K <= 1152, N a multiple of 192 or 256).
+bool gemm_ws_supported(int32_t N, int32_t K);
+int gemm_ws_pick_bn(int32_t N);
+int launch_gemm_ws(const GemmProblem& p, cudaStream_t stream, bool pdl);
 int gemm_init();  // sets kernel attributes, resolves the tensor-map encoder; idempotent
 
 int num_sms();

@@ -29,164 +29,9 @@
 // byte: two logic ops per word instead of a sign-extension); the accumulator is then an exact
 // multiple of 2^(8-b) (|acc| <= 4608*127*128 < 2^31) and the epilogue multiplies by 2^-(8-b),
 // which is exact in fp32, before the scale.
-#include <cuda_bf16.h>
-
-#include "dp_common.cuh"
-#include "dp_internal.h"
+#include "gemm_device.cuh"
 
 namespace dp {
-
-constexpr int BM = 128;
-constexpr int BK = 128;  // int8 elements = bytes = one 128-byte swizzle row
-constexpr int kEpiWarp0 = 2, kEpiWarps = 8, kUnpackWarp0 = kEpiWarp0 + kEpiWarps, kUnpackWarps = 8;
-constexpr int kUnpackThreads = kUnpackWarps * 32;
-__host__ __device__ constexpr int gemm_threads(int bits) {
-  return (kUnpackWarp0 + (bits == 8 ? 0 : kUnpackWarps)) * 32;
-}
-constexpr int kYStageBytes = 32 * 64;  // per epilogue warp: 32 tokens x 32 bf16
-constexpr int kSmemBudget = 200 * 1024;
-constexpr int kPStages = 3;
-
-// bn below is the number of weight rows ONE CTA holds (BN for CG = 1, BN / 2 for a pair).
-__host__ __device__ constexpr int p_stage_bytes(int bn, int bits) {
-  return bits == 8 ? 0 : bn * (BK * bits / 8);
-}
-__host__ __device__ constexpr int ab_stage_bytes(int bn) { return BM * BK + bn * BK; }
-__host__ __device__ constexpr int num_stages(int bn, int bits) {
-  int n = (kSmemBudget - kPStages * p_stage_bytes(bn, bits)) / ab_stage_bytes(bn);
-  return n > 8 ? 8 : n;
-}
-__host__ __device__ constexpr int tmem_cols(int bn) { return bn <= 64 ? 128 : bn <= 128 ? 256 : 512; }
-
-struct GemmParams {
-  const float* s_a;
-  const float* s_w;
-  const uint16_t* bias;
-  uint16_t* y;
-  int64_t ldy;
-  int32_t* dbg_acc;
-  int64_t dbg_ldacc;
-  int64_t M;
-  int32_t N, K;
-  int32_t m_tiles, n_tiles;  // m_tiles counts row tiles of 128 * CG tokens
-  int32_t early_w;  // weights may be fetched before the preceding kernel on the stream has finished
-  int32_t* status;
-};
-
-struct Ring {  // stage index + phase bit of a circular buffer
-  int s = 0;
-  uint32_t ph = 0;
-  __device__ __forceinline__ void next(int n) {
-    if (++s == n) {
-      s = 0;
-      ph ^= 1u;
-    }
-  }
-};
-
-// ---- in-smem weight expansion ------------------------------------------------------------------
-// 4-bit: tile P is [BN][64 bytes]; each thread expands 8 bytes (16 codes) into one 16-byte chunk of
-// the operand tile B = [BN][128 bytes], chunk position XOR-swizzled by (row & 7).
-template <int BN, bool PERM>
-__device__ __forceinline__ void unpack4_tile(const uint8_t* P, uint8_t* B, int tid) {
-#pragma unroll
-  for (int i = 0; i < (BN * 8 + kUnpackThreads - 1) / kUnpackThreads; ++i) {
-    const int idx = tid + i * kUnpackThreads;
-    if (BN * 8 % kUnpackThreads != 0 && idx >= BN * 8) break;
-    const int row = idx >> 3, kc = idx & 7;
-    const uint2 in = *reinterpret_cast<const uint2*>(P + row * 64 + kc * 8);
-    uint4 o;
-    const uint32_t lo0 = ((in.x << 4) & 0xF0F0F0F0u) ^ 0x80808080u;  // even fields
-    const uint32_t hi0 = (in.x & 0xF0F0F0F0u) ^ 0x80808080u;         // odd fields
-    const uint32_t lo1 = ((in.y << 4) & 0xF0F0F0F0u) ^ 0x80808080u;
-    const uint32_t hi1 = (in.y & 0xF0F0F0F0u) ^ 0x80808080u;
-    if constexpr (PERM) {
-      o = make_uint4(lo0, hi0, lo1, hi1);
-    } else {
-      o.x = __byte_perm(lo0, hi0, 0x5140);
-      o.y = __byte_perm(lo0, hi0, 0x7362);
-      o.z = __byte_perm(lo1, hi1, 0x5140);
-      o.w = __byte_perm(lo1, hi1, 0x7362);
-    }
-    *reinterpret_cast<uint4*>(B + row * 128 + ((kc ^ (row & 7)) << 4)) = o;
-  }
-}
-
-// 3-bit: tile P is [BN][48 bytes]; each thread expands 3 words (32 codes) into two 16-byte chunks.
-__device__ __forceinline__ uint32_t spread3(uint32_t v) {  // 4 fields of 3 bits -> top 3 bits of 4 bytes
-  return (((v << 5) & 0x000000E0u) | ((v << 10) & 0x0000E000u) | ((v << 15) & 0x00E00000u) |
-          ((v << 20) & 0xE0000000u)) ^ 0x80808080u;
-}
-template <int BN>
-__device__ __forceinline__ void unpack3_tile(const uint8_t* P, uint8_t* B, int tid) {
-#pragma unroll
-  for (int i = 0; i < (BN * 4 + kUnpackThreads - 1) / kUnpackThreads; ++i) {
-    const int idx = tid + i * kUnpackThreads;
-    if (BN * 4 % kUnpackThreads != 0 && idx >= BN * 4) break;
-    const int row = idx >> 2, g = idx & 3;
-    const uint32_t* src = reinterpret_cast<const uint32_t*>(P + row * 48 + g * 12);
-    const uint32_t s0 = src[0], s1 = src[1], s2 = src[2];
-    uint4 o0, o1;
-    o0.x = spread3(s0);                               // stream bits  0..11
-    o0.y = spread3(s0 >> 12);                         //             12..23
-    o0.z = spread3(__funnelshift_r(s0, s1, 24));      //             24..35
-    o0.w = spread3(s1 >> 4);                          //             36..47
-    o1.x = spread3(s1 >> 16);                         //             48..59
-    o1.y = spread3(__funnelshift_r(s1, s2, 28));      //             60..71
-    o1.z = spread3(s2 >> 8);                          //             72..83
-    o1.w = spread3(s2 >> 20);                         //             84..95
-    uint8_t* brow = B + row * 128;
-    const int sw = row & 7;
-    *reinterpret_cast<uint4*>(brow + (((2 * g) ^ sw) << 4)) = o0;
-    *reinterpret_cast<uint4*>(brow + (((2 * g + 1) ^ sw) << 4)) = o1;
-  }
-}
-
-// ---- epilogue arithmetic -----------------------------------------------------------------------------
-// 32 accumulators of one token -> bf16 into the warp's staging tile [32 tokens][64 bytes], 16-byte
-// chunks XOR-swizzled by ((token >> 1) & 3) so that both the per-token writes and the row-wise
-// read-back are free of bank conflicts. Per element, in this order: t = (float)(acc / 2^SHIFT),
-// sc = s_a * s_w[n], y = fma(t, sc, bias[n]), bf16 round-to-nearest-even.
-template <int SHIFT>
-__device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], float sa,
-                                               const float4* __restrict__ s4,
-                                               const float4* __restrict__ b4,
-                                               uint4* __restrict__ stage_row, int sw,
-                                               int32_t* acc_dst) {
-  // all shared-memory reads and all arithmetic first, the four 16-byte stores last: nothing in the
-  // arithmetic then has to wait behind a store the compiler cannot reorder
-  uint32_t o[16];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const float4 sw4 = s4[j], bb = b4[j];
-    float t0 = __int2float_rn(static_cast<int>(r[4 * j + 0]));
-    float t1 = __int2float_rn(static_cast<int>(r[4 * j + 1]));
-    float t2 = __int2float_rn(static_cast<int>(r[4 * j + 2]));
-    float t3 = __int2float_rn(static_cast<int>(r[4 * j + 3]));
-    if constexpr (SHIFT != 0) {  // exact: the accumulator is a multiple of 2^SHIFT
-      constexpr float kInv = 1.0f / (1 << SHIFT);
-      t0 = __fmul_rn(t0, kInv);
-      t1 = __fmul_rn(t1, kInv);
-      t2 = __fmul_rn(t2, kInv);
-      t3 = __fmul_rn(t3, kInv);
-    }
-    const float y0 = __fmaf_rn(t0, __fmul_rn(sa, sw4.x), bb.x);
-    const float y1 = __fmaf_rn(t1, __fmul_rn(sa, sw4.y), bb.y);
-    const float y2 = __fmaf_rn(t2, __fmul_rn(sa, sw4.z), bb.z);
-    const float y3 = __fmaf_rn(t3, __fmul_rn(sa, sw4.w), bb.w);
-    const __nv_bfloat162 h0 = __floats2bfloat162_rn(y0, y1);
-    const __nv_bfloat162 h1 = __floats2bfloat162_rn(y2, y3);
-    o[2 * j] = *reinterpret_cast<const uint32_t*>(&h0);
-    o[2 * j + 1] = *reinterpret_cast<const uint32_t*>(&h1);
-  }
-#pragma unroll
-  for (int j = 0; j < 4; ++j)
-    stage_row[j ^ sw] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
-  if (acc_dst != nullptr) {
-#pragma unroll
-    for (int j = 0; j < 32; ++j) acc_dst[j] = static_cast<int>(r[j]) >> SHIFT;
-  }
-}
 
 // ---- the kernel ----------------------------------------------------------------------------------
 template <int BN, int BITS, bool PERM, int CG>
@@ -217,12 +62,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint64_t* acc_empty = acc_full + 2;  // CG = 2: the leader's copy collects both CTAs' epilogue warps
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  constexpr int SLABS = BN / 64;            // 64-column slabs per tile
-  constexpr int SLABS_LO = (SLABS + 1) / 2;  // slabs of the first warp of a quadrant; the rest go to the second
-  constexpr int EPI_ACTIVE = SLABS > 1 ? kEpiWarps : kEpiWarps / 2;  // BN = 64: one warp per quadrant
-  float* s_scale = reinterpret_cast<float*>(                 // [warps][64 * SLABS_LO] weight scales
+  using EL = EpiLayout<BN>;
+  float* s_scale = reinterpret_cast<float*>(  // per-warp copies of the tile's weight scales, then biases
       (reinterpret_cast<uintptr_t>(tmem_slot + 4) + 15) & ~uintptr_t(15));
-  float* s_bias = s_scale + kEpiWarps * 64 * SLABS_LO;        // [warps][64 * SLABS_LO]
+  float* s_bias = s_scale + EL::SCALE_FLOATS;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int KB = p.K / BK;
@@ -243,7 +86,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&acc_full[i], 1);
-      mbar_init(&acc_empty[i], CG * EPI_ACTIVE);  // one arrival per epilogue warp
+      mbar_init(&acc_empty[i], CG * EL::ACTIVE);  // one arrival per epilogue warp
     }
     *abort_flag = 0;
     fence_barrier_init();
@@ -287,8 +130,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           if (!a_open && deferred == NS) {  // ring full of weight tiles: now wait for the activations
             pdl_wait();
             a_open = true;
-            for (int d = 0; d < deferred; ++d)
-              tma_load_2d(sA + def_s[d] * A_BYTES, &tmap_a, def_kb[d] * BK, def_m[d], &full_a[def_s[d]]);
+            for (int d = 0; d < deferred; ++d) {
+              int c0, c1;
+              a_tile_coords(p, def_m[d], def_kb[d], c0, c1);
+              tma_load_2d(sA + def_s[d] * A_BYTES, &tmap_a, c0, c1, &full_a[def_s[d]]);
+            }
             deferred = 0;
           }
           if (!(ok = mbar_wait(&empty[st.s], st.ph ^ 1u, abort_flag))) break;
@@ -303,7 +149,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             ps.next(NP);
           }
           if (a_open) {
-            tma_load_2d(sA + st.s * A_BYTES, &tmap_a, kb * BK, m_row, &full_a[st.s]);
+            int c0, c1;
+            a_tile_coords(p, m_row, kb, c0, c1);
+            tma_load_2d(sA + st.s * A_BYTES, &tmap_a, c0, c1, &full_a[st.s]);
           } else {
             def_kb[deferred] = kb;
             def_m[deferred] = m_row;
@@ -315,8 +163,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       }
       if (!a_open) {  // fewer k-blocks than stages in the whole CTA
         pdl_wait();
-        for (int d = 0; d < deferred; ++d)
-          tma_load_2d(sA + def_s[d] * A_BYTES, &tmap_a, def_kb[d] * BK, def_m[d], &full_a[def_s[d]]);
+        for (int d = 0; d < deferred; ++d) {
+          int c0, c1;
+          a_tile_coords(p, def_m[d], def_kb[d], c0, c1);
+          tma_load_2d(sA + def_s[d] * A_BYTES, &tmap_a, c0, c1, &full_a[def_s[d]]);
+        }
       }
       if (!ok) {
         // drain: give copies still in flight a bounded time to land before the CTA exits
@@ -386,86 +237,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
   } else if (warp < kUnpackWarp0) {
     // ================= epilogue =================
-    const int ew = warp - kEpiWarp0;
-    const int qd = warp & 3;                  // TMEM lane quadrant this warp may read
-    const int slab0 = ew < 4 ? 0 : SLABS_LO;  // this warp's slabs: [slab0, slab1)
-    const int slab1 = ew < 4 ? SLABS_LO : SLABS;
-    float* ts = s_scale + ew * 64 * SLABS_LO;  // this warp's private copy: no CTA-wide sync
-    float* tb = s_bias + ew * 64 * SLABS_LO;
-    uint8_t* stage = sY + ew * kYStageBytes;
-    const uint4* stage4 = reinterpret_cast<const uint4*>(stage);
-    uint4* stage_row = reinterpret_cast<uint4*>(stage + lane * 64);
-    uint32_t acc_empty_addr[2];  // where this warp reports a drained accumulator buffer
-#pragma unroll
-    for (int i = 0; i < 2; ++i)
-      acc_empty_addr[i] = CG == 2 ? map_to_cta(&acc_empty[i], 0) : smem_u32(&acc_empty[i]);
-    bool ok = slab0 < slab1;
-    int tcount = 0, staged_n = -1;
-    if (ok && p.early_w) pdl_wait();  // s_a below is written by the preceding kernel
+    EpilogueWarp<BN, SHIFT> epi;
+    epi.init(warp, lane, s_scale, s_bias, sY,
+             CG == 2 ? map_to_cta(&acc_empty[0], 0) : smem_u32(&acc_empty[0]),
+             CG == 2 ? map_to_cta(&acc_empty[1], 0) : smem_u32(&acc_empty[1]));
+    bool ok = epi.active();
+    int tcount = 0;
+    if (ok && p.early_w) pdl_wait();  // s_a is written by the preceding kernel
     for (int tile = first_tile; tile < total_tiles && ok; tile += tile_stride, ++tcount) {
-      const int n_blk = tile % p.n_tiles;  // column tiles of one row strip run together
       const int buf = tcount & 1;
-      const uint32_t aph = (tcount >> 1) & 1;
-      const int n0 = n_blk * BN;
-      const int row0 = (tile / p.n_tiles) * (BM * CG) + static_cast<int>(rank) * BM + qd * 32;
-      const int64_t row = static_cast<int64_t>(row0) + lane;
-      const bool row_ok = row < p.M;
-      // independent loads first, their latency overlaps the wait for the accumulator
-      const float sa = row_ok ? __ldg(p.s_a + row) : 0.0f;
-      if (n_blk != staged_n) {
-        constexpr int NV = 2 * SLABS_LO;  // 32-column groups this warp may need
-        float sv[NV], bv[NV];
-#pragma unroll
-        for (int j = 0; j < NV; ++j) {
-          const int col = slab0 * 64 + lane + 32 * j;
-          sv[j] = col < slab1 * 64 ? __ldg(p.s_w + n0 + col) : 0.0f;
-          bv[j] = (col < slab1 * 64 && p.bias != nullptr)
-                      ? __uint_as_float(static_cast<uint32_t>(__ldg(p.bias + n0 + col)) << 16)
-                      : 0.0f;
-        }
-        __syncwarp();
-#pragma unroll
-        for (int j = 0; j < NV; ++j) {
-          ts[lane + 32 * j] = sv[j];
-          tb[lane + 32 * j] = bv[j];
-        }
-        __syncwarp();
-        staged_n = n_blk;
-      }
-      ok = mbar_wait(&acc_full[buf], aph, abort_flag);
-      ok = __all_sync(0xFFFFFFFFu, ok);
-      if (!ok) break;
-      tc_fence_after();
-      const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + buf * (TCOLS / 2);
-      int32_t* arow = (p.dbg_acc != nullptr && row_ok) ? p.dbg_acc + row * p.dbg_ldacc + n0 : nullptr;
-      for (int c = 2 * slab0; c < 2 * slab1; ++c) {  // 32-column chunks of this warp
-        uint32_t r[32];
-        tmem_ld_32x32(t_addr + c * 32, r);
-        tmem_ld_wait();
-        if (c + 1 == 2 * slab1) {  // this warp's last accumulators are in registers
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(acc_empty_addr[buf]);
-        }
-        const int lc = (c - 2 * slab0) * 32;  // column inside this warp's staged scales
-        epilogue_chunk<SHIFT>(r, sa, reinterpret_cast<const float4*>(ts + lc),
-                              reinterpret_cast<const float4*>(tb + lc), stage_row, (lane >> 1) & 3,
-                              arow ? arow + c * 32 : nullptr);
-        __syncwarp();
-        // staged chunk -> global: every store instruction covers eight 64-byte row segments
-        {
-          const int ch = lane & 3;
-          uint16_t* ycol = p.y + n0 + c * 32 + ch * 8;
-#pragma unroll
-          for (int it = 0; it < 4; ++it) {
-            const int rr = 8 * it + (lane >> 2);
-            const uint4 v = stage4[rr * 4 + (ch ^ ((rr >> 1) & 3))];
-            const int64_t grow = static_cast<int64_t>(row0) + rr;
-            if (grow < p.M) *reinterpret_cast<uint4*>(ycol + grow * p.ldy) = v;
-          }
-        }
-        __syncwarp();  // the staging tile is rewritten by the next chunk
-      }
+      ok = epi.tile(p, tile % p.n_tiles, (tile / p.n_tiles) * (BM * CG) + static_cast<int>(rank) * BM,
+                    tmem_base, buf * (TCOLS / 2), &acc_full[buf], (tcount >> 1) & 1, buf, abort_flag);
     }
   } else {
     // ================= unpack (3/4-bit weights) =================
@@ -589,6 +371,10 @@ static int encode_2d(CUtensorMap* out, const void* base, uint64_t inner_bytes, u
 int gemm_encode_a(CUtensorMap* out, const int8_t* q, int64_t M, int64_t K, int64_t ldq) {
   return encode_2d(out, q, K, M, ldq, BK, BM, true);
 }
+int gemm_encode_a_tiled(CUtensorMap* out, const int8_t* q, int64_t M, int64_t K) {
+  const uint64_t rows = static_cast<uint64_t>((M + BM - 1) / BM) * (K / BK) * BM;
+  return encode_2d(out, q, BK, rows, BK, BK, BM, true);
+}
 
 // The box of the weight descriptor is what ONE CTA fetches per k-block: bn / cg rows.
 int gemm_encode_w(CUtensorMap* out, const void* qweight, int32_t N, int32_t K, int32_t bits,
@@ -664,6 +450,7 @@ int launch_gemm(const GemmProblem& g, cudaStream_t stream, bool pdl) {
   p.K = g.K;
   p.m_tiles = static_cast<int32_t>((g.M + BM * cg - 1) / (BM * cg));
   p.n_tiles = g.N / g.bn;
+  p.a_tiled = g.a_tiled;
   p.early_w = (pdl && g.early_w) ? 1 : 0;
   p.status = g.status;
   const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;

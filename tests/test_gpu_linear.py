@@ -95,6 +95,27 @@ def test_mma_cta_pair_many_tiles():
                x, w, s_w, b, bits)
 
 
+@pytest.mark.parametrize("bits", [8, 4, 3])
+@pytest.mark.parametrize("N,K", [(384, 384), (512, 256), (768, 1152)])
+def test_mma_weight_stationary(bits, N, K):
+    """The CTA-pair kernel that keeps a strip of output channels resident for the whole K and streams
+    only activation tiles: both strip widths (192, 256), short and full K, ragged M."""
+    M = 600
+    x, w, s_w, b = _case(M, K, N, bits, full_range=True)
+    L = DevLayer(w, s_w, b, bits)
+    _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | B.DP_FLAG_WEIGHT_STATIONARY), x, w, s_w, b, bits)
+
+
+def test_mma_weight_stationary_strip_changes():
+    """More work items than CTA pairs, so pairs run several row tiles per strip and some runs cross
+    a strip boundary (the resident strip is replaced while the pipeline is live)."""
+    M, K, N = 2100, 1152, 2304
+    for bits in (8, 4, 3):
+        x, w, s_w, b = _case(M, K, N, bits)
+        L = DevLayer(w, s_w, b, bits)
+        _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | B.DP_FLAG_WEIGHT_STATIONARY), x, w, s_w, b, bits)
+
+
 def test_mma_many_tiles_per_cta():
     """More tiles than SMs, so the persistent loop, both accumulator buffers and the stage ring
     wrap-around are exercised (M = 1300 -> 11 row tiles x 18 column tiles of 64)."""
