@@ -98,6 +98,17 @@ typedef struct dp_debug {
 #define DP_FLAG_WEIGHT_STATIONARY 0x2000u
 #define DP_FLAG_NO_WEIGHT_STATIONARY 0x4000u
 
+/* dp_plan_create only: choose each layer's tensor-core kernel variant (tile width, single CTA /
+ * CTA pair / weight-stationary) by timing the candidates on the device during plan creation
+ * (allocates scratch, launches and synchronises; a few milliseconds per distinct layer shape)
+ * instead of by the built-in cost model. */
+#define DP_FLAG_AUTOTUNE 0x10000u
+/* dp_plan_create only: the caller states that, within one timestep, the inputs of the plan's
+ * small-M layers (M <= 32: in a DiT the adaLN modulation linears, which consume only the
+ * timestep/class embedding) do not depend on any other layer's output. dp_plan_run then runs
+ * those layers first in each step, equal shapes grouped into one launch; results are unchanged. */
+#define DP_FLAG_GROUP_SMALL_M 0x20000u
+
 /* flags for dp_plan_run */
 #define DP_PLAN_SAME_X 1u       /* x_ptrs has n_layers entries reused by every step              */
 #define DP_PLAN_SAME_Y 2u       /* y_ptrs has n_layers entries reused (overwritten) every step   */

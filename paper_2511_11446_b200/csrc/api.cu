@@ -340,9 +340,78 @@ struct dp_plan {
   size_t workspace_bytes;
   size_t x_bytes;
   std::vector<TmapACache> a_cache;
+  std::vector<std::vector<int>> groups;  // small-M layers of equal shape, run first in every step
+  std::vector<char> grouped;             // per layer: member of a group
   cudaStream_t copy_stream;
   cudaEvent_t ev_copied[2], ev_consumed[2];
 };
+
+// Times every kernel variant that can run this layer shape (the whole layer: DAQ + GEMM, as the
+// plan will launch it) and returns the fastest. Plan creation only.
+struct TunedShape {
+  int64_t M;
+  int32_t N, K, bits;
+  int bn, cg, ws;
+};
+static int autotune_shape(const dp_weight& w, int64_t M, uint32_t flags, int* bn_out, int* cg_out, int* ws_out) {
+  struct Cand {
+    int bn, cg, ws;
+  };
+  std::vector<Cand> cands;
+  const int widths[4] = {64, 128, 192, 256};
+  for (int i = 0; i < 4; ++i)
+    if (w.N % widths[i] == 0) {
+      cands.push_back({widths[i], 1, 0});
+      if (widths[i] >= 128) cands.push_back({widths[i], 2, 0});
+      if (widths[i] >= 192 && gemm_ws_supported(w.N, w.K)) cands.push_back({widths[i], 2, 1});
+    }
+  void *x = nullptr, *y = nullptr, *ws = nullptr;
+  cudaStream_t stream = nullptr;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  const size_t xb = static_cast<size_t>(M) * w.K * 2, yb = static_cast<size_t>(M) * w.N * 2;
+  const size_t wb = dp_wq_linear_workspace(M, w.N, w.K, w.bits, 0);
+  cudaError_t e = cudaMalloc(&x, xb);
+  if (e == cudaSuccess) e = cudaMalloc(&y, yb);
+  if (e == cudaSuccess) e = cudaMalloc(&ws, wb);
+  if (e == cudaSuccess) e = cudaMemset(x, 0x3c, xb);  // bf16 0x3c3c = 0.0115: finite, non-zero
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreate(&e0);
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  int st = e == cudaSuccess ? DP_OK : fail(DP_ERR_CUDA, "autotune set-up: %s", cudaGetErrorString(e));
+  float best = 1e30f;
+  for (size_t c = 0; c < cands.size() && st == DP_OK; ++c) {
+    CUtensorMap tw;
+    st = gemm_encode_w(&tw, w.qweight, w.N, w.K, w.bits, cands[c].bn, cands[c].cg);
+    const int warm = 2, reps = 8;
+    for (int it = 0; it < warm + reps && st == DP_OK; ++it) {
+      if (it == warm) cudaEventRecord(e0, stream);
+      st = run_linear(&w, x, w.K, nullptr, M, y, w.N, ws, nullptr, nullptr, flags & DP_FLAG_NO_PDL, stream, &tw,
+                      cands[c].bn, cands[c].cg, cands[c].ws, nullptr, it > 0);
+    }
+    if (st != DP_OK) break;
+    cudaEventRecord(e1, stream);
+    e = cudaEventSynchronize(e1);
+    float ms = 0.0f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    if (e != cudaSuccess) {
+      st = fail(DP_ERR_CUDA, "autotune timing: %s", cudaGetErrorString(e));
+      break;
+    }
+    if (ms < best) {
+      best = ms;
+      *bn_out = cands[c].bn;
+      *cg_out = cands[c].cg;
+      *ws_out = cands[c].ws;
+    }
+  }
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  if (stream) cudaStreamDestroy(stream);
+  cudaFree(x);
+  cudaFree(y);
+  cudaFree(ws);
+  return st;
+}
 
 extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const int64_t* M_per_layer,
                               uint32_t flags, dp_plan** out) {
@@ -350,7 +419,12 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
   *out = nullptr;
   if (!layers || !M_per_layer || n_layers <= 0)
     return fail(DP_ERR_INVALID_ARG, "layers/M_per_layer NULL or n_layers <= 0");
-  if (flags & ~kLinearFlags) return fail(DP_ERR_INVALID_ARG, "unknown flag bits 0x%x", flags);
+  if (flags & ~(kLinearFlags | DP_FLAG_AUTOTUNE | DP_FLAG_GROUP_SMALL_M))
+    return fail(DP_ERR_INVALID_ARG, "unknown flag bits 0x%x", flags);
+  const bool autotune = (flags & DP_FLAG_AUTOTUNE) != 0;
+  const bool group_small = (flags & DP_FLAG_GROUP_SMALL_M) != 0;
+  flags &= ~(DP_FLAG_AUTOTUNE | DP_FLAG_GROUP_SMALL_M);
+  std::vector<TunedShape> tuned;
   int st = check_device();
   if (st != DP_OK) return st;
   dp_plan* p = new (std::nothrow) dp_plan();
@@ -384,6 +458,24 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
       if ((lf & DP_FLAG_CTA_PAIR) && L.w.N % 128) lf &= ~DP_FLAG_CTA_PAIR;
       if ((lf & DP_FLAG_WEIGHT_STATIONARY) && !gemm_ws_supported(L.w.N, L.w.K)) lf &= ~DP_FLAG_WEIGHT_STATIONARY;
       choose_tile(lf, L.M, L.w.N, L.w.K, L.w.bits, &L.bn, &L.cg, &L.ws);
+      if (autotune) {
+        const TunedShape* hit = nullptr;
+        for (const TunedShape& t : tuned)
+          if (t.M == L.M && t.N == L.w.N && t.K == L.w.K && t.bits == L.w.bits) hit = &t;
+        if (hit == nullptr) {
+          TunedShape t = {L.M, L.w.N, L.w.K, L.w.bits, L.bn, L.cg, L.ws};
+          st = autotune_shape(L.w, L.M, flags, &t.bn, &t.cg, &t.ws);
+          if (st != DP_OK) {
+            delete p;
+            return st;
+          }
+          tuned.push_back(t);
+          hit = &tuned.back();
+        }
+        L.bn = hit->bn;
+        L.cg = hit->cg;
+        L.ws = hit->ws;
+      }
       st = gemm_encode_w(&L.tmap_w, L.w.qweight, L.w.N, L.w.K, L.w.bits, L.bn, L.cg);
       if (st != DP_OK) {
         delete p;
@@ -395,6 +487,24 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
     L.x_offset = p->x_bytes;
     p->x_bytes += align256(static_cast<size_t>(L.M) * L.w.K * 2);
     p->layers.push_back(L);
+  }
+  p->grouped.assign(p->layers.size(), 0);
+  if (group_small) {
+    for (size_t l = 0; l < p->layers.size(); ++l) {
+      const PlanLayer& L = p->layers[l];
+      if (!L.simt || L.M == 0) continue;
+      std::vector<int>* home = nullptr;
+      for (auto& g : p->groups) {
+        const PlanLayer& G = p->layers[g[0]];
+        if (G.M == L.M && G.w.N == L.w.N && G.w.K == L.w.K && g.size() < static_cast<size_t>(kSimtGroupMax)) home = &g;
+      }
+      if (home == nullptr) {
+        p->groups.emplace_back();
+        home = &p->groups.back();
+      }
+      home->push_back(static_cast<int>(l));
+      p->grouped[l] = 1;
+    }
   }
   cudaError_t e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
   for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
@@ -441,9 +551,29 @@ static const CUtensorMap* cached_tmap_a(dp_plan* plan, const void* ws, int64_t M
 static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, void* workspace,
                          int32_t* status, cudaStream_t stream, bool* chained) {
   const int n = static_cast<int>(plan->layers.size());
+  for (const std::vector<int>& grp : plan->groups) {
+    const PlanLayer& G = plan->layers[grp[0]];
+    SimtGroupArgs ga;
+    ga.M = G.M;
+    ga.N = G.w.N;
+    ga.K = G.w.K;
+    ga.n_layers = static_cast<int32_t>(grp.size());
+    ga.early_w = *chained ? 1 : 0;
+    for (size_t i = 0; i < grp.size(); ++i) {
+      const int l = grp[i];
+      const PlanLayer& L = plan->layers[l];
+      if (!xs[l] || !ys[l]) return fail(DP_ERR_INVALID_ARG, "layer %d: NULL x or y", l);
+      if (!aligned16(xs[l]) || !aligned16(ys[l])) return fail(DP_ERR_ALIGN, "layer %d: x/y misaligned", l);
+      ga.layer[i] = {xs[l], static_cast<uint16_t*>(ys[l]), L.w.qweight, L.w.s_w,
+                     static_cast<const uint16_t*>(L.w.bias), L.w.bits};
+    }
+    int st = launch_simt_group(ga, stream, !(plan->flags & DP_FLAG_NO_PDL));
+    if (st != DP_OK) return st;
+    *chained = true;
+  }
   for (int l = 0; l < n; ++l) {
     const PlanLayer& L = plan->layers[l];
-    if (L.M == 0) continue;
+    if (L.M == 0 || plan->grouped[l]) continue;
     if (!xs[l] || !ys[l]) return fail(DP_ERR_INVALID_ARG, "layer %d: NULL x or y", l);
     if (!aligned16(xs[l]) || !aligned16(ys[l])) return fail(DP_ERR_ALIGN, "layer %d: x/y misaligned", l);
     const CUtensorMap* ta = nullptr;

@@ -41,6 +41,22 @@ struct SimtArgs {
   int32_t early_w;  // weights may be fetched before the preceding kernel on the stream has finished
 };
 int launch_simt_linear(const SimtArgs& a, cudaStream_t stream, bool pdl);
+// Up to kSimtGroupMax layers of one shape (bf16 inputs [M][K], outputs [M][N], both contiguous).
+constexpr int kSimtGroupMax = 32;
+struct SimtGroupArgs {
+  struct Layer {
+    const void* x;
+    uint16_t* y;
+    const void* qweight;
+    const float* s_w;
+    const uint16_t* bias;
+    int32_t bits;
+  } layer[kSimtGroupMax];
+  int64_t M;
+  int32_t N, K, n_layers;
+  int32_t early_w;
+};
+int launch_simt_group(const SimtGroupArgs& g, cudaStream_t stream, bool pdl);
 size_t simt_max_k();
 
 // gemm_tc.cu — tcgen05 kind::i8 GEMM with in-smem weight unpack and fused dequant epilogue.

@@ -72,17 +72,16 @@ __device__ __forceinline__ void expand_unit(const uint32_t (&pk)[BITS], uint32_t
 }
 
 template <int BITS>
-__global__ void __launch_bounds__(kSimtWarps * 32)
-simt_linear_kernel(SimtArgs a) {
+__device__ __forceinline__ void simt_linear_body(const SimtArgs& a, const int block_x, const int block_y) {
   extern __shared__ __align__(16) uint8_t smem[];
   int8_t* sq = reinterpret_cast<int8_t*>(smem);                       // [kSimtRows][K]
   float* ssa = reinterpret_cast<float*>(smem + kSimtRows * a.K);      // [kSimtRows]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int sub = lane & (kSimtLanesPerCh - 1);
-  const int64_t m0 = static_cast<int64_t>(blockIdx.y) * kSimtRows;
+  const int64_t m0 = static_cast<int64_t>(block_y) * kSimtRows;
   const int K = a.K;
   const int units = K >> 5;
-  const int n = blockIdx.x * kSimtChPerCta + warp * (32 / kSimtLanesPerCh) + (lane >> 3);
+  const int n = block_x * kSimtChPerCta + warp * (32 / kSimtLanesPerCh) + (lane >> 3);
   const bool n_ok = n < a.N;
   const uint32_t* wrow = static_cast<const uint32_t*>(a.qweight) +
                          static_cast<int64_t>(n_ok ? n : 0) * ((K * BITS) >> 5);
@@ -147,7 +146,7 @@ simt_linear_kernel(SimtArgs a) {
       }
       if (lane == 0) ssa[warp] = sc;
     }
-    if (blockIdx.x == 0 && row < a.M) {  // optional taps, written once per token
+    if (block_x == 0 && row < a.M) {  // optional taps, written once per token
       if (a.dbg_sa != nullptr && lane == 0) a.dbg_sa[row] = ssa[warp];
       if (a.dbg_q != nullptr) {
         __syncwarp();
@@ -228,7 +227,61 @@ simt_linear_kernel(SimtArgs a) {
   }
 }
 
+template <int BITS>
+__global__ void __launch_bounds__(kSimtWarps * 32)
+simt_linear_kernel(SimtArgs a) {
+  simt_linear_body<BITS>(a, blockIdx.x, blockIdx.y);
+}
+
+// Several layers of one shape (M, K, N) in one launch: blockIdx.z picks the layer. Used for the
+// adaLN modulation linears of a timestep, which are mutually independent and, one at a time, far
+// too small (3..8 MB of weights) to fill the GPU for longer than a launch takes.
+__global__ void __launch_bounds__(kSimtWarps * 32)
+simt_group_kernel(SimtGroupArgs g) {
+  SimtArgs a;
+  const SimtGroupArgs::Layer& L = g.layer[blockIdx.z];
+  a.x = L.x;
+  a.ldx = g.K;
+  a.s_a_in = nullptr;
+  a.M = g.M;
+  a.N = g.N;
+  a.K = g.K;
+  a.bits = L.bits;
+  a.qweight = L.qweight;
+  a.s_w = L.s_w;
+  a.bias = L.bias;
+  a.y = L.y;
+  a.ldy = g.N;
+  a.dbg_q = nullptr;
+  a.dbg_ldq = 0;
+  a.dbg_sa = nullptr;
+  a.dbg_acc = nullptr;
+  a.dbg_ldacc = 0;
+  a.early_w = g.early_w;
+  if (L.bits == 8) simt_linear_body<8>(a, blockIdx.x, blockIdx.y);
+  else if (L.bits == 4) simt_linear_body<4>(a, blockIdx.x, blockIdx.y);
+  else simt_linear_body<3>(a, blockIdx.x, blockIdx.y);
+}
+
 size_t simt_max_k() { return 16384; }
+
+int launch_simt_group(const SimtGroupArgs& g, cudaStream_t stream, bool pdl) {
+  if (g.M == 0 || g.n_layers == 0) return DP_OK;
+  const size_t smem = static_cast<size_t>(kSimtRows) * g.K + kSimtRows * sizeof(float);
+  const dim3 grid((g.N + kSimtChPerCta - 1) / kSimtChPerCta, static_cast<unsigned>((g.M + kSimtRows - 1) / kSimtRows),
+                  static_cast<unsigned>(g.n_layers));
+  const dim3 block(kSimtWarps * 32);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(simt_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem));
+    if (e != cudaSuccess) return fail(DP_ERR_CUDA, "simt smem attribute: %s", cudaGetErrorString(e));
+  }
+  SimtGroupArgs args = g;
+  if (!pdl) args.early_w = 0;
+  cudaError_t e = launch(simt_group_kernel, grid, block, smem, stream, pdl, args);
+  if (e != cudaSuccess) return fail(DP_ERR_CUDA, "grouped simt launch failed: %s", cudaGetErrorString(e));
+  return DP_OK;
+}
 
 int launch_simt_linear(const SimtArgs& a, cudaStream_t stream, bool pdl) {
   if (a.M == 0) return DP_OK;

@@ -39,8 +39,9 @@ class DevWeights:
 
 class DitStack:
     def __init__(self, seed=synth.BASE_SEED + 4, batch=8, tokens=256, blocks=synth.BLOCKS, T=50, keep=25,
-                 bit_choices=(3, 4, 8), resident_steps=None, flags=0):
-        self.seed, self.T = seed, T
+                 bit_choices=(3, 4, 8), resident_steps=None,
+                 flags=B.DP_FLAG_AUTOTUNE | B.DP_FLAG_GROUP_SMALL_M):
+        self.seed, self.T, self.flags = seed, T, flags
         self.table = synth.dit_layers(batch, tokens, blocks)
         self.bits = synth.bit_plan(seed, len(self.table), bit_choices)
         self.kept = synth.kept_timesteps(seed, T, keep, 0.2)
@@ -76,10 +77,12 @@ class DitStack:
         return tot
 
     def launches_per_timestep(self):
-        n = 0
-        for (_, M, K, N) in self.table:
-            n += 1 if M <= 32 else 2
-        return n
+        """Kernel launches of this library per timestep: DAQ + GEMM per token linear; the small-M
+        (adaLN) linears of a step share one grouped launch per 32 when the plan groups them."""
+        small = sum(1 for (_, M, K, N) in self.table if M <= 32)
+        big = len(self.table) - small
+        grouped = bool(self.flags & B.DP_FLAG_GROUP_SMALL_M)
+        return 2 * big + (-(-small // 32) if grouped else small)
 
     # ---- execution ----
     def ptrs(self, n_steps=None):

@@ -83,6 +83,37 @@ def test_plan_run_matches_oracle_every_step_and_layer():
         B.dp_plan_destroy(plan)
 
 
+def test_plan_autotuned_and_grouped_matches_oracle():
+    """Plan created with the on-device autotuner and with the small-M layers (adaLN) of a step
+    grouped into one launch: every output of every step still equals the oracle's."""
+    table, layers, dev = _mini_plan(tokens=256, batch=3, blocks=3)
+    T = 6
+    kept = [1, 4, 5]
+    nL, nS = len(layers), len(kept)
+    xs = [[synth.activations(SEED, l, t, L["M"], L["K"], synth.sigma_t(t, T), n_out=max(1, L["K"] // 100))
+           for l, L in enumerate(layers)] for t in kept]
+    ref = oracle.plan_run(layers, kept, xs)
+    plan = B.dp_plan_create([d.w for d in dev], [L["M"] for L in layers],
+                            B.DP_FLAG_AUTOTUNE | B.DP_FLAG_GROUP_SMALL_M)
+    try:
+        ws = torch.empty(B.dp_plan_workspace(plan), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        xd = [[to_dev_bf16(xs[i][l]) for l in range(nL)] for i in range(nS)]
+        yd = [[torch.full((L["M"], L["N"]), float("nan"), dtype=torch.bfloat16, device="cuda")
+               for L in layers] for _ in range(nS)]
+        xp = B.ptr_array([xd[i][l].data_ptr() for i in range(nS) for l in range(nL)])
+        yp = B.ptr_array([yd[i][l].data_ptr() for i in range(nS) for l in range(nL)])
+        B.dp_plan_run(plan, kept, 0, xp, yp, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for i in range(nS):
+            for l in range(nL):
+                d = bf16_ulp_dist(bf16_to_np(yd[i][l]), ref[i][l])
+                assert d.max() <= 1, (i, l, table[l], int(d.max()))
+    finally:
+        B.dp_plan_destroy(plan)
+
+
 def test_plan_run_host_inputs():
     table, layers, dev = _mini_plan(tokens=128, batch=2, blocks=1)
     kept = [1, 3, 4]
