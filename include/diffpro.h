@@ -190,6 +190,12 @@ typedef struct dp_plan dp_plan;
 int dp_plan_create(const dp_weight* layers, int32_t n_layers, const int64_t* M_per_layer,
                    uint32_t flags, dp_plan** out);
 size_t dp_plan_workspace(const dp_plan* plan);
+/* Which kernel the plan runs layer `layer` with (for reports and for timing that kernel alone):
+ * *tile_n = tile width in output channels, *cta_group = 1 or 2 CTAs per row tile,
+ * *weight_stationary = 0/1, *small_m = 1 when the CUDA-core small-M kernel is used (the other three
+ * are then 0). Any output pointer may be NULL. */
+int dp_plan_layer_variant(const dp_plan* plan, int32_t layer, int32_t* tile_n, int32_t* cta_group,
+                          int32_t* weight_stationary, int32_t* small_m);
 void dp_plan_destroy(dp_plan* plan);
 
 /*

@@ -31,7 +31,7 @@ def DP_FLAG_TILE_N(bn: int) -> int:
 DP_STATIC_SCRATCH_BYTES = 10 << 20
 
 EXPORTS = ["dp_daq_quantize", "dp_wq_linear_workspace", "dp_wq_linear", "dp_wq_linear_static", "dp_plan_create",
-           "dp_plan_workspace", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
+           "dp_plan_workspace", "dp_plan_layer_variant", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
            "dp_plan_run_host", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_status_string",
            "dp_last_error", "dp_version"]
 
@@ -67,6 +67,7 @@ def lib():
         L.dp_wq_linear_workspace.argtypes = [C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_uint32]
         L.dp_plan_workspace.restype = C.c_size_t
         L.dp_plan_workspace.argtypes = [C.c_void_p]
+        L.dp_plan_layer_variant.argtypes = [C.c_void_p, C.c_int32] + [C.POINTER(C.c_int32)] * 4
         L.dp_plan_x_bytes.restype = C.c_size_t
         L.dp_plan_x_bytes.argtypes = [C.c_void_p]
         L.dp_plan_destroy.restype = None
@@ -148,6 +149,24 @@ def dp_plan_create(weights: list[dp_weight], Ms: list[int], flags=0) -> C.c_void
 
 def dp_plan_workspace(plan) -> int:
     return int(lib().dp_plan_workspace(plan))
+
+
+def dp_plan_layer_variant(plan, layer: int) -> dict:
+    """{'tile_n', 'cta_group', 'weight_stationary', 'small_m'} of one layer of a plan."""
+    v = [C.c_int32() for _ in range(4)]
+    _check(lib().dp_plan_layer_variant(plan, layer, *[C.byref(t) for t in v]), "dp_plan_layer_variant")
+    return dict(tile_n=v[0].value, cta_group=v[1].value, weight_stationary=v[2].value, small_m=v[3].value)
+
+
+def variant_flags(v: dict) -> int:
+    """dp_wq_linear flags that force the kernel variant a plan chose for a layer."""
+    if v["small_m"]:
+        return DP_FLAG_FORCE_SIMT
+    f = DP_FLAG_FORCE_MMA | DP_FLAG_TILE_N(v["tile_n"])
+    if v["weight_stationary"]:
+        return f | DP_FLAG_WEIGHT_STATIONARY
+    f |= DP_FLAG_NO_WEIGHT_STATIONARY
+    return f | (DP_FLAG_CTA_PAIR if v["cta_group"] == 2 else DP_FLAG_NO_CTA_PAIR)
 
 
 def dp_plan_x_bytes(plan) -> int:

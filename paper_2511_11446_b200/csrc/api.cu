@@ -520,6 +520,17 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
 }
 
 extern "C" size_t dp_plan_workspace(const dp_plan* plan) { return plan ? plan->workspace_bytes : 0; }
+extern "C" int dp_plan_layer_variant(const dp_plan* plan, int32_t layer, int32_t* tile_n, int32_t* cta_group,
+                                     int32_t* weight_stationary, int32_t* small_m) {
+  if (!plan || layer < 0 || layer >= static_cast<int32_t>(plan->layers.size()))
+    return fail(DP_ERR_INVALID_ARG, "dp_plan_layer_variant: bad plan or layer index");
+  const PlanLayer& L = plan->layers[layer];
+  if (tile_n) *tile_n = L.simt ? 0 : L.bn;
+  if (cta_group) *cta_group = L.simt ? 0 : L.cg;
+  if (weight_stationary) *weight_stationary = L.simt ? 0 : L.ws;
+  if (small_m) *small_m = L.simt ? 1 : 0;
+  return DP_OK;
+}
 extern "C" size_t dp_plan_x_bytes(const dp_plan* plan) { return plan ? plan->x_bytes : 0; }
 
 extern "C" void dp_plan_destroy(dp_plan* plan) {

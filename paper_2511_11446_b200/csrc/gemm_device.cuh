@@ -129,49 +129,13 @@ __device__ __forceinline__ void unpack3_tile(const uint8_t* P, uint8_t* B, int t
 }
 
 // ---- epilogue arithmetic -----------------------------------------------------------------------------
-// 32 accumulators of one token -> bf16 into the warp's staging tile [32 tokens][64 bytes], 16-byte
-// chunks XOR-swizzled by ((token >> 1) & 3) so that both the per-token writes and the row-wise
-// read-back are free of bank conflicts. Per element, in this order: t = (float)(acc / 2^SHIFT),
-// sc = s_a * s_w[n], y = fma(t, sc, bias[n]), bf16 round-to-nearest-even.
+// One output, in this order: t = (float)(acc / 2^SHIFT) (exact scaling), sc = s_a * s_w[n],
+// y = fma(t, sc, bias[n]); the caller rounds pairs to bf16 (nearest even).
 template <int SHIFT>
-__device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], float sa,
-                                               const float4* __restrict__ s4,
-                                               const float4* __restrict__ b4,
-                                               uint4* __restrict__ stage_row, int sw,
-                                               int32_t* acc_dst) {
-  // all shared-memory reads and all arithmetic first, the four 16-byte stores last: nothing in the
-  // arithmetic then has to wait behind a store the compiler cannot reorder
-  uint32_t o[16];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const float4 sw4 = s4[j], bb = b4[j];
-    float t0 = __int2float_rn(static_cast<int>(r[4 * j + 0]));
-    float t1 = __int2float_rn(static_cast<int>(r[4 * j + 1]));
-    float t2 = __int2float_rn(static_cast<int>(r[4 * j + 2]));
-    float t3 = __int2float_rn(static_cast<int>(r[4 * j + 3]));
-    if constexpr (SHIFT != 0) {  // exact: the accumulator is a multiple of 2^SHIFT
-      constexpr float kInv = 1.0f / (1 << SHIFT);
-      t0 = __fmul_rn(t0, kInv);
-      t1 = __fmul_rn(t1, kInv);
-      t2 = __fmul_rn(t2, kInv);
-      t3 = __fmul_rn(t3, kInv);
-    }
-    const float y0 = __fmaf_rn(t0, __fmul_rn(sa, sw4.x), bb.x);
-    const float y1 = __fmaf_rn(t1, __fmul_rn(sa, sw4.y), bb.y);
-    const float y2 = __fmaf_rn(t2, __fmul_rn(sa, sw4.z), bb.z);
-    const float y3 = __fmaf_rn(t3, __fmul_rn(sa, sw4.w), bb.w);
-    const __nv_bfloat162 h0 = __floats2bfloat162_rn(y0, y1);
-    const __nv_bfloat162 h1 = __floats2bfloat162_rn(y2, y3);
-    o[2 * j] = *reinterpret_cast<const uint32_t*>(&h0);
-    o[2 * j + 1] = *reinterpret_cast<const uint32_t*>(&h1);
-  }
-#pragma unroll
-  for (int j = 0; j < 4; ++j)
-    stage_row[j ^ sw] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
-  if (acc_dst != nullptr) {
-#pragma unroll
-    for (int j = 0; j < 32; ++j) acc_dst[j] = static_cast<int>(r[j]) >> SHIFT;
-  }
+__device__ __forceinline__ float dequant_one(uint32_t acc, float sa, float sw, float bias) {
+  float t = __int2float_rn(static_cast<int>(acc));
+  if constexpr (SHIFT != 0) t = __fmul_rn(t, 1.0f / (1 << SHIFT));  // exact: acc is a multiple of 2^SHIFT
+  return __fmaf_rn(t, __fmul_rn(sa, sw), bias);
 }
 
 // ---- the epilogue of one warp ---------------------------------------------------------------------------
@@ -193,7 +157,6 @@ struct EpilogueWarp {
   int qd, slab0, slab1, lane, staged_n;
   float *ts, *tb;
   const uint4* stage4;
-  uint4* stage_row;
   uint32_t acc_empty_addr[2];  // (cluster) address of the barrier that collects drained buffers
 
   __device__ __forceinline__ void init(int warp, int lane_, float* s_scale, float* s_bias, uint8_t* sY,
@@ -207,7 +170,6 @@ struct EpilogueWarp {
     tb = s_bias + ew * 64 * L::SLABS_LO;
     uint8_t* stage = sY + ew * kYStageBytes;
     stage4 = reinterpret_cast<const uint4*>(stage);
-    stage_row = reinterpret_cast<uint4*>(stage + lane * 64);
     acc_empty_addr[0] = acc_empty0;
     acc_empty_addr[1] = acc_empty1;
     staged_n = -1;
@@ -222,10 +184,16 @@ struct EpilogueWarp {
                                        volatile int* abort_flag) {
     const int n0 = n_blk * BN;
     const int row0 = cta_row0 + qd * 32;
-    const int64_t row = static_cast<int64_t>(row0) + lane;
-    const bool row_ok = row < p.M;
-    // independent loads first, their latency overlaps the wait for the accumulator
-    const float sa = row_ok ? __ldg(p.s_a + row) : 0.0f;
+    // Accumulators are read in the fragment layout: this thread owns tokens row0 + r8 + 8 i
+    // (i = 0..3) and, per 32-column chunk, columns 8 j + 2 t4, + 1 (j = 0..3). Owning columns lets
+    // it fetch its scales and biases with plain (non-broadcast) 8-byte shared loads.
+    const int t4 = lane & 3, r8 = lane >> 2;
+    float sa[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int64_t row = static_cast<int64_t>(row0) + r8 + 8 * i;
+      sa[i] = row < p.M ? __ldg(p.s_a + row) : 0.0f;
+    }
     if (n_blk != staged_n) {
       constexpr int NV = 2 * L::SLABS_LO;  // 32-column groups this warp may need
       float sv[NV], bv[NV];
@@ -251,20 +219,49 @@ struct EpilogueWarp {
     if (!ok) return false;
     tc_fence_after();
     const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + t_cols;
-    int32_t* arow = (p.dbg_acc != nullptr && row_ok) ? p.dbg_acc + row * p.dbg_ldacc + n0 : nullptr;
+    uint32_t* stage32 = reinterpret_cast<uint32_t*>(const_cast<uint4*>(stage4));
     for (int c = 2 * slab0; c < 2 * slab1; ++c) {  // 32-column chunks of this warp
-      uint32_t r[32];
-      tmem_ld_32x32(t_addr + c * 32, r);
-      tmem_ld_wait();
-      if (c + 1 == 2 * slab1) {  // this warp's last accumulators are in registers
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(acc_empty_addr[buf]);
+      const int lc = (c - 2 * slab0) * 32 + 2 * t4;  // this thread's first column inside the staged scales
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {  // tokens r8 + 16 h and r8 + 16 h + 8
+        uint32_t r[16];
+        tmem_ld_16x256b_x4(t_addr + (static_cast<uint32_t>(16 * h) << 16) + c * 32, r);
+        tmem_ld_wait();
+        if (h == 1 && c + 1 == 2 * slab1) {  // this warp's last accumulators are in registers
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(acc_empty_addr[buf]);
+        }
+        // staging tile [32 tokens][64 bytes], 16-byte chunks XOR-swizzled by ((token >> 1) & 3): these
+        // 4-byte stores and the 16-byte row-wise read-back below are both free of bank conflicts
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 sw = *reinterpret_cast<const float2*>(ts + lc + 8 * j);
+          const float2 bb = *reinterpret_cast<const float2*>(tb + lc + 8 * j);
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            const int rr = r8 + 16 * h + 8 * i;
+            const float s = sa[2 * h + i];
+            const __nv_bfloat162 v = __floats2bfloat162_rn(dequant_one<SHIFT>(r[4 * j + 2 * i], s, sw.x, bb.x),
+                                                           dequant_one<SHIFT>(r[4 * j + 2 * i + 1], s, sw.y, bb.y));
+            stage32[rr * 16 + ((j ^ ((rr >> 1) & 3)) << 2) + t4] = *reinterpret_cast<const uint32_t*>(&v);
+          }
+        }
+        if (p.dbg_acc != nullptr) {
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            const int64_t row = static_cast<int64_t>(row0) + r8 + 16 * h + 8 * i;
+            if (row < p.M) {
+              int32_t* arow = p.dbg_acc + row * p.dbg_ldacc + n0 + c * 32 + 2 * t4;
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                arow[8 * j] = static_cast<int>(r[4 * j + 2 * i]) >> SHIFT;
+                arow[8 * j + 1] = static_cast<int>(r[4 * j + 2 * i + 1]) >> SHIFT;
+              }
+            }
+          }
+        }
       }
-      const int lc = (c - 2 * slab0) * 32;  // column inside this warp's staged scales
-      epilogue_chunk<SHIFT>(r, sa, reinterpret_cast<const float4*>(ts + lc),
-                            reinterpret_cast<const float4*>(tb + lc), stage_row, (lane >> 1) & 3,
-                            arow ? arow + c * 32 : nullptr);
       __syncwarp();
       // staged chunk -> global: every store instruction covers eight 64-byte row segments
       {
