@@ -109,6 +109,14 @@ typedef struct dp_debug {
  * those layers first in each step, equal shapes grouped into one launch; results are unchanged. */
 #define DP_FLAG_GROUP_SMALL_M 0x20000u
 
+/* dp_plan_create only: let the plan's tensor-core GEMM kernels quantize their activations
+ * themselves instead of running DAQ as a kernel of its own in front of each GEMM: the CTAs share
+ * the tokens, publish finished 128-token tiles on counters the plan owns, and start the tiles
+ * whose tokens are ready. One launch per layer instead of two; results are identical. Off by
+ * default: on B200 the two-kernel form is faster, because its small DAQ kernel is already resident
+ * (programmatic dependent launch) while the previous GEMM drains. */
+#define DP_FLAG_FUSED_DAQ 0x40000u
+
 /* flags for dp_plan_run */
 #define DP_PLAN_SAME_X 1u       /* x_ptrs has n_layers entries reused by every step              */
 #define DP_PLAN_SAME_Y 2u       /* y_ptrs has n_layers entries reused (overwritten) every step   */

@@ -21,7 +21,7 @@ DP_OK = 0
 DP_FLAG_NONE, DP_FLAG_FORCE_SIMT, DP_FLAG_FORCE_MMA, DP_FLAG_NO_PDL = 0, 1, 2, 4
 DP_FLAG_CTA_PAIR, DP_FLAG_NO_CTA_PAIR = 0x800, 0x1000
 DP_FLAG_WEIGHT_STATIONARY, DP_FLAG_NO_WEIGHT_STATIONARY = 0x2000, 0x4000
-DP_FLAG_AUTOTUNE, DP_FLAG_GROUP_SMALL_M = 0x10000, 0x20000
+DP_FLAG_AUTOTUNE, DP_FLAG_GROUP_SMALL_M, DP_FLAG_FUSED_DAQ = 0x10000, 0x20000, 0x40000
 DP_PLAN_SAME_X, DP_PLAN_SAME_Y = 1, 2
 
 

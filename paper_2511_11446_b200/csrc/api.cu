@@ -124,7 +124,7 @@ static int check_weight(const dp_weight* w) {
 static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_a_in, int64_t M,
                       void* y, int64_t ldy, void* workspace, const dp_debug* dbg, int32_t* status,
                       uint32_t flags, cudaStream_t stream, const CUtensorMap* tmap_w, int bn, int cg, int ws,
-                      const CUtensorMap* tmap_a_cached, bool chained) {
+                      const CUtensorMap* tmap_a_cached, bool chained, int32_t* daq_sync = nullptr) {
   const bool pdl = !(flags & DP_FLAG_NO_PDL);
   if (use_simt(M, w->N, w->K, flags)) {
     if (static_cast<size_t>(w->K) > simt_max_k())
@@ -155,12 +155,15 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
   int64_t ldq;
   int korder = KORDER_NATURAL;
   const bool tiled = s_a_in == nullptr;  // the library's own scratch: stored as contiguous 128 x 128 tiles
+  const bool fused = s_a_in == nullptr && daq_sync != nullptr && dbg == nullptr;  // DAQ inside the GEMM kernel
   if (s_a_in == nullptr) {
     int8_t* wq = static_cast<int8_t*>(workspace);
     float* wsa = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align256(scratch_q_bytes(M, w->K)));
     korder = gemm_korder(w->bits);
-    int st = launch_daq(x, M, w->K, ldx, wq, w->K, wsa, nullptr, korder, true, stream, pdl);
-    if (st != DP_OK) return st;
+    if (!fused) {
+      int st = launch_daq(x, M, w->K, ldx, wq, w->K, wsa, nullptr, korder, true, stream, pdl);
+      if (st != DP_OK) return st;
+    }
     q = wq;
     s_a = wsa;
     ldq = w->K;
@@ -172,7 +175,12 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
   GemmProblem g;
   g.korder = korder;
   g.a_tiled = tiled ? 1 : 0;
-  g.early_w = (s_a_in == nullptr) ? 1 : 0;
+  g.early_w = fused ? (chained ? 1 : 0) : (s_a_in == nullptr ? 1 : 0);
+  g.x = fused ? static_cast<const uint16_t*>(x) : nullptr;
+  g.ldx = ldx;
+  g.q_out = fused ? const_cast<int8_t*>(q) : nullptr;
+  g.s_a_out = fused ? const_cast<float*>(s_a) : nullptr;
+  g.sync = fused ? daq_sync : nullptr;
   if (tmap_a_cached != nullptr) {
     g.tmap_a = *tmap_a_cached;
   } else {
@@ -342,6 +350,7 @@ struct dp_plan {
   std::vector<TmapACache> a_cache;
   std::vector<std::vector<int>> groups;  // small-M layers of equal shape, run first in every step
   std::vector<char> grouped;             // per layer: member of a group
+  int32_t* daq_sync;                     // device counters of the in-kernel DAQ (nullptr: DAQ in its own kernel)
   cudaStream_t copy_stream;
   cudaEvent_t ev_copied[2], ev_consumed[2];
 };
@@ -419,11 +428,12 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
   *out = nullptr;
   if (!layers || !M_per_layer || n_layers <= 0)
     return fail(DP_ERR_INVALID_ARG, "layers/M_per_layer NULL or n_layers <= 0");
-  if (flags & ~(kLinearFlags | DP_FLAG_AUTOTUNE | DP_FLAG_GROUP_SMALL_M))
+  if (flags & ~(kLinearFlags | DP_FLAG_AUTOTUNE | DP_FLAG_GROUP_SMALL_M | DP_FLAG_FUSED_DAQ))
     return fail(DP_ERR_INVALID_ARG, "unknown flag bits 0x%x", flags);
   const bool autotune = (flags & DP_FLAG_AUTOTUNE) != 0;
   const bool group_small = (flags & DP_FLAG_GROUP_SMALL_M) != 0;
-  flags &= ~(DP_FLAG_AUTOTUNE | DP_FLAG_GROUP_SMALL_M);
+  const bool fused_daq = (flags & DP_FLAG_FUSED_DAQ) != 0;
+  flags &= ~(DP_FLAG_AUTOTUNE | DP_FLAG_GROUP_SMALL_M | DP_FLAG_FUSED_DAQ);
   std::vector<TunedShape> tuned;
   int st = check_device();
   if (st != DP_OK) return st;
@@ -433,6 +443,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
   p->workspace_bytes = 256;
   p->x_bytes = 0;
   p->copy_stream = nullptr;
+  p->daq_sync = nullptr;
   for (int i = 0; i < 2; ++i) p->ev_copied[i] = p->ev_consumed[i] = nullptr;
   for (int32_t l = 0; l < n_layers; ++l) {
     st = check_weight(&layers[l]);
@@ -506,7 +517,18 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
       p->grouped[l] = 1;
     }
   }
-  cudaError_t e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
+  cudaError_t e = cudaSuccess;
+  if (fused_daq) {
+    int64_t max_tiles = 0;
+    for (const PlanLayer& L : p->layers)
+      if (!L.simt && (L.M + 127) / 128 > max_tiles) max_tiles = (L.M + 127) / 128;
+    if (max_tiles > 0) {
+      const size_t bytes = sizeof(int32_t) * static_cast<size_t>(max_tiles + 1);
+      e = cudaMalloc(reinterpret_cast<void**>(&p->daq_sync), bytes);
+      if (e == cudaSuccess) e = cudaMemset(p->daq_sync, 0, bytes);
+    }
+  }
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
   for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
     e = cudaEventCreateWithFlags(&p->ev_copied[i], cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_consumed[i], cudaEventDisableTiming);
@@ -540,6 +562,7 @@ extern "C" void dp_plan_destroy(dp_plan* plan) {
     if (plan->ev_consumed[i]) cudaEventDestroy(plan->ev_consumed[i]);
   }
   if (plan->copy_stream) cudaStreamDestroy(plan->copy_stream);
+  if (plan->daq_sync) cudaFree(plan->daq_sync);
   delete plan;
 }
 
@@ -594,7 +617,8 @@ static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, 
       if (st != DP_OK) return st;
     }
     int st = run_linear(&L.w, xs[l], L.w.K, nullptr, L.M, ys[l], L.w.N, workspace, nullptr, status,
-                        plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, L.cg, L.ws, ta, *chained);
+                        plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, L.cg, L.ws, ta, *chained,
+                        L.simt ? nullptr : plan->daq_sync);
     if (st != DP_OK) return st;
     *chained = true;
   }

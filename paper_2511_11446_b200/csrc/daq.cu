@@ -6,86 +6,9 @@
 // max is exact); the quantizer is one fused multiply-add per element: x * fl(127/a) + 1.5*2^23
 // rounds the exact product once, half to even, and leaves the integer in the low mantissa bits.
 // HBM-bound: 2 bytes read + 1 byte written per element.
-#include "dp_common.cuh"
-#include "dp_internal.h"
+#include "daq_device.cuh"
 
 namespace dp {
-
-__device__ __forceinline__ uint32_t ld_nc_u32x4(const uint4* p, uint4& v) {
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
-  return 0;
-}
-
-__device__ __forceinline__ uint32_t absmax_bits2(uint32_t m, uint32_t w) {
-  return __vmaxu2(m, w & 0x7FFF7FFFu);
-}
-
-// Quantizes two bf16 packed in `w` (low half = even k) -> two int8 in the low bytes of result
-// positions chosen by the caller.
-__device__ __forceinline__ uint32_t quant_pair(uint32_t w, float inv) {
-  const float magic = 12582912.0f;  // 1.5 * 2^23
-  float lo = __uint_as_float(w << 16);
-  float hi = __uint_as_float(w & 0xFFFF0000u);
-  uint32_t a = __float_as_uint(__fmaf_rn(lo, inv, magic));
-  uint32_t b = __float_as_uint(__fmaf_rn(hi, inv, magic));
-  return __byte_perm(a, b, 0x0040);  // byte0 = a.byte0, byte1 = b.byte0
-}
-
-// Eight consecutive codes. EO = false: stored in order; EO = true: stored as k = 0,2,4,6,1,3,5,7.
-template <bool EO>
-__device__ __forceinline__ uint2 quant_vec(const uint4& v, float inv) {
-  uint32_t p0 = quant_pair(v.x, inv), p1 = quant_pair(v.y, inv);
-  uint32_t p2 = quant_pair(v.z, inv), p3 = quant_pair(v.w, inv);
-  if constexpr (EO) {
-    const uint32_t t0 = __byte_perm(p0, p1, 0x5140);  // k0 k2 k1 k3
-    const uint32_t t1 = __byte_perm(p2, p3, 0x5140);  // k4 k6 k5 k7
-    return make_uint2(__byte_perm(t0, t1, 0x5410), __byte_perm(t0, t1, 0x7632));
-  } else {
-    return make_uint2(__byte_perm(p0, p1, 0x5410), __byte_perm(p2, p3, 0x5410));
-  }
-}
-
-// Scale and reciprocal of one token from its absmax magnitude bits (a bf16 pattern, sign cleared).
-__device__ __forceinline__ void token_scale(uint32_t abits, float& s_a, float& inv) {
-  float a = __uint_as_float(abits << 16);
-  if (a < 7.888609052210118e-31f) {  // 2^-100: treat the token as all-zero
-    s_a = 0.0f;
-    inv = 0.0f;
-  } else {
-    s_a = __fdiv_rn(a, 127.0f);
-    inv = __fdiv_rn(127.0f, a);
-  }
-}
-
-__device__ __forceinline__ uint32_t warp_max_u32(uint32_t m) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-  return m;
-}
-__device__ __forceinline__ int warp_sum_i32(int s) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
-  return s;
-}
-
-// Where the 8 codes of vector `idx` (k = 8 idx ..) of one token go. Row-major: q[row][k]. Tiled
-// (tiled_kb = K / 128 > 0): the matrix is cut into 128-token x 128-code tiles of 16 KB, stored one
-// after the other ([row tile][k block][128][128]), so that the GEMM's TMA loads of an activation tile
-// read one contiguous 16 KB range instead of 128 rows a whole row pitch apart.
-struct QRow {
-  uint2* base;
-  int tiled;
-  __device__ __forceinline__ QRow(int8_t* q, int64_t row, int64_t ldq, int tiled_kb) : tiled(tiled_kb) {
-    base = tiled_kb ? reinterpret_cast<uint2*>(q + ((row >> 7) * tiled_kb) * 16384 + (row & 127) * 128)
-                    : reinterpret_cast<uint2*>(q + row * ldq);
-  }
-  __device__ __forceinline__ void store(int idx, uint2 v) const {
-    if (tiled) base[(idx >> 4) * 2048 + (idx & 15)] = v;  // next k block: + 16384 bytes
-    else base[idx] = v;
-  }
-};
 
 constexpr int kDaqWarps = 8;
 

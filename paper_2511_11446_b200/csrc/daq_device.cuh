@@ -1,0 +1,140 @@
+// Device-side pieces of dynamic activation quantization (Step 3, Eq. "daq"; b = 8, zero-point 0,
+// clip threshold = the token's absolute maximum) shared by the stand-alone DAQ kernels and by the
+// GEMM kernels that quantize their own activations.
+#pragma once
+
+#include "dp_common.cuh"
+#include "dp_internal.h"
+
+namespace dp {
+
+__device__ __forceinline__ uint32_t ld_nc_u32x4(const uint4* p, uint4& v) {
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return 0;
+}
+
+__device__ __forceinline__ uint32_t absmax_bits2(uint32_t m, uint32_t w) {
+  return __vmaxu2(m, w & 0x7FFF7FFFu);
+}
+
+// Quantizes two bf16 packed in `w` (low half = even k) -> two int8 in the low bytes of result
+// positions chosen by the caller.
+__device__ __forceinline__ uint32_t quant_pair(uint32_t w, float inv) {
+  const float magic = 12582912.0f;  // 1.5 * 2^23
+  float lo = __uint_as_float(w << 16);
+  float hi = __uint_as_float(w & 0xFFFF0000u);
+  uint32_t a = __float_as_uint(__fmaf_rn(lo, inv, magic));
+  uint32_t b = __float_as_uint(__fmaf_rn(hi, inv, magic));
+  return __byte_perm(a, b, 0x0040);  // byte0 = a.byte0, byte1 = b.byte0
+}
+
+// Eight consecutive codes. EO = false: stored in order; EO = true: stored as k = 0,2,4,6,1,3,5,7.
+template <bool EO>
+__device__ __forceinline__ uint2 quant_vec(const uint4& v, float inv) {
+  uint32_t p0 = quant_pair(v.x, inv), p1 = quant_pair(v.y, inv);
+  uint32_t p2 = quant_pair(v.z, inv), p3 = quant_pair(v.w, inv);
+  if constexpr (EO) {
+    const uint32_t t0 = __byte_perm(p0, p1, 0x5140);  // k0 k2 k1 k3
+    const uint32_t t1 = __byte_perm(p2, p3, 0x5140);  // k4 k6 k5 k7
+    return make_uint2(__byte_perm(t0, t1, 0x5410), __byte_perm(t0, t1, 0x7632));
+  } else {
+    return make_uint2(__byte_perm(p0, p1, 0x5410), __byte_perm(p2, p3, 0x5410));
+  }
+}
+
+// Scale and reciprocal of one token from its absmax magnitude bits (a bf16 pattern, sign cleared).
+__device__ __forceinline__ void token_scale(uint32_t abits, float& s_a, float& inv) {
+  float a = __uint_as_float(abits << 16);
+  if (a < 7.888609052210118e-31f) {  // 2^-100: treat the token as all-zero
+    s_a = 0.0f;
+    inv = 0.0f;
+  } else {
+    s_a = __fdiv_rn(a, 127.0f);
+    inv = __fdiv_rn(127.0f, a);
+  }
+}
+
+__device__ __forceinline__ uint32_t warp_max_u32(uint32_t m) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  return m;
+}
+__device__ __forceinline__ int warp_sum_i32(int s) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+  return s;
+}
+
+// Where the 8 codes of vector `idx` (k = 8 idx ..) of one token go. Row-major: q[row][k]. Tiled
+// (tiled_kb = K / 128 > 0): the matrix is cut into 128-token x 128-code tiles of 16 KB, stored one
+// after the other ([row tile][k block][128][128]), so that the GEMM's TMA loads of an activation tile
+// read one contiguous 16 KB range instead of 128 rows a whole row pitch apart.
+struct QRow {
+  uint2* base;
+  int tiled;
+  __device__ __forceinline__ QRow(int8_t* q, int64_t row, int64_t ldq, int tiled_kb) : tiled(tiled_kb) {
+    base = tiled_kb ? reinterpret_cast<uint2*>(q + ((row >> 7) * tiled_kb) * 16384 + (row & 127) * 128)
+                    : reinterpret_cast<uint2*>(q + row * ldq);
+  }
+  __device__ __forceinline__ void store(int idx, uint2 v) const {
+    if (tiled) base[(idx >> 4) * 2048 + (idx & 15)] = v;  // next k block: + 16384 bytes
+    else base[idx] = v;
+  }
+};
+
+// One token by one warp, any K (multiple of 8): two passes over the row, the second served by
+// L1/L2. Writes the codes through `qr` and returns the scale (valid in every lane).
+template <bool EO>
+__device__ __forceinline__ float daq_row_2pass(const uint16_t* __restrict__ x_row, int K, const QRow& qr, int lane) {
+  const int nvec = K >> 3;
+  const uint4* xr = reinterpret_cast<const uint4*>(x_row);
+  uint32_t m = 0;
+#pragma unroll 5
+  for (int idx = lane; idx < nvec; idx += 32) {
+    const uint4 v = xr[idx];
+    m = absmax_bits2(absmax_bits2(absmax_bits2(absmax_bits2(m, v.x), v.y), v.z), v.w);
+  }
+  m = warp_max_u32(max(m & 0xFFFFu, m >> 16));
+  float sc, inv;
+  token_scale(m, sc, inv);
+#pragma unroll 5
+  for (int idx = lane; idx < nvec; idx += 32) qr.store(idx, quant_vec<EO>(xr[idx], inv));
+  return sc;
+}
+
+// Two tokens by one warp at once (the loads of both are in flight together, which matters when the
+// warp has several tokens to do and each costs a full memory round trip). has_b == false: only A.
+template <bool EO>
+__device__ __forceinline__ void daq_two_rows_2pass(const uint16_t* __restrict__ xa, const uint16_t* __restrict__ xb,
+                                                   bool has_b, int K, const QRow& qa, const QRow& qb, int lane,
+                                                   float& sc_a, float& sc_b) {
+  const int nvec = K >> 3;
+  const uint4* ra = reinterpret_cast<const uint4*>(xa);
+  const uint4* rb = reinterpret_cast<const uint4*>(has_b ? xb : xa);
+  uint32_t ma = 0, mb = 0;
+#pragma unroll 5
+  for (int idx = lane; idx < nvec; idx += 32) {
+    const uint4 va = ra[idx], vb = rb[idx];
+    ma = absmax_bits2(absmax_bits2(absmax_bits2(absmax_bits2(ma, va.x), va.y), va.z), va.w);
+    mb = absmax_bits2(absmax_bits2(absmax_bits2(absmax_bits2(mb, vb.x), vb.y), vb.z), vb.w);
+  }
+  ma = max(ma & 0xFFFFu, ma >> 16);
+  mb = max(mb & 0xFFFFu, mb >> 16);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    ma = max(ma, __shfl_xor_sync(0xFFFFFFFFu, ma, o));
+    mb = max(mb, __shfl_xor_sync(0xFFFFFFFFu, mb, o));
+  }
+  float inv_a, inv_b;
+  token_scale(ma, sc_a, inv_a);
+  token_scale(mb, sc_b, inv_b);
+#pragma unroll 5
+  for (int idx = lane; idx < nvec; idx += 32) {
+    qa.store(idx, quant_vec<EO>(ra[idx], inv_a));
+    if (has_b) qb.store(idx, quant_vec<EO>(rb[idx], inv_b));
+  }
+}
+
+}  // namespace dp

@@ -82,6 +82,13 @@ struct GemmProblem {
   int32_t early_w;  // the preceding kernel on the stream is this call's own DAQ: weights may be
                     // fetched before it has finished
   int32_t* status;
+  // In-kernel DAQ (x != nullptr): the GEMM kernel quantizes x into q_out / s_a_out (the buffers
+  // behind tmap_a and s_a) itself; sync = zeroed counters, one per 128-token tile plus one.
+  const uint16_t* x;
+  int64_t ldx;
+  int8_t* q_out;
+  float* s_a_out;
+  int32_t* sync;
 };
 // allow: bit 1 = single-CTA tiles permitted, bit 2 = CTA-pair tiles permitted
 void gemm_pick_tile(int64_t M, int32_t N, int32_t K, int32_t bits, uint32_t allow, int* bn_out, int* cg_out);

@@ -5,8 +5,7 @@
 
 #include <cuda_bf16.h>
 
-#include "dp_common.cuh"
-#include "dp_internal.h"
+#include "daq_device.cuh"
 
 namespace dp {
 
@@ -43,6 +42,16 @@ struct GemmParams {
   int64_t M;
   int32_t N, K;
   int32_t m_tiles, n_tiles;  // m_tiles counts row tiles of 128 * CG tokens
+  // In-kernel DAQ (x != nullptr): the kernel quantizes the bf16 activations itself, into the tiled
+  // scratch q_out / s_a_out that tmap_a and s_a refer to, and its CTAs tell each other through
+  // sync[] (one counter per 128-token tile, then one exit counter; all zero between kernels) which
+  // tiles are complete.
+  const uint16_t* x;
+  int64_t ldx;
+  int8_t* q_out;
+  float* s_a_out;
+  int32_t* sync;
+  int32_t sync_tiles;
   int32_t a_tiled;  // activations are stored as contiguous 128 x 128 tiles
   int32_t early_w;  // weights may be fetched before the preceding kernel on the stream has finished
   int32_t* status;
@@ -56,6 +65,67 @@ __device__ __forceinline__ void a_tile_coords(const GemmParams& p, int m_row, in
   } else {
     c0 = kb * BK;
     c1 = m_row;
+  }
+}
+
+// ---- in-kernel DAQ -------------------------------------------------------------------------------
+// Every CTA of the grid quantizes an equal share of the tokens (its 8 epilogue warps, one token per
+// warp at a time), publishes each finished token on the counter of its 128-token tile, and only
+// then turns to its GEMM tiles; the TMA producer of a tile first waits for that tile's counter.
+template <bool EO>
+__device__ __forceinline__ void daq_phase(const GemmParams& p, int epi_warp, int lane) {
+  const int64_t per_cta = (p.M + gridDim.x - 1) / gridDim.x;
+  const int64_t r0 = static_cast<int64_t>(blockIdx.x) * per_cta;
+  const int64_t r1 = r0 + per_cta < p.M ? r0 + per_cta : p.M;
+  const int kb = p.K / BK;
+  for (int64_t row = r0 + epi_warp; row < r1; row += 2 * kEpiWarps) {  // two tokens per round
+    const int64_t row_b = row + kEpiWarps;
+    const bool has_b = row_b < r1;
+    const QRow qa(p.q_out, row, 0, kb), qb(p.q_out, has_b ? row_b : row, 0, kb);
+    float sc_a, sc_b;
+    daq_two_rows_2pass<EO>(p.x + row * p.ldx, p.x + row_b * p.ldx, has_b, p.K, qa, qb, lane, sc_a, sc_b);
+    if (lane == 0) {
+      p.s_a_out[row] = sc_a;
+      if (has_b) p.s_a_out[row_b] = sc_b;
+    }
+    __syncwarp();
+    if (lane == 0) {
+      __threadfence();  // the tokens' codes and scales are visible device-wide before they are counted
+      if (has_b && (row_b >> 7) == (row >> 7)) {
+        atomicAdd(p.sync + (row >> 7), 2);
+      } else {
+        atomicAdd(p.sync + (row >> 7), 1);
+        if (has_b) atomicAdd(p.sync + (row_b >> 7), 1);
+      }
+    }
+  }
+}
+// One thread: until every token of 128-token tile `t` has been quantized (bounded).
+__device__ __forceinline__ bool wait_tile_quantized(const GemmParams& p, int t, volatile int* abort_flag) {
+  const int64_t left = p.M - static_cast<int64_t>(t) * BM;
+  const int expect = left >= BM ? BM : static_cast<int>(left);
+  if (expect <= 0) return true;  // a tile wholly past M: the loads read the fill value
+  const long long t0 = clock64();
+  uint32_t polls = 0;
+  while (ld_acquire_gpu(p.sync + t) < expect) {
+    if ((++polls & 15u) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitBudgetCycles) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+  fence_proxy_async_all();  // the codes were written with ordinary stores and are read by TMA next
+  return true;
+}
+// Last thing a CTA does (one thread, after all its roles have finished): count itself out; the last
+// CTA of the grid returns every counter to zero for the next kernel.
+__device__ __forceinline__ void daq_sync_exit(const GemmParams& p) {
+  __threadfence();
+  if (atomicAdd(p.sync + p.sync_tiles, 1) == static_cast<int>(gridDim.x) - 1) {
+    for (int i = 0; i <= p.sync_tiles; ++i) p.sync[i] = 0;
+    __threadfence();
   }
 }
 
@@ -189,10 +259,12 @@ struct EpilogueWarp {
     // it fetch its scales and biases with plain (non-broadcast) 8-byte shared loads.
     const int t4 = lane & 3, r8 = lane >> 2;
     float sa[4];
+    if (p.x == nullptr) {  // scales from an earlier kernel: fetch them while waiting for the accumulator
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int64_t row = static_cast<int64_t>(row0) + r8 + 8 * i;
-      sa[i] = row < p.M ? __ldg(p.s_a + row) : 0.0f;
+      for (int i = 0; i < 4; ++i) {
+        const int64_t row = static_cast<int64_t>(row0) + r8 + 8 * i;
+        sa[i] = row < p.M ? __ldg(p.s_a + row) : 0.0f;
+      }
     }
     if (n_blk != staged_n) {
       constexpr int NV = 2 * L::SLABS_LO;  // 32-column groups this warp may need
@@ -218,6 +290,14 @@ struct EpilogueWarp {
     ok = __all_sync(0xFFFFFFFFu, ok);
     if (!ok) return false;
     tc_fence_after();
+    if (p.x != nullptr) {  // scales written by other CTAs of this kernel: their tile is complete by now
+      (void)ld_acquire_gpu(p.sync + (cta_row0 >> 7));
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int64_t row = static_cast<int64_t>(row0) + r8 + 8 * i;
+        sa[i] = row < p.M ? *reinterpret_cast<const volatile float*>(p.s_a + row) : 0.0f;
+      }
+    }
     const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + t_cols;
     uint32_t* stage32 = reinterpret_cast<uint32_t*>(const_cast<uint4*>(stage4));
     for (int c = 2 * slab0; c < 2 * slab1; ++c) {  // 32-column chunks of this warp

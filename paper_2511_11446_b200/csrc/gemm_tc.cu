@@ -119,13 +119,15 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (lane == 0) {
       Ring st, ps;
       bool ok = true;
-      bool a_open = !p.early_w;  // false until griddepcontrol.wait has been executed
+      bool a_open = !p.early_w || p.x != nullptr;  // false until griddepcontrol.wait has been executed
+      int ready_tile = -1;                          // in-kernel DAQ: last 128-token tile seen complete
       int deferred = 0;          // stages whose weight tile is in flight but whose A tile is not
       int def_kb[NS], def_m[NS], def_s[NS];
       for (int tile = first_tile; tile < total_tiles && ok; tile += tile_stride) {
         const int n_blk = tile % p.n_tiles;  // column tiles of one row strip run together
         const int m_row = (tile / p.n_tiles) * (BM * CG) + static_cast<int>(rank) * BM;
         const int w_row = n_blk * BN + static_cast<int>(rank) * BNL;
+        bool a_ready = p.x == nullptr || (m_row >> 7) == ready_tile;
         for (int kb = 0; kb < KB; ++kb) {
           if (!a_open && deferred == NS) {  // ring full of weight tiles: now wait for the activations
             pdl_wait();
@@ -149,6 +151,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             ps.next(NP);
           }
           if (a_open) {
+            if (!a_ready) {  // weights of this stage are already in flight; now the tile's tokens
+              if (p.early_w && ready_tile < 0) pdl_wait();  // until the preceding kernel has exited the
+                                                           // counters still hold ITS tiles' counts
+              if (!(ok = wait_tile_quantized(p, m_row >> 7, abort_flag))) break;
+              ready_tile = m_row >> 7;
+              a_ready = true;
+            }
             int c0, c1;
             a_tile_coords(p, m_row, kb, c0, c1);
             tma_load_2d(sA + st.s * A_BYTES, &tmap_a, c0, c1, &full_a[st.s]);
@@ -241,9 +250,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     epi.init(warp, lane, s_scale, s_bias, sY,
              CG == 2 ? map_to_cta(&acc_empty[0], 0) : smem_u32(&acc_empty[0]),
              CG == 2 ? map_to_cta(&acc_empty[1], 0) : smem_u32(&acc_empty[1]));
+    if (p.x != nullptr) {  // quantize this CTA's share of the tokens first (all eight warps)
+      if (p.early_w) pdl_wait();  // x comes from the preceding kernel, whose GEMM may still read the scratch
+      daq_phase<PERM>(p, warp - kEpiWarp0, lane);
+    }
     bool ok = epi.active();
     int tcount = 0;
-    if (ok && p.early_w) pdl_wait();  // s_a is written by the preceding kernel
+    if (ok && p.early_w && p.x == nullptr) pdl_wait();  // s_a is written by the preceding kernel
     for (int tile = first_tile; tile < total_tiles && ok; tile += tile_stride, ++tcount) {
       const int buf = tcount & 1;
       ok = epi.tile(p, tile % p.n_tiles, (tile / p.n_tiles) * (BM * CG) + static_cast<int>(rank) * BM,
@@ -283,6 +296,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     else tmem_dealloc(tmem_base, TCOLS);
   }
   if (threadIdx.x == 0 && *abort_flag && p.status != nullptr) atomicExch(p.status, DP_ERR_TIMEOUT);
+  if (threadIdx.x == 0 && p.x != nullptr) daq_sync_exit(p);
 }
 
 // ---- host side -------------------------------------------------------------------------------------
@@ -451,6 +465,12 @@ int launch_gemm(const GemmProblem& g, cudaStream_t stream, bool pdl) {
   p.m_tiles = static_cast<int32_t>((g.M + BM * cg - 1) / (BM * cg));
   p.n_tiles = g.N / g.bn;
   p.a_tiled = g.a_tiled;
+  p.x = g.x;
+  p.ldx = g.ldx;
+  p.q_out = g.q_out;
+  p.s_a_out = g.s_a_out;
+  p.sync = g.sync;
+  p.sync_tiles = static_cast<int32_t>((g.M + BM - 1) / BM);
   p.early_w = (pdl && g.early_w) ? 1 : 0;
   p.status = g.status;
   const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;

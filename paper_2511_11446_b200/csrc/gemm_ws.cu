@@ -104,8 +104,8 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     // ================= TMA producer =================
     if (lane == 0) {
       Ring st, pr;
-      bool ok = true, a_open = !p.early_w;
-      int cur_strip = -1, strips = 0;
+      bool ok = true, a_open = !p.early_w || p.x != nullptr;
+      int cur_strip = -1, strips = 0, ready_tile = -1;
       for (int item = item0; item < item1 && ok; ++item) {
         const int strip = strip_of(item);
         if (strip != cur_strip) {
@@ -139,6 +139,12 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           a_open = true;
         }
         const int m_row = mtile_of(item) * (BM * CG) + static_cast<int>(rank) * BM;
+        if (p.x != nullptr && (m_row >> 7) != ready_tile) {  // in-kernel DAQ: this tile's tokens are quantized
+          if (p.early_w && ready_tile < 0) pdl_wait();  // until the preceding kernel has exited the counters
+                                                       // still hold ITS tiles' counts
+          if (!(ok = wait_tile_quantized(p, m_row >> 7, abort_flag))) break;
+          ready_tile = m_row >> 7;
+        }
         for (int kb = 0; kb < KB; ++kb) {
           if (!(ok = mbar_wait(&empty[st.s], st.ph ^ 1u, abort_flag))) break;
           mbar_arrive_expect_tx(&full_a[st.s], A_BYTES);
@@ -214,9 +220,13 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     // ================= epilogue =================
     EpilogueWarp<BN, SHIFT> epi;
     epi.init(warp, lane, s_scale, s_bias, sY, map_to_cta(&acc_empty[0], 0), map_to_cta(&acc_empty[1], 0));
+    if (p.x != nullptr) {  // quantize this CTA's share of the tokens first (all eight warps)
+      if (p.early_w) pdl_wait();
+      daq_phase<PERM>(p, warp - kEpiWarp0, lane);
+    }
     bool ok = epi.active();
     int tcount = 0;
-    if (ok && p.early_w) pdl_wait();  // s_a is written by the preceding kernel
+    if (ok && p.early_w && p.x == nullptr) pdl_wait();  // s_a is written by the preceding kernel
     for (int item = item0; item < item1 && ok; ++item, ++tcount) {
       const int buf = tcount & 1;
       ok = epi.tile(p, strip_of(item), mtile_of(item) * (BM * CG) + static_cast<int>(rank) * BM, tmem_base,
@@ -263,6 +273,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     tmem_dealloc_pair(tmem_base, TCOLS);
   }
   if (threadIdx.x == 0 && *abort_flag && p.status != nullptr) atomicExch(p.status, DP_ERR_TIMEOUT);
+  if (threadIdx.x == 0 && p.x != nullptr) daq_sync_exit(p);
 }
 
 // ---- host side -------------------------------------------------------------------------------------
@@ -337,6 +348,12 @@ int launch_gemm_ws(const GemmProblem& g, cudaStream_t stream, bool pdl) {
   p.m_tiles = static_cast<int32_t>((g.M + 2 * BM - 1) / (2 * BM));
   p.n_tiles = g.N / g.bn;
   p.a_tiled = g.a_tiled;
+  p.x = g.x;
+  p.ldx = g.ldx;
+  p.q_out = g.q_out;
+  p.s_a_out = g.s_a_out;
+  p.sync = g.sync;
+  p.sync_tiles = static_cast<int32_t>((g.M + BM - 1) / BM);
   p.early_w = (pdl && g.early_w) ? 1 : 0;
   p.status = g.status;
   const int64_t items = static_cast<int64_t>(p.m_tiles) * p.n_tiles;

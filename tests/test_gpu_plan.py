@@ -83,9 +83,11 @@ def test_plan_run_matches_oracle_every_step_and_layer():
         B.dp_plan_destroy(plan)
 
 
-def test_plan_autotuned_and_grouped_matches_oracle():
+@pytest.mark.parametrize("extra", [B.DP_FLAG_FUSED_DAQ, 0], ids=["daq_in_gemm", "daq_kernel"])
+def test_plan_autotuned_and_grouped_matches_oracle(extra):
     """Plan created with the on-device autotuner and with the small-M layers (adaLN) of a step
-    grouped into one launch: every output of every step still equals the oracle's."""
+    grouped into one launch, with DAQ inside the GEMM kernels or in its own kernel (default): every
+    output of every step still equals the oracle's."""
     table, layers, dev = _mini_plan(tokens=256, batch=3, blocks=3)
     T = 6
     kept = [1, 4, 5]
@@ -94,7 +96,7 @@ def test_plan_autotuned_and_grouped_matches_oracle():
            for l, L in enumerate(layers)] for t in kept]
     ref = oracle.plan_run(layers, kept, xs)
     plan = B.dp_plan_create([d.w for d in dev], [L["M"] for L in layers],
-                            B.DP_FLAG_AUTOTUNE | B.DP_FLAG_GROUP_SMALL_M)
+                            B.DP_FLAG_AUTOTUNE | B.DP_FLAG_GROUP_SMALL_M | extra)
     try:
         ws = torch.empty(B.dp_plan_workspace(plan), dtype=torch.uint8, device="cuda")
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
