@@ -216,6 +216,34 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const void* tmap, int c0,
         "r"(smem_u32(bar))
       : "memory");
 }
+// CTA-pair form: the copy lands in THIS CTA's shared memory but its bytes are counted on an mbarrier
+// that may live in the pair's other CTA (`cluster_bar` from map_to_cta). No multicast.
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const void* tmap, int c0, int c1, uint32_t cluster_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(cluster_bar)
+      : "memory");
+}
+// arrive + expect_tx on an mbarrier that may live in the pair's other CTA.
+__device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_bar), "r"(bytes) : "memory");
+}
+// Spinning (non-suspending) wait for one polling thread: lowest wake-up latency.
+__device__ __forceinline__ bool mbar_spin_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  const long long t0 = clock64();
+  uint32_t polls = 0;
+  while (!mbar_try_wait_cluster(bar, parity)) {
+    if ((++polls & 255u) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitBudgetCycles) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+  return true;
+}
 // 2-D tiled store shared -> global (bulk async-group completion). Rows past the tensor's extent
 // are clipped by the hardware. Coordinates are never negative here.
 __device__ __forceinline__ void tma_store_2d(const void* tmap, int c0, int c1, const void* src) {

@@ -72,10 +72,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   const int total_tiles = p.m_tiles * p.n_tiles;
   const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;  // 0 = leader of the pair
   const int first_tile = blockIdx.x / CG, tile_stride = gridDim.x / CG;
+  // TMA loads of operand stages: in a pair both CTAs' bytes are counted on the leader's barrier
+  auto stage_expect = [&](uint64_t* bar, uint32_t bytes) {
+    if constexpr (CG == 2) mbar_arrive_expect_tx_cluster(map_to_cta(bar, 0), bytes);
+    else mbar_arrive_expect_tx(bar, bytes);
+  };
+  auto stage_load = [&](void* dst, const CUtensorMap* tm, int c0, int c1, uint64_t* bar) {
+    if constexpr (CG == 2) tma_load_2d_pair(dst, tm, c0, c1, map_to_cta(bar, 0));
+    else tma_load_2d(dst, tm, c0, c1, bar);
+  };
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NS; ++i) {
-      mbar_init(&full_a[i], 1);
+      mbar_init(&full_a[i], CG);  // pair: the leader's copy counts both CTAs' TMA loads
       mbar_init(&bready[i], kUnpackThreads);
       mbar_init(&empty[i], 1);
       mbar_init(&peer_ready[i], 1);
@@ -135,19 +144,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             for (int d = 0; d < deferred; ++d) {
               int c0, c1;
               a_tile_coords(p, def_m[d], def_kb[d], c0, c1);
-              tma_load_2d(sA + def_s[d] * A_BYTES, &tmap_a, c0, c1, &full_a[def_s[d]]);
+              stage_load(sA + def_s[d] * A_BYTES, &tmap_a, c0, c1, &full_a[def_s[d]]);
             }
             deferred = 0;
           }
-          if (!(ok = mbar_wait(&empty[st.s], st.ph ^ 1u, abort_flag))) break;
+          if (!(ok = mbar_spin_wait(&empty[st.s], st.ph ^ 1u, abort_flag))) break;
           if constexpr (BITS == 8) {
-            mbar_arrive_expect_tx(&full_a[st.s], A_BYTES + B_BYTES);
-            tma_load_2d(sB + st.s * B_BYTES, &tmap_w, kb * BK, w_row, &full_a[st.s]);
+            stage_expect(&full_a[st.s], A_BYTES + B_BYTES);
+            stage_load(sB + st.s * B_BYTES, &tmap_w, kb * BK, w_row, &full_a[st.s]);
           } else {
             if (!(ok = mbar_wait(&pempty[ps.s], ps.ph ^ 1u, abort_flag))) break;
             mbar_arrive_expect_tx(&pfull[ps.s], P_BYTES);
             tma_load_2d(sP + ps.s * P_BYTES, &tmap_w, kb * (BK * BITS / 8), w_row, &pfull[ps.s]);
-            mbar_arrive_expect_tx(&full_a[st.s], A_BYTES);
+            stage_expect(&full_a[st.s], A_BYTES);
             ps.next(NP);
           }
           if (a_open) {
@@ -160,7 +169,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
             int c0, c1;
             a_tile_coords(p, m_row, kb, c0, c1);
-            tma_load_2d(sA + st.s * A_BYTES, &tmap_a, c0, c1, &full_a[st.s]);
+            stage_load(sA + st.s * A_BYTES, &tmap_a, c0, c1, &full_a[st.s]);
           } else {
             def_kb[deferred] = kb;
             def_m[deferred] = m_row;
@@ -175,7 +184,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         for (int d = 0; d < deferred; ++d) {
           int c0, c1;
           a_tile_coords(p, def_m[d], def_kb[d], c0, c1);
-          tma_load_2d(sA + def_s[d] * A_BYTES, &tmap_a, c0, c1, &full_a[def_s[d]]);
+          stage_load(sA + def_s[d] * A_BYTES, &tmap_a, c0, c1, &full_a[def_s[d]]);
         }
       }
       if (!ok) {
@@ -188,17 +197,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   } else if (warp == 1) {
     if (lane == 0) {
       if (CG == 2 && rank != 0) {
-        // ================= pair follower: report each loaded stage to the leader =================
-        Ring st;
-        bool ok = true;
-        for (int tile = first_tile; tile < total_tiles && ok; tile += tile_stride) {
-          for (int kb = 0; kb < KB; ++kb) {
-            if (!(ok = mbar_wait(&full_a[st.s], st.ph, abort_flag))) break;
-            if constexpr (BITS != 8) {
+        // ================= pair follower: report each expanded weight stage to the leader =================
+        // (TMA loads of both CTAs are counted on the leader's barrier directly)
+        if constexpr (BITS != 8) {
+          Ring st;
+          bool ok = true;
+          for (int tile = first_tile; tile < total_tiles && ok; tile += tile_stride) {
+            for (int kb = 0; kb < KB; ++kb) {
               if (!(ok = mbar_wait(&bready[st.s], st.ph, abort_flag))) break;
+              mbar_arrive_cluster(map_to_cta(&peer_ready[st.s], 0));
+              st.next(NS);
             }
-            mbar_arrive_cluster(map_to_cta(&peer_ready[st.s], 0));
-            st.next(NS);
           }
         }
       } else {
@@ -216,12 +225,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * (TCOLS / 2);
           for (int kb = 0; kb < KB; ++kb) {
-            if (!(ok = mbar_wait(&full_a[st.s], st.ph, abort_flag))) break;
+            if (!(ok = mbar_spin_wait(&full_a[st.s], st.ph, abort_flag))) break;
             if constexpr (BITS != 8) {
               if (!(ok = mbar_wait(&bready[st.s], st.ph, abort_flag))) break;
-            }
-            if constexpr (CG == 2) {
-              if (!(ok = mbar_wait_cluster(&peer_ready[st.s], st.ph, abort_flag))) break;
+              if constexpr (CG == 2) {
+                if (!(ok = mbar_wait_cluster(&peer_ready[st.s], st.ph, abort_flag))) break;
+              }
             }
             tc_fence_after();
             const uint64_t adesc = smem_desc_sw128(smem_u32(sA + st.s * A_BYTES));

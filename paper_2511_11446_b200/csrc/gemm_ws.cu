@@ -69,7 +69,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NS; ++i) {
-      mbar_init(&full_a[i], 1);
+      mbar_init(&full_a[i], CG);  // leader's copy: one arrival (+ bytes) from each CTA's producer
       mbar_init(&empty[i], 1);
       mbar_init(&peer_ready[i], 1);
       mbar_init(&pfull[i], 1);
@@ -146,11 +146,13 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           ready_tile = m_row >> 7;
         }
         for (int kb = 0; kb < KB; ++kb) {
-          if (!(ok = mbar_wait(&empty[st.s], st.ph ^ 1u, abort_flag))) break;
-          mbar_arrive_expect_tx(&full_a[st.s], A_BYTES);
+          if (!(ok = mbar_spin_wait(&empty[st.s], st.ph ^ 1u, abort_flag))) break;
+          // both CTAs' activation tiles are counted on the LEADER's barrier: the MMA thread waits once
+          const uint32_t bar = map_to_cta(&full_a[st.s], 0);
+          mbar_arrive_expect_tx_cluster(bar, A_BYTES);
           int c0, c1;
           a_tile_coords(p, m_row, kb, c0, c1);
-          tma_load_2d(sA + st.s * A_BYTES, &tmap_a, c0, c1, &full_a[st.s]);
+          tma_load_2d_pair(sA + st.s * A_BYTES, &tmap_a, c0, c1, bar);
           st.next(NS);
         }
       }
@@ -163,8 +165,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   } else if (warp == 1) {
     if (lane == 0) {
       if (rank != 0) {
-        // ================= pair follower: report the strip and each loaded stage to the leader =================
-        Ring st;
+        // ================= pair follower: report each resident strip to the leader =================
         bool ok = true;
         int cur_strip = -1, strips = 0;
         for (int item = item0; item < item1 && ok; ++item) {
@@ -174,11 +175,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             cur_strip = strip_of(item);
             ++strips;
           }
-          for (int kb = 0; kb < KB; ++kb) {
-            if (!(ok = mbar_wait(&full_a[st.s], st.ph, abort_flag))) break;
-            mbar_arrive_cluster(map_to_cta(&peer_ready[st.s], 0));
-            st.next(NS);
-          }
+
         }
       } else {
         // ================= MMA issuer =================
@@ -199,8 +196,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * (TCOLS / 2);
           for (int kb = 0; kb < KB; ++kb) {
-            if (!(ok = mbar_wait(&full_a[st.s], st.ph, abort_flag))) break;
-            if (!(ok = mbar_wait_cluster(&peer_ready[st.s], st.ph, abort_flag))) break;
+            if (!(ok = mbar_spin_wait(&full_a[st.s], st.ph, abort_flag))) break;  // both CTAs' tiles landed
             tc_fence_after();
             const uint64_t adesc = smem_desc_sw128(smem_u32(sA + st.s * A_BYTES));
             const uint64_t bdesc = smem_desc_sw128(smem_u32(sW + kb * B_BYTES));
