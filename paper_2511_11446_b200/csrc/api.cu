@@ -53,7 +53,7 @@ static size_t scratch_q_bytes(int64_t M, int32_t K) { return static_cast<size_t>
 constexpr uint32_t kLinearFlags =
     DP_FLAG_FORCE_SIMT | DP_FLAG_FORCE_MMA | DP_FLAG_NO_PDL | DP_FLAG_TILE_N_MASK | DP_FLAG_CTA_PAIR |
     DP_FLAG_NO_CTA_PAIR | DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_NO_WEIGHT_STATIONARY;
-constexpr int64_t kWsMinRows = 4096;  // from here on a resident weight strip is reused often enough to pay
+constexpr int64_t kWsMinRows = 8192;  // from here on a resident weight strip is reused often enough to pay
 static int forced_bn(uint32_t flags) { return static_cast<int>((flags & DP_FLAG_TILE_N_MASK) >> 8) * 64; }
 
 // Tile width and CTA-group size of the tensor-core kernel for this problem, honouring the tuning

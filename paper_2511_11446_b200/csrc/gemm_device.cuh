@@ -16,7 +16,9 @@ constexpr int kUnpackThreads = kUnpackWarps * 32;
 __host__ __device__ constexpr int gemm_threads(int bits) {
   return (kUnpackWarp0 + (bits == 8 ? 0 : kUnpackWarps)) * 32;
 }
-constexpr int kYStageBytes = 32 * 64;  // per epilogue warp: 32 tokens x 32 bf16
+// Output staging per epilogue warp: 32 tokens x CW bf16 (CW = columns handled per round: 32, or 16
+// where shared memory is short).
+__host__ __device__ constexpr int y_stage_bytes(int cw) { return 32 * cw * 2; }
 constexpr int kSmemBudget = 200 * 1024;
 constexpr int kPStages = 3;
 
@@ -221,7 +223,7 @@ struct EpiLayout {
   static constexpr int SCALE_FLOATS = kEpiWarps * 64 * SLABS_LO;         // per array (scales, biases)
 };
 
-template <int BN, int SHIFT>
+template <int BN, int SHIFT, int CW = 32>
 struct EpilogueWarp {
   using L = EpiLayout<BN>;
   int qd, slab0, slab1, lane, staged_n;
@@ -238,7 +240,7 @@ struct EpilogueWarp {
     slab1 = ew < 4 ? L::SLABS_LO : L::SLABS;
     ts = s_scale + ew * 64 * L::SLABS_LO;
     tb = s_bias + ew * 64 * L::SLABS_LO;
-    uint8_t* stage = sY + ew * kYStageBytes;
+    uint8_t* stage = sY + ew * y_stage_bytes(CW);
     stage4 = reinterpret_cast<const uint4*>(stage);
     acc_empty_addr[0] = acc_empty0;
     acc_empty_addr[1] = acc_empty1;
@@ -300,62 +302,123 @@ struct EpilogueWarp {
     }
     const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + t_cols;
     uint32_t* stage32 = reinterpret_cast<uint32_t*>(const_cast<uint4*>(stage4));
-    for (int c = 2 * slab0; c < 2 * slab1; ++c) {  // 32-column chunks of this warp
-      const int lc = (c - 2 * slab0) * 32 + 2 * t4;  // this thread's first column inside the staged scales
+    if constexpr (CW == 32) {
+      for (int c = 2 * slab0; c < 2 * slab1; ++c) {  // 32-column chunks of this warp
+        const int lc = (c - 2 * slab0) * 32 + 2 * t4;  // this thread's first column inside the staged scales
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {  // tokens r8 + 16 h and r8 + 16 h + 8
-        uint32_t r[16];
-        tmem_ld_16x256b_x4(t_addr + (static_cast<uint32_t>(16 * h) << 16) + c * 32, r);
-        tmem_ld_wait();
-        if (h == 1 && c + 1 == 2 * slab1) {  // this warp's last accumulators are in registers
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(acc_empty_addr[buf]);
-        }
-        // staging tile [32 tokens][64 bytes], 16-byte chunks XOR-swizzled by ((token >> 1) & 3): these
-        // 4-byte stores and the 16-byte row-wise read-back below are both free of bank conflicts
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float2 sw = *reinterpret_cast<const float2*>(ts + lc + 8 * j);
-          const float2 bb = *reinterpret_cast<const float2*>(tb + lc + 8 * j);
-#pragma unroll
-          for (int i = 0; i < 2; ++i) {
-            const int rr = r8 + 16 * h + 8 * i;
-            const float s = sa[2 * h + i];
-            const __nv_bfloat162 v = __floats2bfloat162_rn(dequant_one<SHIFT>(r[4 * j + 2 * i], s, sw.x, bb.x),
-                                                           dequant_one<SHIFT>(r[4 * j + 2 * i + 1], s, sw.y, bb.y));
-            stage32[rr * 16 + ((j ^ ((rr >> 1) & 3)) << 2) + t4] = *reinterpret_cast<const uint32_t*>(&v);
+        for (int h = 0; h < 2; ++h) {  // tokens r8 + 16 h and r8 + 16 h + 8
+          uint32_t r[16];
+          tmem_ld_16x256b_x4(t_addr + (static_cast<uint32_t>(16 * h) << 16) + c * 32, r);
+          tmem_ld_wait();
+          if (h == 1 && c + 1 == 2 * slab1) {  // this warp's last accumulators are in registers
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(acc_empty_addr[buf]);
           }
-        }
-        if (p.dbg_acc != nullptr) {
+          // staging tile [32 tokens][64 bytes], 16-byte chunks XOR-swizzled by ((token >> 1) & 3): these
+          // 4-byte stores and the 16-byte row-wise read-back below are both free of bank conflicts
 #pragma unroll
-          for (int i = 0; i < 2; ++i) {
-            const int64_t row = static_cast<int64_t>(row0) + r8 + 16 * h + 8 * i;
-            if (row < p.M) {
-              int32_t* arow = p.dbg_acc + row * p.dbg_ldacc + n0 + c * 32 + 2 * t4;
+          for (int j = 0; j < 4; ++j) {
+            const float2 sw = *reinterpret_cast<const float2*>(ts + lc + 8 * j);
+            const float2 bb = *reinterpret_cast<const float2*>(tb + lc + 8 * j);
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                arow[8 * j] = static_cast<int>(r[4 * j + 2 * i]) >> SHIFT;
-                arow[8 * j + 1] = static_cast<int>(r[4 * j + 2 * i + 1]) >> SHIFT;
+            for (int i = 0; i < 2; ++i) {
+              const int rr = r8 + 16 * h + 8 * i;
+              const float s = sa[2 * h + i];
+              const __nv_bfloat162 v = __floats2bfloat162_rn(dequant_one<SHIFT>(r[4 * j + 2 * i], s, sw.x, bb.x),
+                                                             dequant_one<SHIFT>(r[4 * j + 2 * i + 1], s, sw.y, bb.y));
+              stage32[rr * 16 + ((j ^ ((rr >> 1) & 3)) << 2) + t4] = *reinterpret_cast<const uint32_t*>(&v);
+            }
+          }
+          if (p.dbg_acc != nullptr) {
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+              const int64_t row = static_cast<int64_t>(row0) + r8 + 16 * h + 8 * i;
+              if (row < p.M) {
+                int32_t* arow = p.dbg_acc + row * p.dbg_ldacc + n0 + c * 32 + 2 * t4;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  arow[8 * j] = static_cast<int>(r[4 * j + 2 * i]) >> SHIFT;
+                  arow[8 * j + 1] = static_cast<int>(r[4 * j + 2 * i + 1]) >> SHIFT;
+                }
               }
             }
           }
         }
-      }
-      __syncwarp();
-      // staged chunk -> global: every store instruction covers eight 64-byte row segments
-      {
-        const int ch = lane & 3;
-        uint16_t* ycol = p.y + n0 + c * 32 + ch * 8;
+        __syncwarp();
+        // staged chunk -> global: every store instruction covers eight 64-byte row segments
+        {
+          const int ch = lane & 3;
+          uint16_t* ycol = p.y + n0 + c * 32 + ch * 8;
 #pragma unroll
-        for (int it = 0; it < 4; ++it) {
-          const int rr = 8 * it + (lane >> 2);
-          const uint4 v = stage4[rr * 4 + (ch ^ ((rr >> 1) & 3))];
-          const int64_t grow = static_cast<int64_t>(row0) + rr;
-          if (grow < p.M) *reinterpret_cast<uint4*>(ycol + grow * p.ldy) = v;
+          for (int it = 0; it < 4; ++it) {
+            const int rr = 8 * it + (lane >> 2);
+            const uint4 v = stage4[rr * 4 + (ch ^ ((rr >> 1) & 3))];
+            const int64_t grow = static_cast<int64_t>(row0) + rr;
+            if (grow < p.M) *reinterpret_cast<uint4*>(ycol + grow * p.ldy) = v;
+          }
         }
+        __syncwarp();  // the staging tile is rewritten by the next chunk
       }
-      __syncwarp();  // the staging tile is rewritten by the next chunk
+    } else {
+      for (int c = 4 * slab0; c < 4 * slab1; ++c) {  // 16-column chunks of this warp
+        const int lc = (c - 4 * slab0) * 16 + 2 * t4;  // this thread's first column inside the staged scales
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {  // tokens r8 + 16 h and r8 + 16 h + 8
+          uint32_t r[8];
+          tmem_ld_16x256b_x2(t_addr + (static_cast<uint32_t>(16 * h) << 16) + c * 16, r);
+          tmem_ld_wait();
+          if (h == 1 && c + 1 == 4 * slab1) {  // this warp's last accumulators are in registers
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(acc_empty_addr[buf]);
+          }
+          // staging tile [32 tokens][32 bytes], the two 16-byte halves of a row swapped for tokens with
+          // bit 2 set: these 4-byte stores and the 16-byte row-wise read-back below are both free of
+          // bank conflicts
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const float2 sw = *reinterpret_cast<const float2*>(ts + lc + 8 * j);
+            const float2 bb = *reinterpret_cast<const float2*>(tb + lc + 8 * j);
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+              const int rr = r8 + 16 * h + 8 * i;
+              const float s = sa[2 * h + i];
+              const __nv_bfloat162 v = __floats2bfloat162_rn(dequant_one<SHIFT>(r[4 * j + 2 * i], s, sw.x, bb.x),
+                                                             dequant_one<SHIFT>(r[4 * j + 2 * i + 1], s, sw.y, bb.y));
+              stage32[rr * 8 + ((j ^ ((rr >> 2) & 1)) << 2) + t4] = *reinterpret_cast<const uint32_t*>(&v);
+            }
+          }
+          if (p.dbg_acc != nullptr) {
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+              const int64_t row = static_cast<int64_t>(row0) + r8 + 16 * h + 8 * i;
+              if (row < p.M) {
+                int32_t* arow = p.dbg_acc + row * p.dbg_ldacc + n0 + c * 16 + 2 * t4;
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                  arow[8 * j] = static_cast<int>(r[4 * j + 2 * i]) >> SHIFT;
+                  arow[8 * j + 1] = static_cast<int>(r[4 * j + 2 * i + 1]) >> SHIFT;
+                }
+              }
+            }
+          }
+        }
+        __syncwarp();
+        // staged chunk -> global: every store instruction covers sixteen 32-byte row segments
+        {
+          const int ch = lane & 1;
+          uint16_t* ycol = p.y + n0 + c * 16 + ch * 8;
+#pragma unroll
+          for (int it = 0; it < 2; ++it) {
+            const int rr = 16 * it + (lane >> 1);
+            const uint4 v = stage4[rr * 2 + (ch ^ ((rr >> 2) & 1))];
+            const int64_t grow = static_cast<int64_t>(row0) + rr;
+            if (grow < p.M) *reinterpret_cast<uint4*>(ycol + grow * p.ldy) = v;
+          }
+        }
+        __syncwarp();  // the staging tile is rewritten by the next chunk
+      }
     }
     return true;
   }

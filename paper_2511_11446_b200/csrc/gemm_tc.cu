@@ -51,7 +51,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint8_t* sB = sA + NS * A_BYTES;
   uint8_t* sP = sB + NS * B_BYTES;
   uint8_t* sY = sP + NP * P_BYTES;  // [epilogue warps][32 tokens][64 bytes] output staging
-  uint8_t* tail = sY + kEpiWarps * kYStageBytes;
+  uint8_t* tail = sY + kEpiWarps * y_stage_bytes(32);
   uint64_t* full_a = reinterpret_cast<uint64_t*>(tail);
   uint64_t* bready = full_a + NS;
   uint64_t* empty = bready + NS;
@@ -312,7 +312,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 template <int BN, int BITS, int CG>
 constexpr size_t gemm_smem_bytes() {
   return 1024 + static_cast<size_t>(num_stages(BN / CG, BITS)) * ab_stage_bytes(BN / CG) +
-         kPStages * p_stage_bytes(BN / CG, BITS) + kEpiWarps * kYStageBytes +
+         kPStages * p_stage_bytes(BN / CG, BITS) + kEpiWarps * y_stage_bytes(32) +
          (4 * 8 + 2 * kPStages + 4) * 8 + 32 + 2 * kEpiWarps * 64 * ((BN / 64 + 1) / 2) * 4 + 64;
 }
 

@@ -21,7 +21,10 @@ namespace dp {
 
 constexpr int kWsMaxKB = 9;   // k-blocks of 128 a resident strip may have (K <= 1152)
 // Activation ring depth: what is left of shared memory beside the resident strip.
-__host__ __device__ constexpr int ws_stages(int bn) { return bn >= 256 ? 3 : 5; }
+// At BN = 256 the epilogue works in 16-column rounds (half the staging memory) to make room for a
+// fourth stage.
+__host__ __device__ constexpr int ws_epi_cols(int bn) { return bn >= 256 ? 16 : 32; }
+__host__ __device__ constexpr int ws_stages(int bn) { return bn >= 256 ? 4 : 5; }
 
 template <int BN, int BITS, bool PERM>
 __global__ void __launch_bounds__(gemm_threads(BITS), 1)
@@ -40,7 +43,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint8_t* sW = smem;                            // [KB][BNL][128] int8, 128-byte swizzled: the strip
   uint8_t* sA = sW + kWsMaxKB * B_BYTES;         // activation ring (and packed-tile staging)
   uint8_t* sY = sA + NS * A_BYTES;
-  uint8_t* tail = sY + kEpiWarps * kYStageBytes;
+  uint8_t* tail = sY + kEpiWarps * y_stage_bytes(ws_epi_cols(BN));
   uint64_t* full_a = reinterpret_cast<uint64_t*>(tail);
   uint64_t* empty = full_a + NS;
   uint64_t* peer_ready = empty + NS;  // leader only
@@ -214,7 +217,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
   } else if (warp < kUnpackWarp0) {
     // ================= epilogue =================
-    EpilogueWarp<BN, SHIFT> epi;
+    EpilogueWarp<BN, SHIFT, ws_epi_cols(BN)> epi;
     epi.init(warp, lane, s_scale, s_bias, sY, map_to_cta(&acc_empty[0], 0), map_to_cta(&acc_empty[1], 0));
     if (p.x != nullptr) {  // quantize this CTA's share of the tokens first (all eight warps)
       if (p.early_w) pdl_wait();
@@ -275,7 +278,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 // ---- host side -------------------------------------------------------------------------------------
 template <int BN>
 constexpr size_t ws_smem_bytes() {
-  return 1024 + static_cast<size_t>(kWsMaxKB) * (BN / 2) * BK + ws_stages(BN) * BM * BK + kEpiWarps * kYStageBytes +
+  return 1024 + static_cast<size_t>(kWsMaxKB) * (BN / 2) * BK + ws_stages(BN) * BM * BK + kEpiWarps * y_stage_bytes(ws_epi_cols(BN)) +
          (5 * ws_stages(BN) + 4 + 3) * 8 + 32 + 2 * EpiLayout<BN>::SCALE_FLOATS * 4 + 64;
 }
 
