@@ -86,7 +86,7 @@ static int check_tile_flags(uint32_t flags, int32_t N) {
   if (fb != 0 && (fb > 256 || N % fb)) return fail(DP_ERR_SHAPE, "forced tile width %d does not divide N=%d", fb, N);
   if ((flags & DP_FLAG_CTA_PAIR) && (flags & DP_FLAG_NO_CTA_PAIR))
     return fail(DP_ERR_INVALID_ARG, "CTA_PAIR and NO_CTA_PAIR are exclusive");
-  if ((flags & DP_FLAG_CTA_PAIR) && ((fb != 0 && fb < 128) || N % 128))
+  if ((flags & DP_FLAG_CTA_PAIR) && ((fb != 0 && fb < 128) || (N % 128 && N % 192)))
     return fail(DP_ERR_SHAPE, "CTA-pair tiles need a tile width of 128, 192 or 256 dividing N=%d", N);
   if ((flags & DP_FLAG_WEIGHT_STATIONARY) && (flags & (DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_NO_CTA_PAIR)))
     return fail(DP_ERR_INVALID_ARG, "WEIGHT_STATIONARY contradicts another flag");
@@ -466,7 +466,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
     }
     if (!L.simt && L.M > 0) {
       uint32_t lf = flags;  // a pair request that this layer's N cannot honour falls back to the default
-      if ((lf & DP_FLAG_CTA_PAIR) && L.w.N % 128) lf &= ~DP_FLAG_CTA_PAIR;
+      if ((lf & DP_FLAG_CTA_PAIR) && L.w.N % 128 && L.w.N % 192) lf &= ~DP_FLAG_CTA_PAIR;
       if ((lf & DP_FLAG_WEIGHT_STATIONARY) && !gemm_ws_supported(L.w.N, L.w.K)) lf &= ~DP_FLAG_WEIGHT_STATIONARY;
       choose_tile(lf, L.M, L.w.N, L.w.K, L.w.bits, &L.bn, &L.cg, &L.ws);
       if (autotune) {

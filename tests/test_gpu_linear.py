@@ -171,6 +171,43 @@ def test_mma_extreme_accumulators(bits):
     _check(out, x, w, s_w, None, bits)
 
 
+@pytest.mark.parametrize("variant", [B.DP_FLAG_NO_CTA_PAIR, B.DP_FLAG_CTA_PAIR | B.DP_FLAG_NO_WEIGHT_STATIONARY,
+                                     B.DP_FLAG_WEIGHT_STATIONARY, B.DP_FLAG_FORCE_SIMT],
+                         ids=["single", "pair", "weight_stationary", "small_m_kernel"])
+def test_padded_row_pitches_and_untouched_padding(variant):
+    """x with ldx > K and y with ldy > N: the padding columns of y keep their contents, rows past M
+    are not written, and the result equals the oracle's."""
+    simt = variant == B.DP_FLAG_FORCE_SIMT
+    M, K, N, bits = (20 if simt else 300), 256, 384, 4
+    ldx, ldy, rows_alloc = K + 64, N + 40, M + 7
+    x, w, s_w, b = _case(M, K, N, bits)
+    L = DevLayer(w, s_w, b, bits)
+    xp = np.full((M, ldx), 0x7FC0, np.uint16)  # NaN in the padding: must never be read into the result
+    xp[:, :K] = x
+    xd = torch.from_numpy(xp.view(np.int16).copy()).cuda().view(torch.bfloat16)
+    y = torch.full((rows_alloc, ldy), 3.0, dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(B.dp_wq_linear_workspace(M, N, K, bits, variant), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    flags = variant if simt else (variant | B.DP_FLAG_FORCE_MMA)
+    B.dp_wq_linear(L.w, xd, ldx, None, M, y, ldy, ws, None, status, flags)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    got = y.view(torch.int16).cpu().numpy().view(np.uint16)
+    ref = oracle.wq_linear(x, oracle.pack(w, bits), s_w, b, bits)
+    assert bf16_ulp_dist(got[:M, :N], ref).max() <= 1
+    assert np.all(got[:M, N:] == 0x4040) and np.all(got[M:, :] == 0x4040)  # bf16(3.0) untouched
+
+
+def test_single_token_and_minimal_k_through_the_tensor_core_path():
+    """M = 1 (one live row in a 128-row tile) and the smallest K (one k-block) on every variant."""
+    for variant in (B.DP_FLAG_NO_CTA_PAIR, B.DP_FLAG_CTA_PAIR | B.DP_FLAG_NO_WEIGHT_STATIONARY,
+                    B.DP_FLAG_WEIGHT_STATIONARY):
+        for bits in (8, 3):
+            x, w, s_w, b = _case(1, 128, 192, bits, full_range=True)
+            L = DevLayer(w, s_w, b, bits)
+            _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | variant), x, w, s_w, b, bits, exact_y=False)
+
+
 @pytest.mark.parametrize("flags", [B.DP_FLAG_FORCE_SIMT, B.DP_FLAG_FORCE_MMA])
 def test_prequantized_input(flags):
     M, K, N, bits = 130, 256, 128, 4
