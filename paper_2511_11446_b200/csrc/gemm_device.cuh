@@ -302,123 +302,77 @@ struct EpilogueWarp {
     }
     const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + t_cols;
     uint32_t* stage32 = reinterpret_cast<uint32_t*>(const_cast<uint4*>(stage4));
-    if constexpr (CW == 32) {
-      for (int c = 2 * slab0; c < 2 * slab1; ++c) {  // 32-column chunks of this warp
-        const int lc = (c - 2 * slab0) * 32 + 2 * t4;  // this thread's first column inside the staged scales
+    // Rounds of CW columns. Per round the warp reads its two 16-token halves from tensor memory (the
+    // next read is in flight while the current one is converted), writes bf16 pairs into its staging
+    // tile [32 tokens][CW * 2 bytes] and copies the tile out row-wise. The staging tile's 16-byte
+    // chunks are XOR-swizzled by the token index so that both the 4-byte writes and the 16-byte
+    // row-wise read-back are free of bank conflicts.
+    constexpr int G = CW / 8;  // 8-column groups per round = 16-byte chunks per staged row
+    auto swz = [](int rr) { return CW == 32 ? ((rr >> 1) & 3) : ((rr >> 2) & 1); };
+    auto tload = [&](int c, int h, uint32_t (&r)[4 * G]) {
+      const uint32_t addr = t_addr + (static_cast<uint32_t>(16 * h) << 16) + c * CW;
+      if constexpr (G == 4) tmem_ld_16x256b_x4(addr, r);
+      else tmem_ld_16x256b_x2(addr, r);
+    };
+    auto convert = [&](const uint32_t (&r)[4 * G], int c, int h, int lc) {  // tokens r8 + 16 h, r8 + 16 h + 8
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {  // tokens r8 + 16 h and r8 + 16 h + 8
-          uint32_t r[16];
-          tmem_ld_16x256b_x4(t_addr + (static_cast<uint32_t>(16 * h) << 16) + c * 32, r);
-          tmem_ld_wait();
-          if (h == 1 && c + 1 == 2 * slab1) {  // this warp's last accumulators are in registers
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(acc_empty_addr[buf]);
-          }
-          // staging tile [32 tokens][64 bytes], 16-byte chunks XOR-swizzled by ((token >> 1) & 3): these
-          // 4-byte stores and the 16-byte row-wise read-back below are both free of bank conflicts
+      for (int j = 0; j < G; ++j) {
+        const float2 sw = *reinterpret_cast<const float2*>(ts + lc + 8 * j);
+        const float2 bb = *reinterpret_cast<const float2*>(tb + lc + 8 * j);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float2 sw = *reinterpret_cast<const float2*>(ts + lc + 8 * j);
-            const float2 bb = *reinterpret_cast<const float2*>(tb + lc + 8 * j);
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-              const int rr = r8 + 16 * h + 8 * i;
-              const float s = sa[2 * h + i];
-              const __nv_bfloat162 v = __floats2bfloat162_rn(dequant_one<SHIFT>(r[4 * j + 2 * i], s, sw.x, bb.x),
-                                                             dequant_one<SHIFT>(r[4 * j + 2 * i + 1], s, sw.y, bb.y));
-              stage32[rr * 16 + ((j ^ ((rr >> 1) & 3)) << 2) + t4] = *reinterpret_cast<const uint32_t*>(&v);
-            }
-          }
-          if (p.dbg_acc != nullptr) {
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-              const int64_t row = static_cast<int64_t>(row0) + r8 + 16 * h + 8 * i;
-              if (row < p.M) {
-                int32_t* arow = p.dbg_acc + row * p.dbg_ldacc + n0 + c * 32 + 2 * t4;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  arow[8 * j] = static_cast<int>(r[4 * j + 2 * i]) >> SHIFT;
-                  arow[8 * j + 1] = static_cast<int>(r[4 * j + 2 * i + 1]) >> SHIFT;
-                }
-              }
-            }
-          }
+        for (int i = 0; i < 2; ++i) {
+          const int rr = r8 + 16 * h + 8 * i;
+          const float s = sa[2 * h + i];
+          const __nv_bfloat162 v = __floats2bfloat162_rn(dequant_one<SHIFT>(r[4 * j + 2 * i], s, sw.x, bb.x),
+                                                         dequant_one<SHIFT>(r[4 * j + 2 * i + 1], s, sw.y, bb.y));
+          stage32[rr * (4 * G) + ((j ^ swz(rr)) << 2) + t4] = *reinterpret_cast<const uint32_t*>(&v);
         }
-        __syncwarp();
-        // staged chunk -> global: every store instruction covers eight 64-byte row segments
-        {
-          const int ch = lane & 3;
-          uint16_t* ycol = p.y + n0 + c * 32 + ch * 8;
-#pragma unroll
-          for (int it = 0; it < 4; ++it) {
-            const int rr = 8 * it + (lane >> 2);
-            const uint4 v = stage4[rr * 4 + (ch ^ ((rr >> 1) & 3))];
-            const int64_t grow = static_cast<int64_t>(row0) + rr;
-            if (grow < p.M) *reinterpret_cast<uint4*>(ycol + grow * p.ldy) = v;
-          }
-        }
-        __syncwarp();  // the staging tile is rewritten by the next chunk
       }
-    } else {
-      for (int c = 4 * slab0; c < 4 * slab1; ++c) {  // 16-column chunks of this warp
-        const int lc = (c - 4 * slab0) * 16 + 2 * t4;  // this thread's first column inside the staged scales
+      if (p.dbg_acc != nullptr) {
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {  // tokens r8 + 16 h and r8 + 16 h + 8
-          uint32_t r[8];
-          tmem_ld_16x256b_x2(t_addr + (static_cast<uint32_t>(16 * h) << 16) + c * 16, r);
-          tmem_ld_wait();
-          if (h == 1 && c + 1 == 4 * slab1) {  // this warp's last accumulators are in registers
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(acc_empty_addr[buf]);
-          }
-          // staging tile [32 tokens][32 bytes], the two 16-byte halves of a row swapped for tokens with
-          // bit 2 set: these 4-byte stores and the 16-byte row-wise read-back below are both free of
-          // bank conflicts
+        for (int i = 0; i < 2; ++i) {
+          const int64_t row = static_cast<int64_t>(row0) + r8 + 16 * h + 8 * i;
+          if (row < p.M) {
+            int32_t* arow = p.dbg_acc + row * p.dbg_ldacc + n0 + c * CW + 2 * t4;
 #pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const float2 sw = *reinterpret_cast<const float2*>(ts + lc + 8 * j);
-            const float2 bb = *reinterpret_cast<const float2*>(tb + lc + 8 * j);
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-              const int rr = r8 + 16 * h + 8 * i;
-              const float s = sa[2 * h + i];
-              const __nv_bfloat162 v = __floats2bfloat162_rn(dequant_one<SHIFT>(r[4 * j + 2 * i], s, sw.x, bb.x),
-                                                             dequant_one<SHIFT>(r[4 * j + 2 * i + 1], s, sw.y, bb.y));
-              stage32[rr * 8 + ((j ^ ((rr >> 2) & 1)) << 2) + t4] = *reinterpret_cast<const uint32_t*>(&v);
-            }
-          }
-          if (p.dbg_acc != nullptr) {
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-              const int64_t row = static_cast<int64_t>(row0) + r8 + 16 * h + 8 * i;
-              if (row < p.M) {
-                int32_t* arow = p.dbg_acc + row * p.dbg_ldacc + n0 + c * 16 + 2 * t4;
-#pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                  arow[8 * j] = static_cast<int>(r[4 * j + 2 * i]) >> SHIFT;
-                  arow[8 * j + 1] = static_cast<int>(r[4 * j + 2 * i + 1]) >> SHIFT;
-                }
-              }
+            for (int j = 0; j < G; ++j) {
+              arow[8 * j] = static_cast<int>(r[4 * j + 2 * i]) >> SHIFT;
+              arow[8 * j + 1] = static_cast<int>(r[4 * j + 2 * i + 1]) >> SHIFT;
             }
           }
         }
-        __syncwarp();
-        // staged chunk -> global: every store instruction covers sixteen 32-byte row segments
-        {
-          const int ch = lane & 1;
-          uint16_t* ycol = p.y + n0 + c * 16 + ch * 8;
-#pragma unroll
-          for (int it = 0; it < 2; ++it) {
-            const int rr = 16 * it + (lane >> 1);
-            const uint4 v = stage4[rr * 2 + (ch ^ ((rr >> 2) & 1))];
-            const int64_t grow = static_cast<int64_t>(row0) + rr;
-            if (grow < p.M) *reinterpret_cast<uint4*>(ycol + grow * p.ldy) = v;
-          }
-        }
-        __syncwarp();  // the staging tile is rewritten by the next chunk
       }
+    };
+    const int c_begin = (64 / CW) * slab0, c_end = (64 / CW) * slab1;
+    uint32_t ra[4 * G], rb[4 * G];
+    tload(c_begin, 0, ra);
+    for (int c = c_begin; c < c_end; ++c) {
+      const int lc = (c - c_begin) * CW + 2 * t4;  // this thread's first column inside the staged scales
+      tmem_ld_wait();
+      tload(c, 1, rb);
+      convert(ra, c, 0, lc);
+      tmem_ld_wait();
+      if (c + 1 < c_end) {
+        tload(c + 1, 0, ra);
+      } else {  // this warp's last accumulators are in registers: hand the buffer back
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(acc_empty_addr[buf]);
+      }
+      convert(rb, c, 1, lc);
+      __syncwarp();
+      {  // staged round -> global: every store instruction covers whole row segments of CW * 2 bytes
+        const int ch = lane % G;
+        uint16_t* ycol = p.y + n0 + c * CW + ch * 8;
+#pragma unroll
+        for (int it = 0; it < G; ++it) {
+          const int rr = it * (32 / G) + lane / G;
+          const uint4 v = stage4[rr * G + (ch ^ swz(rr))];
+          const int64_t grow = static_cast<int64_t>(row0) + rr;
+          if (grow < p.M) *reinterpret_cast<uint4*>(ycol + grow * p.ldy) = v;
+        }
+      }
+      __syncwarp();  // the staging tile is rewritten by the next round
     }
     return true;
   }
