@@ -210,6 +210,7 @@ def run_ours(args):
                                 "int8_peak_tops_used": int8_peak, "hbm_gbs_used": peaks["hbm_gbs"],
                                 "peaks": peaks["source"]}
         out["mma_i8_peak_tops_measured"] = measure_mma_peak()
+        out["roofline_hbm_kernels"] = hbm_kernel_rooflines(stack, peaks)
         out["e2e"] = e2e(stack, ops_step, world)
         tops, dt, desc, cores = oracle_sample()
         out["cpu_baseline"] = {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
@@ -272,6 +273,64 @@ def gemm_roofline(stack, peaks):
             "frac_of_nominal": achieved / NOMINAL_INT8_TOPS, "launches": len(idx),
             "avg_launch_us": 1e3 * ms / len(idx), "variants": dict(variants),
             "traffic": GEMM_DRAM_BYTES_PER_LAUNCH}
+
+
+def hbm_kernel_rooflines(stack, peaks):
+    """The HBM-bound kernels of the path against the measured copy bandwidth: (a) the adaLN
+    modulation linears of one timestep (28 layers, M = batch, mixed bits) as the plan runs them, one
+    grouped launch, bytes = packed weights + inputs + outputs; (b) dp_daq_quantize at M = 32768."""
+    import torch
+    from paper_2511_11446_b200 import binding as B, synth_cuda, synth
+
+    def graph_time(fn, reps=5):
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            fn()
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); g.replay(); e1.record(); torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return statistics.median(ts[1:]) * 1e-3
+
+    out = {}
+    idx = [l for l, (_, M, K, N) in enumerate(stack.table) if M <= 32]
+    plan = B.dp_plan_create([stack.layers[l].w for l in idx], [stack.table[l][1] for l in idx],
+                            B.DP_FLAG_GROUP_SMALL_M)
+    try:
+        ws = torch.empty(B.dp_plan_workspace(plan), dtype=torch.uint8, device="cuda")
+        # two input/output sets so that consecutive replays do not find the (small) activations in L2;
+        # the weights (140 MB per pass) exceed L2 by themselves
+        xp = B.ptr_array([stack.x[0][l].data_ptr() for l in idx])
+        yp = B.ptr_array([stack.y[l].data_ptr() for l in idx])
+        t = graph_time(lambda: B.dp_plan_run(plan, [0], 0, xp, yp, ws, stack.status,
+                                             flags=B.DP_PLAN_SAME_X | B.DP_PLAN_SAME_Y))
+        by = sum(stack.layers[l].packed_bytes() + 6 * stack.table[l][3] + 2 * stack.table[l][1] * (stack.table[l][2] + stack.table[l][3])
+                 for l in idx)
+        out["adaln_group"] = {"layers": len(idx), "bytes": by, "us": t * 1e6, "achieved": by / t / 1e9,
+                              "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": by / t / 1e9 / peaks["hbm_gbs"]}
+    finally:
+        B.dp_plan_destroy(plan)
+    for K in (1152, 4608):
+        M = 32768
+        x = synth_cuda.activations(synth.BASE_SEED, 0, 0, M, K, 1.0, n_out=K // 100)
+        q = torch.empty((M, K), dtype=torch.int8, device="cuda")
+        sa = torch.empty(M, dtype=torch.float32, device="cuda")
+        x2 = x.clone(); q2 = torch.empty_like(q)  # 2 sets: 2 x (75 + 38) MB or 2 x (302 + 151) MB, past L2
+        def run():
+            B.dp_daq_quantize(x, M, K, K, q, K, sa)
+            B.dp_daq_quantize(x2, M, K, K, q2, K, sa)
+        t = graph_time(run) / 2
+        by = 3 * M * K + 4 * M
+        out[f"daq_M32768_K{K}"] = {"bytes": by, "us": t * 1e6, "achieved": by / t / 1e9, "peak": peaks["hbm_gbs"],
+                                   "unit": "GB/s", "frac": by / t / 1e9 / peaks["hbm_gbs"]}
+        del x, x2, q, q2
+    return out
 
 
 def measure_mma_peak():

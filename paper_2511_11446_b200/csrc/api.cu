@@ -516,6 +516,11 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
       home->push_back(static_cast<int>(l));
       p->grouped[l] = 1;
     }
+    for (const auto& g : p->groups) {
+      const PlanLayer& G = p->layers[g[0]];
+      const size_t need = simt_group_scratch_bytes(G.M, G.w.K, static_cast<int32_t>(g.size()));
+      if (need > p->workspace_bytes) p->workspace_bytes = need;
+    }
   }
   cudaError_t e = cudaSuccess;
   if (fused_daq) {
@@ -593,6 +598,9 @@ static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, 
     ga.K = G.w.K;
     ga.n_layers = static_cast<int32_t>(grp.size());
     ga.early_w = *chained ? 1 : 0;
+    ga.q_scratch = static_cast<int8_t*>(workspace);
+    ga.sa_scratch = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) +
+                                             align256(static_cast<size_t>(ga.n_layers) * ga.M * ga.K));
     for (size_t i = 0; i < grp.size(); ++i) {
       const int l = grp[i];
       const PlanLayer& L = plan->layers[l];

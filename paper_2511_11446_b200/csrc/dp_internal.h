@@ -55,7 +55,13 @@ struct SimtGroupArgs {
   int64_t M;
   int32_t N, K, n_layers;
   int32_t early_w;
+  // Scratch for the group's int8 tokens [n_layers][M][K] and scales [n_layers][M]: when given, one
+  // small kernel quantizes all tokens of the group first and the main kernel's CTAs only fetch the
+  // codes; when null every CTA quantizes its tokens itself.
+  int8_t* q_scratch;
+  float* sa_scratch;
 };
+size_t simt_group_scratch_bytes(int64_t M, int32_t K, int32_t n_layers);
 int launch_simt_group(const SimtGroupArgs& g, cudaStream_t stream, bool pdl);
 size_t simt_max_k();
 

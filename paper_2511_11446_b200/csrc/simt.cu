@@ -10,8 +10,7 @@
 // with token j's sum) and sent through the dequant epilogue.
 #include <cuda_bf16.h>
 
-#include "dp_common.cuh"
-#include "dp_internal.h"
+#include "daq_device.cuh"
 
 namespace dp {
 
@@ -236,6 +235,21 @@ simt_linear_kernel(SimtArgs a) {
 // Several layers of one shape (M, K, N) in one launch: blockIdx.z picks the layer. Used for the
 // adaLN modulation linears of a timestep, which are mutually independent and, one at a time, far
 // too small (3..8 MB of weights) to fill the GPU for longer than a launch takes.
+// DAQ of every token of a group (one warp per token; grid = (ceil(M / 8), layers)).
+__global__ void __launch_bounds__(kSimtWarps * 32)
+daq_group_kernel(SimtGroupArgs g) {
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t row = static_cast<int64_t>(blockIdx.x) * kSimtWarps + warp;
+  pdl_wait();
+  if (row >= g.M) return;
+  const int layer = blockIdx.y;
+  const uint16_t* x = static_cast<const uint16_t*>(g.layer[layer].x) + row * g.K;
+  const QRow qr(g.q_scratch + static_cast<int64_t>(layer) * g.M * g.K, row, g.K, 0);
+  const float sc = daq_row_2pass<false>(x, g.K, qr, lane);
+  if (lane == 0) g.sa_scratch[static_cast<int64_t>(layer) * g.M + row] = sc;
+}
+
 __global__ void __launch_bounds__(kSimtWarps * 32)
 simt_group_kernel(SimtGroupArgs g) {
   SimtArgs a;
@@ -243,6 +257,10 @@ simt_group_kernel(SimtGroupArgs g) {
   a.x = L.x;
   a.ldx = g.K;
   a.s_a_in = nullptr;
+  if (g.q_scratch != nullptr) {  // tokens already quantized by daq_group_kernel
+    a.x = g.q_scratch + static_cast<int64_t>(blockIdx.z) * g.M * g.K;
+    a.s_a_in = g.sa_scratch + static_cast<int64_t>(blockIdx.z) * g.M;
+  }
   a.M = g.M;
   a.N = g.N;
   a.K = g.K;
@@ -265,8 +283,18 @@ simt_group_kernel(SimtGroupArgs g) {
 
 size_t simt_max_k() { return 16384; }
 
+size_t simt_group_scratch_bytes(int64_t M, int32_t K, int32_t n_layers) {
+  const size_t q = (static_cast<size_t>(n_layers) * M * K + 255) & ~static_cast<size_t>(255);
+  return q + ((sizeof(float) * n_layers * M + 255) & ~static_cast<size_t>(255));
+}
+
 int launch_simt_group(const SimtGroupArgs& g, cudaStream_t stream, bool pdl) {
   if (g.M == 0 || g.n_layers == 0) return DP_OK;
+  if (g.q_scratch != nullptr) {
+    const dim3 dgrid(static_cast<unsigned>((g.M + kSimtWarps - 1) / kSimtWarps), static_cast<unsigned>(g.n_layers));
+    cudaError_t e = launch(daq_group_kernel, dgrid, dim3(kSimtWarps * 32), 0, stream, pdl, g);
+    if (e != cudaSuccess) return fail(DP_ERR_CUDA, "grouped DAQ launch failed: %s", cudaGetErrorString(e));
+  }
   const size_t smem = static_cast<size_t>(kSimtRows) * g.K + kSimtRows * sizeof(float);
   const dim3 grid((g.N + kSimtChPerCta - 1) / kSimtChPerCta, static_cast<unsigned>((g.M + kSimtRows - 1) / kSimtRows),
                   static_cast<unsigned>(g.n_layers));
@@ -278,6 +306,7 @@ int launch_simt_group(const SimtGroupArgs& g, cudaStream_t stream, bool pdl) {
   }
   SimtGroupArgs args = g;
   if (!pdl) args.early_w = 0;
+  if (g.q_scratch != nullptr && pdl) args.early_w = 1;  // the preceding kernel is the group's own DAQ
   cudaError_t e = launch(simt_group_kernel, grid, block, smem, stream, pdl, args);
   if (e != cudaSuccess) return fail(DP_ERR_CUDA, "grouped simt launch failed: %s", cudaGetErrorString(e));
   return DP_OK;
