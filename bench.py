@@ -304,12 +304,14 @@ def hbm_kernel_rooflines(stack, peaks):
                             B.DP_FLAG_GROUP_SMALL_M)
     try:
         ws = torch.empty(B.dp_plan_workspace(plan), dtype=torch.uint8, device="cuda")
-        # two input/output sets so that consecutive replays do not find the (small) activations in L2;
-        # the weights (140 MB per pass) exceed L2 by themselves
         xp = B.ptr_array([stack.x[0][l].data_ptr() for l in idx])
         yp = B.ptr_array([stack.y[l].data_ptr() for l in idx])
-        t = graph_time(lambda: B.dp_plan_run(plan, [0], 0, xp, yp, ws, stack.status,
-                                             flags=B.DP_PLAN_SAME_X | B.DP_PLAN_SAME_Y))
+        # four passes per graph replay: the 133 MB of packed weights exceed L2, so each pass streams
+        # them from HBM again
+        def passes():
+            for _ in range(4):
+                B.dp_plan_run(plan, [0], 0, xp, yp, ws, stack.status, flags=B.DP_PLAN_SAME_X | B.DP_PLAN_SAME_Y)
+        t = graph_time(passes) / 4
         by = sum(stack.layers[l].packed_bytes() + 6 * stack.table[l][3] + 2 * stack.table[l][1] * (stack.table[l][2] + stack.table[l][3])
                  for l in idx)
         out["adaln_group"] = {"layers": len(idx), "bytes": by, "us": t * 1e6, "achieved": by / t / 1e9,
@@ -402,7 +404,18 @@ def main():
     ap.add_argument("--only", default=None, choices=["layer", "gemm", "daq"])
     ap.add_argument("--iters", type=int, default=None)
     ap.add_argument("--flags", type=lambda v: int(v, 0), default=0, help="dp_wq_linear tuning flags for --sweep")
+    ap.add_argument("--hbm-kernels", action="store_true",
+                    help="time only the HBM-bound kernels (grouped adaLN launch, DAQ at M=32768) and print their rooflines")
     args = ap.parse_args()
+    if args.hbm_kernels:
+        import torch
+        from paper_2511_11446_b200 import synth
+        from paper_2511_11446_b200.workloads import DitStack
+        torch.cuda.set_device(0)
+        from paper_2511_11446_b200 import binding as B
+        stack = DitStack(seed=synth.BASE_SEED + 4, flags=B.DP_FLAG_GROUP_SMALL_M)  # no autotuning needed here
+        print(json.dumps(hbm_kernel_rooflines(stack, measured_peaks())))
+        return
     if args.sweep:
         import torch
         from paper_2511_11446_b200 import sweep

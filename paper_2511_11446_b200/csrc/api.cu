@@ -148,6 +148,7 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
     a.dbg_acc = dbg ? dbg->acc : nullptr;
     a.dbg_ldacc = dbg ? dbg->ldacc : 0;
     a.early_w = chained ? 1 : 0;
+    a.status = status;
     return launch_simt_linear(a, stream, pdl);
   }
   const int8_t* q;
@@ -598,6 +599,7 @@ static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, 
     ga.K = G.w.K;
     ga.n_layers = static_cast<int32_t>(grp.size());
     ga.early_w = *chained ? 1 : 0;
+    ga.status = status;
     ga.q_scratch = static_cast<int8_t*>(workspace);
     ga.sa_scratch = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) +
                                              align256(static_cast<size_t>(ga.n_layers) * ga.M * ga.K));

@@ -244,6 +244,19 @@ __device__ __forceinline__ bool mbar_spin_wait(uint64_t* bar, uint32_t parity, v
   }
   return true;
 }
+// Untiled bulk copy global -> shared (both addresses 16-byte aligned, size a multiple of 16 bytes),
+// completion counted in bytes on an mbarrier of this CTA.
+__device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+// Asks L2 to fetch `bytes` (a multiple of 16) from 16-byte aligned `gsrc`; nothing lands in the SM.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* gsrc, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gsrc), "r"(bytes) : "memory");
+}
+
 // 2-D tiled store shared -> global (bulk async-group completion). Rows past the tensor's extent
 // are clipped by the hardware. Coordinates are never negative here.
 __device__ __forceinline__ void tma_store_2d(const void* tmap, int c0, int c1, const void* src) {

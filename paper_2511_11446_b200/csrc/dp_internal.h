@@ -39,6 +39,7 @@ struct SimtArgs {
   int32_t* dbg_acc;
   int64_t dbg_ldacc;
   int32_t early_w;  // weights may be fetched before the preceding kernel on the stream has finished
+  int32_t* status;  // device word raised to DP_ERR_TIMEOUT when a bounded wait expires (may be null)
 };
 int launch_simt_linear(const SimtArgs& a, cudaStream_t stream, bool pdl);
 // Up to kSimtGroupMax layers of one shape (bf16 inputs [M][K], outputs [M][N], both contiguous).
@@ -60,6 +61,10 @@ struct SimtGroupArgs {
   // codes; when null every CTA quantizes its tokens itself.
   int8_t* q_scratch;
   float* sa_scratch;
+  int32_t* status;  // as SimtArgs::status
+  // Matrix-instruction form: CTAs [cta_begin[l], cta_begin[l + 1]) of grid.x work on layer l (filled
+  // by launch_simt_group: more CTAs for the layers that take longer).
+  int32_t cta_begin[kSimtGroupMax + 1];
 };
 size_t simt_group_scratch_bytes(int64_t M, int32_t K, int32_t n_layers);
 int launch_simt_group(const SimtGroupArgs& g, cudaStream_t stream, bool pdl);

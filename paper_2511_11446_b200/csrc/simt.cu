@@ -10,13 +10,20 @@
 // with token j's sum) and sent through the dequant epilogue.
 //
 // For K <= 1152 (every adaLN layer) the contraction instead runs on warp-level int8 matrix
-// instructions (m16n8k32: 16 channels x 8 tokens per warp), which removes almost all shared-memory
-// reads and integer issue slots of the dp4a form and leaves the kernel bound by the weight stream:
-// a warp owns 16 channels; lane (g, t) = (lane / 4, lane % 4) fetches the units 4j + t of rows g
-// and g + 8, and because a dot product may visit k in any order as long as both operands agree,
-// those registers serve directly as the A fragments while the B fragments are the same units of
-// token g, read from shared memory (row pitch K + 8 keeps the 64-bit reads conflict-free).
+// instructions (m16n8k32 with the tokens as the 16 rows and 8 output channels as the columns), and
+// the weights reach the SM as bulk asynchronous copies: eight consecutive weight rows are one
+// contiguous run of the packed matrix, which each warp streams through a private ring of
+// shared-memory stages (3- and 4-bit: one copy of eight whole rows per stage; 8-bit: one copy per
+// row and third of K; completion counted in bytes on the stage's mbarrier), so
+// HBM sees a few thousand long sequential streams and the bytes in flight do not depend on
+// registers. Lane (g, t) = (lane / 4, lane % 4) reads the units 4j + t of row g from the stage,
+// expands them to int8 and feeds them as B fragments; because a dot product may visit k in any
+// order as long as both operands agree, the A fragments are simply the same units of tokens g and
+// g + 8 from shared memory (row pitch K + 16 keeps those 128-bit reads conflict-free).
 #include <cuda_bf16.h>
+
+#include <algorithm>
+#include <type_traits>
 
 #include "daq_device.cuh"
 
@@ -27,11 +34,18 @@ constexpr int kSimtWarps = 8;
 constexpr int kSimtLanesPerCh = 8;  // lanes sharing one output channel
 constexpr int kSimtChPerCta = kSimtWarps * (32 / kSimtLanesPerCh);
 constexpr int kSimtSlots = 5;       // units a lane holds per pass (K = 1152: 36 units / 8 lanes)
-constexpr int kMmaChPerWarp = 16;   // matrix-instruction form: channels per warp (the M of m16n8k32)
-constexpr int kMmaChPerCta = kSimtWarps * kMmaChPerWarp;
+// Matrix-instruction form (K <= kMmaMaxK).
 constexpr int kMmaMaxK = 1152;
-// 128-k steps whose packed units a lane keeps in flight at once (two rows each).
-template <int BITS> __host__ __device__ constexpr int mma_batch() { return BITS == 8 ? 3 : (BITS == 4 ? 5 : 9); }
+constexpr int kMmaWarps = 8;
+constexpr int kMmaRows = 16;          // tokens per CTA (the M of m16n8k32)
+constexpr int kMmaCh = 8;             // output channels per block (the N of m16n8k32)
+constexpr int kMmaMaxStages = 8;
+constexpr int kMmaRingBytes = 9600;   // per warp
+// 128-k steps per ring stage. Low-bit rows are short enough for a stage to hold eight whole rows,
+// which are contiguous in the packed matrix: one copy per stage. 8-bit rows go in thirds, one copy
+// per row, 16 bytes of padding per staged row so that the lanes' reads spread over all banks.
+template <int BITS> __host__ __device__ constexpr int mma_chunk_j() { return BITS == 8 ? 3 : 9; }
+constexpr int kMmaPitch8 = 3 * 128 + 16;
 
 // Packed form of one unit (32 consecutive k of one weight row): BITS words.
 template <int BITS>
@@ -83,11 +97,11 @@ __device__ __forceinline__ void expand_unit(const uint32_t (&pk)[BITS], uint32_t
   }
 }
 
-// This CTA's tokens -> int8 in shared memory, one warp per token (rows `pitch` bytes apart), and
-// their scales: DAQ here (Step 3, Eq. "daq"), or a copy when the caller passes quantized tokens.
+// Token `warp` of this CTA -> int8 in shared memory, by one warp (rows `pitch` bytes apart), and
+// its scale: DAQ here (Step 3, Eq. "daq"), or a copy when the caller passes quantized tokens.
 __device__ __forceinline__ void stage_tokens(const SimtArgs& a, const int64_t m0, const int block_x,
-                                             int8_t* sq, const int pitch, float* ssa) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+                                             int8_t* sq, const int pitch, float* ssa, const int warp) {
+  const int lane = threadIdx.x & 31;
   const int K = a.K;
   {
     const int64_t row = m0 + warp;
@@ -174,7 +188,7 @@ __device__ __forceinline__ void simt_linear_body(const SimtArgs& a, const int bl
   }
   if (a.early_w) pdl_wait();  // the tokens come from the preceding kernel on the stream
 
-  stage_tokens(a, m0, block_x, sq, K, ssa);
+  stage_tokens(a, m0, block_x, sq, K, ssa, warp);
   __syncthreads();
 
   // ---- contraction: passes of kSimtSlots units per lane ----
@@ -255,88 +269,237 @@ __device__ __forceinline__ void mma_m16n8k32_s8(int (&c)[4], uint32_t a0, uint32
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Matrix-instruction form (K <= kMmaMaxK). Fragment roles of m16n8k32: A row = channel (g and g + 8),
-// B column = token g, D element (row, column pair 2t, 2t + 1). The instruction's k index of a
-// register is immaterial here: lane (g, t) supplies, for step s of its unit, words 2s and 2s + 1 of
-// the unit as the (k-low, k-high) registers of BOTH operands, so every k meets its partner once.
+// Packed unit -> 8 words of 4 int8 holding w * 2^(8 - BITS) (the code, sign bit flipped, in the top
+// bits of its byte), k ascending: cheaper than true values, and the int32 sums come out as exact
+// multiples of 2^(8 - BITS) that the epilogue shifts back.
 template <int BITS>
-__device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block_x, const int block_y) {
-  extern __shared__ __align__(16) uint8_t smem[];
-  const int K = a.K, pitch = K + 8;
-  int8_t* sq = reinterpret_cast<int8_t*>(smem);                       // [kSimtRows][pitch]
-  float* ssa = reinterpret_cast<float*>(smem + kSimtRows * pitch);    // [kSimtRows]
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = lane >> 2, t = lane & 3;
-  const int64_t m0 = static_cast<int64_t>(block_y) * kSimtRows;
-  const int n0 = block_x * kMmaChPerCta + warp * kMmaChPerWarp;
-  const bool n_ok = n0 < a.N;  // N is a multiple of 16: a warp's channels exist together
-  const int64_t wpitch = (K * BITS) >> 5;
-  const uint32_t* w_lo = static_cast<const uint32_t*>(a.qweight) + (n_ok ? n0 + g : 0) * wpitch;
-  const uint32_t* w_hi = w_lo + (n_ok ? 8 * wpitch : 0);
-  const int kj = K >> 7;
-  constexpr int BJ = mma_batch<BITS>();
-  uint32_t pk[BJ][2][BITS];
-  pdl_launch_dependents();
-  if (!a.early_w) pdl_wait();
-  auto fetch_batch = [&](const int j0) {
+__device__ __forceinline__ void expand_unit_top(const uint32_t (&pk)[BITS], uint32_t (&w)[8]) {
+  if constexpr (BITS == 8) {
 #pragma unroll
-    for (int i = 0; i < BJ; ++i) {
-      if (n_ok && j0 + i < kj) {
-        fetch_unit<BITS>(w_lo, 4 * (j0 + i) + t, pk[i][0]);
-        fetch_unit<BITS>(w_hi, 4 * (j0 + i) + t, pk[i][1]);
-      }
+    for (int i = 0; i < 8; ++i) w[i] = pk[i];
+  } else if constexpr (BITS == 4) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t v = pk[i] ^ 0x88888888u;
+      const uint32_t lo = (v << 4) & 0xF0F0F0F0u, hi = v & 0xF0F0F0F0u;
+      w[2 * i] = __byte_perm(lo, hi, 0x5140);
+      w[2 * i + 1] = __byte_perm(lo, hi, 0x7362);
     }
-  };
-  fetch_batch(0);  // in flight across the prologue
-  if (a.early_w) pdl_wait();
-  stage_tokens(a, m0, block_x, sq, pitch, ssa);
-  __syncthreads();
-
-  int c[4] = {0, 0, 0, 0};
-  const int8_t* qrow = sq + g * pitch + t * 32;
-  for (int j0 = 0; j0 < kj; j0 += BJ) {
-    if (j0 != 0) fetch_batch(j0);
+  } else {
+    // sign bits (bit 2 of every 3-bit field of the 96-bit unit) flipped first
+    const uint32_t p0 = pk[0] ^ 0x24924924u, p1 = pk[1] ^ 0x49249249u, p2 = pk[2] ^ 0x92492492u;
 #pragma unroll
-    for (int i = 0; i < BJ; ++i) {
-      if (n_ok && j0 + i < kj) {
-        uint32_t wl[8], wh[8];
-        expand_unit<BITS>(pk[i][0], wl);
-        expand_unit<BITS>(pk[i][1], wh);
-        const uint2* qp = reinterpret_cast<const uint2*>(qrow + (j0 + i) * 128);
-#pragma unroll
-        for (int s = 0; s < 4; ++s) {
-          const uint2 q = qp[s];
-          mma_m16n8k32_s8(c, wl[2 * s], wh[2 * s], wl[2 * s + 1], wh[2 * s + 1], q.x, q.y);
-        }
-      }
+    for (int j = 0; j < 8; ++j) {
+      const int bit = 12 * j;  // the word's four fields start here
+      uint32_t x;
+      if (bit == 0) x = p0;
+      else if (bit < 24) x = p0 >> bit;
+      else if (bit < 32) x = __funnelshift_r(p0, p1, bit);
+      else if (bit < 56) x = p1 >> (bit - 32);
+      else if (bit < 64) x = __funnelshift_r(p1, p2, bit - 32);
+      else x = p2 >> (bit - 64);
+      // fields 0, 2 and fields 1, 3 move to the tops of their bytes by one multiplication each
+      // (the two shifted copies inside a product do not overlap, so nothing carries)
+      const uint32_t e = (x & 0x1C7u) * 0x8020u, o = (x & 0xE38u) * 0x100400u;
+      w[j] = (e & 0x00E000E0u) | (o & 0xE000E000u);
     }
   }
+}
 
-  if (n_ok) {
+// Packed unit `unit` of a staged weight row.
+template <int BITS>
+__device__ __forceinline__ void stage_unit(const uint8_t* row, int unit, uint32_t (&pk)[BITS]) {
+  if constexpr (BITS == 8) {
+    const uint4 u = reinterpret_cast<const uint4*>(row)[unit * 2], v = reinterpret_cast<const uint4*>(row)[unit * 2 + 1];
+    pk[0] = u.x; pk[1] = u.y; pk[2] = u.z; pk[3] = u.w;
+    pk[4] = v.x; pk[5] = v.y; pk[6] = v.z; pk[7] = v.w;
+  } else if constexpr (BITS == 4) {
+    const uint4 u = reinterpret_cast<const uint4*>(row)[unit];
+    pk[0] = u.x; pk[1] = u.y; pk[2] = u.z; pk[3] = u.w;
+  } else {
+    const uint32_t* p = reinterpret_cast<const uint32_t*>(row) + unit * 3;
+    pk[0] = p[0]; pk[1] = p[1]; pk[2] = p[2];
+  }
+}
+
+// Bounded wait without the abort shortcut: lets copies already issued land before a warp that gave
+// up leaves its ring.
+__device__ __forceinline__ void mbar_drain(uint64_t* bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > (1ll << 26)) return;
+  }
+}
+
+// Matrix-instruction form (K <= kMmaMaxK). Fragment roles of m16n8k32: A row = token (g and g + 8),
+// B column = channel g of the block, D element (token g or g + 8, channels 2t and 2t + 1). The
+// instruction's k index of a register is immaterial here: lane (g, t) supplies, for step s of its
+// unit, words 2s and 2s + 1 of the unit as the (k-low, k-high) registers of BOTH operands, so every
+// k meets its partner exactly once.
+template <int BITS>
+__device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block_x, const int block_y,
+                                              const int grid_x) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  const int K = a.K, qpitch = K + 16;
+  int8_t* sq = reinterpret_cast<int8_t*>(smem);                             // [kMmaRows][qpitch]
+  float* ssa = reinterpret_cast<float*>(smem + kMmaRows * qpitch);          // [kMmaRows]
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ssa + kMmaRows);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ssa + kMmaRows + 4);         // [kMmaWarps][kMmaMaxStages]
+  uint8_t* ring = reinterpret_cast<uint8_t*>(bars + kMmaWarps * kMmaMaxStages);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int64_t m0 = static_cast<int64_t>(block_y) * kMmaRows;
+  const bool two = a.M - m0 > 8;  // tokens g + 8 exist
+  constexpr int CJ = mma_chunk_j<BITS>();
+  const int64_t rowbytes = (static_cast<int64_t>(K) * BITS) >> 3;
+  const int pitch = BITS == 8 ? kMmaPitch8 : static_cast<int>(rowbytes);  // of a staged row
+  const int stage = kMmaCh * pitch;
+  const int S = min(kMmaMaxStages, kMmaRingBytes / stage);
+  uint64_t* bar = bars + warp * kMmaMaxStages;
+  uint8_t* myring = ring + warp * kMmaRingBytes;
+  const uint8_t* wbase = static_cast<const uint8_t*>(a.qweight);
+  const int kj = K >> 7;
+  const int nc = (kj + CJ - 1) / CJ;  // 1 for the low-bit forms (K <= kMmaMaxK)
+  // 8-channel blocks of this warp: blk0, blk0 + stride, ... The grid is sized to one wave, so a warp
+  // streams several blocks back to back.
+  const int nblocks = a.N / kMmaCh;
+  const int stride = grid_x * kMmaWarps;
+  const int blk0 = block_x * kMmaWarps + warp;
+  const int total = blk0 < nblocks ? ((nblocks - blk0 + stride - 1) / stride) * nc : 0;
+
+  if (threadIdx.x == 0) *abort_flag = 0;
+  if (lane == 0) {
+    for (int s = 0; s < S; ++s) mbar_init(&bar[s], 1);
+    fence_barrier_init();
+  }
+  __syncwarp();
+  pdl_launch_dependents();
+  if (!a.early_w) pdl_wait();
+
+  // Producer side of the ring (lane 0): item = (block, chunk); the copy of item i lands in stage i % S.
+  int f_it = 0, f_c = 0, f_blk = blk0, f_s = 0;
+  auto issue = [&]() {
+    if (f_it < total) {
+      if (lane == 0) {
+        const uint8_t* src = wbase + static_cast<int64_t>(f_blk) * kMmaCh * rowbytes;
+        uint8_t* dst = myring + f_s * stage;
+
+        if constexpr (BITS < 8) {
+          const uint32_t bytes = static_cast<uint32_t>(kMmaCh * rowbytes);
+          mbar_arrive_expect_tx(&bar[f_s], bytes);
+          bulk_load_1d(dst, src, bytes, &bar[f_s]);
+        } else {
+          const uint32_t bytes = static_cast<uint32_t>(min(CJ, kj - f_c * CJ) * 128);
+          mbar_arrive_expect_tx(&bar[f_s], kMmaCh * bytes);
+          src += f_c * (CJ * 128);
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int n = n0 + g + 8 * h;
-      const float sw = a.s_w[n];
-      const float b = a.bias != nullptr ? __uint_as_float(static_cast<uint32_t>(a.bias[n]) << 16) : 0.0f;
+          for (int r = 0; r < kMmaCh; ++r) bulk_load_1d(dst + r * kMmaPitch8, src + r * rowbytes, bytes, &bar[f_s]);
+        }
+      }
+      ++f_it;
+      if (++f_s == S) f_s = 0;
+      if (++f_c == nc) { f_c = 0; f_blk += stride; }
+    }
+  };
+#pragma unroll 1
+  for (int s = 0; s < S; ++s) issue();  // in flight across the prologue
+  if (a.early_w) pdl_wait();
+  for (int r = warp; r < (two ? kMmaRows : kMmaRows / 2); r += kMmaWarps)
+    stage_tokens(a, m0, block_x, sq, qpitch, ssa, r);
+  __syncthreads();
+
+  // Four accumulator sets, one per matrix instruction of a unit: consecutive instructions never
+  // wait on each other's results.
+  int c[4][4];
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int tok = 2 * t + e;
+  for (int i = 0; i < 4; ++i) c[i][0] = c[i][1] = c[i][2] = c[i][3] = 0;
+  int c_c = 0, c_blk = blk0, st = 0;
+  uint32_t ph = 0;
+  const int8_t* qrow = sq + g * qpitch + t * 32;
+  float sw[2] = {0.0f, 0.0f}, bs[2] = {0.0f, 0.0f};  // of channels 2t, 2t + 1 of the current block
+  auto epilogue = [&]() {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int n = c_blk * kMmaCh + 2 * t + e;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int tok = g + 8 * h;
         const int64_t row = m0 + tok;
         if (row < a.M) {
-          const int mine = c[2 * h + e];
-          const float y = __fmaf_rn(static_cast<float>(mine), __fmul_rn(ssa[tok], sw), b);
+          const int i = 2 * h + e;  // exact shift: the sum is a multiple of 2^(8 - BITS)
+          const int mine = (c[0][i] + c[1][i] + c[2][i] + c[3][i]) >> (8 - BITS);
+          const float y = __fmaf_rn(static_cast<float>(mine), __fmul_rn(ssa[tok], sw[e]), bs[e]);
           a.y[row * a.ldy + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
           if (a.dbg_acc != nullptr) a.dbg_acc[row * a.dbg_ldacc + n] = mine;
         }
       }
     }
+  };
+  // One unit of the staged chunk against tokens g (and g + 8 when TWO).
+  auto unit_step = [&](const uint8_t* srow, const int8_t* qu, const int u, auto two_tag) {
+    constexpr bool TWO = decltype(two_tag)::value;
+    uint32_t pk[BITS], w[8];
+    stage_unit<BITS>(srow, u, pk);
+    expand_unit_top<BITS>(pk, w);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const uint4 lo = *reinterpret_cast<const uint4*>(qu + 16 * h);
+      uint4 hi = make_uint4(0u, 0u, 0u, 0u);
+      if constexpr (TWO) hi = *reinterpret_cast<const uint4*>(qu + 8 * qpitch + 16 * h);
+      mma_m16n8k32_s8(c[2 * h], lo.x, hi.x, lo.y, hi.y, w[4 * h], w[4 * h + 1]);
+      mma_m16n8k32_s8(c[2 * h + 1], lo.z, hi.z, lo.w, hi.w, w[4 * h + 2], w[4 * h + 3]);
+    }
+  };
+  int it = 0;
+  for (; it < total; ++it) {
+    if (c_c == 0) {  // the block's scales and biases: in flight while its chunks are contracted
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int n = c_blk * kMmaCh + 2 * t + e;
+        sw[e] = a.s_w[n];
+        bs[e] = a.bias != nullptr ? __uint_as_float(static_cast<uint32_t>(a.bias[n]) << 16) : 0.0f;
+      }
+    }
+    if (!mbar_wait(&bar[st], ph, abort_flag)) break;
+    const int nj = min(CJ, kj - c_c * CJ);
+    const uint8_t* srow = myring + st * stage + g * pitch;
+    const int8_t* qc = qrow + c_c * (CJ * 128);
+    if (nj == CJ && !two) {  // the common case, free of per-unit tests
+#pragma unroll
+      for (int jj = 0; jj < CJ; ++jj) unit_step(srow, qc + jj * 128, 4 * jj + t, std::false_type{});
+    } else if (two) {
+#pragma unroll
+      for (int jj = 0; jj < CJ; ++jj)
+        if (jj < nj) unit_step(srow, qc + jj * 128, 4 * jj + t, std::true_type{});
+    } else {
+#pragma unroll
+      for (int jj = 0; jj < CJ; ++jj)
+        if (jj < nj) unit_step(srow, qc + jj * 128, 4 * jj + t, std::false_type{});
+    }
+    __syncwarp();  // every lane has consumed the stage: refill it
+    issue();
+    if (++c_c == nc) {
+      epilogue();
+#pragma unroll
+      for (int i = 0; i < 4; ++i) c[i][0] = c[i][1] = c[i][2] = c[i][3] = 0;
+      c_c = 0;
+      c_blk += stride;
+    }
+    if (++st == S) { st = 0; ph ^= 1u; }
   }
+  // A warp that gave up lets the copies it still has in flight land before the CTA may exit.
+  for (; it < f_it; ++it) {
+    mbar_drain(&bar[st], ph);
+    if (++st == S) { st = 0; ph ^= 1u; }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag && a.status != nullptr) atomicExch(a.status, DP_ERR_TIMEOUT);
 }
 
 template <int BITS, bool MMA>
-__global__ void __launch_bounds__(kSimtWarps * 32)
+__global__ void __launch_bounds__(kSimtWarps * 32, MMA ? 2 : 0)
 simt_linear_kernel(SimtArgs a) {
-  if constexpr (MMA) simt_mma_body<BITS>(a, blockIdx.x, blockIdx.y);
+  if constexpr (MMA) simt_mma_body<BITS>(a, blockIdx.x, blockIdx.y, gridDim.x);
   else simt_linear_body<BITS>(a, blockIdx.x, blockIdx.y);
 }
 
@@ -359,16 +522,23 @@ daq_group_kernel(SimtGroupArgs g) {
 }
 
 template <bool MMA>
-__global__ void __launch_bounds__(kSimtWarps * 32)
+__global__ void __launch_bounds__(kSimtWarps * 32, MMA ? 2 : 0)
 simt_group_kernel(SimtGroupArgs g) {
   SimtArgs a;
-  const SimtGroupArgs::Layer& L = g.layer[blockIdx.z];
+  int layer = blockIdx.z, block_x = blockIdx.x, grid_x = gridDim.x;
+  if constexpr (MMA) {  // grid.x enumerates (layer, CTA of the layer)
+    layer = 0;
+    while (static_cast<int>(blockIdx.x) >= g.cta_begin[layer + 1]) ++layer;
+    block_x = blockIdx.x - g.cta_begin[layer];
+    grid_x = g.cta_begin[layer + 1] - g.cta_begin[layer];
+  }
+  const SimtGroupArgs::Layer& L = g.layer[layer];
   a.x = L.x;
   a.ldx = g.K;
   a.s_a_in = nullptr;
   if (g.q_scratch != nullptr) {  // tokens already quantized by daq_group_kernel
-    a.x = g.q_scratch + static_cast<int64_t>(blockIdx.z) * g.M * g.K;
-    a.s_a_in = g.sa_scratch + static_cast<int64_t>(blockIdx.z) * g.M;
+    a.x = g.q_scratch + static_cast<int64_t>(layer) * g.M * g.K;
+    a.s_a_in = g.sa_scratch + static_cast<int64_t>(layer) * g.M;
   }
   a.M = g.M;
   a.N = g.N;
@@ -385,10 +555,11 @@ simt_group_kernel(SimtGroupArgs g) {
   a.dbg_acc = nullptr;
   a.dbg_ldacc = 0;
   a.early_w = g.early_w;
+  a.status = g.status;
   if constexpr (MMA) {
-    if (L.bits == 8) simt_mma_body<8>(a, blockIdx.x, blockIdx.y);
-    else if (L.bits == 4) simt_mma_body<4>(a, blockIdx.x, blockIdx.y);
-    else simt_mma_body<3>(a, blockIdx.x, blockIdx.y);
+    if (L.bits == 8) simt_mma_body<8>(a, block_x, blockIdx.y, grid_x);
+    else if (L.bits == 4) simt_mma_body<4>(a, block_x, blockIdx.y, grid_x);
+    else simt_mma_body<3>(a, block_x, blockIdx.y, grid_x);
   } else {
     if (L.bits == 8) simt_linear_body<8>(a, blockIdx.x, blockIdx.y);
     else if (L.bits == 4) simt_linear_body<4>(a, blockIdx.x, blockIdx.y);
@@ -398,8 +569,24 @@ simt_group_kernel(SimtGroupArgs g) {
 
 static bool simt_use_mma(int32_t K) { return K <= kMmaMaxK; }
 static size_t simt_smem_bytes(int32_t K) {
-  return static_cast<size_t>(kSimtRows) * (K + 8) + kSimtRows * sizeof(float);
+  if (!simt_use_mma(K)) return static_cast<size_t>(kSimtRows) * K + kSimtRows * sizeof(float);
+  return static_cast<size_t>(kMmaRows) * (K + 16) + kMmaRows * sizeof(float) + 16 +
+         sizeof(uint64_t) * kMmaWarps * kMmaMaxStages + static_cast<size_t>(kMmaWarps) * kMmaRingBytes;
 }
+
+// grid.x of the matrix-instruction form: all CTAs of the launch resident at once (one wave), each
+// warp walking its strided share of the 8-channel blocks.
+template <typename Kern>
+static int mma_grid_x(Kern kern, size_t smem, int32_t N, int64_t other_ctas) {
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kMmaWarps * 32, smem) != cudaSuccess || per_sm < 1)
+    per_sm = 1;
+  const int64_t slots = static_cast<int64_t>(num_sms()) * per_sm;
+  const int64_t full = (N / kMmaCh + kMmaWarps - 1) / kMmaWarps;
+  return static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(full, slots / std::max<int64_t>(1, other_ctas))));
+}
+
+static_assert(kMmaWarps == kSimtWarps, "both forms launch kSimtWarps warps");
 
 size_t simt_max_k() { return 16384; }
 
@@ -417,9 +604,10 @@ int launch_simt_group(const SimtGroupArgs& g, cudaStream_t stream, bool pdl) {
   }
   const size_t smem = simt_smem_bytes(g.K);
   const bool mma = simt_use_mma(g.K);
-  const int ch = mma ? kMmaChPerCta : kSimtChPerCta;
-  const dim3 grid((g.N + ch - 1) / ch, static_cast<unsigned>((g.M + kSimtRows - 1) / kSimtRows),
-                  static_cast<unsigned>(g.n_layers));
+  const int rows = mma ? kMmaRows : kSimtRows;
+  const int64_t m_groups = (g.M + rows - 1) / rows;
+  dim3 grid((g.N + kSimtChPerCta - 1) / kSimtChPerCta, static_cast<unsigned>(m_groups),
+            static_cast<unsigned>(g.n_layers));
   const dim3 block(kSimtWarps * 32);
   void (*kern)(SimtGroupArgs) = mma ? simt_group_kernel<true> : simt_group_kernel<false>;
   if (smem > 48 * 1024) {
@@ -428,6 +616,31 @@ int launch_simt_group(const SimtGroupArgs& g, cudaStream_t stream, bool pdl) {
     if (e != cudaSuccess) return fail(DP_ERR_CUDA, "simt smem attribute: %s", cudaGetErrorString(e));
   }
   SimtGroupArgs args = g;
+  if (mma) {
+    // One wave: the resident-CTA slots are shared out in proportion to the time a CTA of each
+    // bit-width needs per channel block (measured: the 8-bit form is bound by its copies, the 3-bit
+    // form by the expansion arithmetic), every layer getting at least one CTA.
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kMmaWarps * 32, smem) != cudaSuccess || per_sm < 1)
+      per_sm = 1;
+    const int64_t slots = std::max<int64_t>(g.n_layers, static_cast<int64_t>(num_sms()) * per_sm / m_groups);
+    const int full = (g.N / kMmaCh + kMmaWarps - 1) / kMmaWarps;
+    double cost[kSimtGroupMax], total = 0.0;
+    for (int l = 0; l < g.n_layers; ++l) {
+      cost[l] = g.layer[l].bits == 8 ? 1.6 : g.layer[l].bits == 4 ? 1.0 : 1.2;
+      total += cost[l];
+    }
+    int begin = 0;
+    double acc = 0.0;
+    for (int l = 0; l < g.n_layers; ++l) {  // cumulative rounding: the counts sum to `slots`
+      args.cta_begin[l] = begin;
+      acc += cost[l];
+      const int end = static_cast<int>(acc / total * static_cast<double>(slots) + 0.5);
+      begin = std::min(begin + full, std::max(begin + 1, end));
+    }
+    args.cta_begin[g.n_layers] = begin;
+    grid = dim3(static_cast<unsigned>(begin), static_cast<unsigned>(m_groups), 1);
+  }
   if (!pdl) args.early_w = 0;
   if (g.q_scratch != nullptr && pdl) args.early_w = 1;  // the preceding kernel is the group's own DAQ
   cudaError_t e = launch(kern, grid, block, smem, stream, pdl, args);
@@ -439,8 +652,9 @@ int launch_simt_linear(const SimtArgs& a, cudaStream_t stream, bool pdl) {
   if (a.M == 0) return DP_OK;
   const size_t smem = simt_smem_bytes(a.K);
   const bool mma = simt_use_mma(a.K);
-  const int ch = mma ? kMmaChPerCta : kSimtChPerCta;
-  const dim3 grid((a.N + ch - 1) / ch, static_cast<unsigned>((a.M + kSimtRows - 1) / kSimtRows));
+  const int rows = mma ? kMmaRows : kSimtRows;
+  const int64_t m_groups = (a.M + rows - 1) / rows;
+  dim3 grid((a.N + kSimtChPerCta - 1) / kSimtChPerCta, static_cast<unsigned>(m_groups));
   const dim3 block(kSimtWarps * 32);
   void (*kern)(SimtArgs);
   if (mma) kern = a.bits == 8 ? simt_linear_kernel<8, true> : a.bits == 4 ? simt_linear_kernel<4, true>
@@ -452,6 +666,7 @@ int launch_simt_linear(const SimtArgs& a, cudaStream_t stream, bool pdl) {
                                          static_cast<int>(smem));
     if (e != cudaSuccess) return fail(DP_ERR_CUDA, "simt smem attribute: %s", cudaGetErrorString(e));
   }
+  if (mma) grid.x = mma_grid_x(kern, smem, a.N, m_groups);
   SimtArgs args = a;
   if (!pdl) args.early_w = 0;
   cudaError_t e = launch(kern, grid, block, smem, stream, pdl, args);
