@@ -78,11 +78,12 @@ class DitStack:
 
     def launches_per_timestep(self):
         """Kernel launches of this library per timestep: DAQ + GEMM per token linear; the small-M
-        (adaLN) linears of a step share one grouped launch per 32 when the plan groups them."""
+        (adaLN) linears of a step share, per 32 of them, one grouped DAQ launch and one grouped
+        linear launch when the plan groups them."""
         small = sum(1 for (_, M, K, N) in self.table if M <= 32)
         big = len(self.table) - small
         grouped = bool(self.flags & B.DP_FLAG_GROUP_SMALL_M)
-        return 2 * big + (-(-small // 32) if grouped else small)
+        return 2 * big + (2 * -(-small // 32) if grouped else small)
 
     # ---- execution ----
     def ptrs(self, n_steps=None):
