@@ -225,13 +225,15 @@ def gemm_roofline(stack, peaks):
     GEMM launches of one timestep, each with the kernel variant the plan chose for its layer, on
     pre-quantized activations (so no DAQ launch in between), captured in one CUDA graph and timed
     with CUDA events on the replay stream. One timestep's operands (0.4 GB of int8 activations,
-    0.4 GB of weights, 1.1 GB of outputs) exceed L2, so every launch streams from HBM."""
+    0.4 GB of weights, 1.1 GB of outputs) exceed L2, so every launch streams from HBM. A layer the
+    plan runs in the unpack-first form launches the 8-bit kernel on an int8 copy of its weights:
+    here that copy is generated directly (same seeded values), so the launch is that GEMM alone."""
     import collections
     import torch
-    from paper_2511_11446_b200 import binding as B
+    from paper_2511_11446_b200 import binding as B, synth_cuda
     x0 = stack.x[0]
     idx = [l for l, (_, M, K, N) in enumerate(stack.table) if M > 32]
-    qs, sas, flags, variants = {}, {}, {}, collections.Counter()
+    qs, sas, flags, variants, weights, keep = {}, {}, {}, collections.Counter(), {}, []
     for l in idx:
         _, M, K, N = stack.table[l]
         qs[l] = torch.empty((M, K), dtype=torch.int8, device="cuda")
@@ -239,12 +241,19 @@ def gemm_roofline(stack, peaks):
         B.dp_daq_quantize(x0[l], M, K, K, qs[l], K, sas[l])
         v = B.dp_plan_layer_variant(stack.plan, l)
         flags[l] = B.variant_flags(v)
-        variants[("ws" if v["weight_stationary"] else "pair" if v["cta_group"] == 2 else "single") + str(v["tile_n"])] += 1
+        weights[l] = stack.layers[l].w
+        if v["unpack_first"]:
+            w8, _ = synth_cuda.weights(stack.seed, l, N, K, stack.bits[l])
+            keep.append(w8)
+            weights[l] = B.make_weight(w8, stack.layers[l].s_w, stack.layers[l].bias, N, K, 8)
+            flags[l] &= ~B.DP_FLAG_UNPACK_FIRST
+        variants[("ws" if v["weight_stationary"] else "pair" if v["cta_group"] == 2 else "single") + str(v["tile_n"])
+                 + ("+unpack_first" if v["unpack_first"] else "")] += 1
 
     def run():
         for l in idx:
             _, M, K, N = stack.table[l]
-            B.dp_wq_linear(stack.layers[l].w, qs[l], K, sas[l], M, stack.y[l], N, None, None, stack.status, flags[l])
+            B.dp_wq_linear(weights[l], qs[l], K, sas[l], M, stack.y[l], N, None, None, stack.status, flags[l])
 
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())

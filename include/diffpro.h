@@ -117,6 +117,16 @@ typedef struct dp_debug {
  * (programmatic dependent launch) while the previous GEMM drains. */
 #define DP_FLAG_FUSED_DAQ 0x40000u
 
+/* dp_wq_linear and dp_plan_create, packed bit-widths (3, 4) on the tensor-core path: expand the
+ * packed weights once per call to int8 [N][K] in the workspace (extra CTAs of the DAQ launch; a
+ * launch of its own when the activations arrive quantized) and run the 8-bit kernel on that copy,
+ * instead of expanding the tiles in shared memory inside the GEMM (Step 4's unpack, hoisted). Pays
+ * when a weight tile is consumed by many row tiles but each CTA sees it only once or twice (M of a
+ * few thousand): there the in-kernel expansion is repeated M/128 times across CTAs. The copy lives
+ * only for the call, the weights stay packed in memory, results are identical. Adds N*K bytes to
+ * the workspace. With DP_FLAG_AUTOTUNE the plan times both forms per layer shape. */
+#define DP_FLAG_UNPACK_FIRST 0x80000u
+
 /* flags for dp_plan_run */
 #define DP_PLAN_SAME_X 1u       /* x_ptrs has n_layers entries reused by every step              */
 #define DP_PLAN_SAME_Y 2u       /* y_ptrs has n_layers entries reused (overwritten) every step   */
@@ -204,6 +214,9 @@ size_t dp_plan_workspace(const dp_plan* plan);
  * are then 0). Any output pointer may be NULL. */
 int dp_plan_layer_variant(const dp_plan* plan, int32_t layer, int32_t* tile_n, int32_t* cta_group,
                           int32_t* weight_stationary, int32_t* small_m);
+/* *unpack_first = 1 when the plan runs layer `layer` in the DP_FLAG_UNPACK_FIRST form (the
+ * variant dp_plan_layer_variant reports is then the 8-bit kernel's). No counterpart in the paper. */
+int dp_plan_layer_unpack_first(const dp_plan* plan, int32_t layer, int32_t* unpack_first);
 void dp_plan_destroy(dp_plan* plan);
 
 /*

@@ -22,6 +22,7 @@ DP_FLAG_NONE, DP_FLAG_FORCE_SIMT, DP_FLAG_FORCE_MMA, DP_FLAG_NO_PDL = 0, 1, 2, 4
 DP_FLAG_CTA_PAIR, DP_FLAG_NO_CTA_PAIR = 0x800, 0x1000
 DP_FLAG_WEIGHT_STATIONARY, DP_FLAG_NO_WEIGHT_STATIONARY = 0x2000, 0x4000
 DP_FLAG_AUTOTUNE, DP_FLAG_GROUP_SMALL_M, DP_FLAG_FUSED_DAQ = 0x10000, 0x20000, 0x40000
+DP_FLAG_UNPACK_FIRST = 0x80000
 DP_PLAN_SAME_X, DP_PLAN_SAME_Y = 1, 2
 
 
@@ -31,7 +32,7 @@ def DP_FLAG_TILE_N(bn: int) -> int:
 DP_STATIC_SCRATCH_BYTES = 10 << 20
 
 EXPORTS = ["dp_daq_quantize", "dp_wq_linear_workspace", "dp_wq_linear", "dp_wq_linear_static", "dp_plan_create",
-           "dp_plan_workspace", "dp_plan_layer_variant", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
+           "dp_plan_workspace", "dp_plan_layer_variant", "dp_plan_layer_unpack_first", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
            "dp_plan_run_host", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_status_string",
            "dp_last_error", "dp_version"]
 
@@ -68,6 +69,7 @@ def lib():
         L.dp_plan_workspace.restype = C.c_size_t
         L.dp_plan_workspace.argtypes = [C.c_void_p]
         L.dp_plan_layer_variant.argtypes = [C.c_void_p, C.c_int32] + [C.POINTER(C.c_int32)] * 4
+        L.dp_plan_layer_unpack_first.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
         L.dp_plan_x_bytes.restype = C.c_size_t
         L.dp_plan_x_bytes.argtypes = [C.c_void_p]
         L.dp_plan_destroy.restype = None
@@ -152,10 +154,13 @@ def dp_plan_workspace(plan) -> int:
 
 
 def dp_plan_layer_variant(plan, layer: int) -> dict:
-    """{'tile_n', 'cta_group', 'weight_stationary', 'small_m'} of one layer of a plan."""
+    """{'tile_n', 'cta_group', 'weight_stationary', 'small_m', 'unpack_first'} of one layer of a plan."""
     v = [C.c_int32() for _ in range(4)]
     _check(lib().dp_plan_layer_variant(plan, layer, *[C.byref(t) for t in v]), "dp_plan_layer_variant")
-    return dict(tile_n=v[0].value, cta_group=v[1].value, weight_stationary=v[2].value, small_m=v[3].value)
+    u = C.c_int32(0)
+    _check(lib().dp_plan_layer_unpack_first(plan, layer, C.byref(u)), "dp_plan_layer_unpack_first")
+    return dict(tile_n=v[0].value, cta_group=v[1].value, weight_stationary=v[2].value, small_m=v[3].value,
+                unpack_first=u.value)
 
 
 def variant_flags(v: dict) -> int:
@@ -163,6 +168,8 @@ def variant_flags(v: dict) -> int:
     if v["small_m"]:
         return DP_FLAG_FORCE_SIMT
     f = DP_FLAG_FORCE_MMA | DP_FLAG_TILE_N(v["tile_n"])
+    if v.get("unpack_first"):
+        f |= DP_FLAG_UNPACK_FIRST
     if v["weight_stationary"]:
         return f | DP_FLAG_WEIGHT_STATIONARY
     f |= DP_FLAG_NO_WEIGHT_STATIONARY

@@ -52,7 +52,7 @@ static size_t scratch_q_bytes(int64_t M, int32_t K) { return static_cast<size_t>
 
 constexpr uint32_t kLinearFlags =
     DP_FLAG_FORCE_SIMT | DP_FLAG_FORCE_MMA | DP_FLAG_NO_PDL | DP_FLAG_TILE_N_MASK | DP_FLAG_CTA_PAIR |
-    DP_FLAG_NO_CTA_PAIR | DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_NO_WEIGHT_STATIONARY;
+    DP_FLAG_NO_CTA_PAIR | DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_UNPACK_FIRST;
 constexpr int64_t kWsMinRows = 8192;  // from here on a resident weight strip is reused often enough to pay
 static int forced_bn(uint32_t flags) { return static_cast<int>((flags & DP_FLAG_TILE_N_MASK) >> 8) * 64; }
 
@@ -124,7 +124,8 @@ static int check_weight(const dp_weight* w) {
 static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_a_in, int64_t M,
                       void* y, int64_t ldy, void* workspace, const dp_debug* dbg, int32_t* status,
                       uint32_t flags, cudaStream_t stream, const CUtensorMap* tmap_w, int bn, int cg, int ws,
-                      const CUtensorMap* tmap_a_cached, bool chained, int32_t* daq_sync = nullptr) {
+                      const CUtensorMap* tmap_a_cached, bool chained, int32_t* daq_sync = nullptr,
+                      int pre = -1) {
   const bool pdl = !(flags & DP_FLAG_NO_PDL);
   if (use_simt(M, w->N, w->K, flags)) {
     if (static_cast<size_t>(w->K) > simt_max_k())
@@ -155,6 +156,23 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
   const float* s_a;
   int64_t ldq;
   int korder = KORDER_NATURAL;
+  // Unpack-first variant: the packed weights are expanded once to int8 [N][K] in the workspace (by
+  // extra CTAs of the DAQ launch) and the 8-bit kernel runs on that copy, instead of every CTA
+  // expanding the weight tiles it needs in shared memory.
+  if (pre < 0) pre = (flags & DP_FLAG_UNPACK_FIRST) ? 1 : 0;
+  const bool unpack_first = pre > 0 && w->bits < 8;
+  dp_weight w8 = *w;
+  UnpackJob job{nullptr, nullptr, 0, 0, 0};
+  if (unpack_first) {
+    int8_t* dst = reinterpret_cast<int8_t*>(static_cast<uint8_t*>(workspace) + align256(scratch_q_bytes(M, w->K)) +
+                                            align256(sizeof(float) * static_cast<size_t>(M)));
+    job = UnpackJob{static_cast<const uint32_t*>(w->qweight), dst, static_cast<int64_t>(w->N) * w->K / 32, w->bits, 0};
+    w8.bits = 8;
+    w8.qweight = dst;
+    w = &w8;
+    tmap_w = nullptr;  // the caller's descriptor covers the packed matrix
+    daq_sync = nullptr;
+  }
   const bool tiled = s_a_in == nullptr;  // the library's own scratch: stored as contiguous 128 x 128 tiles
   const bool fused = s_a_in == nullptr && daq_sync != nullptr && dbg == nullptr;  // DAQ inside the GEMM kernel
   if (s_a_in == nullptr) {
@@ -162,7 +180,8 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
     float* wsa = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align256(scratch_q_bytes(M, w->K)));
     korder = gemm_korder(w->bits);
     if (!fused) {
-      int st = launch_daq(x, M, w->K, ldx, wq, w->K, wsa, nullptr, korder, true, stream, pdl);
+      int st = launch_daq(x, M, w->K, ldx, wq, w->K, wsa, nullptr, korder, true, stream, pdl,
+                          unpack_first ? &job : nullptr);
       if (st != DP_OK) return st;
     }
     q = wq;
@@ -172,11 +191,16 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
     q = static_cast<const int8_t*>(x);
     s_a = s_a_in;
     ldq = ldx;
+    if (unpack_first) {
+      int st = launch_unpack(job, stream, pdl);
+      if (st != DP_OK) return st;
+    }
   }
   GemmProblem g;
   g.korder = korder;
   g.a_tiled = tiled ? 1 : 0;
   g.early_w = fused ? (chained ? 1 : 0) : (s_a_in == nullptr ? 1 : 0);
+  if (unpack_first) g.early_w = 0;  // the weights come from the kernel just before this one
   g.x = fused ? static_cast<const uint16_t*>(x) : nullptr;
   g.ldx = ldx;
   g.q_out = fused ? const_cast<int8_t*>(q) : nullptr;
@@ -250,7 +274,9 @@ static int check_linear_args(const dp_weight* w, const void* x, int64_t ldx, con
     if (dbg->acc && (dbg->ldacc < w->N || (reinterpret_cast<uintptr_t>(dbg->acc) & 3u)))
       return fail(DP_ERR_ALIGN, "dbg.acc misaligned or too narrow");
   }
-  if (!use_simt(M, w->N, w->K, flags) && s_a_in == nullptr) {
+  // scratch users: the library's own DAQ, and the int8 copy of the weights of the unpack-first form
+  if (!use_simt(M, w->N, w->K, flags) &&
+      (s_a_in == nullptr || ((flags & DP_FLAG_UNPACK_FIRST) && w->bits < 8))) {
     const size_t need = dp_wq_linear_workspace(M, w->N, w->K, w->bits, flags);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))
       return fail(DP_ERR_WORKSPACE, "workspace needs %zu bytes, 256-byte aligned (got %zu)", need,
@@ -265,10 +291,11 @@ static int check_linear_args(const dp_weight* w, const void* x, int64_t ldx, con
 using namespace dp;
 
 extern "C" size_t dp_wq_linear_workspace(int64_t M, int32_t N, int32_t K, int32_t bits, uint32_t flags) {
-  (void)bits;
   if (M <= 0 || K <= 0) return 256;
   if (use_simt(M, N, K, flags)) return 256;
-  return align256(scratch_q_bytes(M, K)) + align256(sizeof(float) * static_cast<size_t>(M));
+  size_t need = align256(scratch_q_bytes(M, K)) + align256(sizeof(float) * static_cast<size_t>(M));
+  if ((flags & DP_FLAG_UNPACK_FIRST) && bits < 8) need += align256(static_cast<size_t>(N) * K);
+  return need;
 }
 
 extern "C" int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_a_in,
@@ -335,6 +362,7 @@ struct PlanLayer {
   int64_t M;
   bool simt;
   int bn, cg, ws;
+  int pre;  // weights expanded to int8 scratch first, 8-bit kernel on the copy
   CUtensorMap tmap_w;
   size_t x_offset;  // byte offset of this layer's input inside one staged step (host-input path)
 };
@@ -361,25 +389,27 @@ struct dp_plan {
 struct TunedShape {
   int64_t M;
   int32_t N, K, bits;
-  int bn, cg, ws;
+  int bn, cg, ws, pre;
 };
-static int autotune_shape(const dp_weight& w, int64_t M, uint32_t flags, int* bn_out, int* cg_out, int* ws_out) {
+static int autotune_shape(const dp_weight& w, int64_t M, uint32_t flags, int* bn_out, int* cg_out, int* ws_out,
+                          int* pre_out) {
   struct Cand {
-    int bn, cg, ws;
+    int bn, cg, ws, pre;
   };
   std::vector<Cand> cands;
   const int widths[4] = {64, 128, 192, 256};
-  for (int i = 0; i < 4; ++i)
-    if (w.N % widths[i] == 0) {
-      cands.push_back({widths[i], 1, 0});
-      if (widths[i] >= 128) cands.push_back({widths[i], 2, 0});
-      if (widths[i] >= 192 && gemm_ws_supported(w.N, w.K)) cands.push_back({widths[i], 2, 1});
-    }
+  for (int pre = 0; pre <= (w.bits < 8 ? 1 : 0); ++pre)
+    for (int i = 0; i < 4; ++i)
+      if (w.N % widths[i] == 0) {
+        cands.push_back({widths[i], 1, 0, pre});
+        if (widths[i] >= 128) cands.push_back({widths[i], 2, 0, pre});
+        if (widths[i] >= 192 && gemm_ws_supported(w.N, w.K)) cands.push_back({widths[i], 2, 1, pre});
+      }
   void *x = nullptr, *y = nullptr, *ws = nullptr;
   cudaStream_t stream = nullptr;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   const size_t xb = static_cast<size_t>(M) * w.K * 2, yb = static_cast<size_t>(M) * w.N * 2;
-  const size_t wb = dp_wq_linear_workspace(M, w.N, w.K, w.bits, 0);
+  const size_t wb = dp_wq_linear_workspace(M, w.N, w.K, w.bits, DP_FLAG_UNPACK_FIRST);
   cudaError_t e = cudaMalloc(&x, xb);
   if (e == cudaSuccess) e = cudaMalloc(&y, yb);
   if (e == cudaSuccess) e = cudaMalloc(&ws, wb);
@@ -396,7 +426,7 @@ static int autotune_shape(const dp_weight& w, int64_t M, uint32_t flags, int* bn
     for (int it = 0; it < warm + reps && st == DP_OK; ++it) {
       if (it == warm) cudaEventRecord(e0, stream);
       st = run_linear(&w, x, w.K, nullptr, M, y, w.N, ws, nullptr, nullptr, flags & DP_FLAG_NO_PDL, stream, &tw,
-                      cands[c].bn, cands[c].cg, cands[c].ws, nullptr, it > 0);
+                      cands[c].bn, cands[c].cg, cands[c].ws, nullptr, it > 0, nullptr, cands[c].pre);
     }
     if (st != DP_OK) break;
     cudaEventRecord(e1, stream);
@@ -412,6 +442,7 @@ static int autotune_shape(const dp_weight& w, int64_t M, uint32_t flags, int* bn
       *bn_out = cands[c].bn;
       *cg_out = cands[c].cg;
       *ws_out = cands[c].ws;
+      *pre_out = cands[c].pre;
     }
   }
   if (e0) cudaEventDestroy(e0);
@@ -460,6 +491,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
     L.bn = 0;
     L.cg = 1;
     L.ws = 0;
+    L.pre = 0;
     memset(&L.tmap_w, 0, sizeof(L.tmap_w));
     if (L.simt && static_cast<size_t>(L.w.K) > simt_max_k()) {
       delete p;
@@ -469,14 +501,15 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
       uint32_t lf = flags;  // a pair request that this layer's N cannot honour falls back to the default
       if ((lf & DP_FLAG_CTA_PAIR) && L.w.N % 128 && L.w.N % 192) lf &= ~DP_FLAG_CTA_PAIR;
       if ((lf & DP_FLAG_WEIGHT_STATIONARY) && !gemm_ws_supported(L.w.N, L.w.K)) lf &= ~DP_FLAG_WEIGHT_STATIONARY;
-      choose_tile(lf, L.M, L.w.N, L.w.K, L.w.bits, &L.bn, &L.cg, &L.ws);
+      L.pre = ((lf & DP_FLAG_UNPACK_FIRST) && L.w.bits < 8) ? 1 : 0;
+      choose_tile(lf, L.M, L.w.N, L.w.K, L.pre ? 8 : L.w.bits, &L.bn, &L.cg, &L.ws);
       if (autotune) {
         const TunedShape* hit = nullptr;
         for (const TunedShape& t : tuned)
           if (t.M == L.M && t.N == L.w.N && t.K == L.w.K && t.bits == L.w.bits) hit = &t;
         if (hit == nullptr) {
-          TunedShape t = {L.M, L.w.N, L.w.K, L.w.bits, L.bn, L.cg, L.ws};
-          st = autotune_shape(L.w, L.M, flags, &t.bn, &t.cg, &t.ws);
+          TunedShape t = {L.M, L.w.N, L.w.K, L.w.bits, L.bn, L.cg, L.ws, L.pre};
+          st = autotune_shape(L.w, L.M, flags, &t.bn, &t.cg, &t.ws, &t.pre);
           if (st != DP_OK) {
             delete p;
             return st;
@@ -487,6 +520,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
         L.bn = hit->bn;
         L.cg = hit->cg;
         L.ws = hit->ws;
+        L.pre = hit->pre;
       }
       st = gemm_encode_w(&L.tmap_w, L.w.qweight, L.w.N, L.w.K, L.w.bits, L.bn, L.cg);
       if (st != DP_OK) {
@@ -494,7 +528,8 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
         return st;
       }
     }
-    const size_t ws = dp_wq_linear_workspace(L.M, L.w.N, L.w.K, L.w.bits, flags);
+    const size_t ws = dp_wq_linear_workspace(L.M, L.w.N, L.w.K, L.w.bits,
+                                             (flags & ~DP_FLAG_UNPACK_FIRST) | (L.pre ? DP_FLAG_UNPACK_FIRST : 0));
     if (ws > p->workspace_bytes) p->workspace_bytes = ws;
     L.x_offset = p->x_bytes;
     p->x_bytes += align256(static_cast<size_t>(L.M) * L.w.K * 2);
@@ -548,6 +583,13 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
 }
 
 extern "C" size_t dp_plan_workspace(const dp_plan* plan) { return plan ? plan->workspace_bytes : 0; }
+extern "C" int dp_plan_layer_unpack_first(const dp_plan* plan, int32_t layer, int32_t* unpack_first) {
+  if (!plan || layer < 0 || layer >= static_cast<int32_t>(plan->layers.size()) || !unpack_first)
+    return fail(DP_ERR_INVALID_ARG, "dp_plan_layer_unpack_first: bad plan, layer index or NULL output");
+  const PlanLayer& L = plan->layers[layer];
+  *unpack_first = (!L.simt && L.pre) ? 1 : 0;
+  return DP_OK;
+}
 extern "C" int dp_plan_layer_variant(const dp_plan* plan, int32_t layer, int32_t* tile_n, int32_t* cta_group,
                                      int32_t* weight_stationary, int32_t* small_m) {
   if (!plan || layer < 0 || layer >= static_cast<int32_t>(plan->layers.size()))
@@ -628,7 +670,7 @@ static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, 
     }
     int st = run_linear(&L.w, xs[l], L.w.K, nullptr, L.M, ys[l], L.w.N, workspace, nullptr, status,
                         plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, L.cg, L.ws, ta, *chained,
-                        L.simt ? nullptr : plan->daq_sync);
+                        L.simt ? nullptr : plan->daq_sync, L.simt ? 0 : L.pre);
     if (st != DP_OK) return st;
     *chained = true;
   }

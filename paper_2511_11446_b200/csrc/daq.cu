@@ -17,11 +17,15 @@ template <int MAXV, bool EO>
 __global__ void __launch_bounds__(kDaqWarps * 32)
 daq_rows_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t ldx,
                 int8_t* __restrict__ q, int64_t ldq, float* __restrict__ s_a,
-                int32_t* __restrict__ rowsum, int tiled_kb) {
+                int32_t* __restrict__ rowsum, int tiled_kb, const UnpackJob job) {
   pdl_launch_dependents();
   const int64_t row = static_cast<int64_t>(blockIdx.x) * kDaqWarps + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   pdl_wait();
+  if (static_cast<int>(blockIdx.x) >= job.first_block) {  // the launch's weight-expansion CTAs
+    unpack_units(job, blockIdx.x - job.first_block);
+    return;
+  }
   if (row >= M) return;
   const int nvec = K >> 3;
   const uint4* xr = reinterpret_cast<const uint4*>(x + row * ldx);
@@ -67,11 +71,15 @@ template <bool EO>
 __global__ void __launch_bounds__(kDaqWarps * 32)
 daq_rows_2pass_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t ldx,
                       int8_t* __restrict__ q, int64_t ldq, float* __restrict__ s_a,
-                      int32_t* __restrict__ rowsum, int tiled_kb) {
+                      int32_t* __restrict__ rowsum, int tiled_kb, const UnpackJob job) {
   pdl_launch_dependents();
   const int64_t row = static_cast<int64_t>(blockIdx.x) * kDaqWarps + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   pdl_wait();
+  if (static_cast<int>(blockIdx.x) >= job.first_block) {  // the launch's weight-expansion CTAs
+    unpack_units(job, blockIdx.x - job.first_block);
+    return;
+  }
   if (row >= M) return;
   const int nvec = K >> 3;
   const uint4* xr = reinterpret_cast<const uint4*>(x + row * ldx);
@@ -98,30 +106,52 @@ daq_rows_2pass_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t 
   }
 }
 
+__global__ void __launch_bounds__(kDaqWarps * 32)
+unpack_kernel(const UnpackJob job) {
+  pdl_launch_dependents();
+  pdl_wait();
+  unpack_units(job, blockIdx.x);
+}
+
 template <bool EO>
 static cudaError_t launch_daq_t(const uint16_t* xp, int64_t M, int k, int64_t ldx, int8_t* q, int64_t ldq,
-                                float* s_a, int32_t* rowsum, int tiled_kb, cudaStream_t stream, bool pdl) {
-  const dim3 grid(static_cast<unsigned>((M + kDaqWarps - 1) / kDaqWarps));
+                                float* s_a, int32_t* rowsum, int tiled_kb, cudaStream_t stream, bool pdl,
+                                UnpackJob job) {
+  const unsigned daq_blocks = static_cast<unsigned>((M + kDaqWarps - 1) / kDaqWarps);
+  job.first_block = static_cast<int32_t>(daq_blocks);
+  const unsigned extra = static_cast<unsigned>((job.units + kDaqWarps * 32 - 1) / (kDaqWarps * 32));
+  const dim3 grid(daq_blocks + extra);
   const dim3 block(kDaqWarps * 32);
   if (k <= 256 * 5)
-    return launch(daq_rows_kernel<5, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb);
+    return launch(daq_rows_kernel<5, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb, job);
   if (k <= 256 * 9)
-    return launch(daq_rows_kernel<9, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb);
+    return launch(daq_rows_kernel<9, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb, job);
   if (k <= 256 * 18)
-    return launch(daq_rows_kernel<18, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb);
-  return launch(daq_rows_2pass_kernel<EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb);
+    return launch(daq_rows_kernel<18, EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb, job);
+  return launch(daq_rows_2pass_kernel<EO>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb, job);
 }
 
 int launch_daq(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq,
-               float* s_a, int32_t* rowsum, int korder, bool tiled, cudaStream_t stream, bool pdl) {
+               float* s_a, int32_t* rowsum, int korder, bool tiled, cudaStream_t stream, bool pdl,
+               const UnpackJob* unpack) {
   if (M == 0) return DP_OK;
   const uint16_t* xp = static_cast<const uint16_t*>(x);
   const int k = static_cast<int>(K);
   const int tiled_kb = tiled ? k / 128 : 0;
+  UnpackJob job{nullptr, nullptr, 0, 0, 0};
+  if (unpack != nullptr) job = *unpack;
   const cudaError_t e = korder == KORDER_EVEN_ODD
-                            ? launch_daq_t<true>(xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb, stream, pdl)
-                            : launch_daq_t<false>(xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb, stream, pdl);
+                            ? launch_daq_t<true>(xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb, stream, pdl, job)
+                            : launch_daq_t<false>(xp, M, k, ldx, q, ldq, s_a, rowsum, tiled_kb, stream, pdl, job);
   if (e != cudaSuccess) return fail(DP_ERR_CUDA, "DAQ launch failed: %s", cudaGetErrorString(e));
+  return DP_OK;
+}
+
+int launch_unpack(const UnpackJob& job, cudaStream_t stream, bool pdl) {
+  if (job.units == 0) return DP_OK;
+  const dim3 grid(static_cast<unsigned>((job.units + kDaqWarps * 32 - 1) / (kDaqWarps * 32)));
+  const cudaError_t e = launch(unpack_kernel, grid, dim3(kDaqWarps * 32), 0, stream, pdl, job);
+  if (e != cudaSuccess) return fail(DP_ERR_CUDA, "weight expansion launch failed: %s", cudaGetErrorString(e));
   return DP_OK;
 }
 

@@ -137,4 +137,49 @@ __device__ __forceinline__ void daq_two_rows_2pass(const uint16_t* __restrict__ 
   }
 }
 
+// Packed unit -> 8 words of 4 int8 (true values, k ascending).
+template <int BITS>
+__device__ __forceinline__ void expand_unit(const uint32_t (&pk)[BITS], uint32_t (&w)[8]) {
+  if constexpr (BITS == 8) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) w[i] = pk[i];
+  } else if constexpr (BITS == 4) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t lo = pk[i] & 0x0F0F0F0Fu, hi = (pk[i] >> 4) & 0x0F0F0F0Fu;
+      w[2 * i] = __vsub4(__byte_perm(lo, hi, 0x5140), 0x08080808u);
+      w[2 * i + 1] = __vsub4(__byte_perm(lo, hi, 0x7362), 0x08080808u);
+    }
+  } else {
+    const uint64_t lo64 = (static_cast<uint64_t>(pk[1]) << 32) | pk[0];
+    const uint64_t hi64 = (static_cast<uint64_t>(pk[2]) << 32) | pk[1];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int bit = 12 * j;
+      const uint32_t x = static_cast<uint32_t>(bit < 32 ? (lo64 >> bit) : (hi64 >> (bit - 32))) & 0xFFFu;
+      const uint32_t o = (x & 7u) | ((x & 0x38u) << 5) | ((x & 0x1C0u) << 10) | ((x & 0xE00u) << 15);
+      w[j] = __vsub4(o, 0x04040404u);
+    }
+  }
+}
+
+// CTA `block` of an unpack job: one thread per unit of 32 codes (12 or 16 bytes in, 32 bytes out).
+__device__ __forceinline__ void unpack_units(const UnpackJob& job, const int block) {
+  const int64_t u = static_cast<int64_t>(block) * blockDim.x + threadIdx.x;
+  if (u >= job.units) return;
+  uint32_t w[8];
+  if (job.bits == 4) {
+    const uint4 v = reinterpret_cast<const uint4*>(job.packed)[u];
+    const uint32_t pk[4] = {v.x, v.y, v.z, v.w};
+    expand_unit<4>(pk, w);
+  } else {
+    const uint32_t* p = job.packed + u * 3;
+    const uint32_t pk[3] = {p[0], p[1], p[2]};
+    expand_unit<3>(pk, w);
+  }
+  uint4* o = reinterpret_cast<uint4*>(job.out) + u * 2;
+  o[0] = make_uint4(w[0], w[1], w[2], w[3]);
+  o[1] = make_uint4(w[4], w[5], w[6], w[7]);
+}
+
 }  // namespace dp

@@ -18,8 +18,19 @@ enum KOrder {
 int gemm_korder(int32_t bits);
 
 // daq.cu
+// Expansion of a packed weight matrix to int8 [N][K] (true values, k ascending) in global scratch,
+// run by extra CTAs of a DAQ launch or on its own: `units` = N * K / 32 units of 32 codes.
+struct UnpackJob {
+  const uint32_t* packed;
+  int8_t* out;
+  int64_t units;
+  int32_t bits;         // 3 or 4
+  int32_t first_block;  // filled by the launcher: CTAs from here on unpack
+};
 int launch_daq(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq,
-               float* s_a, int32_t* rowsum, int korder, bool tiled, cudaStream_t stream, bool pdl);
+               float* s_a, int32_t* rowsum, int korder, bool tiled, cudaStream_t stream, bool pdl,
+               const UnpackJob* unpack = nullptr);
+int launch_unpack(const UnpackJob& job, cudaStream_t stream, bool pdl);
 
 // simt.cu — CUDA-core weight-streaming linear for small M (DAQ fused in the CTA prologue).
 struct SimtArgs {

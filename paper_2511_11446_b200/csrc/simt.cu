@@ -71,32 +71,6 @@ __device__ __forceinline__ void fetch_unit(const uint32_t* __restrict__ row, int
   }
 }
 
-// Packed unit -> 8 words of 4 int8 (true values, k ascending).
-template <int BITS>
-__device__ __forceinline__ void expand_unit(const uint32_t (&pk)[BITS], uint32_t (&w)[8]) {
-  if constexpr (BITS == 8) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) w[i] = pk[i];
-  } else if constexpr (BITS == 4) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint32_t lo = pk[i] & 0x0F0F0F0Fu, hi = (pk[i] >> 4) & 0x0F0F0F0Fu;
-      w[2 * i] = __vsub4(__byte_perm(lo, hi, 0x5140), 0x08080808u);
-      w[2 * i + 1] = __vsub4(__byte_perm(lo, hi, 0x7362), 0x08080808u);
-    }
-  } else {
-    const uint64_t lo64 = (static_cast<uint64_t>(pk[1]) << 32) | pk[0];
-    const uint64_t hi64 = (static_cast<uint64_t>(pk[2]) << 32) | pk[1];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int bit = 12 * j;
-      const uint32_t x = static_cast<uint32_t>(bit < 32 ? (lo64 >> bit) : (hi64 >> (bit - 32))) & 0xFFFu;
-      const uint32_t o = (x & 7u) | ((x & 0x38u) << 5) | ((x & 0x1C0u) << 10) | ((x & 0xE00u) << 15);
-      w[j] = __vsub4(o, 0x04040404u);
-    }
-  }
-}
-
 // Token `warp` of this CTA -> int8 in shared memory, by one warp (rows `pitch` bytes apart), and
 // its scale: DAQ here (Step 3, Eq. "daq"), or a copy when the caller passes quantized tokens.
 __device__ __forceinline__ void stage_tokens(const SimtArgs& a, const int64_t m0, const int block_x,

@@ -208,7 +208,23 @@ def test_single_token_and_minimal_k_through_the_tensor_core_path():
             _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | variant), x, w, s_w, b, bits, exact_y=False)
 
 
-@pytest.mark.parametrize("flags", [B.DP_FLAG_FORCE_SIMT, B.DP_FLAG_FORCE_MMA])
+@pytest.mark.parametrize("bits", [4, 3])
+@pytest.mark.parametrize("variant", [0, B.DP_FLAG_CTA_PAIR | B.DP_FLAG_NO_WEIGHT_STATIONARY,
+                                     B.DP_FLAG_WEIGHT_STATIONARY])
+@pytest.mark.parametrize("M,K,N", [(300, 1152, 384), (2048, 384, 768), (77, 128, 192)])
+def test_mma_unpack_first(bits, variant, M, K, N):
+    """Packed weights expanded once to int8 in the workspace (extra CTAs of the DAQ launch), then the
+    8-bit kernel on the copy: every code value, ragged M, single-CTA / pair / weight-stationary."""
+    x, w, s_w, b = _case(M, K, N, bits, full_range=True)
+    L = DevLayer(w, s_w, b, bits)
+    flags = B.DP_FLAG_FORCE_MMA | B.DP_FLAG_UNPACK_FIRST | variant
+    assert (B.dp_wq_linear_workspace(M, N, K, bits, flags) - B.dp_wq_linear_workspace(M, N, K, bits, flags & ~B.DP_FLAG_UNPACK_FIRST)
+            >= N * K)
+    _check(run_linear(L, x, flags=flags), x, w, s_w, b, bits)
+
+
+@pytest.mark.parametrize("flags", [B.DP_FLAG_FORCE_SIMT, B.DP_FLAG_FORCE_MMA,
+                                   B.DP_FLAG_FORCE_MMA | B.DP_FLAG_UNPACK_FIRST])
 def test_prequantized_input(flags):
     M, K, N, bits = 130, 256, 128, 4
     x, w, s_w, b = _case(M, K, N, bits)
@@ -217,6 +233,20 @@ def test_prequantized_input(flags):
     out = run_linear(L, x, flags=flags, prequant=(q, s_a), taps=False)
     y = oracle.wq_linear(x, oracle.pack(w, bits), s_w, b, bits)
     assert out["status"] == 0 and bf16_ulp_dist(out["y"], y).max() <= 1
+
+
+def test_unpack_first_without_workspace_is_refused():
+    """Quantized activations need no scratch, the int8 copy of the weights does: no launch without it."""
+    M, K, N, bits = 130, 256, 128, 4
+    x, w, s_w, b = _case(M, K, N, bits)
+    q, s_a, _ = oracle.daq(x)
+    L = DevLayer(w, s_w, b, bits)
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.DiffproError) as e:
+        B.dp_wq_linear(L.w, torch.from_numpy(q.copy()).cuda(), K, torch.from_numpy(s_a.copy()).cuda(), M, y, N, None,
+                       None, status, B.DP_FLAG_FORCE_MMA | B.DP_FLAG_UNPACK_FIRST)
+    assert e.value.status == B.DP_ERR_WORKSPACE
 
 
 def test_default_dispatch_and_argument_errors():
