@@ -154,7 +154,14 @@ def run_ours(args):
     peaks = measured_peaks()
 
     seed = D.rank_seed(synth.BASE_SEED + 4, rank)
-    stack = DitStack(seed=seed)
+    variants = None
+    if args.load_variants:
+        with open(args.load_variants) as f:
+            variants = json.load(f)
+    stack = DitStack(seed=seed, variants=variants)
+    if args.save_variants and rank == 0:
+        with open(args.save_variants, "w") as f:
+            json.dump(stack.layer_variants(), f)
     nL, nS = len(stack.table), len(stack.kept)
     ops_step = stack.ops_per_timestep() * nS
     graph = stack.capture()
@@ -413,6 +420,11 @@ def main():
     ap.add_argument("--only", default=None, choices=["layer", "gemm", "daq"])
     ap.add_argument("--iters", type=int, default=None)
     ap.add_argument("--flags", type=lambda v: int(v, 0), default=0, help="dp_wq_linear tuning flags for --sweep")
+    ap.add_argument("--save-variants", default=None,
+                    help="write the per-layer kernel variants the autotuner chose to this JSON file")
+    ap.add_argument("--load-variants", default=None,
+                    help="apply per-layer kernel variants from this JSON file instead of autotuning (a run "
+                         "under a profiler times variants differently, so profiles reuse a plain run's choice)")
     ap.add_argument("--hbm-kernels", action="store_true",
                     help="time only the HBM-bound kernels (grouped adaLN launch, DAQ at M=32768) and print their rooflines")
     args = ap.parse_args()

@@ -217,6 +217,14 @@ int dp_plan_layer_variant(const dp_plan* plan, int32_t layer, int32_t* tile_n, i
 /* *unpack_first = 1 when the plan runs layer `layer` in the DP_FLAG_UNPACK_FIRST form (the
  * variant dp_plan_layer_variant reports is then the 8-bit kernel's). No counterpart in the paper. */
 int dp_plan_layer_unpack_first(const dp_plan* plan, int32_t layer, int32_t* unpack_first);
+/* Replaces the kernel variant of layer `layer` by the one `flags` names (the tuning flags of
+ * dp_wq_linear: DP_FLAG_TILE_N, [NO_]CTA_PAIR, [NO_]WEIGHT_STATIONARY, UNPACK_FIRST; anything left
+ * open is chosen as dp_wq_linear would): lets a deployment keep the outcome of one
+ * DP_FLAG_AUTOTUNE run and apply it to later plans. Host only; may raise dp_plan_workspace, so ask
+ * again afterwards. Small-M layers and unknown bits are refused (DP_ERR_INVALID_ARG), tile widths
+ * that do not fit the layer with DP_ERR_SHAPE; the plan is unchanged on error. Not to be called
+ * while a dp_plan_run of the plan is being issued. No counterpart in the paper. */
+int dp_plan_set_layer_flags(dp_plan* plan, int32_t layer, uint32_t flags);
 void dp_plan_destroy(dp_plan* plan);
 
 /*

@@ -583,6 +583,26 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
 }
 
 extern "C" size_t dp_plan_workspace(const dp_plan* plan) { return plan ? plan->workspace_bytes : 0; }
+extern "C" int dp_plan_set_layer_flags(dp_plan* plan, int32_t layer, uint32_t flags) {
+  if (!plan || layer < 0 || layer >= static_cast<int32_t>(plan->layers.size()))
+    return fail(DP_ERR_INVALID_ARG, "dp_plan_set_layer_flags: bad plan or layer index");
+  PlanLayer& L = plan->layers[layer];
+  constexpr uint32_t kVariantFlags = DP_FLAG_TILE_N_MASK | DP_FLAG_CTA_PAIR | DP_FLAG_NO_CTA_PAIR |
+                                     DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_UNPACK_FIRST;
+  if (flags & ~kVariantFlags) return fail(DP_ERR_INVALID_ARG, "dp_plan_set_layer_flags: flag bits 0x%x do not name a variant", flags);
+  if (L.simt || L.M == 0) return fail(DP_ERR_INVALID_ARG, "layer %d runs the small-M kernel: it has no variants", layer);
+  if (int st = check_tile_flags(flags, L.w.N)) return st;
+  if ((flags & DP_FLAG_WEIGHT_STATIONARY) && !gemm_ws_supported(L.w.N, L.w.K))
+    return fail(DP_ERR_SHAPE, "layer %d: the weight-stationary kernel does not take N=%d K=%d", layer, L.w.N, L.w.K);
+  PlanLayer T = L;
+  T.pre = ((flags & DP_FLAG_UNPACK_FIRST) && T.w.bits < 8) ? 1 : 0;
+  choose_tile(flags, T.M, T.w.N, T.w.K, T.pre ? 8 : T.w.bits, &T.bn, &T.cg, &T.ws);
+  if (int st = gemm_encode_w(&T.tmap_w, T.w.qweight, T.w.N, T.w.K, T.w.bits, T.bn, T.cg)) return st;
+  L = T;
+  const size_t ws = dp_wq_linear_workspace(L.M, L.w.N, L.w.K, L.w.bits, L.pre ? DP_FLAG_UNPACK_FIRST : 0);
+  if (ws > plan->workspace_bytes) plan->workspace_bytes = ws;
+  return DP_OK;
+}
 extern "C" int dp_plan_layer_unpack_first(const dp_plan* plan, int32_t layer, int32_t* unpack_first) {
   if (!plan || layer < 0 || layer >= static_cast<int32_t>(plan->layers.size()) || !unpack_first)
     return fail(DP_ERR_INVALID_ARG, "dp_plan_layer_unpack_first: bad plan, layer index or NULL output");

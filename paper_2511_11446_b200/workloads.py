@@ -40,7 +40,11 @@ class DevWeights:
 class DitStack:
     def __init__(self, seed=synth.BASE_SEED + 4, batch=8, tokens=256, blocks=synth.BLOCKS, T=50, keep=25,
                  bit_choices=(3, 4, 8), resident_steps=None,
-                 flags=B.DP_FLAG_AUTOTUNE | B.DP_FLAG_GROUP_SMALL_M):
+                 flags=B.DP_FLAG_AUTOTUNE | B.DP_FLAG_GROUP_SMALL_M, variants=None):
+        """variants: per-layer tuning flags from an earlier autotuned stack's layer_variants() (None
+        entries: small-M layers); given, the plan applies them instead of timing variants itself."""
+        if variants is not None:
+            flags &= ~B.DP_FLAG_AUTOTUNE
         self.seed, self.T, self.flags = seed, T, flags
         self.table = synth.dit_layers(batch, tokens, blocks)
         self.bits = synth.bit_plan(seed, len(self.table), bit_choices)
@@ -48,6 +52,10 @@ class DitStack:
         self.layers = [DevWeights(seed, l, N, K, self.bits[l]) for l, (_, M, K, N) in enumerate(self.table)]
         self.Ms = [M for (_, M, K, N) in self.table]
         self.plan = B.dp_plan_create([L.w for L in self.layers], self.Ms, flags)
+        if variants is not None:
+            for l, f in enumerate(variants):
+                if f is not None:
+                    B.dp_plan_set_layer_flags(self.plan, l, f)
         self.workspace = torch.empty(B.dp_plan_workspace(self.plan), dtype=torch.uint8, device="cuda")
         self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
         self.y = [torch.empty((M, N), dtype=torch.bfloat16, device="cuda") for (_, M, K, N) in self.table]
@@ -65,6 +73,15 @@ class DitStack:
         _, M, K, _ = self.table[l]
         return synth.activations(self.seed, l, t, M, K, synth.sigma_t(t, self.T), n_out=max(1, K // 100),
                                  rows=rows)
+
+    def layer_variants(self):
+        """Per layer: the tuning flags naming the kernel variant the plan runs (None: small-M kernel)."""
+        out = []
+        for l in range(len(self.table)):
+            v = B.dp_plan_layer_variant(self.plan, l)
+            out.append(None if v["small_m"] else
+                       B.variant_flags(v) & ~(B.DP_FLAG_FORCE_MMA | B.DP_FLAG_FORCE_SIMT))
+        return out
 
     # ---- accounting ----
     def ops_per_timestep(self):

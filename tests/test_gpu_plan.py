@@ -116,6 +116,53 @@ def test_plan_autotuned_and_grouped_matches_oracle(extra):
         B.dp_plan_destroy(plan)
 
 
+def test_plan_with_variants_set_per_layer_matches_oracle():
+    """dp_plan_set_layer_flags: every tensor-core layer switched to another variant after creation
+    (unpack-first for the packed ones, CTA pairs / forced widths for the rest), workspace asked again,
+    every output still the oracle's; small-M layers and nonsense flags are refused."""
+    table, layers, dev = _mini_plan(tokens=256, batch=2, blocks=2)
+    T, kept = 6, [2, 5]
+    nL, nS = len(layers), len(kept)
+    xs = [[synth.activations(SEED, l, t, L["M"], L["K"], synth.sigma_t(t, T), n_out=max(1, L["K"] // 100))
+           for l, L in enumerate(layers)] for t in kept]
+    ref = oracle.plan_run(layers, kept, xs)
+    plan = B.dp_plan_create([d.w for d in dev], [L["M"] for L in layers], B.DP_FLAG_GROUP_SMALL_M)
+    try:
+        before = B.dp_plan_workspace(plan)
+        choices = [B.DP_FLAG_UNPACK_FIRST | B.DP_FLAG_TILE_N(128) | B.DP_FLAG_NO_CTA_PAIR,
+                   B.DP_FLAG_CTA_PAIR | B.DP_FLAG_NO_WEIGHT_STATIONARY | B.DP_FLAG_UNPACK_FIRST,
+                   B.DP_FLAG_TILE_N(64) | B.DP_FLAG_NO_CTA_PAIR]
+        n_set = 0
+        for l, L in enumerate(layers):
+            if B.dp_plan_layer_variant(plan, l)["small_m"]:
+                with pytest.raises(B.DiffproError):
+                    B.dp_plan_set_layer_flags(plan, l, B.DP_FLAG_UNPACK_FIRST)
+                continue
+            B.dp_plan_set_layer_flags(plan, l, choices[n_set % 3])
+            v = B.dp_plan_layer_variant(plan, l)
+            assert v["unpack_first"] == (1 if (choices[n_set % 3] & B.DP_FLAG_UNPACK_FIRST) and L["bits"] < 8 else 0)
+            n_set += 1
+        with pytest.raises(B.DiffproError):
+            B.dp_plan_set_layer_flags(plan, 0, B.DP_FLAG_FORCE_MMA)
+        assert n_set >= 8 and B.dp_plan_workspace(plan) > before
+        ws = torch.empty(B.dp_plan_workspace(plan), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        xd = [[to_dev_bf16(xs[i][l]) for l in range(nL)] for i in range(nS)]
+        yd = [[torch.full((L["M"], L["N"]), float("nan"), dtype=torch.bfloat16, device="cuda")
+               for L in layers] for _ in range(nS)]
+        xp = B.ptr_array([xd[i][l].data_ptr() for i in range(nS) for l in range(nL)])
+        yp = B.ptr_array([yd[i][l].data_ptr() for i in range(nS) for l in range(nL)])
+        B.dp_plan_run(plan, kept, 0, xp, yp, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for i in range(nS):
+            for l in range(nL):
+                d = bf16_ulp_dist(bf16_to_np(yd[i][l]), ref[i][l])
+                assert d.max() <= 1, (i, l, table[l], int(d.max()))
+    finally:
+        B.dp_plan_destroy(plan)
+
+
 def test_plan_run_host_inputs():
     table, layers, dev = _mini_plan(tokens=128, batch=2, blocks=1)
     kept = [1, 3, 4]
