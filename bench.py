@@ -29,7 +29,8 @@ UNIT = "TOPS"
 NOMINAL_INT8_TOPS = 4500.0
 # dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch, averaged over the four M = 2048 layer
 # shapes, from the ncu capture summarised in profiles/ (None until that capture matches the kernels).
-GEMM_DRAM_BYTES_PER_LAUNCH = 5.09e6  # 4-bit layers; reads only: the bf16 outputs stay in L2 past the kernel's end
+GEMM_DRAM_BYTES_PER_LAUNCH = 6.99e6  # 8-bit kernel on int8 activations + int8 weights, cold L2; reads only: the
+                                     # bf16 outputs stay in L2 past the kernel's end
 
 
 def measured_peaks():
