@@ -117,15 +117,20 @@ typedef struct dp_debug {
  * (programmatic dependent launch) while the previous GEMM drains. */
 #define DP_FLAG_FUSED_DAQ 0x40000u
 
-/* dp_wq_linear and dp_plan_create, packed bit-widths (3, 4) on the tensor-core path: expand the
- * packed weights once per call to int8 [N][K] in the workspace (extra CTAs of the DAQ launch; a
- * launch of its own when the activations arrive quantized) and run the 8-bit kernel on that copy,
- * instead of expanding the tiles in shared memory inside the GEMM (Step 4's unpack, hoisted). Pays
- * when a weight tile is consumed by many row tiles but each CTA sees it only once or twice (M of a
- * few thousand): there the in-kernel expansion is repeated M/128 times across CTAs. The copy lives
- * only for the call, the weights stay packed in memory, results are identical. Adds N*K bytes to
- * the workspace. With DP_FLAG_AUTOTUNE the plan times both forms per layer shape. */
+/* dp_wq_linear and dp_plan_create, packed bit-widths (3, 4) on the tensor-core path: where the
+ * packed weights are expanded (Step 4's unpack). UNPACK_FIRST: once per call to int8 [N][K] in the
+ * workspace (extra CTAs of the DAQ launch; a launch of its own when the activations arrive
+ * quantized), the 8-bit kernel then runs on that copy. NO_UNPACK_FIRST: tile by tile in shared memory
+ * inside the GEMM. The first form avoids repeating the expansion in every CTA that needs a weight
+ * tile (M/128 of them) and was faster on B200 at every size measured except where the
+ * weight-stationary kernel applies (there equal), so it is the default whenever the library runs DAQ
+ * itself; with quantized activations (s_a given) the default is the in-GEMM form, which needs no
+ * workspace. The copy lives only for the call, the weights stay packed in memory, results are
+ * identical. Adds N*K bytes to the workspace (dp_wq_linear_workspace counts them unless
+ * NO_UNPACK_FIRST is given). With DP_FLAG_AUTOTUNE the plan times both forms per layer shape.
+ * Giving both flags is an error. */
 #define DP_FLAG_UNPACK_FIRST 0x80000u
+#define DP_FLAG_NO_UNPACK_FIRST 0x100000u
 
 /* flags for dp_plan_run */
 #define DP_PLAN_SAME_X 1u       /* x_ptrs has n_layers entries reused by every step              */

@@ -22,7 +22,8 @@ DP_FLAG_NONE, DP_FLAG_FORCE_SIMT, DP_FLAG_FORCE_MMA, DP_FLAG_NO_PDL = 0, 1, 2, 4
 DP_FLAG_CTA_PAIR, DP_FLAG_NO_CTA_PAIR = 0x800, 0x1000
 DP_FLAG_WEIGHT_STATIONARY, DP_FLAG_NO_WEIGHT_STATIONARY = 0x2000, 0x4000
 DP_FLAG_AUTOTUNE, DP_FLAG_GROUP_SMALL_M, DP_FLAG_FUSED_DAQ = 0x10000, 0x20000, 0x40000
-DP_FLAG_UNPACK_FIRST = 0x80000
+DP_FLAG_UNPACK_FIRST, DP_FLAG_NO_UNPACK_FIRST = 0x80000, 0x100000
+DP_FLAG_TILE_N_MASK = 0x700
 DP_PLAN_SAME_X, DP_PLAN_SAME_Y = 1, 2
 
 
@@ -173,8 +174,7 @@ def variant_flags(v: dict) -> int:
     if v["small_m"]:
         return DP_FLAG_FORCE_SIMT
     f = DP_FLAG_FORCE_MMA | DP_FLAG_TILE_N(v["tile_n"])
-    if v.get("unpack_first"):
-        f |= DP_FLAG_UNPACK_FIRST
+    f |= DP_FLAG_UNPACK_FIRST if v.get("unpack_first") else DP_FLAG_NO_UNPACK_FIRST
     if v["weight_stationary"]:
         return f | DP_FLAG_WEIGHT_STATIONARY
     f |= DP_FLAG_NO_WEIGHT_STATIONARY

@@ -52,7 +52,8 @@ static size_t scratch_q_bytes(int64_t M, int32_t K) { return static_cast<size_t>
 
 constexpr uint32_t kLinearFlags =
     DP_FLAG_FORCE_SIMT | DP_FLAG_FORCE_MMA | DP_FLAG_NO_PDL | DP_FLAG_TILE_N_MASK | DP_FLAG_CTA_PAIR |
-    DP_FLAG_NO_CTA_PAIR | DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_UNPACK_FIRST;
+    DP_FLAG_NO_CTA_PAIR | DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_UNPACK_FIRST |
+    DP_FLAG_NO_UNPACK_FIRST;
 constexpr int64_t kWsMinRows = 8192;  // from here on a resident weight strip is reused often enough to pay
 static int forced_bn(uint32_t flags) { return static_cast<int>((flags & DP_FLAG_TILE_N_MASK) >> 8) * 64; }
 
@@ -91,6 +92,14 @@ static int check_tile_flags(uint32_t flags, int32_t N) {
   if ((flags & DP_FLAG_WEIGHT_STATIONARY) && (flags & (DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_NO_CTA_PAIR)))
     return fail(DP_ERR_INVALID_ARG, "WEIGHT_STATIONARY contradicts another flag");
   return DP_OK;
+}
+
+// Whether a packed layer runs in the unpack-first form: the flags decide; by default it does when
+// the library quantizes the activations itself (a workspace exists and the expansion rides in the
+// DAQ launch).
+static bool want_unpack_first(uint32_t flags, int32_t bits, bool library_daq) {
+  if (bits >= 8 || (flags & DP_FLAG_NO_UNPACK_FIRST)) return false;
+  return (flags & DP_FLAG_UNPACK_FIRST) || library_daq;
 }
 
 constexpr int64_t kSimtMaxRows = 32;  // at or below this the CUDA-core streaming kernel is used
@@ -159,7 +168,7 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
   // Unpack-first variant: the packed weights are expanded once to int8 [N][K] in the workspace (by
   // extra CTAs of the DAQ launch) and the 8-bit kernel runs on that copy, instead of every CTA
   // expanding the weight tiles it needs in shared memory.
-  if (pre < 0) pre = (flags & DP_FLAG_UNPACK_FIRST) ? 1 : 0;
+  if (pre < 0) pre = want_unpack_first(flags, w->bits, s_a_in == nullptr) ? 1 : 0;
   const bool unpack_first = pre > 0 && w->bits < 8;
   dp_weight w8 = *w;
   UnpackJob job{nullptr, nullptr, 0, 0, 0};
@@ -262,6 +271,8 @@ static int check_linear_args(const dp_weight* w, const void* x, int64_t ldx, con
   if (int tst = check_tile_flags(flags, w->N)) return tst;
   if ((flags & DP_FLAG_FORCE_SIMT) && (flags & DP_FLAG_FORCE_MMA))
     return fail(DP_ERR_INVALID_ARG, "FORCE_SIMT and FORCE_MMA are exclusive");
+  if ((flags & DP_FLAG_UNPACK_FIRST) && (flags & DP_FLAG_NO_UNPACK_FIRST))
+    return fail(DP_ERR_INVALID_ARG, "UNPACK_FIRST and NO_UNPACK_FIRST are exclusive");
   if (M == 0) return DP_OK;
   if (!x || !y) return fail(DP_ERR_INVALID_ARG, "x or y is NULL");
   if (ldx < w->K || ldy < w->N) return fail(DP_ERR_SHAPE, "leading dimension smaller than the row");
@@ -276,7 +287,7 @@ static int check_linear_args(const dp_weight* w, const void* x, int64_t ldx, con
   }
   // scratch users: the library's own DAQ, and the int8 copy of the weights of the unpack-first form
   if (!use_simt(M, w->N, w->K, flags) &&
-      (s_a_in == nullptr || ((flags & DP_FLAG_UNPACK_FIRST) && w->bits < 8))) {
+      (s_a_in == nullptr || want_unpack_first(flags, w->bits, false))) {
     const size_t need = dp_wq_linear_workspace(M, w->N, w->K, w->bits, flags);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))
       return fail(DP_ERR_WORKSPACE, "workspace needs %zu bytes, 256-byte aligned (got %zu)", need,
@@ -294,7 +305,7 @@ extern "C" size_t dp_wq_linear_workspace(int64_t M, int32_t N, int32_t K, int32_
   if (M <= 0 || K <= 0) return 256;
   if (use_simt(M, N, K, flags)) return 256;
   size_t need = align256(scratch_q_bytes(M, K)) + align256(sizeof(float) * static_cast<size_t>(M));
-  if ((flags & DP_FLAG_UNPACK_FIRST) && bits < 8) need += align256(static_cast<size_t>(N) * K);
+  if (want_unpack_first(flags, bits, true)) need += align256(static_cast<size_t>(N) * K);
   return need;
 }
 
@@ -337,6 +348,9 @@ static int static_scratch_address(void** out) {
 extern "C" int dp_wq_linear_static(const dp_weight* w, const void* x_bf16, int64_t ldx, int64_t M,
                                    void* y_bf16, int64_t ldy, int32_t* device_status, uint32_t flags,
                                    dp_stream stream) {
+  // The built-in scratch is sized for the activations only: weights are expanded inside the GEMM
+  // unless the caller asks otherwise (and the copy fits).
+  if (!(flags & DP_FLAG_UNPACK_FIRST)) flags |= DP_FLAG_NO_UNPACK_FIRST;
   int st = check_weight(w);
   if (st != DP_OK) return st;
   const size_t need = dp_wq_linear_workspace(M, w->N, w->K, w->bits, flags);
@@ -398,7 +412,9 @@ static int autotune_shape(const dp_weight& w, int64_t M, uint32_t flags, int* bn
   };
   std::vector<Cand> cands;
   const int widths[4] = {64, 128, 192, 256};
-  for (int pre = 0; pre <= (w.bits < 8 ? 1 : 0); ++pre)
+  const int pre_lo = (flags & DP_FLAG_UNPACK_FIRST) ? 1 : 0;
+  const int pre_hi = (w.bits < 8 && !(flags & (DP_FLAG_NO_UNPACK_FIRST | DP_FLAG_FUSED_DAQ))) ? 1 : 0;
+  for (int pre = pre_lo < pre_hi ? pre_lo : pre_hi; pre <= pre_hi; ++pre)
     for (int i = 0; i < 4; ++i)
       if (w.N % widths[i] == 0) {
         cands.push_back({widths[i], 1, 0, pre});
@@ -499,9 +515,11 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
     }
     if (!L.simt && L.M > 0) {
       uint32_t lf = flags;  // a pair request that this layer's N cannot honour falls back to the default
+      // DAQ inside the GEMM kernel and a DAQ launch that also expands the weights exclude each other
+      if ((lf & DP_FLAG_FUSED_DAQ) && !(lf & DP_FLAG_UNPACK_FIRST)) lf |= DP_FLAG_NO_UNPACK_FIRST;
       if ((lf & DP_FLAG_CTA_PAIR) && L.w.N % 128 && L.w.N % 192) lf &= ~DP_FLAG_CTA_PAIR;
       if ((lf & DP_FLAG_WEIGHT_STATIONARY) && !gemm_ws_supported(L.w.N, L.w.K)) lf &= ~DP_FLAG_WEIGHT_STATIONARY;
-      L.pre = ((lf & DP_FLAG_UNPACK_FIRST) && L.w.bits < 8) ? 1 : 0;
+      L.pre = want_unpack_first(lf, L.w.bits, true) ? 1 : 0;
       choose_tile(lf, L.M, L.w.N, L.w.K, L.pre ? 8 : L.w.bits, &L.bn, &L.cg, &L.ws);
       if (autotune) {
         const TunedShape* hit = nullptr;
@@ -529,7 +547,8 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
       }
     }
     const size_t ws = dp_wq_linear_workspace(L.M, L.w.N, L.w.K, L.w.bits,
-                                             (flags & ~DP_FLAG_UNPACK_FIRST) | (L.pre ? DP_FLAG_UNPACK_FIRST : 0));
+                                             (flags & ~(DP_FLAG_UNPACK_FIRST | DP_FLAG_NO_UNPACK_FIRST)) |
+                                                 (L.pre ? DP_FLAG_UNPACK_FIRST : DP_FLAG_NO_UNPACK_FIRST));
     if (ws > p->workspace_bytes) p->workspace_bytes = ws;
     L.x_offset = p->x_bytes;
     p->x_bytes += align256(static_cast<size_t>(L.M) * L.w.K * 2);
@@ -588,18 +607,22 @@ extern "C" int dp_plan_set_layer_flags(dp_plan* plan, int32_t layer, uint32_t fl
     return fail(DP_ERR_INVALID_ARG, "dp_plan_set_layer_flags: bad plan or layer index");
   PlanLayer& L = plan->layers[layer];
   constexpr uint32_t kVariantFlags = DP_FLAG_TILE_N_MASK | DP_FLAG_CTA_PAIR | DP_FLAG_NO_CTA_PAIR |
-                                     DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_UNPACK_FIRST;
+                                     DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_UNPACK_FIRST |
+    DP_FLAG_NO_UNPACK_FIRST;
   if (flags & ~kVariantFlags) return fail(DP_ERR_INVALID_ARG, "dp_plan_set_layer_flags: flag bits 0x%x do not name a variant", flags);
   if (L.simt || L.M == 0) return fail(DP_ERR_INVALID_ARG, "layer %d runs the small-M kernel: it has no variants", layer);
   if (int st = check_tile_flags(flags, L.w.N)) return st;
   if ((flags & DP_FLAG_WEIGHT_STATIONARY) && !gemm_ws_supported(L.w.N, L.w.K))
     return fail(DP_ERR_SHAPE, "layer %d: the weight-stationary kernel does not take N=%d K=%d", layer, L.w.N, L.w.K);
   PlanLayer T = L;
-  T.pre = ((flags & DP_FLAG_UNPACK_FIRST) && T.w.bits < 8) ? 1 : 0;
+  if ((flags & DP_FLAG_UNPACK_FIRST) && (flags & DP_FLAG_NO_UNPACK_FIRST))
+    return fail(DP_ERR_INVALID_ARG, "UNPACK_FIRST and NO_UNPACK_FIRST are exclusive");
+  T.pre = want_unpack_first(flags, T.w.bits, true) ? 1 : 0;
   choose_tile(flags, T.M, T.w.N, T.w.K, T.pre ? 8 : T.w.bits, &T.bn, &T.cg, &T.ws);
   if (int st = gemm_encode_w(&T.tmap_w, T.w.qweight, T.w.N, T.w.K, T.w.bits, T.bn, T.cg)) return st;
   L = T;
-  const size_t ws = dp_wq_linear_workspace(L.M, L.w.N, L.w.K, L.w.bits, L.pre ? DP_FLAG_UNPACK_FIRST : 0);
+  const size_t ws = dp_wq_linear_workspace(L.M, L.w.N, L.w.K, L.w.bits,
+                                           L.pre ? DP_FLAG_UNPACK_FIRST : DP_FLAG_NO_UNPACK_FIRST);
   if (ws > plan->workspace_bytes) plan->workspace_bytes = ws;
   return DP_OK;
 }

@@ -14,6 +14,10 @@ from helpers import bf16_ulp_dist
 
 pytestmark = pytest.mark.gpu
 SEED = synth.BASE_SEED
+# the tensor-core kernels that expand packed weights themselves (the default for packed layers is the
+# unpack-first form, which runs the 8-bit kernel on an int8 copy: test_mma_path and
+# test_mma_unpack_first cover it)
+MMA_PACKED = B.DP_FLAG_FORCE_MMA | B.DP_FLAG_NO_UNPACK_FIRST
 
 
 def _case(M, K, N, bits, layer=0, n_out=None, bias=True, full_range=False):
@@ -54,10 +58,13 @@ def test_simt_path(bits, M, K, N):
 @pytest.mark.parametrize("M,K,N", [(128, 128, 64), (128, 256, 128), (256, 1152, 1152),
                                    (300, 1152, 384), (1000, 4608, 1152), (77, 384, 192),
                                    (2048, 1152, 4608)])
-def test_mma_path(bits, M, K, N):
+@pytest.mark.parametrize("unpack", [0, B.DP_FLAG_NO_UNPACK_FIRST], ids=["default", "in_gemm"])
+def test_mma_path(bits, M, K, N, unpack):
+    if bits == 8 and unpack:
+        pytest.skip("8-bit weights have one form")
     x, w, s_w, b = _case(M, K, N, bits, full_range=(N in (64, 192)), bias=(N != 384))
     L = DevLayer(w, s_w, b, bits)
-    _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA), x, w, s_w, b, bits)
+    _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | unpack), x, w, s_w, b, bits)
 
 
 @pytest.mark.parametrize("bits", [8, 4, 3])
@@ -68,7 +75,7 @@ def test_mma_every_tile_width(bits, bn):
     M, K, N = 200, 384, 2 * bn
     x, w, s_w, b = _case(M, K, N, bits, full_range=True)
     L = DevLayer(w, s_w, b, bits)
-    _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | B.DP_FLAG_TILE_N(bn)), x, w, s_w, b, bits)
+    _check(run_linear(L, x, flags=MMA_PACKED | B.DP_FLAG_TILE_N(bn)), x, w, s_w, b, bits)
 
 
 @pytest.mark.parametrize("bits", [8, 4, 3])
@@ -80,7 +87,7 @@ def test_mma_cta_pair_tiles(bits, bn):
         K, N = 384, 2 * bn
         x, w, s_w, b = _case(M, K, N, bits, full_range=True)
         L = DevLayer(w, s_w, b, bits)
-        _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | B.DP_FLAG_CTA_PAIR | B.DP_FLAG_TILE_N(bn)),
+        _check(run_linear(L, x, flags=MMA_PACKED | B.DP_FLAG_CTA_PAIR | B.DP_FLAG_TILE_N(bn)),
                x, w, s_w, b, bits)
 
 
@@ -91,7 +98,7 @@ def test_mma_cta_pair_many_tiles():
     for bits in (8, 4, 3):
         x, w, s_w, b = _case(M, K, N, bits)
         L = DevLayer(w, s_w, b, bits)
-        _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | B.DP_FLAG_CTA_PAIR | B.DP_FLAG_TILE_N(128)),
+        _check(run_linear(L, x, flags=MMA_PACKED | B.DP_FLAG_CTA_PAIR | B.DP_FLAG_TILE_N(128)),
                x, w, s_w, b, bits)
 
 
@@ -103,7 +110,7 @@ def test_mma_weight_stationary(bits, N, K):
     M = 600
     x, w, s_w, b = _case(M, K, N, bits, full_range=True)
     L = DevLayer(w, s_w, b, bits)
-    _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | B.DP_FLAG_WEIGHT_STATIONARY), x, w, s_w, b, bits)
+    _check(run_linear(L, x, flags=MMA_PACKED | B.DP_FLAG_WEIGHT_STATIONARY), x, w, s_w, b, bits)
 
 
 def test_mma_weight_stationary_strip_changes():
@@ -113,7 +120,7 @@ def test_mma_weight_stationary_strip_changes():
     for bits in (8, 4, 3):
         x, w, s_w, b = _case(M, K, N, bits)
         L = DevLayer(w, s_w, b, bits)
-        _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | B.DP_FLAG_WEIGHT_STATIONARY), x, w, s_w, b, bits)
+        _check(run_linear(L, x, flags=MMA_PACKED | B.DP_FLAG_WEIGHT_STATIONARY), x, w, s_w, b, bits)
 
 
 def test_mma_many_tiles_per_cta():
@@ -123,7 +130,7 @@ def test_mma_many_tiles_per_cta():
     for bits in (8, 4, 3):
         x, w, s_w, b = _case(M, K, N, bits)
         L = DevLayer(w, s_w, b, bits)
-        _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | B.DP_FLAG_TILE_N(64)), x, w, s_w, b, bits)
+        _check(run_linear(L, x, flags=MMA_PACKED | B.DP_FLAG_TILE_N(64)), x, w, s_w, b, bits)
 
 
 @pytest.mark.parametrize("bits", [8, 4, 3])
@@ -138,13 +145,13 @@ def test_mma_one_hot_and_constant_inputs(bits):
     w = rng.integers(-(1 << (bits - 1)), 1 << (bits - 1), size=(N, K)).astype(np.int8)
     s_w = np.ones(N, np.float32)
     L = DevLayer(w, s_w, None, bits)
-    out = run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA)
+    out = run_linear(L, x, flags=MMA_PACKED)
     _check(out, x, w, s_w, None, bits)
     km = (np.arange(M) * 7) % K
     sign = np.where(np.arange(M) % 2 == 0, 127, -127)
     assert np.array_equal(out["acc"], sign[:, None] * w[:, km].T.astype(np.int32))
     xc = synth.f32_to_bf16_bits(np.full((M, K), 0.75, np.float32))
-    _check(run_linear(L, xc, flags=B.DP_FLAG_FORCE_MMA), xc, w, s_w, None, bits)
+    _check(run_linear(L, xc, flags=MMA_PACKED), xc, w, s_w, None, bits)
 
 
 @pytest.mark.parametrize("bits", [8, 4, 3])
@@ -166,7 +173,7 @@ def test_mma_extreme_accumulators(bits):
     w[2::4, : K // 2] = lo
     s_w = np.full(N, 2.0 ** -10, np.float32)
     L = DevLayer(w, s_w, None, bits)
-    out = run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA)
+    out = run_linear(L, x, flags=MMA_PACKED)
     assert np.abs(out["acc"]).max() == 4608 * 127 * (1 << (bits - 1))
     _check(out, x, w, s_w, None, bits)
 
@@ -188,7 +195,7 @@ def test_padded_row_pitches_and_untouched_padding(variant):
     y = torch.full((rows_alloc, ldy), 3.0, dtype=torch.bfloat16, device="cuda")
     ws = torch.empty(B.dp_wq_linear_workspace(M, N, K, bits, variant), dtype=torch.uint8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    flags = variant if simt else (variant | B.DP_FLAG_FORCE_MMA)
+    flags = variant if simt else (variant | MMA_PACKED)
     B.dp_wq_linear(L.w, xd, ldx, None, M, y, ldy, ws, None, status, flags)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
@@ -205,7 +212,7 @@ def test_single_token_and_minimal_k_through_the_tensor_core_path():
         for bits in (8, 3):
             x, w, s_w, b = _case(1, 128, 192, bits, full_range=True)
             L = DevLayer(w, s_w, b, bits)
-            _check(run_linear(L, x, flags=B.DP_FLAG_FORCE_MMA | variant), x, w, s_w, b, bits, exact_y=False)
+            _check(run_linear(L, x, flags=MMA_PACKED | variant), x, w, s_w, b, bits, exact_y=False)
 
 
 @pytest.mark.parametrize("bits", [4, 3])
@@ -218,8 +225,8 @@ def test_mma_unpack_first(bits, variant, M, K, N):
     x, w, s_w, b = _case(M, K, N, bits, full_range=True)
     L = DevLayer(w, s_w, b, bits)
     flags = B.DP_FLAG_FORCE_MMA | B.DP_FLAG_UNPACK_FIRST | variant
-    assert (B.dp_wq_linear_workspace(M, N, K, bits, flags) - B.dp_wq_linear_workspace(M, N, K, bits, flags & ~B.DP_FLAG_UNPACK_FIRST)
-            >= N * K)
+    in_gemm = (flags & ~B.DP_FLAG_UNPACK_FIRST) | B.DP_FLAG_NO_UNPACK_FIRST
+    assert B.dp_wq_linear_workspace(M, N, K, bits, flags) - B.dp_wq_linear_workspace(M, N, K, bits, in_gemm) >= N * K
     _check(run_linear(L, x, flags=flags), x, w, s_w, b, bits)
 
 

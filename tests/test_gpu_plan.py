@@ -126,12 +126,13 @@ def test_plan_with_variants_set_per_layer_matches_oracle():
     xs = [[synth.activations(SEED, l, t, L["M"], L["K"], synth.sigma_t(t, T), n_out=max(1, L["K"] // 100))
            for l, L in enumerate(layers)] for t in kept]
     ref = oracle.plan_run(layers, kept, xs)
-    plan = B.dp_plan_create([d.w for d in dev], [L["M"] for L in layers], B.DP_FLAG_GROUP_SMALL_M)
+    plan = B.dp_plan_create([d.w for d in dev], [L["M"] for L in layers],
+                            B.DP_FLAG_GROUP_SMALL_M | B.DP_FLAG_NO_UNPACK_FIRST)
     try:
         before = B.dp_plan_workspace(plan)
         choices = [B.DP_FLAG_UNPACK_FIRST | B.DP_FLAG_TILE_N(128) | B.DP_FLAG_NO_CTA_PAIR,
                    B.DP_FLAG_CTA_PAIR | B.DP_FLAG_NO_WEIGHT_STATIONARY | B.DP_FLAG_UNPACK_FIRST,
-                   B.DP_FLAG_TILE_N(64) | B.DP_FLAG_NO_CTA_PAIR]
+                   B.DP_FLAG_TILE_N(64) | B.DP_FLAG_NO_CTA_PAIR | B.DP_FLAG_NO_UNPACK_FIRST]
         n_set = 0
         for l, L in enumerate(layers):
             if B.dp_plan_layer_variant(plan, l)["small_m"]:
@@ -141,6 +142,8 @@ def test_plan_with_variants_set_per_layer_matches_oracle():
             B.dp_plan_set_layer_flags(plan, l, choices[n_set % 3])
             v = B.dp_plan_layer_variant(plan, l)
             assert v["unpack_first"] == (1 if (choices[n_set % 3] & B.DP_FLAG_UNPACK_FIRST) and L["bits"] < 8 else 0)
+            if choices[n_set % 3] & B.DP_FLAG_TILE_N_MASK:
+                assert v["tile_n"] == ((choices[n_set % 3] & B.DP_FLAG_TILE_N_MASK) >> 8) * 64
             n_set += 1
         with pytest.raises(B.DiffproError):
             B.dp_plan_set_layer_flags(plan, 0, B.DP_FLAG_FORCE_MMA)
