@@ -12,7 +12,7 @@ import torch
 import oracle
 from paper_2511_11446_b200 import binding as B, synth, synth_cuda
 from paper_2511_11446_b200.workloads import DitStack, DevWeights
-from gpu_util import bf16_to_np
+from gpu_util import bf16_to_np, to_dev_bf16
 from helpers import bf16_ulp_dist
 
 pytestmark = pytest.mark.gpu
@@ -59,6 +59,49 @@ def test_c4_plan_run_as_benchmarked_sampled_rows():
         x_rows = stack.host_input_rows(l, t, rows)
         _check_rows(stack.y[l], x_rows, rows, stack.seed, l, N, K, stack.bits[l],
                     (l, name, stack.bits[l], B.dp_plan_layer_variant(stack.plan, l)))
+
+
+def _run_layer(W, x_bits_or_dev, M, K, N, bits, flags=0):
+    x = x_bits_or_dev if torch.is_tensor(x_bits_or_dev) else to_dev_bf16(x_bits_or_dev)
+    y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(B.dp_wq_linear_workspace(M, N, K, bits, flags), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.dp_wq_linear(W.w, x, K, None, M, y, N, ws, None, status, flags)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return y
+
+
+def test_c1_single_proj_linear_whole_output():
+    """M = 256 tokens, 1152 -> 1152, int8 weights, 8 outlier channels: every output element."""
+    seed, layer, M, K, N, bits = synth.BASE_SEED + 1, 0, 256, 1152, 1152, 8
+    x = synth.activations(seed, layer, 0, M, K, 1.0, n_out=8)
+    y = _run_layer(DevWeights(seed, layer, N, K, bits), x, M, K, N, bits)
+    _check_rows(y, x, list(range(M)), seed, layer, N, K, bits, "c1")
+
+
+def test_c2_fc1_4bit_whole_output():
+    """M = 2048, 1152 -> 4608 at 4 bits, 1 % outlier channels: every output element."""
+    seed, layer, M, K, N, bits = synth.BASE_SEED + 2, 0, 2048, 1152, 4608, 4
+    x = synth.activations(seed, layer, 0, M, K, 1.0, n_out=K // 100)
+    y = _run_layer(DevWeights(seed, layer, N, K, bits), x, M, K, N, bits)
+    _check_rows(y, x, list(range(M)), seed, layer, N, K, bits, "c2")
+
+
+def test_c3_block_at_m4096_with_gelu_input_sampled_rows():
+    """One block's linears at M = 4096 (adaLN M = 16), bits from {4, 8}; fc2 reads GELU(N(0,1)):
+    non-negative, heavy-tailed, the case where absmax scaling wastes half the code range."""
+    seed = synth.BASE_SEED + 3
+    table = [("qkv", 4096, 1152, 3456), ("proj", 4096, 1152, 1152), ("fc1", 4096, 1152, 4608),
+             ("fc2", 4096, 4608, 1152), ("adaln", 16, 1152, 6912)]
+    bits = synth.bit_plan(seed, len(table), (4, 8))
+    rng = np.random.default_rng(3)
+    for l, (name, M, K, N) in enumerate(table):
+        x = (synth.gelu_activations(seed, l, 0, M, K) if name == "fc2"
+             else synth.activations(seed, l, 0, M, K, 1.0, n_out=K // 100))
+        y = _run_layer(DevWeights(seed, l, N, K, bits[l]), x, M, K, N, bits[l])
+        rows = _sample_rows(M, rng, n=12)
+        _check_rows(y, x[rows], rows, seed, l, N, K, bits[l], ("c3", name, bits[l]))
 
 
 @pytest.mark.parametrize("name,K,N,M,bits", [("qkv", 1152, 3456, 32768, 4), ("proj", 1152, 1152, 32768, 3),
