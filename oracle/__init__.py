@@ -74,6 +74,30 @@ def daq(x: np.ndarray):
     return q, s_a, rowsum
 
 
+def clip_rank(p, K: int) -> int:
+    """Rank from the top of the nearest-rank p-th percentile of K values (p = 100 -> 1): the
+    ceil(p K / 100)-th smallest is the (K - ceil(p K / 100) + 1)-th largest. p may be a str/Fraction."""
+    from fractions import Fraction
+    import math
+    f = Fraction(str(p)) * K / 100
+    return K - max(1, math.ceil(f)) + 1
+
+
+def daq_robust(x: np.ndarray, rank: int, act_bits: int = 8):
+    """Eq. "daq" with the clip threshold at the rank-th largest magnitude of each token and
+    act_bits-bit codes: x uint16 (bf16 bits) [M, K] -> (q int8, s_a fp32 [M], rowsum int32 [M])."""
+    _chk(x, np.uint16, "x")
+    M, K = x.shape
+    q = np.empty((M, K), np.int8)
+    s_a = np.empty(M, np.float32)
+    rowsum = np.empty(M, np.int32)
+    st = lib().orc_daq_robust(_p(x), _i64(M), _i64(K), _i64(K), C.c_int(rank), C.c_int(act_bits), _p(q), _i64(K),
+                              _p(s_a), _p(rowsum))
+    if st != 0:
+        raise ValueError(f"bad clip rank {rank} (K = {K}) or activation bits {act_bits}")
+    return q, s_a, rowsum
+
+
 def pack(w: np.ndarray, bits: int) -> np.ndarray:
     """w int8 [N,K] -> packed: int8 [N,K] (bits 8) or uint32 [N, K*bits/32]."""
     _chk(w, np.int8, "w")

@@ -12,6 +12,12 @@
  *                  the absolute maximum of one token's K activations (p = 100, one group); round is
  *                  half-to-even; the division by alpha is evaluated as a multiplication by
  *                  fl(127 / tau) whose exact product is rounded once.
+ *   orc_daq_robust Step 3, Eq. "daq" with its percentile clip (p < 100) and Step 6 / Algorithm 2
+ *                  Phase B's activation bits per time bin: tau = Percentile(|v|, p) read as the
+ *                  nearest-rank percentile of one token's K magnitudes and passed as its rank from
+ *                  the top (rank 1 = maximum, rank r = r-th largest counting repeats;
+ *                  r = K - ceil(p K / 100) + 1), alpha = tau / (2^(a-1) - 1) for a activation bits,
+ *                  values beyond tau clip to the extreme codes. rank 1, a = 8 is orc_daq.
  *   orc_pack/orc_unpack   "GPTQ packed" low-bit weights (Step 1 calibration text, Step 3): a
  *                  little-endian bit stream of b-bit offset-binary codes per output channel. The
  *                  paper fixes no layout; this is the layout the library's header documents.
@@ -103,6 +109,53 @@ void orc_daq(const uint16_t* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, in
 #pragma omp parallel for schedule(static)
   for (int64_t m = 0; m < M; ++m)
     daq_row(x + m * ldx, K, q + m * ldq, s_a + m, rowsum ? rowsum + m : 0);
+}
+
+/* ---- DAQ with percentile clip and a-bit codes (Eq. "daq", p < 100; Step 6) ------------------- */
+
+static int cmp_float_desc(const void* a, const void* b) {
+  const float fa = *(const float*)a, fb = *(const float*)b;
+  return (fa < fb) - (fa > fb);
+}
+
+/* One token. clip_rank in [1, K]; act_bits in [2, 8]. */
+static void daq_row_robust(const uint16_t* x, int64_t K, int clip_rank, int act_bits, int8_t* q, float* s_a,
+                           int32_t* rowsum) {
+  float* mag = (float*)malloc((size_t)K * sizeof(float));
+  for (int64_t k = 0; k < K; ++k) mag[k] = fabsf(bf16_to_f32(x[k]));
+  qsort(mag, (size_t)K, sizeof(float), cmp_float_desc);
+  const float tau = mag[clip_rank - 1]; /* the clip_rank-th largest magnitude */
+  free(mag);
+  const float qmax = (float)((1 << (act_bits - 1)) - 1);
+  int32_t sum = 0;
+  if (tau < 0x1p-100f) {
+    *s_a = 0.0f;
+    for (int64_t k = 0; k < K; ++k) q[k] = 0;
+  } else {
+    const float alpha = tau / qmax;
+    const float inv_alpha = qmax / tau;
+    *s_a = alpha;
+    for (int64_t k = 0; k < K; ++k) {
+      /* clip(v, -tau, tau) / alpha and then round is the same as round and then clamp to +-qmax,
+         because tau / alpha rounds to qmax; the product is exact in double as in daq_row */
+      double r = nearbyint((double)bf16_to_f32(x[k]) * (double)inv_alpha);
+      if (r > (double)qmax) r = (double)qmax;
+      if (r < -(double)qmax) r = -(double)qmax;
+      q[k] = (int8_t)r;
+      sum += (int32_t)q[k];
+    }
+  }
+  if (rowsum) *rowsum = sum;
+}
+
+/* Returns 0, or -1 on a bad clip_rank / act_bits (nothing is written then). */
+int orc_daq_robust(const uint16_t* x, int64_t M, int64_t K, int64_t ldx, int clip_rank, int act_bits, int8_t* q,
+                   int64_t ldq, float* s_a, int32_t* rowsum) {
+  if (clip_rank < 1 || clip_rank > K || act_bits < 2 || act_bits > 8) return -1;
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m)
+    daq_row_robust(x + m * ldx, K, clip_rank, act_bits, q + m * ldq, s_a + m, rowsum ? rowsum + m : 0);
+  return 0;
 }
 
 /* ---- packed weights ------------------------------------------------------------------------- */
