@@ -154,6 +154,24 @@ typedef struct dp_debug {
 int dp_daq_quantize(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq,
                     float* s_a, int32_t* rowsum, dp_stream stream);
 
+/*
+ * The same with the equation's percentile clip and with fewer activation bits.
+ *   Step 3, Eq. "daq": tau = Percentile(|v|, p); Step 6 / Algorithm 2 Phase B: the activation bits of
+ *   a forward pass come from the time bin of its step. Reading: the percentile is the nearest-rank one
+ *   over the K magnitudes of a token and is passed as its rank from the top,
+ *     clip_rank = K - ceil(p K / 100) + 1     (p = 100 -> 1; p = 99.9 -> 2 at K = 1152, 5 at K = 4608),
+ *   so tau = the clip_rank-th largest |x[m,k]|, repeats counted. With qmax = 2^(act_bits-1) - 1:
+ *     s_a[m] = tau / qmax,   q[m,k] = clamp(RNE(x[m,k] * (qmax/tau)), -qmax, qmax)
+ *   (values beyond tau land on the extreme codes, which is what clipping to [-tau, tau] before the
+ *   division gives); tau < 2^-100: s_a[m] = 0, q[m,:] = 0. clip_rank = 1, act_bits = 8 is dp_daq_quantize.
+ * Arguments and layouts as dp_daq_quantize; 1 <= clip_rank <= min(K, 64) (DP_ERR_INVALID_ARG),
+ * 2 <= act_bits <= 8 (DP_ERR_BITS), K % 8 == 0 and 8 <= K <= 4608 (DP_ERR_SHAPE). The codes are
+ * ordinary int8, so dp_wq_linear takes them with their scales as quantized activations.
+ */
+int dp_daq_quantize_robust(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq,
+                           float* s_a, int32_t* rowsum, int32_t clip_rank, int32_t act_bits,
+                           dp_stream stream);
+
 /* Bytes of device scratch dp_wq_linear needs for this problem (holds the int8 activations and
  * their scales between the two kernels of the large-M path). Never 0; multiple of 256. */
 size_t dp_wq_linear_workspace(int64_t M, int32_t N, int32_t K, int32_t bits, uint32_t flags);

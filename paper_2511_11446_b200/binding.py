@@ -32,7 +32,7 @@ def DP_FLAG_TILE_N(bn: int) -> int:
 
 DP_STATIC_SCRATCH_BYTES = 10 << 20
 
-EXPORTS = ["dp_daq_quantize", "dp_wq_linear_workspace", "dp_wq_linear", "dp_wq_linear_static", "dp_plan_create",
+EXPORTS = ["dp_daq_quantize", "dp_daq_quantize_robust", "dp_wq_linear_workspace", "dp_wq_linear", "dp_wq_linear_static", "dp_plan_create",
            "dp_plan_workspace", "dp_plan_layer_variant", "dp_plan_layer_unpack_first", "dp_plan_set_layer_flags", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
            "dp_plan_run_host", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_status_string",
            "dp_last_error", "dp_version"]
@@ -78,6 +78,8 @@ def lib():
         L.dp_plan_destroy.argtypes = [C.c_void_p]
         L.dp_status_string.restype = C.c_char_p
         L.dp_last_error.restype = C.c_char_p
+        L.dp_daq_quantize_robust.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_int64,
+                                             C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]
         L.dp_daq_quantize.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
                                       C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
         L.dp_wq_linear.argtypes = [C.POINTER(dp_weight), C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
@@ -126,6 +128,19 @@ def dp_daq_quantize(x, M, K, ldx, q, ldq, s_a, rowsum=None, stream=None):
 
 def dp_wq_linear_workspace(M, N, K, bits, flags=0) -> int:
     return int(lib().dp_wq_linear_workspace(M, N, K, bits, flags))
+
+
+def clip_rank(p, K: int) -> int:
+    """Rank from the top of the nearest-rank p-th percentile of K values (argument marshalling for
+    dp_daq_quantize_robust: K - ceil(p K / 100) + 1)."""
+    from fractions import Fraction
+    f = Fraction(str(p)) * K / 100
+    return K - max(1, -((-f.numerator) // f.denominator)) + 1
+
+
+def dp_daq_quantize_robust(x, M, K, ldx, q, ldq, s_a, rank, act_bits=8, rowsum=None, stream=None):
+    _check(lib().dp_daq_quantize_robust(_ptr(x), M, K, ldx, _ptr(q), ldq, _ptr(s_a), _ptr(rowsum), rank, act_bits,
+                                        _stream(stream)), "dp_daq_quantize_robust")
 
 
 def dp_wq_linear(w: dp_weight, x, ldx, s_a_in, M, y, ldy, workspace, dbg: dp_debug | None = None,

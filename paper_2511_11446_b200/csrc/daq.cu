@@ -106,6 +106,115 @@ daq_rows_2pass_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t 
   }
 }
 
+// ---- DAQ with a percentile clip and a-bit codes -------------------------------------------------------
+// Eq. "daq" with tau = Percentile(|v|, p) below the maximum (nearest-rank reading: the clip_rank-th
+// largest magnitude of the token, repeats counted) and alpha = tau / qmax, qmax = 2^(a-1) - 1 for the
+// activation bits a of the step's time bin (Step 6). One warp per token, row in registers as above.
+// The threshold is found by peeling maxima: each round takes the largest magnitude below the
+// previous one together with its multiplicity until clip_rank values are covered (for p = 99.9: 2
+// rounds at K = 1152, 5 at K = 4608). A lane keeps the maximum of each of its 8-element vectors, so
+// a round is a max over those few numbers plus a rescan of only the vectors that held the peeled
+// value. Values beyond tau land on +-qmax: the rounded product is clamped while it still sits in
+// the fp32 mantissa.
+// Packed helpers on words of two 15-bit magnitudes (bit 15 of each half clear):
+// number of halves equal to the value replicated in t2
+__device__ __forceinline__ int count_eq2(uint32_t e, uint32_t t2) {
+  const uint32_t z = ((e ^ t2) | 0x80008000u) - 0x00010001u;  // bit 15 of a half stays set unless the half was 0
+  return __popc(~z & 0x80008000u);
+}
+// the halves that are below the bound replicated in b2 (<= 0x8000 per half), the others zeroed
+__device__ __forceinline__ uint32_t keep_below2(uint32_t e, uint32_t b2) {
+  const uint32_t ge = ((e | 0x80008000u) - b2) & 0x80008000u;  // bit 15 set where half >= bound; no borrow
+  return e & ~(ge - (ge >> 15));
+}
+__device__ __forceinline__ uint32_t fold_max2(uint32_t m2) { return max(m2 & 0xFFFFu, m2 >> 16); }
+__device__ __forceinline__ uint32_t quant_pair_clamped(uint32_t w, float inv, float lo, float hi) {
+  const float magic = 12582912.0f;  // 1.5 * 2^23
+  const float a = fminf(fmaxf(__fmaf_rn(__uint_as_float(w << 16), inv, magic), lo), hi);
+  const float b = fminf(fmaxf(__fmaf_rn(__uint_as_float(w & 0xFFFF0000u), inv, magic), lo), hi);
+  return __byte_perm(__float_as_uint(a), __float_as_uint(b), 0x0040);
+}
+
+template <int MAXV>
+__global__ void __launch_bounds__(kDaqWarps * 32)
+daq_rows_robust_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t ldx, int8_t* __restrict__ q,
+                       int64_t ldq, float* __restrict__ s_a, int32_t* __restrict__ rowsum, int clip_rank,
+                       float qmax) {
+  const int64_t row = static_cast<int64_t>(blockIdx.x) * kDaqWarps + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= M) return;
+  const int nvec = K >> 3;
+  const uint4* xr = reinterpret_cast<const uint4*>(x + row * ldx);
+  uint4 v[MAXV];
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int idx = lane + 32 * i;
+    if (idx < nvec) ld_nc_u32x4(xr + idx, v[i]);
+    else v[i] = make_uint4(0, 0, 0, 0);
+  }
+  // threshold: magnitude bits (bf16 pattern, sign cleared) of the clip_rank-th largest element
+  uint32_t gmax[MAXV];  // per vector: its largest magnitude not yet peeled (padding vectors: 0)
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i)
+    gmax[i] = fold_max2(absmax_bits2(absmax_bits2(absmax_bits2(absmax_bits2(0u, v[i].x), v[i].y), v[i].z), v[i].w));
+  uint32_t tau_bits = 0;
+  int remaining = clip_rank;
+  for (int round = 0; round < clip_rank; ++round) {
+    uint32_t mx = 0;
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) mx = max(mx, gmax[i]);
+    const uint32_t wmx = warp_max_u32(mx);
+    tau_bits = wmx;
+    if (wmx == 0) break;  // all that is left are zeros
+    const uint32_t t2 = wmx | (wmx << 16);
+    int cnt = 0;
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) {
+      if (gmax[i] == wmx) {  // this vector holds the value: count it and find the vector's next maximum
+        const uint32_t w[4] = {v[i].x & 0x7FFF7FFFu, v[i].y & 0x7FFF7FFFu, v[i].z & 0x7FFF7FFFu,
+                               v[i].w & 0x7FFF7FFFu};
+        uint32_t m2 = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          cnt += count_eq2(w[j], t2);
+          m2 = __vmaxu2(m2, keep_below2(w[j], t2));
+        }
+        gmax[i] = fold_max2(m2);
+      }
+    }
+    const int wcnt = warp_sum_i32(cnt);
+    if (wcnt >= remaining) break;
+    remaining -= wcnt;
+  }
+  const float tau = __uint_as_float(tau_bits << 16);
+  float sc = 0.0f, inv = 0.0f;
+  if (!(tau < 7.888609052210118e-31f)) {  // 2^-100, as in the absmax form
+    sc = __fdiv_rn(tau, qmax);
+    inv = __fdiv_rn(qmax, tau);
+  }
+  const float magic = 12582912.0f;
+  const float lo = magic - qmax, hi = magic + qmax;
+  uint2* out = reinterpret_cast<uint2*>(q + row * ldq);
+  int sum = 0;
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int idx = lane + 32 * i;
+    if (idx < nvec) {
+      const uint32_t p0 = quant_pair_clamped(v[i].x, inv, lo, hi), p1 = quant_pair_clamped(v[i].y, inv, lo, hi);
+      const uint32_t p2 = quant_pair_clamped(v[i].z, inv, lo, hi), p3 = quant_pair_clamped(v[i].w, inv, lo, hi);
+      const uint2 o = make_uint2(__byte_perm(p0, p1, 0x5410), __byte_perm(p2, p3, 0x5410));
+      out[idx] = o;
+      sum = __dp4a(static_cast<int>(o.x), 0x01010101, sum);
+      sum = __dp4a(static_cast<int>(o.y), 0x01010101, sum);
+    }
+  }
+  if (lane == 0) s_a[row] = sc;
+  if (rowsum != nullptr) {
+    sum = warp_sum_i32(sum);
+    if (lane == 0) rowsum[row] = sum;
+  }
+}
+
 __global__ void __launch_bounds__(kDaqWarps * 32)
 unpack_kernel(const UnpackJob job) {
   pdl_launch_dependents();
@@ -147,6 +256,24 @@ int launch_daq(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int6
   return DP_OK;
 }
 
+int launch_daq_robust(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq, float* s_a,
+                      int32_t* rowsum, int clip_rank, int act_bits, cudaStream_t stream) {
+  if (M == 0) return DP_OK;
+  const uint16_t* xp = static_cast<const uint16_t*>(x);
+  const int k = static_cast<int>(K);
+  const float qmax = static_cast<float>((1 << (act_bits - 1)) - 1);
+  const dim3 grid(static_cast<unsigned>((M + kDaqWarps - 1) / kDaqWarps)), block(kDaqWarps * 32);
+  cudaError_t e;
+  if (k <= 256 * 5)
+    e = launch(daq_rows_robust_kernel<5>, grid, block, 0, stream, false, xp, M, k, ldx, q, ldq, s_a, rowsum, clip_rank, qmax);
+  else if (k <= 256 * 9)
+    e = launch(daq_rows_robust_kernel<9>, grid, block, 0, stream, false, xp, M, k, ldx, q, ldq, s_a, rowsum, clip_rank, qmax);
+  else
+    e = launch(daq_rows_robust_kernel<18>, grid, block, 0, stream, false, xp, M, k, ldx, q, ldq, s_a, rowsum, clip_rank, qmax);
+  if (e != cudaSuccess) return fail(DP_ERR_CUDA, "robust DAQ launch failed: %s", cudaGetErrorString(e));
+  return DP_OK;
+}
+
 int launch_unpack(const UnpackJob& job, cudaStream_t stream, bool pdl) {
   if (job.units == 0) return DP_OK;
   const dim3 grid(static_cast<unsigned>((job.units + kDaqWarps * 32 - 1) / (kDaqWarps * 32)));
@@ -173,4 +300,26 @@ extern "C" int dp_daq_quantize(const void* x_bf16, int64_t M, int64_t K, int64_t
   if (st != DP_OK) return st;
   return launch_daq(x_bf16, M, K, ldx, q, ldq, s_a, rowsum, KORDER_NATURAL, false,
                     static_cast<cudaStream_t>(stream), false);
+}
+
+extern "C" int dp_daq_quantize_robust(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int8_t* q,
+                                      int64_t ldq, float* s_a, int32_t* rowsum, int32_t clip_rank,
+                                      int32_t act_bits, dp_stream stream) {
+  using namespace dp;
+  if (M < 0 || K < 8 || K > 4608 || (K % 8))
+    return fail(DP_ERR_SHAPE, "dp_daq_quantize_robust: need M >= 0 and K a multiple of 8 in [8, 4608] (M=%lld K=%lld)",
+                (long long)M, (long long)K);
+  if (clip_rank < 1 || clip_rank > 64 || clip_rank > K)
+    return fail(DP_ERR_INVALID_ARG, "dp_daq_quantize_robust: clip_rank=%d not in [1, min(K, 64)]", clip_rank);
+  if (act_bits < 2 || act_bits > 8)
+    return fail(DP_ERR_BITS, "dp_daq_quantize_robust: act_bits=%d not in [2, 8]", act_bits);
+  if (M == 0) return DP_OK;
+  if (!x_bf16 || !q || !s_a) return fail(DP_ERR_INVALID_ARG, "dp_daq_quantize_robust: NULL pointer");
+  if (ldx < K || ldq < K) return fail(DP_ERR_SHAPE, "dp_daq_quantize_robust: leading dimension < K");
+  if (!aligned16(x_bf16) || !aligned16(q) || (ldx % 8) || (ldq % 16) || (reinterpret_cast<uintptr_t>(s_a) & 3u))
+    return fail(DP_ERR_ALIGN, "dp_daq_quantize_robust: pointers/pitches must be 16-byte aligned");
+  int st = check_device();
+  if (st != DP_OK) return st;
+  return launch_daq_robust(x_bf16, M, K, ldx, q, ldq, s_a, rowsum, clip_rank, act_bits,
+                           static_cast<cudaStream_t>(stream));
 }
