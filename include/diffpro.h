@@ -248,6 +248,20 @@ int dp_plan_layer_unpack_first(const dp_plan* plan, int32_t layer, int32_t* unpa
  * that do not fit the layer with DP_ERR_SHAPE; the plan is unchanged on error. Not to be called
  * while a dp_plan_run of the plan is being issued. No counterpart in the paper. */
 int dp_plan_set_layer_flags(dp_plan* plan, int32_t layer, uint32_t flags);
+/* DAQ policy of a plan (Eq. "daq" with its percentile clip; Step 6 and Algorithm 2 Phase B:
+ * "bin in {early, mid, late}; a_bits <- P_DAQ(bin)"). From the next dp_plan_run on, every layer
+ * quantizes its activations as dp_daq_quantize_robust does, with
+ *   clip_rank = K - ceil(p K / 100) + 1,  p = clip_percentile_e3 / 1000 percent (100000 = the maximum),
+ *   act_bits  = act_bits_by_bin[min(2, 3 t / n_timesteps)] for a step with timestep value t
+ * (reading: the three bins are thirds of [0, n_timesteps), bin 0 holding the smallest timestep
+ * values; n_timesteps = 0: 8 bits at every step, act_bits_by_bin may be NULL). Under a policy other
+ * than (100000, 8 bits) packed layers run in the unpack-first form, small-M layers run one by one
+ * behind a quantization launch of their own, and DP_FLAG_FUSED_DAQ is ignored. May raise
+ * dp_plan_workspace: ask again afterwards. Limits: K <= 4608 and clip_rank <= 64 for every layer
+ * (DP_ERR_SHAPE), bits in [2, 8] (DP_ERR_BITS); the plan is unchanged on error. Host only; not to
+ * be called while a dp_plan_run of the plan is being issued. */
+int dp_plan_set_daq(dp_plan* plan, int32_t clip_percentile_e3, int32_t n_timesteps,
+                    const int32_t* act_bits_by_bin);
 void dp_plan_destroy(dp_plan* plan);
 
 /*

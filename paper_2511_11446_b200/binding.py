@@ -33,7 +33,7 @@ def DP_FLAG_TILE_N(bn: int) -> int:
 DP_STATIC_SCRATCH_BYTES = 10 << 20
 
 EXPORTS = ["dp_daq_quantize", "dp_daq_quantize_robust", "dp_wq_linear_workspace", "dp_wq_linear", "dp_wq_linear_static", "dp_plan_create",
-           "dp_plan_workspace", "dp_plan_layer_variant", "dp_plan_layer_unpack_first", "dp_plan_set_layer_flags", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
+           "dp_plan_workspace", "dp_plan_layer_variant", "dp_plan_layer_unpack_first", "dp_plan_set_layer_flags", "dp_plan_set_daq", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
            "dp_plan_run_host", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_status_string",
            "dp_last_error", "dp_version"]
 
@@ -72,6 +72,7 @@ def lib():
         L.dp_plan_layer_variant.argtypes = [C.c_void_p, C.c_int32] + [C.POINTER(C.c_int32)] * 4
         L.dp_plan_layer_unpack_first.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
         L.dp_plan_set_layer_flags.argtypes = [C.c_void_p, C.c_int32, C.c_uint32]
+        L.dp_plan_set_daq.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int32)]
         L.dp_plan_x_bytes.restype = C.c_size_t
         L.dp_plan_x_bytes.argtypes = [C.c_void_p]
         L.dp_plan_destroy.restype = None
@@ -182,6 +183,11 @@ def dp_plan_layer_variant(plan, layer: int) -> dict:
 
 def dp_plan_set_layer_flags(plan, layer: int, flags: int):
     _check(lib().dp_plan_set_layer_flags(plan, layer, flags), "dp_plan_set_layer_flags")
+
+
+def dp_plan_set_daq(plan, clip_percentile_e3: int, n_timesteps: int = 0, act_bits_by_bin=None):
+    bins = None if act_bits_by_bin is None else (C.c_int32 * 3)(*act_bits_by_bin)
+    _check(lib().dp_plan_set_daq(plan, clip_percentile_e3, n_timesteps, bins), "dp_plan_set_daq")
 
 
 def variant_flags(v: dict) -> int:

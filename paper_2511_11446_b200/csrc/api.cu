@@ -102,6 +102,12 @@ static bool want_unpack_first(uint32_t flags, int32_t bits, bool library_daq) {
   return (flags & DP_FLAG_UNPACK_FIRST) || library_daq;
 }
 
+// Rank from the top of the nearest-rank percentile p (in 1/1000 %) of K values: K - ceil(p K / 100) + 1.
+static int clip_rank_of(int32_t p_e3, int32_t K) {
+  const int64_t c = (static_cast<int64_t>(p_e3) * K + 99999) / 100000;
+  return static_cast<int>(K - (c < 1 ? 1 : c) + 1);
+}
+
 constexpr int64_t kSimtMaxRows = 32;  // at or below this the CUDA-core streaming kernel is used
 
 static bool use_simt(int64_t M, int32_t N, int32_t K, uint32_t flags) {
@@ -134,8 +140,10 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
                       void* y, int64_t ldy, void* workspace, const dp_debug* dbg, int32_t* status,
                       uint32_t flags, cudaStream_t stream, const CUtensorMap* tmap_w, int bn, int cg, int ws,
                       const CUtensorMap* tmap_a_cached, bool chained, int32_t* daq_sync = nullptr,
-                      int pre = -1) {
+                      int pre = -1, int daq_rank = 1, int daq_bits = 8) {
   const bool pdl = !(flags & DP_FLAG_NO_PDL);
+  // DAQ policy of a plan (dp_plan_set_daq): clip threshold below the maximum and/or fewer activation bits
+  const bool robust = s_a_in == nullptr && (daq_rank > 1 || daq_bits < 8);
   if (use_simt(M, w->N, w->K, flags)) {
     if (static_cast<size_t>(w->K) > simt_max_k())
       return fail(DP_ERR_SHAPE, "K=%d too large for the small-M kernel", w->K);
@@ -143,6 +151,16 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
     a.x = x;
     a.ldx = ldx;
     a.s_a_in = s_a_in;
+    if (robust) {  // quantize into the workspace first; the kernel then takes the codes as they are
+      int8_t* wq = static_cast<int8_t*>(workspace);
+      float* wsa = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align256(scratch_q_bytes(M, w->K)));
+      int st = launch_daq_robust(x, M, w->K, ldx, wq, w->K, wsa, nullptr, daq_rank, daq_bits, false, stream, pdl,
+                                 nullptr);
+      if (st != DP_OK) return st;
+      a.x = wq;
+      a.ldx = w->K;
+      a.s_a_in = wsa;
+    }
     a.M = M;
     a.N = w->N;
     a.K = w->K;
@@ -169,6 +187,10 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
   // extra CTAs of the DAQ launch) and the 8-bit kernel runs on that copy, instead of every CTA
   // expanding the weight tiles it needs in shared memory.
   if (pre < 0) pre = want_unpack_first(flags, w->bits, s_a_in == nullptr) ? 1 : 0;
+  if (robust) {  // that kernel writes codes in natural k order only: packed layers run on the int8 copy
+    pre = 1;
+    daq_sync = nullptr;
+  }
   const bool unpack_first = pre > 0 && w->bits < 8;
   dp_weight w8 = *w;
   UnpackJob job{nullptr, nullptr, 0, 0, 0};
@@ -188,7 +210,11 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
     int8_t* wq = static_cast<int8_t*>(workspace);
     float* wsa = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align256(scratch_q_bytes(M, w->K)));
     korder = gemm_korder(w->bits);
-    if (!fused) {
+    if (robust) {
+      int st = launch_daq_robust(x, M, w->K, ldx, wq, w->K, wsa, nullptr, daq_rank, daq_bits, true, stream, pdl,
+                                 unpack_first ? &job : nullptr);
+      if (st != DP_OK) return st;
+    } else if (!fused) {
       int st = launch_daq(x, M, w->K, ldx, wq, w->K, wsa, nullptr, korder, true, stream, pdl,
                           unpack_first ? &job : nullptr);
       if (st != DP_OK) return st;
@@ -394,6 +420,9 @@ struct dp_plan {
   std::vector<std::vector<int>> groups;  // small-M layers of equal shape, run first in every step
   std::vector<char> grouped;             // per layer: member of a group
   int32_t* daq_sync;                     // device counters of the in-kernel DAQ (nullptr: DAQ in its own kernel)
+  // DAQ policy (dp_plan_set_daq): clip percentile in 1/1000 %, 100000 = the maximum; activation bits
+  // of the three time bins of [0, daq_timesteps)
+  int32_t daq_p_e3, daq_timesteps, daq_bits[3];
   cudaStream_t copy_stream;
   cudaEvent_t ev_copied[2], ev_consumed[2];
 };
@@ -492,6 +521,9 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
   p->x_bytes = 0;
   p->copy_stream = nullptr;
   p->daq_sync = nullptr;
+  p->daq_p_e3 = 100000;
+  p->daq_timesteps = 0;
+  p->daq_bits[0] = p->daq_bits[1] = p->daq_bits[2] = 8;
   for (int i = 0; i < 2; ++i) p->ev_copied[i] = p->ev_consumed[i] = nullptr;
   for (int32_t l = 0; l < n_layers; ++l) {
     st = check_weight(&layers[l]);
@@ -602,6 +634,34 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
 }
 
 extern "C" size_t dp_plan_workspace(const dp_plan* plan) { return plan ? plan->workspace_bytes : 0; }
+extern "C" int dp_plan_set_daq(dp_plan* plan, int32_t clip_percentile_e3, int32_t n_timesteps,
+                               const int32_t* act_bits_by_bin) {
+  if (!plan) return fail(DP_ERR_INVALID_ARG, "dp_plan_set_daq: plan is NULL");
+  if (clip_percentile_e3 < 1 || clip_percentile_e3 > 100000)
+    return fail(DP_ERR_INVALID_ARG, "dp_plan_set_daq: percentile %d/1000 %% not in (0, 100]", clip_percentile_e3);
+  if (n_timesteps < 0 || (n_timesteps > 0 && !act_bits_by_bin))
+    return fail(DP_ERR_INVALID_ARG, "dp_plan_set_daq: bad n_timesteps / act_bits_by_bin");
+  for (int b = 0; b < 3 && n_timesteps > 0; ++b)
+    if (act_bits_by_bin[b] < 2 || act_bits_by_bin[b] > 8)
+      return fail(DP_ERR_BITS, "dp_plan_set_daq: activation bits %d not in [2, 8]", act_bits_by_bin[b]);
+  size_t need = plan->workspace_bytes;
+  for (const PlanLayer& L : plan->layers) {
+    if (L.M == 0) continue;
+    const int rank = clip_rank_of(clip_percentile_e3, L.w.K);
+    if (rank > 64 || L.w.K > 4608)
+      return fail(DP_ERR_SHAPE, "dp_plan_set_daq: a layer with K=%d would need clip rank %d (limits: K <= 4608, rank <= 64)",
+                  L.w.K, rank);
+    // every layer quantizes into the workspace under a policy; packed ones run on their int8 copy
+    size_t ws = align256(scratch_q_bytes(L.M, L.w.K)) + align256(sizeof(float) * static_cast<size_t>(L.M));
+    if (!L.simt && L.w.bits < 8) ws += align256(static_cast<size_t>(L.w.N) * L.w.K);
+    if (ws > need) need = ws;
+  }
+  plan->workspace_bytes = need;
+  plan->daq_p_e3 = clip_percentile_e3;
+  plan->daq_timesteps = n_timesteps;
+  for (int b = 0; b < 3; ++b) plan->daq_bits[b] = n_timesteps > 0 ? act_bits_by_bin[b] : 8;
+  return DP_OK;
+}
 extern "C" int dp_plan_set_layer_flags(dp_plan* plan, int32_t layer, uint32_t flags) {
   if (!plan || layer < 0 || layer >= static_cast<int32_t>(plan->layers.size()))
     return fail(DP_ERR_INVALID_ARG, "dp_plan_set_layer_flags: bad plan or layer index");
@@ -673,10 +733,18 @@ static const CUtensorMap* cached_tmap_a(dp_plan* plan, const void* ws, int64_t M
   return &plan->a_cache.back().map;
 }
 
-static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, void* workspace,
+static int plan_run_step(dp_plan* plan, int32_t t, const void* const* xs, void* const* ys, void* workspace,
                          int32_t* status, cudaStream_t stream, bool* chained) {
   const int n = static_cast<int>(plan->layers.size());
+  // DAQ policy of this step: the activation bits of the time bin t falls into (thirds of the range)
+  int act_bits = 8;
+  if (plan->daq_timesteps > 0) {
+    int64_t bin = static_cast<int64_t>(t < 0 ? 0 : t) * 3 / plan->daq_timesteps;
+    act_bits = plan->daq_bits[bin > 2 ? 2 : bin];
+  }
+  const bool robust = plan->daq_p_e3 < 100000 || act_bits < 8;
   for (const std::vector<int>& grp : plan->groups) {
+    if (robust) break;  // the grouped launch quantizes with the plain rule: such layers run one by one below
     const PlanLayer& G = plan->layers[grp[0]];
     SimtGroupArgs ga;
     ga.M = G.M;
@@ -702,7 +770,7 @@ static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, 
   }
   for (int l = 0; l < n; ++l) {
     const PlanLayer& L = plan->layers[l];
-    if (L.M == 0 || plan->grouped[l]) continue;
+    if (L.M == 0 || (plan->grouped[l] && !robust)) continue;
     if (!xs[l] || !ys[l]) return fail(DP_ERR_INVALID_ARG, "layer %d: NULL x or y", l);
     if (!aligned16(xs[l]) || !aligned16(ys[l])) return fail(DP_ERR_ALIGN, "layer %d: x/y misaligned", l);
     const CUtensorMap* ta = nullptr;
@@ -713,7 +781,8 @@ static int plan_run_step(dp_plan* plan, const void* const* xs, void* const* ys, 
     }
     int st = run_linear(&L.w, xs[l], L.w.K, nullptr, L.M, ys[l], L.w.N, workspace, nullptr, status,
                         plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, L.cg, L.ws, ta, *chained,
-                        L.simt ? nullptr : plan->daq_sync, L.simt ? 0 : L.pre);
+                        L.simt ? nullptr : plan->daq_sync, L.simt ? 0 : L.pre,
+                        robust ? clip_rank_of(plan->daq_p_e3, L.w.K) : 1, act_bits);
     if (st != DP_OK) return st;
     *chained = true;
   }
@@ -745,7 +814,7 @@ extern "C" int dp_plan_run(const dp_plan* plan_c, const int32_t* steps, int32_t 
   for (int32_t i = n_steps - 1 - start_index; i >= 0; --i) {  // reverse(K*)
     const void* const* xs = x_ptrs + ((flags & DP_PLAN_SAME_X) ? 0 : i * n);
     void* const* ys = y_ptrs + ((flags & DP_PLAN_SAME_Y) ? 0 : i * n);
-    st = plan_run_step(plan, xs, ys, workspace, device_status, static_cast<cudaStream_t>(stream), &chained);
+    st = plan_run_step(plan, steps[i], xs, ys, workspace, device_status, static_cast<cudaStream_t>(stream), &chained);
     if (st != DP_OK) return st;
   }
   return DP_OK;
@@ -785,7 +854,7 @@ extern "C" int dp_plan_run_host(const dp_plan* plan_c, const int32_t* steps, int
     DP_CUDA_OK(cudaEventRecord(plan->ev_copied[h], plan->copy_stream));
     DP_CUDA_OK(cudaStreamWaitEvent(stream, plan->ev_copied[h], 0));
     bool chained = false;  // an event wait precedes every step's first launch
-    st = plan_run_step(plan, xs.data(), y_dev, workspace, device_status, stream, &chained);
+    st = plan_run_step(plan, steps[i], xs.data(), y_dev, workspace, device_status, stream, &chained);
     if (st != DP_OK) return st;
     DP_CUDA_OK(cudaEventRecord(plan->ev_consumed[h], stream));
     if (d2h_layer >= 0) {

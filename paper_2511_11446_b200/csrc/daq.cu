@@ -139,9 +139,15 @@ template <int MAXV>
 __global__ void __launch_bounds__(kDaqWarps * 32)
 daq_rows_robust_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t ldx, int8_t* __restrict__ q,
                        int64_t ldq, float* __restrict__ s_a, int32_t* __restrict__ rowsum, int clip_rank,
-                       float qmax) {
+                       float qmax, int tiled_kb, const UnpackJob job) {
+  pdl_launch_dependents();
   const int64_t row = static_cast<int64_t>(blockIdx.x) * kDaqWarps + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
+  pdl_wait();
+  if (static_cast<int>(blockIdx.x) >= job.first_block) {  // the launch's weight-expansion CTAs
+    unpack_units(job, blockIdx.x - job.first_block);
+    return;
+  }
   if (row >= M) return;
   const int nvec = K >> 3;
   const uint4* xr = reinterpret_cast<const uint4*>(x + row * ldx);
@@ -194,7 +200,7 @@ daq_rows_robust_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t
   }
   const float magic = 12582912.0f;
   const float lo = magic - qmax, hi = magic + qmax;
-  uint2* out = reinterpret_cast<uint2*>(q + row * ldq);
+  const QRow qr(q, row, ldq, tiled_kb);
   int sum = 0;
 #pragma unroll
   for (int i = 0; i < MAXV; ++i) {
@@ -203,7 +209,7 @@ daq_rows_robust_kernel(const uint16_t* __restrict__ x, int64_t M, int K, int64_t
       const uint32_t p0 = quant_pair_clamped(v[i].x, inv, lo, hi), p1 = quant_pair_clamped(v[i].y, inv, lo, hi);
       const uint32_t p2 = quant_pair_clamped(v[i].z, inv, lo, hi), p3 = quant_pair_clamped(v[i].w, inv, lo, hi);
       const uint2 o = make_uint2(__byte_perm(p0, p1, 0x5410), __byte_perm(p2, p3, 0x5410));
-      out[idx] = o;
+      qr.store(idx, o);
       sum = __dp4a(static_cast<int>(o.x), 0x01010101, sum);
       sum = __dp4a(static_cast<int>(o.y), 0x01010101, sum);
     }
@@ -257,19 +263,29 @@ int launch_daq(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int6
 }
 
 int launch_daq_robust(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq, float* s_a,
-                      int32_t* rowsum, int clip_rank, int act_bits, cudaStream_t stream) {
+                      int32_t* rowsum, int clip_rank, int act_bits, bool tiled, cudaStream_t stream, bool pdl,
+                      const UnpackJob* unpack) {
   if (M == 0) return DP_OK;
   const uint16_t* xp = static_cast<const uint16_t*>(x);
   const int k = static_cast<int>(K);
+  const int tiled_kb = tiled ? k / 128 : 0;
   const float qmax = static_cast<float>((1 << (act_bits - 1)) - 1);
-  const dim3 grid(static_cast<unsigned>((M + kDaqWarps - 1) / kDaqWarps)), block(kDaqWarps * 32);
+  UnpackJob job{nullptr, nullptr, 0, 0, 0};
+  if (unpack != nullptr) job = *unpack;
+  const unsigned daq_blocks = static_cast<unsigned>((M + kDaqWarps - 1) / kDaqWarps);
+  job.first_block = static_cast<int32_t>(daq_blocks);
+  const unsigned extra = static_cast<unsigned>((job.units + kDaqWarps * 32 - 1) / (kDaqWarps * 32));
+  const dim3 grid(daq_blocks + extra), block(kDaqWarps * 32);
   cudaError_t e;
   if (k <= 256 * 5)
-    e = launch(daq_rows_robust_kernel<5>, grid, block, 0, stream, false, xp, M, k, ldx, q, ldq, s_a, rowsum, clip_rank, qmax);
+    e = launch(daq_rows_robust_kernel<5>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, clip_rank,
+               qmax, tiled_kb, job);
   else if (k <= 256 * 9)
-    e = launch(daq_rows_robust_kernel<9>, grid, block, 0, stream, false, xp, M, k, ldx, q, ldq, s_a, rowsum, clip_rank, qmax);
+    e = launch(daq_rows_robust_kernel<9>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, clip_rank,
+               qmax, tiled_kb, job);
   else
-    e = launch(daq_rows_robust_kernel<18>, grid, block, 0, stream, false, xp, M, k, ldx, q, ldq, s_a, rowsum, clip_rank, qmax);
+    e = launch(daq_rows_robust_kernel<18>, grid, block, 0, stream, pdl, xp, M, k, ldx, q, ldq, s_a, rowsum, clip_rank,
+               qmax, tiled_kb, job);
   if (e != cudaSuccess) return fail(DP_ERR_CUDA, "robust DAQ launch failed: %s", cudaGetErrorString(e));
   return DP_OK;
 }
@@ -320,6 +336,6 @@ extern "C" int dp_daq_quantize_robust(const void* x_bf16, int64_t M, int64_t K, 
     return fail(DP_ERR_ALIGN, "dp_daq_quantize_robust: pointers/pitches must be 16-byte aligned");
   int st = check_device();
   if (st != DP_OK) return st;
-  return launch_daq_robust(x_bf16, M, K, ldx, q, ldq, s_a, rowsum, clip_rank, act_bits,
-                           static_cast<cudaStream_t>(stream));
+  return launch_daq_robust(x_bf16, M, K, ldx, q, ldq, s_a, rowsum, clip_rank, act_bits, false,
+                           static_cast<cudaStream_t>(stream), false, nullptr);
 }

@@ -32,7 +32,8 @@ int launch_daq(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int6
                const UnpackJob* unpack = nullptr);
 int launch_unpack(const UnpackJob& job, cudaStream_t stream, bool pdl);
 int launch_daq_robust(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq, float* s_a,
-                      int32_t* rowsum, int clip_rank, int act_bits, cudaStream_t stream);
+                      int32_t* rowsum, int clip_rank, int act_bits, bool tiled, cudaStream_t stream, bool pdl,
+                      const UnpackJob* unpack);
 
 // simt.cu — CUDA-core weight-streaming linear for small M (DAQ fused in the CTA prologue).
 struct SimtArgs {

@@ -166,6 +166,57 @@ def test_plan_with_variants_set_per_layer_matches_oracle():
         B.dp_plan_destroy(plan)
 
 
+@pytest.mark.parametrize("flags", [B.DP_FLAG_GROUP_SMALL_M, B.DP_FLAG_NO_UNPACK_FIRST | B.DP_FLAG_FUSED_DAQ],
+                         ids=["grouped", "in_gemm_fused"])
+def test_plan_with_daq_policy_matches_oracle_composition(flags):
+    """dp_plan_set_daq: percentile clip (p = 99.9) and activation bits per time bin (8 / 6 / 4 for
+    the thirds of 12 timesteps) on every layer, whatever variants the plan was created with; the
+    oracle composes its pinned pieces step by step. Setting the policy back restores the plain rule."""
+    table, layers, dev = _mini_plan(tokens=256, batch=2, blocks=1)
+    T, kept, by_bin = 12, [1, 5, 6, 11], [8, 6, 4]
+    nL, nS = len(layers), len(kept)
+    xs = [[synth.activations(SEED, l, t, L["M"], L["K"], synth.sigma_t(t, T), n_out=max(1, L["K"] // 100))
+           for l, L in enumerate(layers)] for t in kept]
+
+    def compose(p, bins):
+        out = []
+        for i, t in enumerate(kept):
+            bits = bins[min(2, 3 * t // T)]
+            row = []
+            for l, L in enumerate(layers):
+                q, s_a, _ = oracle.daq_robust(xs[i][l], oracle.clip_rank(p, L["K"]), bits)
+                w = oracle.unpack(L["qweight"], L["K"], L["bits"])
+                row.append(oracle.epilogue(oracle.gemm_i32(q, w), s_a, L["s_w"], L["bias"]))
+            out.append(row)
+        return out
+
+    plan = B.dp_plan_create([d.w for d in dev], [L["M"] for L in layers], flags)
+    try:
+        xd = [[to_dev_bf16(xs[i][l]) for l in range(nL)] for i in range(nS)]
+        xp = B.ptr_array([xd[i][l].data_ptr() for i in range(nS) for l in range(nL)])
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for p_e3, p, bins in ((99900, "99.9", by_bin), (100000, "100", [8, 8, 8])):
+            B.dp_plan_set_daq(plan, p_e3, T, bins)
+            ws = torch.empty(B.dp_plan_workspace(plan), dtype=torch.uint8, device="cuda")
+            yd = [[torch.full((L["M"], L["N"]), float("nan"), dtype=torch.bfloat16, device="cuda")
+                   for L in layers] for _ in range(nS)]
+            yp = B.ptr_array([yd[i][l].data_ptr() for i in range(nS) for l in range(nL)])
+            B.dp_plan_run(plan, kept, 0, xp, yp, ws, status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            ref = compose(p, bins)
+            for i in range(nS):
+                for l in range(nL):
+                    d = bf16_ulp_dist(bf16_to_np(yd[i][l]), ref[i][l])
+                    assert d.max() <= 1, (p, i, l, table[l], int(d.max()))
+        with pytest.raises(B.DiffproError):
+            B.dp_plan_set_daq(plan, 99900, T, [8, 9, 4])
+        with pytest.raises(B.DiffproError):
+            B.dp_plan_set_daq(plan, 90000, T, by_bin)  # K = 1152 would need rank 116
+    finally:
+        B.dp_plan_destroy(plan)
+
+
 def test_plan_run_host_inputs():
     table, layers, dev = _mini_plan(tokens=128, batch=2, blocks=1)
     kept = [1, 3, 4]
