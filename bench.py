@@ -206,8 +206,7 @@ def run_ours(args):
                    "daq_policy": args.daq_policy or "absmax, 8 bits (the metric's definition)"},
         "us_per_dit_step": 1e3 * ms_per_step / nS,
         "roofline_step": {"ideal_us_per_dit_step_nominal": None},
-        # under a DAQ policy every layer, small-M ones included, is a quantization launch plus a linear launch
-        "gpu_launches": (2 * nL if args.daq_policy else stack.launches_per_timestep()) * nS * args.steps,
+        "gpu_launches": stack.launches_per_timestep() * nS * args.steps,
         "clocks": clocks,
     }
 

@@ -255,8 +255,9 @@ int dp_plan_set_layer_flags(dp_plan* plan, int32_t layer, uint32_t flags);
  *   act_bits  = act_bits_by_bin[min(2, 3 t / n_timesteps)] for a step with timestep value t
  * (reading: the three bins are thirds of [0, n_timesteps), bin 0 holding the smallest timestep
  * values; n_timesteps = 0: 8 bits at every step, act_bits_by_bin may be NULL). Under a policy other
- * than (100000, 8 bits) packed layers run in the unpack-first form, small-M layers run one by one
- * behind a quantization launch of their own, and DP_FLAG_FUSED_DAQ is ignored. May raise
+ * than (100000, 8 bits) packed layers run in the unpack-first form, grouped small-M layers keep their
+ * shared launches for K <= 1280 (longer rows run one by one behind a quantization launch of their
+ * own), and DP_FLAG_FUSED_DAQ is ignored. May raise
  * dp_plan_workspace: ask again afterwards. Limits: K <= 4608 and clip_rank <= 64 for every layer
  * (DP_ERR_SHAPE), bits in [2, 8] (DP_ERR_BITS); the plan is unchanged on error. Host only; not to
  * be called while a dp_plan_run of the plan is being issued. */

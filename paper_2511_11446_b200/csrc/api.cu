@@ -743,9 +743,11 @@ static int plan_run_step(dp_plan* plan, int32_t t, const void* const* xs, void* 
     act_bits = plan->daq_bits[bin > 2 ? 2 : bin];
   }
   const bool robust = plan->daq_p_e3 < 100000 || act_bits < 8;
+  // a group whose rows are too long for the grouped policy DAQ (register-resident, K <= 1280) runs layer by layer
+  auto group_splits = [&](int l) { return robust && plan->layers[l].w.K > 1280; };
   for (const std::vector<int>& grp : plan->groups) {
-    if (robust) break;  // the grouped launch quantizes with the plain rule: such layers run one by one below
     const PlanLayer& G = plan->layers[grp[0]];
+    if (group_splits(grp[0])) continue;
     SimtGroupArgs ga;
     ga.M = G.M;
     ga.N = G.w.N;
@@ -753,6 +755,8 @@ static int plan_run_step(dp_plan* plan, int32_t t, const void* const* xs, void* 
     ga.n_layers = static_cast<int32_t>(grp.size());
     ga.early_w = *chained ? 1 : 0;
     ga.status = status;
+    ga.daq_rank = robust ? clip_rank_of(plan->daq_p_e3, G.w.K) : 1;
+    ga.daq_bits = act_bits;
     ga.q_scratch = static_cast<int8_t*>(workspace);
     ga.sa_scratch = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) +
                                              align256(static_cast<size_t>(ga.n_layers) * ga.M * ga.K));
@@ -770,7 +774,7 @@ static int plan_run_step(dp_plan* plan, int32_t t, const void* const* xs, void* 
   }
   for (int l = 0; l < n; ++l) {
     const PlanLayer& L = plan->layers[l];
-    if (L.M == 0 || (plan->grouped[l] && !robust)) continue;
+    if (L.M == 0 || (plan->grouped[l] && !group_splits(l))) continue;
     if (!xs[l] || !ys[l]) return fail(DP_ERR_INVALID_ARG, "layer %d: NULL x or y", l);
     if (!aligned16(xs[l]) || !aligned16(ys[l])) return fail(DP_ERR_ALIGN, "layer %d: x/y misaligned", l);
     const CUtensorMap* ta = nullptr;

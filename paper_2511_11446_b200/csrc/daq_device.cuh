@@ -137,6 +137,105 @@ __device__ __forceinline__ void daq_two_rows_2pass(const uint16_t* __restrict__ 
   }
 }
 
+// ---- DAQ with a percentile clip and a-bit codes -------------------------------------------------------
+// Eq. "daq" with tau = Percentile(|v|, p) below the maximum (nearest-rank reading: the clip_rank-th
+// largest magnitude of the token, repeats counted) and alpha = tau / qmax, qmax = 2^(a-1) - 1 for the
+// activation bits a of the step's time bin (Step 6). One warp per token, row in registers as above.
+// The threshold is found by peeling maxima: each round takes the largest magnitude below the
+// previous one together with its multiplicity until clip_rank values are covered (for p = 99.9: 2
+// rounds at K = 1152, 5 at K = 4608). A lane keeps the maximum of each of its 8-element vectors, so
+// a round is a max over those few numbers plus a rescan of only the vectors that held the peeled
+// value. Values beyond tau are clipped to it before the multiplication and so land on +-qmax.
+// Packed helpers on words of two 15-bit magnitudes (bit 15 of each half clear):
+// number of halves equal to the value replicated in t2
+__device__ __forceinline__ int count_eq2(uint32_t e, uint32_t t2) {
+  const uint32_t z = ((e ^ t2) | 0x80008000u) - 0x00010001u;  // bit 15 of a half stays set unless the half was 0
+  return __popc(~z & 0x80008000u);
+}
+// the halves that are below the bound replicated in b2 (<= 0x8000 per half), the others zeroed
+__device__ __forceinline__ uint32_t keep_below2(uint32_t e, uint32_t b2) {
+  const uint32_t ge = ((e | 0x80008000u) - b2) & 0x80008000u;  // bit 15 set where half >= bound; no borrow
+  return e & ~(ge - (ge >> 15));
+}
+__device__ __forceinline__ uint32_t fold_max2(uint32_t m2) { return max(m2 & 0xFFFFu, m2 >> 16); }
+// Two bf16 clipped to [-tau, tau] (tau2 = tau's magnitude bits in both halves): the magnitudes are
+// 15-bit integers ordered like the values, so one packed minimum does it; then quantized as usual.
+// Clipping first and rounding after is the equation's own order and cannot leave +-qmax.
+__device__ __forceinline__ uint32_t quant_pair_clipped(uint32_t w, uint32_t tau2, float inv) {
+  return quant_pair((w & 0x80008000u) | __vminu2(w & 0x7FFF7FFFu, tau2), inv);
+}
+
+// One token by one warp: x[K] bf16 (16-byte aligned) -> codes through `qr`, scale in `sc`, the lane's
+// partial code sum in `sum`. K <= 256 * MAXV.
+template <int MAXV>
+__device__ __forceinline__ void robust_row(const uint16_t* __restrict__ x, int K, int lane, int clip_rank, float qmax,
+                                           const QRow& qr, float& sc, int& sum) {
+  const int nvec = K >> 3;
+  const uint4* xr = reinterpret_cast<const uint4*>(x);
+  uint4 v[MAXV];
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int idx = lane + 32 * i;
+    if (idx < nvec) ld_nc_u32x4(xr + idx, v[i]);
+    else v[i] = make_uint4(0, 0, 0, 0);
+  }
+  // threshold: magnitude bits (bf16 pattern, sign cleared) of the clip_rank-th largest element
+  uint32_t gmax[MAXV];  // per vector: its largest magnitude not yet peeled (padding vectors: 0)
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i)
+    gmax[i] = fold_max2(absmax_bits2(absmax_bits2(absmax_bits2(absmax_bits2(0u, v[i].x), v[i].y), v[i].z), v[i].w));
+  uint32_t tau_bits = 0;
+  int remaining = clip_rank;
+  for (int round = 0; round < clip_rank; ++round) {
+    uint32_t mx = 0;
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) mx = max(mx, gmax[i]);
+    const uint32_t wmx = __reduce_max_sync(0xFFFFFFFFu, mx);
+    tau_bits = wmx;
+    if (wmx == 0) break;  // all that is left are zeros
+    const uint32_t t2 = wmx | (wmx << 16);
+    int cnt = 0;
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) {
+      if (gmax[i] == wmx) {  // this vector holds the value: count it and find the vector's next maximum
+        const uint32_t w[4] = {v[i].x & 0x7FFF7FFFu, v[i].y & 0x7FFF7FFFu, v[i].z & 0x7FFF7FFFu,
+                               v[i].w & 0x7FFF7FFFu};
+        uint32_t m2 = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          cnt += count_eq2(w[j], t2);
+          m2 = __vmaxu2(m2, keep_below2(w[j], t2));
+        }
+        gmax[i] = fold_max2(m2);
+      }
+    }
+    const int wcnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+    if (wcnt >= remaining) break;
+    remaining -= wcnt;
+  }
+  const float tau = __uint_as_float(tau_bits << 16);
+  float inv = 0.0f;
+  sc = 0.0f;
+  if (!(tau < 7.888609052210118e-31f)) {  // 2^-100, as in the absmax form
+    sc = __fdiv_rn(tau, qmax);
+    inv = __fdiv_rn(qmax, tau);
+  }
+  const uint32_t tau2 = tau_bits | (tau_bits << 16);
+  sum = 0;
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int idx = lane + 32 * i;
+    if (idx < nvec) {
+      const uint32_t p0 = quant_pair_clipped(v[i].x, tau2, inv), p1 = quant_pair_clipped(v[i].y, tau2, inv);
+      const uint32_t p2 = quant_pair_clipped(v[i].z, tau2, inv), p3 = quant_pair_clipped(v[i].w, tau2, inv);
+      const uint2 o = make_uint2(__byte_perm(p0, p1, 0x5410), __byte_perm(p2, p3, 0x5410));
+      qr.store(idx, o);
+      sum = __dp4a(static_cast<int>(o.x), 0x01010101, sum);
+      sum = __dp4a(static_cast<int>(o.y), 0x01010101, sum);
+    }
+  }
+}
+
 // Packed unit -> 8 words of 4 int8 (true values, k ascending).
 template <int BITS>
 __device__ __forceinline__ void expand_unit(const uint32_t (&pk)[BITS], uint32_t (&w)[8]) {

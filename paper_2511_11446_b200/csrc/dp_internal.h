@@ -76,6 +76,7 @@ struct SimtGroupArgs {
   int8_t* q_scratch;
   float* sa_scratch;
   int32_t* status;  // as SimtArgs::status
+  int32_t daq_rank, daq_bits;  // the group's DAQ rule: (1, 8) = absmax, 8 bits; else percentile clip / a-bit codes
   // Matrix-instruction form: CTAs [cta_begin[l], cta_begin[l + 1]) of grid.x work on layer l (filled
   // by launch_simt_group: more CTAs for the layers that take longer).
   int32_t cta_begin[kSimtGroupMax + 1];

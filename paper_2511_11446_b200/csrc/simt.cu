@@ -495,6 +495,23 @@ daq_group_kernel(SimtGroupArgs g) {
   if (lane == 0) g.sa_scratch[static_cast<int64_t>(layer) * g.M + row] = sc;
 }
 
+// The same under a DAQ policy (percentile clip, a-bit codes): rows of up to 1280 elements in registers.
+__global__ void __launch_bounds__(kSimtWarps * 32)
+daq_group_robust_kernel(SimtGroupArgs g) {
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t row = static_cast<int64_t>(blockIdx.x) * kSimtWarps + warp;
+  pdl_wait();
+  if (row >= g.M) return;
+  const int layer = blockIdx.y;
+  const uint16_t* x = static_cast<const uint16_t*>(g.layer[layer].x) + row * g.K;
+  const QRow qr(g.q_scratch + static_cast<int64_t>(layer) * g.M * g.K, row, g.K, 0);
+  float sc;
+  int sum;
+  robust_row<5>(x, g.K, lane, g.daq_rank, static_cast<float>((1 << (g.daq_bits - 1)) - 1), qr, sc, sum);
+  if (lane == 0) g.sa_scratch[static_cast<int64_t>(layer) * g.M + row] = sc;
+}
+
 template <bool MMA>
 __global__ void __launch_bounds__(kSimtWarps * 32, MMA ? 2 : 0)
 simt_group_kernel(SimtGroupArgs g) {
@@ -573,7 +590,10 @@ int launch_simt_group(const SimtGroupArgs& g, cudaStream_t stream, bool pdl) {
   if (g.M == 0 || g.n_layers == 0) return DP_OK;
   if (g.q_scratch != nullptr) {
     const dim3 dgrid(static_cast<unsigned>((g.M + kSimtWarps - 1) / kSimtWarps), static_cast<unsigned>(g.n_layers));
-    cudaError_t e = launch(daq_group_kernel, dgrid, dim3(kSimtWarps * 32), 0, stream, pdl, g);
+    const bool robust = g.daq_rank > 1 || g.daq_bits < 8;
+    if (robust && g.K > 1280) return fail(DP_ERR_SHAPE, "grouped DAQ policy: K=%d above 1280", g.K);
+    cudaError_t e = robust ? launch(daq_group_robust_kernel, dgrid, dim3(kSimtWarps * 32), 0, stream, pdl, g)
+                           : launch(daq_group_kernel, dgrid, dim3(kSimtWarps * 32), 0, stream, pdl, g);
     if (e != cudaSuccess) return fail(DP_ERR_CUDA, "grouped DAQ launch failed: %s", cudaGetErrorString(e));
   }
   const size_t smem = simt_smem_bytes(g.K);
