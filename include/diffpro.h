@@ -10,7 +10,8 @@
  *   -> INT8 x INT8 -> INT32 GEMM with per-output-channel weight scales (Step 5; Implementation)
  *   -> dequantisation y = acc * s_a[m] * s_w[n] + bias[n], stored as bf16.
  * dp_plan_run is Phase B of Algorithm 2: for t in reverse(K*), run every wrapped linear per the
- * bit plan.
+ * bit plan. dp_daq_quantize_robust / dp_plan_set_daq add the equation's percentile clip (p < 100)
+ * and Phase B's activation bits per time bin.
  *
  * Conventions for every entry point
  *   - All tensor pointers are DEVICE pointers owned by the caller unless the name says `host`.
