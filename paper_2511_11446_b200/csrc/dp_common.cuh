@@ -252,11 +252,6 @@ __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, u
                : "memory");
 }
 
-// Asks L2 to fetch `bytes` (a multiple of 16) from 16-byte aligned `gsrc`; nothing lands in the SM.
-__device__ __forceinline__ void bulk_prefetch_l2(const void* gsrc, uint32_t bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gsrc), "r"(bytes) : "memory");
-}
-
 // 2-D tiled store shared -> global (bulk async-group completion). Rows past the tensor's extent
 // are clipped by the hardware. Coordinates are never negative here.
 __device__ __forceinline__ void tma_store_2d(const void* tmap, int c0, int c1, const void* src) {

@@ -1,7 +1,7 @@
-// CUDA-core path of the quantized linear for small row counts (adaLN modulation: M = batch).
+// Weight-streaming path of the quantized linear for small row counts (adaLN modulation: M = batch).
 //
 // The whole layer in one launch, bound by the weight bytes (M <= 32: 2..144 int8 ops per weight
-// byte). A CTA owns 32 output channels and up to 8 tokens. Eight lanes share one channel: each
+// byte). Form for K > 1152: a CTA owns 32 output channels and up to 8 tokens. Eight lanes share one channel: each
 // lane fetches its 32-code units of the packed weight row straight into registers, all loads of a
 // pass issued back to back and BEFORE the CTA quantizes its tokens (DAQ, Step 3 Eq. "daq", one
 // warp per token, codes to shared memory), so the HBM latency of the weights overlaps the
