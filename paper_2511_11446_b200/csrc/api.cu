@@ -108,6 +108,7 @@ static int clip_rank_of(int32_t p_e3, int32_t K) {
   return static_cast<int>(K - (c < 1 ? 1 : c) + 1);
 }
 
+constexpr int64_t kEarlyWeightsMaxRows = 512;  // see run_linear
 constexpr int64_t kSimtMaxRows = 32;  // at or below this the CUDA-core streaming kernel is used
 
 static bool use_simt(int64_t M, int32_t N, int32_t K, uint32_t flags) {
@@ -236,6 +237,11 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
   g.a_tiled = tiled ? 1 : 0;
   g.early_w = fused ? (chained ? 1 : 0) : (s_a_in == nullptr ? 1 : 0);
   if (unpack_first) g.early_w = 0;  // the weights come from the kernel just before this one
+  // Fetching weight tiles while the DAQ launch still runs pays only for small M: measured on B200,
+  // it shortens a layer by ~0.3 us at M = 256 but lengthens it by 1-1.5 us at M = 2048..4096 (the
+  // prefetch of every CTA competes with the DAQ launch for bandwidth, and the ring then starts with
+  // a burst of activation loads instead of a steady stream); no effect at M = 32768.
+  if (M > kEarlyWeightsMaxRows) g.early_w = 0;
   g.x = fused ? static_cast<const uint16_t*>(x) : nullptr;
   g.ldx = ldx;
   g.q_out = fused ? const_cast<int8_t*>(q) : nullptr;
