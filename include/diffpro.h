@@ -119,8 +119,8 @@ typedef struct dp_debug {
 #define DP_FLAG_FUSED_DAQ 0x40000u
 
 /* dp_wq_linear and dp_plan_create, packed bit-widths (3, 4) on the tensor-core path: where the
- * packed weights are expanded (Step 4's unpack). UNPACK_FIRST: once per call to int8 [N][K] in the
- * workspace (extra CTAs of the DAQ launch; a launch of its own when the activations arrive
+ * packed weights are expanded (the unpack of the "GPTQ packed" weights of Step 3). UNPACK_FIRST: once
+ * per call to int8 [N][K] in the workspace (extra CTAs of the DAQ launch; a launch of its own when the activations arrive
  * quantized), the 8-bit kernel then runs on that copy. NO_UNPACK_FIRST: tile by tile in shared memory
  * inside the GEMM. The first form avoids repeating the expansion in every CTA that needs a weight
  * tile (M/128 of them) and was faster on B200 at every size measured except where the
