@@ -217,6 +217,45 @@ def test_plan_with_daq_policy_matches_oracle_composition(flags):
         B.dp_plan_destroy(plan)
 
 
+def test_daq_policy_on_grouped_small_m_layers_with_long_rows():
+    """Small-M layers of equal shape are grouped; under a DAQ policy a group with K = 4608 cannot use
+    the grouped quantization kernel (rows up to 1280) and falls back to layer-by-layer launches, a
+    group with K = 1152 keeps its shared launch: both must equal the oracle's composition."""
+    shapes = [(8, 4608, 256, 4), (8, 4608, 256, 8), (8, 1152, 96, 3), (8, 1152, 96, 4), (16, 1152, 96, 8)]
+    layers, dev = [], []
+    for l, (M, K, N, bits) in enumerate(shapes):
+        w, s_w = synth.weights(SEED, 40 + l, N, K, bits)
+        b = synth.bias(SEED, 40 + l, N)
+        dev.append(DevLayer(w, s_w, b, bits))
+        layers.append(dict(M=M, N=N, K=K, bits=bits, w=w, s_w=s_w, bias=b))
+    T, kept, bins = 9, [0, 4, 8], [8, 5, 3]
+    xs = [[synth.activations(SEED, 40 + l, t, L["M"], L["K"], 1.0, n_out=max(1, L["K"] // 100))
+           for l, L in enumerate(layers)] for t in kept]
+    plan = B.dp_plan_create([d.w for d in dev], [L["M"] for L in layers], B.DP_FLAG_GROUP_SMALL_M)
+    try:
+        B.dp_plan_set_daq(plan, 99900, T, bins)
+        ws = torch.empty(B.dp_plan_workspace(plan), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        nL, nS = len(layers), len(kept)
+        xd = [[to_dev_bf16(xs[i][l]) for l in range(nL)] for i in range(nS)]
+        yd = [[torch.full((L["M"], L["N"]), float("nan"), dtype=torch.bfloat16, device="cuda")
+               for L in layers] for _ in range(nS)]
+        xp = B.ptr_array([xd[i][l].data_ptr() for i in range(nS) for l in range(nL)])
+        yp = B.ptr_array([yd[i][l].data_ptr() for i in range(nS) for l in range(nL)])
+        B.dp_plan_run(plan, kept, 0, xp, yp, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for i, t in enumerate(kept):
+            bits = bins[min(2, 3 * t // T)]
+            for l, L in enumerate(layers):
+                q, s_a, _ = oracle.daq_robust(xs[i][l], oracle.clip_rank("99.9", L["K"]), bits)
+                ref = oracle.epilogue(oracle.gemm_i32(q, L["w"]), s_a, L["s_w"], L["bias"])
+                d = bf16_ulp_dist(bf16_to_np(yd[i][l]), ref)
+                assert d.max() <= 1, (t, l, shapes[l], int(d.max()))
+    finally:
+        B.dp_plan_destroy(plan)
+
+
 def test_plan_run_host_inputs():
     table, layers, dev = _mini_plan(tokens=128, batch=2, blocks=1)
     kept = [1, 3, 4]
