@@ -8,7 +8,7 @@ import torch
 
 import oracle
 from paper_2511_11446_b200 import synth
-from helpers import bf16_bits, bf16_ulp_dist
+from helpers import bf16_bits, bf16_ulp_dist, f32_frac, round_frac_to_f32
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -129,6 +129,71 @@ def test_epilogue_exact_bound_and_bf16_rounding():
     a = np.arange(-256, 256, dtype=np.int32).reshape(1, -1)
     y1 = oracle.epilogue(a, np.ones(1, np.float32), np.ones(a.shape[1], np.float32), None)
     assert np.array_equal(synth.bf16_bits_to_f32(y1)[0], a[0].astype(np.float32))
+
+
+def _bf16_rne_bits(v: np.float32) -> int:
+    """bf16 bit pattern of a finite float32, round to nearest, ties to even, in exact rationals."""
+    u = int(np.float32(v).view(np.uint32))
+    lo = u & 0xFFFF0000                      # truncation toward zero (same sign)
+    hi = lo + 0x10000                        # next bf16 away from zero
+    f = lambda b: Fraction(float(np.uint32(b).view(np.float32)))
+    x = Fraction(float(v))
+    dl, dh = abs(x - f(lo)), abs(f(hi) - x)
+    if dl < dh or (dl == dh and ((lo >> 16) & 1) == 0):
+        return lo >> 16
+    return hi >> 16
+
+
+def _epilogue_sequences(acc: int, s_a, s_w, bias_f32):
+    """Step 5's dequantisation of one accumulator in exact rationals, each fp32 operation rounded
+    once to nearest-even: the defined sequence and two plausible wrong ones."""
+    A, SA, SW, B = Fraction(acc), f32_frac(s_a), f32_frac(s_w), f32_frac(bias_f32)
+    t = f32_frac(round_frac_to_f32(A))                         # int32 -> fp32
+    sc = f32_frac(round_frac_to_f32(SA * SW))                  # s_a[m] * s_w[n]
+    defined = round_frac_to_f32(t * sc + B)                    # one fused multiply-add
+    other_assoc = round_frac_to_f32(f32_frac(round_frac_to_f32(t * SA)) * SW + B)   # (t*s_a)*s_w + bias
+    unfused = round_frac_to_f32(f32_frac(round_frac_to_f32(t * sc)) + B)            # mul, then add
+    return [_bf16_rne_bits(v) for v in (defined, other_assoc, unfused)]
+
+
+def test_epilogue_exact_fp32_sequence():
+    """orc_epilogue is exactly cvt(RN) -> s_a*s_w (RN) -> fma (RN) -> bf16 (RNE), evaluated here in
+    exact rationals and compared for EQUALITY: random cases, |acc| > 2^24 (where the conversion
+    rounds) and constructed cancellation cases acc*s_a*s_w ~ -bias, where the association
+    (t*s_a)*s_w + bias and an unfused multiply-then-add land on other bf16 values. The test also
+    checks that those two wrong sequences do differ from the oracle on its cases, so an oracle that
+    computed either would fail here."""
+    rng = np.random.default_rng(2511)
+    cases = []
+    for _ in range(300):                                        # random, full accumulator range
+        cases.append((int(rng.integers(-(75 * 10**6), 75 * 10**6)),
+                      np.float32(abs(rng.standard_normal()) * 0.05 + 1e-3),
+                      np.float32(abs(rng.standard_normal()) * 1e-3 + 1e-5),
+                      np.float32(rng.standard_normal() * 0.5)))
+    for a in (2**24 + 1, -(2**24 + 3), 2**25 + 2, 2**26 - 1, 74907648, -74907648, 2**24 + 2, 33554433):
+        cases.append((a, np.float32(0.0123), np.float32(3.3e-4), np.float32(-0.75)))
+    for _ in range(400):                                        # cancellation: t*sc ~ -bias
+        s_a = np.float32(abs(rng.standard_normal()) * 0.05 + 1e-3)
+        s_w = np.float32(abs(rng.standard_normal()) * 1e-3 + 1e-5)
+        b = np.float32(rng.standard_normal() * 2.0)
+        b = np.float32(synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(np.array([b], np.float32)))[0])
+        a = int(round(-float(b) / (float(s_a) * float(s_w))))
+        if abs(a) > 74907648 or a == 0:
+            continue
+        cases.append((a + int(rng.integers(-1, 2)), s_a, s_w, b))
+    acc = np.array([[c[0] for c in cases]], np.int32).T.copy()          # [P, 1]: one row per case
+    got = np.empty(len(cases), np.uint16)
+    n_assoc = n_unfused = 0
+    for i, (a, s_a, s_w, b) in enumerate(cases):
+        bias_bits = synth.f32_to_bf16_bits(np.array([b], np.float32))
+        bias_f32 = synth.bf16_bits_to_f32(bias_bits)[0]
+        y = oracle.epilogue(acc[i:i + 1], np.array([s_a], np.float32), np.array([s_w], np.float32), bias_bits)
+        got[i] = y[0, 0]
+        want, assoc, unfused = _epilogue_sequences(a, s_a, s_w, bias_f32)
+        assert int(got[i]) == want, (i, a, float(s_a), float(s_w), float(b))
+        n_assoc += assoc != want
+        n_unfused += unfused != want
+    assert n_assoc >= 10 and n_unfused >= 10, (n_assoc, n_unfused)
 
 
 def test_bf16_rounding_matches_torch_exhaustively_sampled():
