@@ -353,7 +353,7 @@ def hbm_kernel_rooflines(stack, peaks):
         by = 3 * M * K + 4 * M
         out[f"daq_M32768_K{K}"] = {"bytes": by, "us": t * 1e6, "achieved": by / t / 1e9, "peak": peaks["hbm_gbs"],
                                    "unit": "GB/s", "frac": by / t / 1e9 / peaks["hbm_gbs"]}
-        rank = B.clip_rank("99.9", K)  # the equation's percentile clip, 8-bit codes
+        rank = B.dp_clip_rank(99900, K)  # the equation's percentile clip, 8-bit codes
 
         def run_robust():
             B.dp_daq_quantize_robust(x, M, K, K, q, K, sa, rank, 8)

@@ -5,8 +5,8 @@
  * One call of the hot path =
  *   DAQ (Step 3, Eq. "daq": symmetric INT8, zero-point 0, scale tau/(2^(b-1)-1) with b = 8; here
  *        tau = per-token absmax over K, i.e. the p = 100, one-group case of the equation)
- *   -> unpack of the GPTQ-style packed b-bit weights (Step 1/Step 3: "pack int8/int4 weights";
- *        Algorithm 1 names W3/W4/W8)
+ *   -> unpack of the GPTQ-style packed b-bit weights (Step 1/Step 3: weights are stored packed;
+ *        Algorithm 1 names the widths 3, 4 and 8)
  *   -> INT8 x INT8 -> INT32 GEMM with per-output-channel weight scales (Step 5; Implementation)
  *   -> dequantisation y = acc * s_a[m] * s_w[n] + bias[n], stored as bf16.
  * dp_plan_run is Phase B of Algorithm 2: for t in reverse(K*), run every wrapped linear per the
@@ -58,7 +58,7 @@ typedef void* dp_stream;
  *               little-endian bit stream (8 values per 32-bit word), code u = w + 8.
  *   bits == 3 : qweight is uint32 [N][3K/32]; field k = bits [3k, 3k+3) of the row's bit stream
  *               (32 values per 3 words; fields 10 and 21 of each group straddle words), u = w + 4.
- * s_w  : fp32 [N] per-output-channel scale (Step 5: "per output channel weight scales").
+ * s_w  : fp32 [N], one scale per output channel (Step 5).
  * bias : bf16 [N] or NULL.
  * Requirements: K % 128 == 0, N % 16 == 0, N,K >= 128.
  */
@@ -119,7 +119,7 @@ typedef struct dp_debug {
 #define DP_FLAG_FUSED_DAQ 0x40000u
 
 /* dp_wq_linear and dp_plan_create, packed bit-widths (3, 4) on the tensor-core path: where the
- * packed weights are expanded (the unpack of the "GPTQ packed" weights of Step 3). UNPACK_FIRST: once
+ * packed weights are expanded (the unpack of the GPTQ-style packed weights of Step 3). UNPACK_FIRST: once
  * per call to int8 [N][K] in the workspace (extra CTAs of the DAQ launch; a launch of its own when the activations arrive
  * quantized), the 8-bit kernel then runs on that copy. NO_UNPACK_FIRST: tile by tile in shared memory
  * inside the GEMM. The first form avoids repeating the expansion in every CTA that needs a weight
@@ -173,6 +173,14 @@ int dp_daq_quantize_robust(const void* x_bf16, int64_t M, int64_t K, int64_t ldx
                            float* s_a, int32_t* rowsum, int32_t clip_rank, int32_t act_bits,
                            dp_stream stream);
 
+/*
+ * The rank, counted from the largest, of the nearest-rank percentile that dp_daq_quantize_robust takes
+ * as clip_rank: K - ceil(p K / 100) + 1 for p = clip_percentile_e3 / 1000 percent (Eq. "daq":
+ * tau = Percentile(|v|, p); 100000 -> 1, the maximum). Host arithmetic only; returns 0 when
+ * clip_percentile_e3 is outside [1, 100000] or K < 1.
+ */
+int32_t dp_clip_rank(int32_t clip_percentile_e3, int32_t K);
+
 /* Bytes of device scratch dp_wq_linear needs for this problem (holds the int8 activations and
  * their scales between the two kernels of the large-M path). Never 0; multiple of 256. */
 size_t dp_wq_linear_workspace(int64_t M, int32_t N, int32_t K, int32_t bits, uint32_t flags);
@@ -214,7 +222,9 @@ int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_
  *   - All calls on a device share the one array, on every stream: two calls whose kernels may
  *     overlap on the GPU race on it. Issue them on one stream, or order them yourself.
  *   - The array keeps whatever the previous call left. Nothing in it has to start at zero: the
- *     quantization kernel overwrites every byte the GEMM reads before the GEMM runs.
+ *     quantization kernel overwrites every byte that reaches a stored output before the GEMM runs
+ *     (rows past M of the last 128-token tile are read by the GEMM's tile loads but belong to
+ *     outputs that are never stored).
  *   - No cudaMalloc, cudaFree or other allocating routine is called; x is always bf16 (the
  *     pre-quantized form of dp_wq_linear needs no scratch and is not offered here).
  */
@@ -223,8 +233,8 @@ int dp_wq_linear_static(const dp_weight* w, const void* x_bf16, int64_t ldx, int
                         int64_t ldy, int32_t* device_status, uint32_t flags, dp_stream stream);
 
 /*
- * A deployed plan (Algorithm 2, Phase B: "wrap layers per the bit plan"): n_layers quantized
- * linears with their row counts. Creation validates every layer, chooses kernel variants, encodes
+ * A deployed plan (Algorithm 2, Phase B, whose first step wraps every linear according to the bit
+ * plan): n_layers quantized linears with their row counts. Creation validates every layer, chooses kernel variants, encodes
  * TMA descriptors and may allocate/synchronise; it is not on the timed path. The dp_weight array is
  * copied; the device buffers it points to must outlive the plan.
  */
@@ -249,8 +259,9 @@ int dp_plan_layer_unpack_first(const dp_plan* plan, int32_t layer, int32_t* unpa
  * that do not fit the layer with DP_ERR_SHAPE; the plan is unchanged on error. Not to be called
  * while a dp_plan_run of the plan is being issued. No counterpart in the paper. */
 int dp_plan_set_layer_flags(dp_plan* plan, int32_t layer, uint32_t flags);
-/* DAQ policy of a plan (Eq. "daq" with its percentile clip; Step 6 and Algorithm 2 Phase B:
- * "bin in {early, mid, late}; a_bits <- P_DAQ(bin)"). From the next dp_plan_run on, every layer
+/* DAQ policy of a plan (Eq. "daq" with its percentile clip; Step 6 and Algorithm 2 Phase B, where
+ * the activation bits of a forward pass are looked up by the time bin of its step: early, middle or
+ * late). From the next dp_plan_run on, every layer
  * quantizes its activations as dp_daq_quantize_robust does, with
  *   clip_rank = K - ceil(p K / 100) + 1,  p = clip_percentile_e3 / 1000 percent (100000 = the maximum),
  *   act_bits  = act_bits_by_bin[min(2, 3 t / n_timesteps)] for a step with timestep value t
@@ -314,6 +325,18 @@ int dp_pack_weights_host(const int8_t* w, int32_t N, int32_t K, int32_t bits, vo
  */
 int dp_bench_mma_i8(int32_t ctas, int32_t iters, int32_t tile_n, int32_t* device_status,
                     dp_stream stream);
+
+/*
+ * Test hook for the bounded device waits (no counterpart in the paper). The next launch of the
+ * single-CTA tensor-core kernel made by the calling thread leaves out, in every CTA, the loads of
+ * k-block `k_block` of the CTA's first tile: nothing is issued for that pipeline stage, so nothing is
+ * in flight and no address is touched, and the stage's barrier is never completed. The MMA role's
+ * bounded wait on it runs out (about 0.15 s), every role of the CTA leaves its loop, tensor memory is
+ * freed, the kernel exits normally and `device_status` of that call reads DP_ERR_TIMEOUT; the
+ * outputs of the call are undefined. The hook clears itself when that launch is made; k_block < 0
+ * clears it without a launch. Host state is per thread.
+ */
+void dp_debug_skip_stage_load(int32_t k_block);
 
 const char* dp_status_string(int status);
 const char* dp_last_error(void);

@@ -34,7 +34,8 @@ DP_STATIC_SCRATCH_BYTES = 10 << 20
 
 EXPORTS = ["dp_daq_quantize", "dp_daq_quantize_robust", "dp_wq_linear_workspace", "dp_wq_linear", "dp_wq_linear_static", "dp_plan_create",
            "dp_plan_workspace", "dp_plan_layer_variant", "dp_plan_layer_unpack_first", "dp_plan_set_layer_flags", "dp_plan_set_daq", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
-           "dp_plan_run_host", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_status_string",
+           "dp_plan_run_host", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_clip_rank", "dp_debug_skip_stage_load",
+           "dp_status_string",
            "dp_last_error", "dp_version"]
 
 
@@ -99,6 +100,10 @@ def lib():
                                        C.c_void_p, C.c_size_t, C.c_void_p, C.c_uint32, C.c_void_p]
         L.dp_pack_weights_host.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         L.dp_bench_mma_i8.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.dp_clip_rank.restype = C.c_int32
+        L.dp_clip_rank.argtypes = [C.c_int32, C.c_int32]
+        L.dp_debug_skip_stage_load.restype = None
+        L.dp_debug_skip_stage_load.argtypes = [C.c_int32]
         _lib = L
     return _lib
 
@@ -131,12 +136,13 @@ def dp_wq_linear_workspace(M, N, K, bits, flags=0) -> int:
     return int(lib().dp_wq_linear_workspace(M, N, K, bits, flags))
 
 
-def clip_rank(p, K: int) -> int:
-    """Rank from the top of the nearest-rank p-th percentile of K values (argument marshalling for
-    dp_daq_quantize_robust: K - ceil(p K / 100) + 1)."""
-    from fractions import Fraction
-    f = Fraction(str(p)) * K / 100
-    return K - max(1, -((-f.numerator) // f.denominator)) + 1
+def dp_clip_rank(clip_percentile_e3: int, K: int) -> int:
+    """The clip_rank dp_daq_quantize_robust takes for a percentile given in 1/1000 percent."""
+    return int(lib().dp_clip_rank(clip_percentile_e3, K))
+
+
+def dp_debug_skip_stage_load(k_block: int):
+    lib().dp_debug_skip_stage_load(k_block)
 
 
 def dp_daq_quantize_robust(x, M, K, ldx, q, ldq, s_a, rank, act_bits=8, rowsum=None, stream=None):

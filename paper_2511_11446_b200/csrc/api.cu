@@ -2,6 +2,8 @@
 #include <stdarg.h>
 #include <string.h>
 
+#include <atomic>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -27,23 +29,65 @@ int fail(int status, const char* fmt, ...) {
   return status;
 }
 
+// ---- per-device state ----------------------------------------------------------------------------
+// Everything the library caches about a device (architecture check, SM count, resident CTA pairs,
+// the kernels' shared-memory attributes, which CUDA keeps per device) is set up on the first call
+// made with that device current, under a lock, and published with a release store, so that threads
+// that use different devices, or race on their first call, see consistent state.
+constexpr int kMaxDevices = 64;
+struct DeviceInfo {
+  int status;  // DP_OK or DP_ERR_ARCH
+  int num_sms, max_pairs;
+};
+static DeviceInfo g_dev[kMaxDevices];
+static std::atomic<int> g_dev_ready[kMaxDevices];
+static std::mutex g_dev_mutex;
+
+static int current_device(int* dev) {
+  cudaError_t e = cudaGetDevice(dev);
+  if (e != cudaSuccess) return fail(DP_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  if (*dev < 0 || *dev >= kMaxDevices) return fail(DP_ERR_INVALID_ARG, "device ordinal %d not supported", *dev);
+  return DP_OK;
+}
+
 int check_device() {
   int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return fail(DP_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
-  static int cached_dev = -1, cached_status = DP_OK;
-  if (dev == cached_dev) {
-    if (cached_status != DP_OK) set_error("device %d is not compute capability 10.x", dev);
-    return cached_status;
+  int st = current_device(&dev);
+  if (st != DP_OK) return st;
+  if (!g_dev_ready[dev].load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    if (!g_dev_ready[dev].load(std::memory_order_relaxed)) {
+      DeviceInfo d = {DP_OK, 0, 0};
+      int major = 0;
+      cudaError_t e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+      if (e != cudaSuccess) return fail(DP_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
+      if (major != 10) {
+        d.status = DP_ERR_ARCH;
+      } else {  // a failure here is reported and NOT cached: the next call tries again
+        st = gemm_init_device(dev, &d.num_sms, &d.max_pairs);
+        if (st != DP_OK) return st;
+      }
+      g_dev[dev] = d;
+      g_dev_ready[dev].store(1, std::memory_order_release);
+    }
   }
-  int major = 0;
-  e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
-  if (e != cudaSuccess) return fail(DP_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
-  cached_dev = dev;
-  cached_status = (major == 10) ? DP_OK : DP_ERR_ARCH;
-  if (cached_status != DP_OK)
-    return fail(DP_ERR_ARCH, "device %d has compute capability %d.x; sm_100 required", dev, major);
-  return gemm_init();
+  if (g_dev[dev].status != DP_OK)
+    return fail(g_dev[dev].status, "device %d is not compute capability 10.x; sm_100 required", dev);
+  return DP_OK;
+}
+
+static const DeviceInfo* ready_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  return g_dev_ready[dev].load(std::memory_order_acquire) ? &g_dev[dev] : nullptr;
+}
+int num_sms() {
+  const DeviceInfo* d = ready_device();
+  return d ? d->num_sms : 0;
+}
+int gemm_max_pairs() {
+  const DeviceInfo* d = ready_device();
+  return d ? d->max_pairs : 0;
 }
 
 static size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
@@ -359,21 +403,23 @@ extern "C" int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, cons
 // kernels receive.
 static __device__ __align__(256) unsigned char g_static_scratch[DP_STATIC_SCRATCH_BYTES];
 
-constexpr int kMaxDevices = 64;
-static void* g_static_scratch_ptr[kMaxDevices];  // device address per device ordinal, nullptr = not yet queried
+// device address per device ordinal, nullptr = not yet queried (a cudaDeviceReset invalidates it:
+// the library does not support resetting a device it has been used on)
+static std::atomic<void*> g_static_scratch_ptr[kMaxDevices];
 
 static int static_scratch_address(void** out) {
   int dev = 0;
-  DP_CUDA_OK(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= kMaxDevices) return fail(DP_ERR_INVALID_ARG, "device ordinal %d not supported", dev);
-  if (g_static_scratch_ptr[dev] == nullptr) {
-    void* p = nullptr;
+  int st = current_device(&dev);
+  if (st != DP_OK) return st;
+  void* p = g_static_scratch_ptr[dev].load(std::memory_order_acquire);
+  if (p == nullptr) {
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
     DP_CUDA_OK(cudaGetSymbolAddress(&p, g_static_scratch));
     if (p == nullptr || (reinterpret_cast<uintptr_t>(p) & 255u))
       return fail(DP_ERR_CUDA, "static scratch has no usable device address on device %d", dev);
-    g_static_scratch_ptr[dev] = p;
+    g_static_scratch_ptr[dev].store(p, std::memory_order_release);
   }
-  *out = g_static_scratch_ptr[dev];
+  *out = p;
   return DP_OK;
 }
 
@@ -905,6 +951,13 @@ extern "C" int dp_pack_weights_host(const int8_t* w, int32_t N, int32_t K, int32
     }
   }
   return DP_OK;
+}
+
+extern "C" void dp_debug_skip_stage_load(int32_t k_block) { dp::gemm_debug_skip_stage_load(k_block); }
+
+extern "C" int32_t dp_clip_rank(int32_t clip_percentile_e3, int32_t K) {
+  if (clip_percentile_e3 < 1 || clip_percentile_e3 > 100000 || K < 1) return 0;
+  return dp::clip_rank_of(clip_percentile_e3, K);
 }
 
 extern "C" const char* dp_status_string(int s) {

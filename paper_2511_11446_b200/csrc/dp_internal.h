@@ -125,12 +125,16 @@ int gemm_encode_a_tiled(CUtensorMap* out, const int8_t* q, int64_t M, int64_t K)
 int gemm_encode_w(CUtensorMap* out, const void* qweight, int32_t N, int32_t K, int32_t bits,
                   int32_t bn, int32_t cg);
 int launch_gemm(const GemmProblem& p, cudaStream_t stream, bool pdl);
+void gemm_debug_skip_stage_load(int32_t kb);  // see dp_debug_skip_stage_load
 
 // gemm_ws.cu -- weight-stationary CTA-pair kernel (K <= 1152, N a multiple of 192 or 256).
 bool gemm_ws_supported(int32_t N, int32_t K);
 int gemm_ws_pick_bn(int32_t N);
 int launch_gemm_ws(const GemmProblem& p, cudaStream_t stream, bool pdl);
-int gemm_init();  // sets kernel attributes, resolves the tensor-map encoder; idempotent
+// Per-device set-up (kernel attributes, tensor-map encoder, SM and CTA-pair counts), called once per
+// device by check_device() with that device current.
+int gemm_init_device(int dev, int* num_sms_out, int* max_pairs_out);
+int gemm_ws_init_device();
 
 int num_sms();
 

@@ -57,6 +57,7 @@ struct GemmParams {
   int32_t a_tiled;  // activations are stored as contiguous 128 x 128 tiles
   int32_t early_w;  // weights may be fetched before the preceding kernel on the stream has finished
   int32_t* status;
+  int32_t dbg_skip_kb = -1;  // test hook (dp_debug_skip_stage_load): k-block whose loads are left out, or -1
 };
 
 // TMA coordinates of the activation tile (token row m_row, a multiple of 128; k block kb).

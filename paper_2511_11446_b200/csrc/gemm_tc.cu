@@ -138,6 +138,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int w_row = n_blk * BN + static_cast<int>(rank) * BNL;
         bool a_ready = p.x == nullptr || (m_row >> 7) == ready_tile;
         for (int kb = 0; kb < KB; ++kb) {
+          if constexpr (CG == 1 && BITS == 8) {
+            // test hook: this stage gets no loads and no arrival, so its barrier never completes and
+            // the bounded waits of the other roles run out
+            if (kb == p.dbg_skip_kb && tile == first_tile) {
+              st.next(NS);
+              continue;
+            }
+          }
           if (!a_open && deferred == NS) {  // ring full of weight tiles: now wait for the activations
             pdl_wait();
             a_open = true;
@@ -320,9 +328,7 @@ using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, voi
                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                               CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                               CUtensorMapFloatOOBfill);
-static EncodeFn g_encode = nullptr;
-static int g_num_sms = 0;
-static int g_max_pairs = 0;  // CTA pairs of the widest pair kernel that can be resident at once
+static EncodeFn g_encode = nullptr;  // the driver's tensor-map encoder (one per process)
 
 template <int BN, int BITS, bool PERM, int CG>
 static cudaError_t set_attr() {
@@ -330,22 +336,22 @@ static cudaError_t set_attr() {
                               static_cast<int>(gemm_smem_bytes<BN, BITS, CG>()));
 }
 
-int num_sms() { return g_num_sms; }
-
 int gemm_korder(int32_t bits) { return bits == 4 ? KORDER_EVEN_ODD : KORDER_NATURAL; }
 
-int gemm_init() {
-  static int state = -1;  // -1 not tried, else status
-  if (state >= 0) return state;
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-  if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess)
-    return fail(DP_ERR_CUDA, "cuTensorMapEncodeTiled not available: %s", cudaGetErrorString(e));
-  g_encode = reinterpret_cast<EncodeFn>(fn);
-  int dev = 0;
-  DP_CUDA_OK(cudaGetDevice(&dev));
-  DP_CUDA_OK(cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev));
+// First use of device `dev` (current; called under the library's device lock): the kernels'
+// shared-memory attributes, the SM count and how many CTA pairs of the widest pair kernel can be
+// resident at once.
+int gemm_init_device(int dev, int* num_sms_out, int* max_pairs_out) {
+  if (g_encode == nullptr) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess)
+      return fail(DP_ERR_CUDA, "cuTensorMapEncodeTiled not available: %s", cudaGetErrorString(e));
+    g_encode = reinterpret_cast<EncodeFn>(fn);
+  }
+  int sms = 0;
+  DP_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
 #define DP_SET(BN, CG)                               \
   DP_CUDA_OK((set_attr<BN, 8, false, CG>()));        \
   DP_CUDA_OK((set_attr<BN, 4, false, CG>()));        \
@@ -354,9 +360,10 @@ int gemm_init() {
   DP_SET(64, 1) DP_SET(128, 1) DP_SET(192, 1) DP_SET(256, 1)
   DP_SET(128, 2) DP_SET(192, 2) DP_SET(256, 2)
 #undef DP_SET
+  int pairs = 0;
   {  // how many CTA pairs fit on the device at once (one CTA per SM)
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(g_num_sms & ~1));
+    cfg.gridDim = dim3(static_cast<unsigned>(sms & ~1));
     cfg.blockDim = dim3(gemm_threads(4));
     cfg.dynamicSmemBytes = gemm_smem_bytes<256, 4, 2>();
     cudaLaunchAttribute attr[1];
@@ -366,16 +373,15 @@ int gemm_init() {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, gemm_i8_kernel<256, 4, true, 2>, &cfg);
+    cudaError_t e = cudaOccupancyMaxActiveClusters(&pairs, gemm_i8_kernel<256, 4, true, 2>, &cfg);
     if (e != cudaSuccess) return fail(DP_ERR_CUDA, "cudaOccupancyMaxActiveClusters: %s", cudaGetErrorString(e));
-    g_max_pairs = n;
   }
-  state = DP_OK;
-  return state;
+  int st = gemm_ws_init_device();
+  if (st != DP_OK) return st;
+  *num_sms_out = sms;
+  *max_pairs_out = pairs;
+  return DP_OK;
 }
-
-int gemm_max_pairs() { return g_max_pairs; }
 
 static int encode_2d(CUtensorMap* out, const void* base, uint64_t inner_bytes, uint64_t rows,
                      uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows, bool swizzle128) {
@@ -412,8 +418,8 @@ int gemm_encode_w(CUtensorMap* out, const void* qweight, int32_t N, int32_t K, i
 void gemm_pick_tile(int64_t M, int32_t N, int32_t K, int32_t bits, uint32_t allow, int* bn_out, int* cg_out) {
   (void)K;
   (void)bits;
-  const int sms = g_num_sms > 0 ? g_num_sms : 148;
-  const int pairs = g_max_pairs > 0 ? g_max_pairs : sms / 2;
+  const int sms = num_sms() > 0 ? num_sms() : 148;
+  const int pairs = gemm_max_pairs() > 0 ? gemm_max_pairs() : sms / 2;
   const int cand[4] = {256, 192, 128, 64};
   int best_bn = 0, best_cg = 1;
   double best_cost = 1e30;
@@ -457,10 +463,18 @@ static cudaError_t launch_bn(const GemmProblem& g, const GemmParams& p, dim3 gri
   }
 }
 
+// dp_debug_skip_stage_load: consumed by the calling thread's next single-CTA 8-bit launch.
+static thread_local int32_t g_skip_kb = -1;
+void gemm_debug_skip_stage_load(int32_t kb) { g_skip_kb = kb < 0 ? -1 : kb; }
+
 int launch_gemm(const GemmProblem& g, cudaStream_t stream, bool pdl) {
   if (g.M == 0) return DP_OK;
   const int cg = g.cg == 2 ? 2 : 1;
   GemmParams p;
+  if (cg == 1 && g.bits == 8) {
+    p.dbg_skip_kb = g_skip_kb;
+    g_skip_kb = -1;
+  }
   p.s_a = g.s_a;
   p.s_w = g.s_w;
   p.bias = g.bias;
@@ -483,7 +497,7 @@ int launch_gemm(const GemmProblem& g, cudaStream_t stream, bool pdl) {
   p.early_w = (pdl && g.early_w) ? 1 : 0;
   p.status = g.status;
   const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
-  const int64_t slots = cg == 2 ? (g_max_pairs > 0 ? g_max_pairs : g_num_sms / 2) : g_num_sms;
+  const int64_t slots = cg == 2 ? (gemm_max_pairs() > 0 ? gemm_max_pairs() : num_sms() / 2) : num_sms();
   const dim3 grid(static_cast<unsigned>((tiles < slots ? tiles : slots) * cg));
   cudaError_t e;
   if (cg == 2) {

@@ -288,9 +288,7 @@ static cudaError_t ws_set_attr() {
                               static_cast<int>(ws_smem_bytes<BN>()));
 }
 
-int gemm_ws_init() {
-  static int state = -1;
-  if (state >= 0) return state;
+int gemm_ws_init_device() {  // per device, from gemm_init_device
 #define DP_SET(BN)                                \
   DP_CUDA_OK((ws_set_attr<BN, 8, false>()));      \
   DP_CUDA_OK((ws_set_attr<BN, 4, false>()));      \
@@ -298,8 +296,7 @@ int gemm_ws_init() {
   DP_CUDA_OK((ws_set_attr<BN, 3, false>()));
   DP_SET(192) DP_SET(256)
 #undef DP_SET
-  state = DP_OK;
-  return state;
+  return DP_OK;
 }
 
 bool gemm_ws_supported(int32_t N, int32_t K) { return K <= kWsMaxKB * BK && (N % 256 == 0 || N % 192 == 0); }
@@ -331,8 +328,6 @@ int launch_gemm_ws(const GemmProblem& g, cudaStream_t stream, bool pdl) {
   if (g.M == 0) return DP_OK;
   if (!gemm_ws_supported(g.N, g.K) || g.N % g.bn)
     return fail(DP_ERR_SHAPE, "weight-stationary kernel: unsupported N=%d K=%d bn=%d", g.N, g.K, g.bn);
-  int st = gemm_ws_init();
-  if (st != DP_OK) return st;
   GemmParams p;
   p.s_a = g.s_a;
   p.s_w = g.s_w;

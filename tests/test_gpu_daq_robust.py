@@ -49,7 +49,7 @@ def test_matches_oracle(M, K, rank, bits):
 def test_percentile_of_the_paper_on_the_benchmark_shapes():
     """p = 99.9: rank 2 at K = 1152, rank 5 at K = 4608 (outlier channels x20 make the clip bite)."""
     for K in (1152, 4608):
-        rank = B.clip_rank("99.9", K)
+        rank = B.dp_clip_rank(99900, K)
         assert rank == oracle.clip_rank("99.9", K) == (2 if K == 1152 else 5)
         x = synth.activations(synth.BASE_SEED, 1, 3, 512, K, 1.0, n_out=K // 100)
         got = _run(x, rank, 8)
@@ -79,7 +79,7 @@ def test_pipeline_with_the_linear_matches_the_oracle_composition():
         x = synth.activations(synth.BASE_SEED, 6, 4, M, K, 1.0, n_out=11)
         w, s_w = synth.weights(synth.BASE_SEED, 6, N, K, wbits)
         b = synth.bias(synth.BASE_SEED, 6, N)
-        rank = B.clip_rank("99.9", K)
+        rank = B.dp_clip_rank(99900, K)
         oq, osa, _ = oracle.daq_robust(x, rank, 6)
         ref = oracle.epilogue(oracle.gemm_i32(oq, w), osa, s_w, b)
         L = DevLayer(w, s_w, b, wbits)

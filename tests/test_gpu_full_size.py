@@ -1,10 +1,16 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py times.
 
-The oracle cannot redo a whole 45 TOP plan run, but DAQ and the linear are row-wise: for sampled
-token rows it recomputes complete output rows one by one (all N channels) from inputs regenerated
-on the host from the seed, and those must match what the GPU path wrote. Same tolerance as the
-small cases: bf16 outputs within 1 ulp (the fp32 sequences are identical, so almost all are equal).
+The oracle cannot redo a whole 45 TOP plan run element by element, but DAQ and the linear are
+row-wise, so it can redo (i) the quantization of every call in full (O(MK)), (ii) complete output
+rows of sampled tokens -- one from every 128-token tile, so that every row tile and both halves of
+every 256-token CTA-pair tile, and with them every column tile, is visited -- and (iii) seeded
+(m, n) points one by one. Inputs are regenerated from the seed (the CUDA generator is bit-identical
+to the numpy one; sampled rows are re-checked against numpy here). Same tolerance as the small
+cases: int8 codes and fp32 scales bit-exact, bf16 outputs within 1 ulp (the fp32 sequences are
+identical, so almost all are equal).
 """
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import pytest
 import torch
@@ -18,47 +24,91 @@ from helpers import bf16_ulp_dist
 pytestmark = pytest.mark.gpu
 
 
-def _sample_rows(M, rng, n=6):
-    """Rows from the first, last and interior 128-token tiles (ragged ends included)."""
-    fixed = {0, M - 1, min(M - 1, 127), min(M - 1, 128), M // 2}
-    while len(fixed) < min(M, n + 4):
-        fixed.add(int(rng.integers(0, M)))
-    return sorted(fixed)
+def _tile_rows(M, rng, extra=4):
+    """One token from every 128-token tile (ragged last tile included), the first and the last token,
+    and a few more."""
+    rows = {0, M - 1}
+    for t0 in range(0, M, 128):
+        rows.add(int(rng.integers(t0, min(M, t0 + 128))))
+    for _ in range(extra):
+        rows.add(int(rng.integers(0, M)))
+    return sorted(rows)
 
 
-def _check_rows(y_dev, x_rows, rows, seed, layer, N, K, bits, what):
+def _host_layer(seed, layer, N, K, bits):
+    """Host copy of a layer's constants: integer weights from the numpy generator, packed and
+    unpacked again by the oracle's codec."""
     w, s_w = synth.weights(seed, layer, N, K, bits)
-    b = synth.bias(seed, layer, N)
-    ref = oracle.wq_linear(x_rows, oracle.pack(w, bits), s_w, b, bits)
-    got = bf16_to_np(y_dev[torch.tensor(rows, device="cuda")])
+    packed = oracle.pack(w, bits)
+    return dict(packed=packed, w=oracle.unpack(packed, K, bits), s_w=s_w, bias=synth.bias(seed, layer, N), bits=bits)
+
+
+def _assert_close(got, ref, what):
     d = bf16_ulp_dist(got, ref)
     assert d.max() <= 1, (what, int(d.max()))
     assert (d != 0).mean() < 1e-3, what
 
 
-def test_c4_plan_run_as_benchmarked_sampled_rows():
-    """The benchmark's plan (140 layers, M = 2048 / adaLN M = 8, mixed {3,4,8} bits, autotuned variants,
-    grouped adaLN launch), one retained timestep: sampled rows of layers covering every shape and
-    bit-width, and every adaLN layer of the first blocks."""
+def _check_rows(y_dev, x_rows, rows, H, what):
+    """Complete output rows of the sampled tokens against the oracle's layer."""
+    ref = oracle.wq_linear(np.ascontiguousarray(x_rows), H["packed"], H["s_w"], H["bias"], H["bits"])
+    got = bf16_to_np(y_dev[torch.tensor(rows, device="cuda")])
+    _assert_close(got, ref, what)
+
+
+def test_c4_plan_run_every_retained_step_every_call():
+    """The benchmark's plan (140 layers, M = 2048 / adaLN M = 8, mixed {3,4,8} bits, autotuned
+    variants, grouped adaLN launch) over ALL 25 retained timesteps (sigma(t) and the outlier set
+    drift with t). For every one of the 3500 calls: the int8 codes and scales of the whole input
+    (dp_daq_quantize on the same buffer against the oracle's DAQ); one complete output row from every
+    128-token tile; 4096 seeded (m, n) points recomputed one by one."""
     stack = DitStack(resident_steps=1)  # bench.py's defaults: DP_FLAG_AUTOTUNE | DP_FLAG_GROUP_SMALL_M
-    stack.run(1)
-    torch.cuda.synchronize()
-    assert int(stack.status.item()) == 0
-    t = stack.kept[0]
+    nL = len(stack.table)
+    with ThreadPoolExecutor(8) as ex:
+        host = list(ex.map(lambda l: _host_layer(stack.seed, l, stack.table[l][3], stack.table[l][2], stack.bits[l]),
+                           range(nL)))
+    for l in range(nL):  # the device weights are the same bytes (generator and host packer at full size)
+        dev = stack.layers[l].qweight.cpu().numpy().view(np.uint8).reshape(-1)
+        assert np.array_equal(dev, host[l]["packed"].view(np.uint8).reshape(-1)), l
     rng = np.random.default_rng(7)
-    seen, chosen = set(), []
-    for l, (name, M, K, N) in enumerate(stack.table):
-        key = (name, stack.bits[l], B.dp_plan_layer_variant(stack.plan, l)["unpack_first"])
-        if key not in seen or (M <= 32 and l < 15):
-            seen.add(key)
-            chosen.append(l)
-    assert len(chosen) >= 15
-    for l in chosen:
-        name, M, K, N = stack.table[l]
-        rows = _sample_rows(M, rng)
-        x_rows = stack.host_input_rows(l, t, rows)
-        _check_rows(stack.y[l], x_rows, rows, stack.seed, l, N, K, stack.bits[l],
-                    (l, name, stack.bits[l], B.dp_plan_layer_variant(stack.plan, l)))
+    xp, yp = stack.ptrs(1)
+    calls = 0
+    for t in stack.kept:
+        for l in range(nL):
+            stack.gen_input(l, t, out=stack.x[0][l])
+        for y in stack.y:
+            y.fill_(float("nan"))
+        B.dp_plan_run(stack.plan, [t], 0, xp, yp, stack.workspace, stack.status, flags=B.DP_PLAN_SAME_Y)
+        torch.cuda.synchronize()
+        assert int(stack.status.item()) == 0
+        for l, (name, M, K, N) in enumerate(stack.table):
+            H = host[l]
+            what = (t, l, name, stack.bits[l], B.dp_plan_layer_variant(stack.plan, l))
+            x_host = bf16_to_np(stack.x[0][l])
+            probe = sorted({0, M - 1, int(rng.integers(0, M))})
+            assert np.array_equal(x_host[probe], stack.host_input_rows(l, t, probe)), what
+            # a1-a3 in full
+            q_ref, sa_ref, _ = oracle.daq(x_host)
+            q = torch.empty((M, K), dtype=torch.int8, device="cuda")
+            s_a = torch.empty(M, dtype=torch.float32, device="cuda")
+            B.dp_daq_quantize(stack.x[0][l], M, K, K, q, K, s_a)
+            assert np.array_equal(q.cpu().numpy(), q_ref), what
+            assert np.array_equal(s_a.cpu().numpy().view(np.uint32), sa_ref.view(np.uint32)), what
+            # a4-a6: complete rows, one per 128-token tile
+            rows = _tile_rows(M, rng, extra=2)
+            acc = oracle.gemm_i32(np.ascontiguousarray(q_ref[rows]), H["w"])
+            ref = oracle.epilogue(acc, np.ascontiguousarray(sa_ref[rows]), H["s_w"], H["bias"])
+            ydev = stack.y[l]
+            _assert_close(bf16_to_np(ydev[torch.tensor(rows, device="cuda")]), ref, what)
+            # seeded points, each from the packed weights and the bf16 input
+            pm, pn = rng.integers(0, M, 4096), rng.integers(0, N, 4096)
+            _, py = oracle.wq_linear_points(x_host, H["packed"], H["s_w"], H["bias"], H["bits"], pm, pn)
+            got = bf16_to_np(ydev[torch.from_numpy(pm).cuda(), torch.from_numpy(pn).cuda()])
+            _assert_close(got, py, what)
+            calls += 1
+        assert not any(torch.isnan(y.float()).any().item() for y in stack.y), t
+    assert calls == 25 * 140
+    stack.close()
 
 
 def _run_layer(W, x_bits_or_dev, M, K, N, bits, flags=0):
@@ -77,7 +127,7 @@ def test_c1_single_proj_linear_whole_output():
     seed, layer, M, K, N, bits = synth.BASE_SEED + 1, 0, 256, 1152, 1152, 8
     x = synth.activations(seed, layer, 0, M, K, 1.0, n_out=8)
     y = _run_layer(DevWeights(seed, layer, N, K, bits), x, M, K, N, bits)
-    _check_rows(y, x, list(range(M)), seed, layer, N, K, bits, "c1")
+    _check_rows(y, x, list(range(M)), _host_layer(seed, layer, N, K, bits), "c1")
 
 
 def test_c2_fc1_4bit_whole_output():
@@ -85,31 +135,39 @@ def test_c2_fc1_4bit_whole_output():
     seed, layer, M, K, N, bits = synth.BASE_SEED + 2, 0, 2048, 1152, 4608, 4
     x = synth.activations(seed, layer, 0, M, K, 1.0, n_out=K // 100)
     y = _run_layer(DevWeights(seed, layer, N, K, bits), x, M, K, N, bits)
-    _check_rows(y, x, list(range(M)), seed, layer, N, K, bits, "c2")
+    _check_rows(y, x, list(range(M)), _host_layer(seed, layer, N, K, bits), "c2")
 
 
-def test_c3_block_at_m4096_with_gelu_input_sampled_rows():
-    """One block's linears at M = 4096 (adaLN M = 16), bits from {4, 8}; fc2 reads GELU(N(0,1)):
-    non-negative, heavy-tailed, the case where absmax scaling wastes half the code range."""
+@pytest.mark.parametrize("bits", [4, 8])
+def test_c3_block_at_m4096_with_gelu_input(bits):
+    """One block's linears at M = 4096 (adaLN M = 16), every shape at both widths the config's plan
+    draws from ({4, 8}); fc2 reads GELU(N(0,1)): non-negative, heavy-tailed, the case where absmax
+    scaling wastes half the code range. One complete output row from every 128-token tile."""
     seed = synth.BASE_SEED + 3
     table = [("qkv", 4096, 1152, 3456), ("proj", 4096, 1152, 1152), ("fc1", 4096, 1152, 4608),
              ("fc2", 4096, 4608, 1152), ("adaln", 16, 1152, 6912)]
-    bits = synth.bit_plan(seed, len(table), (4, 8))
-    rng = np.random.default_rng(3)
+    drawn = synth.bit_plan(seed, len(table), (4, 8))
+    assert set(drawn) <= {4, 8}
+    rng = np.random.default_rng(3 + bits)
     for l, (name, M, K, N) in enumerate(table):
         x = (synth.gelu_activations(seed, l, 0, M, K) if name == "fc2"
              else synth.activations(seed, l, 0, M, K, 1.0, n_out=K // 100))
-        y = _run_layer(DevWeights(seed, l, N, K, bits[l]), x, M, K, N, bits[l])
-        rows = _sample_rows(M, rng, n=12)
-        _check_rows(y, x[rows], rows, seed, l, N, K, bits[l], ("c3", name, bits[l]))
+        y = _run_layer(DevWeights(seed, l, N, K, bits), x, M, K, N, bits)
+        rows = _tile_rows(M, rng, extra=8)
+        _check_rows(y, x[rows], rows, _host_layer(seed, l, N, K, bits), ("c3", name, bits, "drawn", drawn[l]))
+        assert not torch.isnan(y.float()).any()
 
 
-@pytest.mark.parametrize("name,K,N,M,bits", [("qkv", 1152, 3456, 32768, 4), ("proj", 1152, 1152, 32768, 3),
-                                             ("fc1", 1152, 4608, 32768, 8), ("fc2", 4608, 1152, 32768, 4),
-                                             ("fc2", 4608, 1152, 32768, 3), ("adaln", 1152, 6912, 32, 3),
-                                             ("adaln", 1152, 6912, 32, 8)])
-def test_c5_large_m_layers_sampled_rows(name, K, N, M, bits):
-    """M = 32768 (batch 32 at 512 px; adaLN M = 32), default dispatch of dp_wq_linear."""
+C5_SHAPES = [("qkv", 1152, 3456, 32768), ("proj", 1152, 1152, 32768), ("fc1", 1152, 4608, 32768),
+             ("fc2", 4608, 1152, 32768), ("adaln", 1152, 6912, 32)]
+
+
+@pytest.mark.parametrize("bits", [3, 4, 8])
+@pytest.mark.parametrize("name,K,N,M", C5_SHAPES)
+def test_c5_large_m_layers_every_row_tile(name, K, N, M, bits):
+    """M = 32768 (batch 32 at 512 px; adaLN M = 32), all five shapes at all three widths, default
+    dispatch of dp_wq_linear (persistent, multi-wave schedules): one complete output row from every
+    one of the 256 128-token tiles (both halves of every 256-token CTA-pair tile), every column."""
     seed, layer = synth.BASE_SEED + 5, 3
     n_out = max(1, K // 100)
     W = DevWeights(seed, layer, N, K, bits)
@@ -120,8 +178,10 @@ def test_c5_large_m_layers_sampled_rows(name, K, N, M, bits):
     B.dp_wq_linear(W.w, x, K, None, M, y, N, ws, None, status, 0)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    rows = _sample_rows(M, np.random.default_rng(M + N + bits), n=10)
+    rows = _tile_rows(M, np.random.default_rng(M + N + bits), extra=6)
+    assert len(rows) >= (M + 127) // 128
     x_rows = synth.activations(seed, layer, 0, M, K, 1.0, n_out=n_out, rows=rows)
-    _check_rows(y, x_rows, rows, seed, layer, N, K, bits, (name, M, bits))
+    assert np.array_equal(bf16_to_np(x[torch.tensor(rows, device="cuda")]), x_rows)
+    _check_rows(y, x_rows, rows, _host_layer(seed, layer, N, K, bits), (name, M, bits))
     # every row was written (no NaN sentinel left) -- a property that holds at any size
     assert not torch.isnan(y.float()).any()

@@ -3,7 +3,8 @@
 Such callers (a custom-op slot of a runtime that owns all device memory, code running during a
 stream capture, a loop that cannot afford an allocation's device stall) get the scratch from a
 fixed array inside the library instead of a `workspace` argument. The result must be the one
-dp_wq_linear gives with a caller-provided workspace. Calls in a row on different problems check
+dp_wq_linear gives with a caller-provided workspace, and both must be the CPU oracle's layer (so the
+check does not rest on the library agreeing with itself). Calls in a row on different problems check
 that the shared array, which keeps the previous call's contents, is fully re-initialised by each
 call. This file is collected last so a failure here cannot mask any other test.
 """
@@ -11,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2511_11446_b200 import binding as B, synth
 from gpu_util import DevLayer, to_dev_bf16, bf16_to_np
 from helpers import bf16_ulp_dist
@@ -33,17 +35,20 @@ def _both(M, K, N, bits, layer):
     B.dp_wq_linear_static(L.w, xd, K, M, y_new, N, status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    return bf16_to_np(y_new), bf16_to_np(y_ref)
+    y_orc = oracle.wq_linear(x, oracle.pack(w, bits), s_w, b, bits)
+    return bf16_to_np(y_new), bf16_to_np(y_ref), y_orc
 
 
 def test_static_scratch_matches_workspace_variant_on_calls_in_a_row():
     # first call: a larger problem fills much of the array; the following, smaller ones with other
     # widths must not see anything of it
     for (M, K, N, bits, layer) in [(1000, 1152, 384, 4, 0), (300, 256, 128, 8, 1), (16, 1152, 96, 3, 2)]:
-        got, ref = _both(M, K, N, bits, layer)
+        got, ref, orc = _both(M, K, N, bits, layer)
         assert not np.any(got == 0x7FC0), "output not fully written"
         assert bf16_ulp_dist(got, ref).max() <= 1
         assert np.array_equal(got, ref)
+        d = bf16_ulp_dist(got, orc)       # the oracle's layer: within 1 bf16 ulp, almost all equal
+        assert d.max() <= 1 and (d != 0).mean() < 1e-3
 
 
 def test_static_scratch_rejects_oversized_problems():
