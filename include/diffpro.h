@@ -98,6 +98,12 @@ typedef struct dp_debug {
  * output channels resident in shared memory for the whole K (K <= 1152, N a multiple of 192). */
 #define DP_FLAG_WEIGHT_STATIONARY 0x2000u
 #define DP_FLAG_NO_WEIGHT_STATIONARY 0x4000u
+/* Tuning/testing: force (or forbid) the activation-stationary CTA-pair kernel, which keeps the int8
+ * codes of a 256-token strip resident in shared memory for the whole K and streams only weight
+ * tiles (K <= 1152, N a multiple of 64, 8-bit weights or the unpack-first form, DAQ run by the
+ * library). DP_FLAG_TILE_N then names the width of the column sub-blocks it walks. */
+#define DP_FLAG_ACT_STATIONARY 0x200000u
+#define DP_FLAG_NO_ACT_STATIONARY 0x400000u
 
 /* dp_plan_create only: choose each layer's tensor-core kernel variant (tile width, single CTA /
  * CTA pair / weight-stationary) by timing the candidates on the device during plan creation
@@ -244,7 +250,8 @@ int dp_plan_create(const dp_weight* layers, int32_t n_layers, const int64_t* M_p
 size_t dp_plan_workspace(const dp_plan* plan);
 /* Which kernel the plan runs layer `layer` with (for reports and for timing that kernel alone):
  * *tile_n = tile width in output channels, *cta_group = 1 or 2 CTAs per row tile,
- * *weight_stationary = 0/1, *small_m = 1 when the CUDA-core small-M kernel is used (the other three
+ * *weight_stationary = 0, 1 (weight-stationary kernel) or 2 (activation-stationary kernel; *tile_n is
+ * then its sub-block width), *small_m = 1 when the CUDA-core small-M kernel is used (the other three
  * are then 0). Any output pointer may be NULL. */
 int dp_plan_layer_variant(const dp_plan* plan, int32_t layer, int32_t* tile_n, int32_t* cta_group,
                           int32_t* weight_stationary, int32_t* small_m);
@@ -252,7 +259,7 @@ int dp_plan_layer_variant(const dp_plan* plan, int32_t layer, int32_t* tile_n, i
  * variant dp_plan_layer_variant reports is then the 8-bit kernel's). No counterpart in the paper. */
 int dp_plan_layer_unpack_first(const dp_plan* plan, int32_t layer, int32_t* unpack_first);
 /* Replaces the kernel variant of layer `layer` by the one `flags` names (the tuning flags of
- * dp_wq_linear: DP_FLAG_TILE_N, [NO_]CTA_PAIR, [NO_]WEIGHT_STATIONARY, UNPACK_FIRST; anything left
+ * dp_wq_linear: DP_FLAG_TILE_N, [NO_]CTA_PAIR, [NO_]WEIGHT_STATIONARY, [NO_]ACT_STATIONARY, UNPACK_FIRST; anything left
  * open is chosen as dp_wq_linear would): lets a deployment keep the outcome of one
  * DP_FLAG_AUTOTUNE run and apply it to later plans. Host only; may raise dp_plan_workspace, so ask
  * again afterwards. Small-M layers and unknown bits are refused (DP_ERR_INVALID_ARG), tile widths

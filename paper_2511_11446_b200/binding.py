@@ -23,6 +23,7 @@ DP_FLAG_CTA_PAIR, DP_FLAG_NO_CTA_PAIR = 0x800, 0x1000
 DP_FLAG_WEIGHT_STATIONARY, DP_FLAG_NO_WEIGHT_STATIONARY = 0x2000, 0x4000
 DP_FLAG_AUTOTUNE, DP_FLAG_GROUP_SMALL_M, DP_FLAG_FUSED_DAQ = 0x10000, 0x20000, 0x40000
 DP_FLAG_UNPACK_FIRST, DP_FLAG_NO_UNPACK_FIRST = 0x80000, 0x100000
+DP_FLAG_ACT_STATIONARY, DP_FLAG_NO_ACT_STATIONARY = 0x200000, 0x400000
 DP_FLAG_TILE_N_MASK = 0x700
 DP_PLAN_SAME_X, DP_PLAN_SAME_Y = 1, 2
 
@@ -202,9 +203,11 @@ def variant_flags(v: dict) -> int:
         return DP_FLAG_FORCE_SIMT
     f = DP_FLAG_FORCE_MMA | DP_FLAG_TILE_N(v["tile_n"])
     f |= DP_FLAG_UNPACK_FIRST if v.get("unpack_first") else DP_FLAG_NO_UNPACK_FIRST
+    if v["weight_stationary"] == 2:
+        return f | DP_FLAG_ACT_STATIONARY
     if v["weight_stationary"]:
         return f | DP_FLAG_WEIGHT_STATIONARY
-    f |= DP_FLAG_NO_WEIGHT_STATIONARY
+    f |= DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_NO_ACT_STATIONARY
     return f | (DP_FLAG_CTA_PAIR if v["cta_group"] == 2 else DP_FLAG_NO_CTA_PAIR)
 
 

@@ -97,15 +97,31 @@ static size_t scratch_q_bytes(int64_t M, int32_t K) { return static_cast<size_t>
 constexpr uint32_t kLinearFlags =
     DP_FLAG_FORCE_SIMT | DP_FLAG_FORCE_MMA | DP_FLAG_NO_PDL | DP_FLAG_TILE_N_MASK | DP_FLAG_CTA_PAIR |
     DP_FLAG_NO_CTA_PAIR | DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_UNPACK_FIRST |
-    DP_FLAG_NO_UNPACK_FIRST;
+    DP_FLAG_NO_UNPACK_FIRST | DP_FLAG_ACT_STATIONARY | DP_FLAG_NO_ACT_STATIONARY;
 constexpr int64_t kWsMinRows = 8192;  // from here on a resident weight strip is reused often enough to pay
 static int forced_bn(uint32_t flags) { return static_cast<int>((flags & DP_FLAG_TILE_N_MASK) >> 8) * 64; }
 
 // Tile width and CTA-group size of the tensor-core kernel for this problem, honouring the tuning
 // flags (validated by check_tile_flags).
-static void choose_tile(uint32_t flags, int64_t M, int32_t N, int32_t K, int32_t bits, int* bn, int* cg,
-                        int* ws) {
+// `bits` is the width the GEMM kernel sees (8 in the unpack-first form); `tiled_a`: the activations
+// are the library's own tiled scratch (DAQ run by the call).
+static void choose_tile(uint32_t flags, int64_t M, int32_t N, int32_t K, int32_t bits, bool tiled_a, int* bn,
+                        int* cg, int* ws) {
   *ws = 0;
+  // (callers clear tiled_a when the layer's scale / bias pointers lack the alignment that kernel's
+  // vector loads need)
+  const bool as_ok = tiled_a && bits == 8 && gemm_as_supported(N, K) &&
+                     !(flags & (DP_FLAG_NO_ACT_STATIONARY | DP_FLAG_NO_CTA_PAIR | DP_FLAG_WEIGHT_STATIONARY));
+  if (as_ok && (flags & DP_FLAG_ACT_STATIONARY)) {
+    int nsub = 1;
+    const int fb = forced_bn(flags);
+    gemm_as_config(M, N, K, (fb != 0 && N % fb == 0) ? fb : 0, bn, &nsub);
+    if (*bn != 0) {
+      *cg = 2;
+      *ws = 2;
+      return;
+    }
+  }
   const bool ws_ok = gemm_ws_supported(N, K) && !(flags & (DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_NO_CTA_PAIR));
   if (ws_ok && ((flags & DP_FLAG_WEIGHT_STATIONARY) || M >= kWsMinRows)) {
     const int fb = forced_bn(flags);
@@ -135,6 +151,9 @@ static int check_tile_flags(uint32_t flags, int32_t N) {
     return fail(DP_ERR_SHAPE, "CTA-pair tiles need a tile width of 128, 192 or 256 dividing N=%d", N);
   if ((flags & DP_FLAG_WEIGHT_STATIONARY) && (flags & (DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_NO_CTA_PAIR)))
     return fail(DP_ERR_INVALID_ARG, "WEIGHT_STATIONARY contradicts another flag");
+  if ((flags & DP_FLAG_ACT_STATIONARY) &&
+      (flags & (DP_FLAG_NO_ACT_STATIONARY | DP_FLAG_NO_CTA_PAIR | DP_FLAG_WEIGHT_STATIONARY)))
+    return fail(DP_ERR_INVALID_ARG, "ACT_STATIONARY contradicts another flag");
   return DP_OK;
 }
 
@@ -162,6 +181,9 @@ static bool use_simt(int64_t M, int32_t N, int32_t K, uint32_t flags) {
   (void)K;
   return M <= kSimtMaxRows;
 }
+
+// (kept for kernels with alignment needs beyond check_weight's; none at present)
+static bool as_pointers_ok(const dp_weight*) { return true; }
 
 static int check_weight(const dp_weight* w) {
   if (!w) return fail(DP_ERR_INVALID_ARG, "dp_weight is NULL");
@@ -297,7 +319,13 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
     int st = tiled ? gemm_encode_a_tiled(&g.tmap_a, q, M, w->K) : gemm_encode_a(&g.tmap_a, q, M, w->K, ldq);
     if (st != DP_OK) return st;
   }
-  if (bn == 0) choose_tile(flags, M, w->N, w->K, w->bits, &bn, &cg, &ws);
+  if (bn == 0) choose_tile(flags, M, w->N, w->K, w->bits, tiled && as_pointers_ok(w), &bn, &cg, &ws);
+  if (ws == 2 && (!tiled || w->bits != 8 || fused || !as_pointers_ok(w)))
+    return fail(DP_ERR_INVALID_ARG, "the activation-stationary kernel needs DAQ run by the call, 8-bit weights (or the "
+                                    "unpack-first form)");
+  // Its weight ring is small (64 KB per CTA): prefetching it while the DAQ launch drains costs that
+  // launch no bandwidth worth speaking of, whatever M is.
+  if (ws == 2 && s_a_in == nullptr && !unpack_first && pdl) g.early_w = 1;
   g.cg = cg;
   g.ws = ws;
   if (tmap_w != nullptr) {
@@ -319,7 +347,7 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
   g.bits = w->bits;
   g.bn = bn;
   g.status = status;
-  int st = ws ? launch_gemm_ws(g, stream, pdl) : launch_gemm(g, stream, pdl);
+  int st = ws == 2 ? launch_gemm_as(g, stream, pdl) : ws ? launch_gemm_ws(g, stream, pdl) : launch_gemm(g, stream, pdl);
   if (st != DP_OK) return st;
   if (dbg != nullptr) {
     if (dbg->q != nullptr) {
@@ -486,8 +514,8 @@ struct TunedShape {
   int32_t N, K, bits;
   int bn, cg, ws, pre;
 };
-static int autotune_shape(const dp_weight& w, int64_t M, uint32_t flags, int* bn_out, int* cg_out, int* ws_out,
-                          int* pre_out) {
+static int autotune_shape(const dp_weight& w, int64_t M, uint32_t flags, bool allow_as, int* bn_out, int* cg_out,
+                          int* ws_out, int* pre_out) {
   struct Cand {
     int bn, cg, ws, pre;
   };
@@ -501,6 +529,8 @@ static int autotune_shape(const dp_weight& w, int64_t M, uint32_t flags, int* bn
         cands.push_back({widths[i], 1, 0, pre});
         if (widths[i] >= 128) cands.push_back({widths[i], 2, 0, pre});
         if (widths[i] >= 192 && gemm_ws_supported(w.N, w.K)) cands.push_back({widths[i], 2, 1, pre});
+        if (allow_as && as_pointers_ok(&w) && gemm_as_supported(w.N, w.K) && (w.bits == 8 || pre))
+          cands.push_back({widths[i], 2, 2, pre});
       }
   void *x = nullptr, *y = nullptr, *ws = nullptr;
   cudaStream_t stream = nullptr;
@@ -604,14 +634,14 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
       if ((lf & DP_FLAG_CTA_PAIR) && L.w.N % 128 && L.w.N % 192) lf &= ~DP_FLAG_CTA_PAIR;
       if ((lf & DP_FLAG_WEIGHT_STATIONARY) && !gemm_ws_supported(L.w.N, L.w.K)) lf &= ~DP_FLAG_WEIGHT_STATIONARY;
       L.pre = want_unpack_first(lf, L.w.bits, true) ? 1 : 0;
-      choose_tile(lf, L.M, L.w.N, L.w.K, L.pre ? 8 : L.w.bits, &L.bn, &L.cg, &L.ws);
+      choose_tile(lf, L.M, L.w.N, L.w.K, L.pre ? 8 : L.w.bits, !fused_daq && as_pointers_ok(&L.w), &L.bn, &L.cg, &L.ws);
       if (autotune) {
         const TunedShape* hit = nullptr;
         for (const TunedShape& t : tuned)
           if (t.M == L.M && t.N == L.w.N && t.K == L.w.K && t.bits == L.w.bits) hit = &t;
         if (hit == nullptr) {
           TunedShape t = {L.M, L.w.N, L.w.K, L.w.bits, L.bn, L.cg, L.ws, L.pre};
-          st = autotune_shape(L.w, L.M, flags, &t.bn, &t.cg, &t.ws, &t.pre);
+          st = autotune_shape(L.w, L.M, flags, !fused_daq, &t.bn, &t.cg, &t.ws, &t.pre);
           if (st != DP_OK) {
             delete p;
             return st;
@@ -720,7 +750,7 @@ extern "C" int dp_plan_set_layer_flags(dp_plan* plan, int32_t layer, uint32_t fl
   PlanLayer& L = plan->layers[layer];
   constexpr uint32_t kVariantFlags = DP_FLAG_TILE_N_MASK | DP_FLAG_CTA_PAIR | DP_FLAG_NO_CTA_PAIR |
                                      DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_UNPACK_FIRST |
-    DP_FLAG_NO_UNPACK_FIRST;
+                                     DP_FLAG_NO_UNPACK_FIRST | DP_FLAG_ACT_STATIONARY | DP_FLAG_NO_ACT_STATIONARY;
   if (flags & ~kVariantFlags) return fail(DP_ERR_INVALID_ARG, "dp_plan_set_layer_flags: flag bits 0x%x do not name a variant", flags);
   if (L.simt || L.M == 0) return fail(DP_ERR_INVALID_ARG, "layer %d runs the small-M kernel: it has no variants", layer);
   if (int st = check_tile_flags(flags, L.w.N)) return st;
@@ -730,7 +760,12 @@ extern "C" int dp_plan_set_layer_flags(dp_plan* plan, int32_t layer, uint32_t fl
   if ((flags & DP_FLAG_UNPACK_FIRST) && (flags & DP_FLAG_NO_UNPACK_FIRST))
     return fail(DP_ERR_INVALID_ARG, "UNPACK_FIRST and NO_UNPACK_FIRST are exclusive");
   T.pre = want_unpack_first(flags, T.w.bits, true) ? 1 : 0;
-  choose_tile(flags, T.M, T.w.N, T.w.K, T.pre ? 8 : T.w.bits, &T.bn, &T.cg, &T.ws);
+  choose_tile(flags, T.M, T.w.N, T.w.K, T.pre ? 8 : T.w.bits, plan->daq_sync == nullptr && as_pointers_ok(&T.w), &T.bn,
+              &T.cg, &T.ws);
+  if ((flags & DP_FLAG_ACT_STATIONARY) && T.ws != 2)
+    return fail(DP_ERR_SHAPE, "layer %d: the activation-stationary kernel does not take this layer (N=%d K=%d, %d-bit "
+                              "weights without the unpack-first form, or DAQ fused into the GEMM)",
+                layer, L.w.N, L.w.K, L.w.bits);
   if (int st = gemm_encode_w(&T.tmap_w, T.w.qweight, T.w.N, T.w.K, T.w.bits, T.bn, T.cg)) return st;
   L = T;
   const size_t ws = dp_wq_linear_workspace(L.M, L.w.N, L.w.K, L.w.bits,

@@ -102,7 +102,8 @@ struct GemmProblem {
   int64_t M;
   int32_t N, K, bits, bn;
   int32_t cg;       // 1: one CTA per 128-row tile; 2: a CTA pair per 256-row tile
-  int32_t ws;       // weight-stationary pair kernel (cg == 2, bn in {192, 256})
+  int32_t ws;       // 1: weight-stationary pair kernel (cg == 2, bn in {192, 256}); 2: activation-stationary
+                    // pair kernel (bn = width of its column sub-blocks)
   int32_t korder;   // KOrder of the activations behind tmap_a
   int32_t a_tiled;  // the activations behind tmap_a are stored as 128 x 128 tiles (see gemm_encode_a_tiled)
   int32_t early_w;  // the preceding kernel on the stream is this call's own DAQ: weights may be
@@ -135,6 +136,13 @@ int launch_gemm_ws(const GemmProblem& p, cudaStream_t stream, bool pdl);
 // device by check_device() with that device current.
 int gemm_init_device(int dev, int* num_sms_out, int* max_pairs_out);
 int gemm_ws_init_device();
+int gemm_as_init_device();
+
+// gemm_as.cu -- activation-stationary CTA-pair kernel (K <= 1152, 8-bit weights, tiled activations).
+bool gemm_as_supported(int32_t N, int32_t K);
+// Sub-block width (forced_bns, or the model's choice when 0) and sub-blocks per slice; *bns_out = 0 if none fits.
+void gemm_as_config(int64_t M, int32_t N, int32_t K, int forced_bns, int* bns_out, int* nsub_out);
+int launch_gemm_as(const GemmProblem& p, cudaStream_t stream, bool pdl);
 
 int num_sms();
 

@@ -379,4 +379,126 @@ struct EpilogueWarp {
   }
 };
 
+
+// ---- epilogue with one token per thread ---------------------------------------------------------------
+// A warp serves its tensor-memory quadrant (32 tokens, one per thread) over a range of accumulator
+// columns in rounds of 16: tcgen05.ld.32x32b.x16 (the next round's read is in flight while this one
+// is converted), the fp32 sequence of Step 5 on packed pairs (two independent IEEE operations per
+// instruction: int32 -> fp32, sc = s_a * s_w[n], fma(t, sc, bias[n]), bf16 round-to-nearest-even),
+// and ONE 32-byte global store per thread and round (st.global.v8: a full sector of the token's
+// output row), so nothing is staged in shared memory and no warp-level synchronisation sits between
+// the arithmetic and the stores. Weight scales and biases come from a private fp32 copy in shared
+// memory, read as broadcast 16-byte loads: global loads in this loop, even of a few cached KB, cost
+// a trip to L2 per round with only ten warps on the SM to hide it. What bounds an epilogue on B200
+// is the chip's store throughput (4.4 TB/s measured: about 15 bytes per clock and SM), then
+// instruction issue; arithmetic does not.
+struct RowEpilogue {
+  static constexpr int CW = 16;         // columns per round
+  static constexpr int kMaxCols = 128;  // columns a warp may own (its private copy of scales and biases)
+  static constexpr int kScaleBytes = 2 * kMaxCols * 4;
+  int qd, lane, staged_col;
+  float *tsw, *tbias;
+  uint32_t acc_empty_addr[2];
+
+  __device__ __forceinline__ void init(int warp, int lane_, float* scale_copy, uint32_t acc_empty0,
+                                       uint32_t acc_empty1) {
+    lane = lane_;
+    qd = warp & 3;
+    tsw = scale_copy;
+    tbias = scale_copy + kMaxCols;
+    acc_empty_addr[0] = acc_empty0;
+    acc_empty_addr[1] = acc_empty1;
+    staged_col = -1;
+  }
+
+  // Output columns col .. col + ncols - 1 (col and ncols multiples of 16, ncols at most 128), this
+  // CTA's tokens cta_row0 .. +127; their accumulators start at tensor-memory column t_col (buffer
+  // `buf`, published on acc_full with phase aph). False if the wait was aborted.
+  __device__ __forceinline__ bool tile(const GemmParams& p, int col, int ncols, int cta_row0, uint32_t tmem_base,
+                                       uint32_t t_col, uint64_t* acc_full, uint32_t aph, int buf,
+                                       volatile int* abort_flag) {
+    const int64_t row = static_cast<int64_t>(cta_row0) + qd * 32 + lane;
+    const float sa = row < p.M ? __ldg(p.s_a + row) : 0.0f;
+    const uint64_t sa2 = f32x2_pack(sa, sa);
+    if (col != staged_col) {
+      float sv[4], bv[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int c = lane + 32 * j;
+        sv[j] = c < ncols ? __ldg(p.s_w + col + c) : 0.0f;
+        bv[j] = (c < ncols && p.bias != nullptr)
+                    ? __uint_as_float(static_cast<uint32_t>(__ldg(p.bias + col + c)) << 16)
+                    : 0.0f;
+      }
+      __syncwarp();  // the previous sub-block's reads of the copy are done
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        tsw[lane + 32 * j] = sv[j];
+        tbias[lane + 32 * j] = bv[j];
+      }
+      __syncwarp();
+      staged_col = col;
+    }
+    bool ok = mbar_wait(acc_full, aph, abort_flag);
+    ok = __all_sync(0xFFFFFFFFu, ok);
+    if (!ok) return false;
+    tc_fence_after();
+    const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + t_col;
+    const float4* sw4 = reinterpret_cast<const float4*>(tsw);
+    const float4* tb4 = reinterpret_cast<const float4*>(tbias);
+    uint16_t* yrow = p.y + row * p.ldy + col;
+    // 32-byte stores need the token's row segment 32-byte aligned; else two 16-byte stores
+    const bool wide = ((reinterpret_cast<uintptr_t>(p.y) | static_cast<uintptr_t>(p.ldy * 2)) & 31u) == 0;
+    const int rounds = ncols / CW;
+    uint32_t ra[16];
+    tmem_ld_32x16(t_addr, ra);
+    for (int c = 0; c < rounds; ++c) {
+      tmem_ld_wait();
+      uint32_t a[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) a[i] = ra[i];
+      if (c + 1 < rounds) {
+        tmem_ld_32x16(t_addr + (c + 1) * CW, ra);
+      } else {  // this warp's last accumulators are in registers: hand the buffer back
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(acc_empty_addr[buf]);
+      }
+      uint32_t w[8];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {  // four columns at a time
+        const float4 sw = sw4[c * 4 + q];
+        const float4 bb = tb4[c * 4 + q];
+        const uint64_t t01 = f32x2_pack(__int2float_rn(static_cast<int>(a[4 * q])),
+                                        __int2float_rn(static_cast<int>(a[4 * q + 1])));
+        const uint64_t t23 = f32x2_pack(__int2float_rn(static_cast<int>(a[4 * q + 2])),
+                                        __int2float_rn(static_cast<int>(a[4 * q + 3])));
+        const uint64_t y01 = f32x2_fma(t01, f32x2_mul(sa2, f32x2_pack(sw.x, sw.y)), f32x2_pack(bb.x, bb.y));
+        const uint64_t y23 = f32x2_fma(t23, f32x2_mul(sa2, f32x2_pack(sw.z, sw.w)), f32x2_pack(bb.z, bb.w));
+        float y0, y1, y2, y3;
+        f32x2_unpack(y01, y0, y1);
+        f32x2_unpack(y23, y2, y3);
+        const __nv_bfloat162 v01 = __floats2bfloat162_rn(y0, y1), v23 = __floats2bfloat162_rn(y2, y3);
+        w[2 * q] = *reinterpret_cast<const uint32_t*>(&v01);
+        w[2 * q + 1] = *reinterpret_cast<const uint32_t*>(&v23);
+      }
+      if (row < p.M) {
+        if (p.dbg_acc != nullptr) {
+          int32_t* arow = p.dbg_acc + row * p.dbg_ldacc + col + c * CW;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) arow[i] = static_cast<int>(a[i]);
+        }
+        if (wide) {
+          st_global_v8(yrow + c * CW, w);
+        } else {
+          uint4* y4 = reinterpret_cast<uint4*>(yrow + c * CW);
+          y4[0] = make_uint4(w[0], w[1], w[2], w[3]);
+          y4[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+      }
+    }
+    return true;
+  }
+};
+
 }  // namespace dp

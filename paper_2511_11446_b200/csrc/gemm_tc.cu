@@ -378,6 +378,8 @@ int gemm_init_device(int dev, int* num_sms_out, int* max_pairs_out) {
   }
   int st = gemm_ws_init_device();
   if (st != DP_OK) return st;
+  st = gemm_as_init_device();
+  if (st != DP_OK) return st;
   *num_sms_out = sms;
   *max_pairs_out = pairs;
   return DP_OK;

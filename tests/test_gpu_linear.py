@@ -123,6 +123,44 @@ def test_mma_weight_stationary_strip_changes():
         _check(run_linear(L, x, flags=MMA_PACKED | B.DP_FLAG_WEIGHT_STATIONARY), x, w, s_w, b, bits)
 
 
+AS = B.DP_FLAG_FORCE_MMA | B.DP_FLAG_ACT_STATIONARY
+
+
+@pytest.mark.parametrize("bits", [8, 4, 3])
+@pytest.mark.parametrize("bn", [64, 128, 192, 256])
+@pytest.mark.parametrize("M,K", [(200, 384), (100, 1152), (600, 128)])
+def test_mma_activation_stationary(bits, bn, M, K):
+    """The CTA-pair kernel that keeps a 256-token strip of int8 codes resident for the whole K and
+    streams only weight tiles: every sub-block width, short and full K (more and fewer k-blocks than
+    ring stages), ragged M (the second CTA's tokens partly / wholly past M), several column
+    sub-blocks per unit. Packed widths reach it through the unpack-first form."""
+    N = 3 * bn
+    x, w, s_w, b = _case(M, K, N, bits, full_range=True, bias=(bn != 128))
+    L = DevLayer(w, s_w, b, bits)
+    _check(run_linear(L, x, flags=AS | B.DP_FLAG_TILE_N(bn)), x, w, s_w, b, bits)
+
+
+def test_mma_activation_stationary_several_units_and_strips_per_pair():
+    """More units than CTA pairs: pairs run several units in a row, keep the resident strip across
+    units of one strip and replace it while the weight ring is live when a run crosses strips; both
+    accumulator buffers and the ring wrap around many times (M = 2100 -> 9 strips)."""
+    for (M, K, N, bits, bn) in [(2100, 1152, 2304, 8, 64), (2100, 640, 2304, 4, 128), (5000, 1152, 1152, 3, 128),
+                                (2100, 256, 4608, 8, 256)]:
+        x, w, s_w, b = _case(M, K, N, bits)
+        L = DevLayer(w, s_w, b, bits)
+        _check(run_linear(L, x, flags=AS | B.DP_FLAG_TILE_N(bn)), x, w, s_w, b, bits)
+
+
+@pytest.mark.parametrize("name,K,N", [("qkv", 1152, 3456), ("proj", 1152, 1152), ("fc1", 1152, 4608)])
+def test_mma_activation_stationary_dit_shapes_default_sub_blocks(name, K, N):
+    """The DiT-XL/2 shapes with K = 1152 at M = 2048, sub-block width chosen by the library (one unit
+    per pair: 8 strips x 9 slices), 8-bit and packed weights."""
+    for bits in (8, 4):
+        x, w, s_w, b = _case(2048, K, N, bits, layer=3)
+        L = DevLayer(w, s_w, b, bits)
+        _check(run_linear(L, x, flags=AS), x, w, s_w, b, bits)
+
+
 def test_mma_many_tiles_per_cta():
     """More tiles than SMs, so the persistent loop, both accumulator buffers and the stage ring
     wrap-around are exercised (M = 1300 -> 11 row tiles x 18 column tiles of 64)."""
