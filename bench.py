@@ -27,10 +27,10 @@ sys.path.insert(0, ROOT)
 METRIC = "fused DAQ+WbA8 linear int8 TOPS (dp_plan_run, DiT-XL/2 linear stack)"
 UNIT = "TOPS"
 NOMINAL_INT8_TOPS = 4500.0
-# dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch, averaged over the four M = 2048 layer
-# shapes, from the ncu capture summarised in profiles/ (None until that capture matches the kernels).
-GEMM_DRAM_BYTES_PER_LAUNCH = 6.99e6  # 8-bit kernel on int8 activations + int8 weights, cold L2; reads only: the
-                                     # bf16 outputs stay in L2 past the kernel's end
+# dram__bytes_read.sum + dram__bytes_write.sum of one whole layer at M = 2048 (its DAQ launch, which for
+# packed layers also expands the weights, plus its GEMM launch), per (shape, weight bits), from the ncu
+# capture summarised in profiles/layer_dram_traffic_M2048.txt. None = no capture of the current kernels.
+LAYER_DRAM_BYTES = None
 
 
 def measured_peaks():
@@ -212,18 +212,21 @@ def run_ours(args):
 
     if rank == 0:
         # ---- roofline of the dominant kernel (tcgen05 GEMM), timed alone with CUDA events ----
-        out["roofline"] = gemm_roofline(stack, peaks)
-        # ideal time of a timestep: per layer max(ops / int8 peak, bytes / HBM)
-        int8_peak = 2.0 * peaks["bf16_sustained"]
+        mma_peak = measure_mma_peak()
+        out["roofline"] = gemm_roofline(stack, peaks, mma_peak)
+        # ideal time of a timestep: per layer max(ops / int8 peak, bytes / HBM); the int8 peak is the
+        # larger of sustained bf16 x2 (the step is seconds of back-to-back work) and the measured
+        # instruction ceiling
+        int8_peak = max(2.0 * peaks["bf16_sustained"], mma_peak or 0.0)
         ideal = 0.0
-        for L, (_, M, K, N) in zip(stack.layers, stack.table):
-            by = 2 * M * K + L.packed_bytes() + 6 * N + 2 * M * N
-            ideal += max(2.0 * M * N * K / (int8_peak * 1e12), by / (peaks["hbm_gbs"] * 1e9))
+        for l, (_, M, K, N) in enumerate(stack.table):
+            ideal += max(2.0 * M * N * K / (int8_peak * 1e12), layer_alg_bytes(stack, l) / (peaks["hbm_gbs"] * 1e9))
         out["roofline_step"] = {"ideal_us_per_dit_step": ideal * 1e6, "frac": ideal * 1e6 / out["us_per_dit_step"],
                                 "int8_peak_tops_used": int8_peak, "hbm_gbs_used": peaks["hbm_gbs"],
                                 "peaks": peaks["source"]}
-        out["mma_i8_peak_tops_measured"] = measure_mma_peak()
+        out["mma_i8_peak_tops_measured"] = mma_peak
         out["roofline_hbm_kernels"] = hbm_kernel_rooflines(stack, peaks)
+        out["roofline_large_m"] = large_m_rooflines(peaks, mma_peak)
         out["e2e"] = e2e(stack, ops_step, world)
         tops, dt, desc, cores = oracle_sample()
         out["cpu_baseline"] = {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
@@ -233,7 +236,13 @@ def run_ours(args):
     D.barrier()
 
 
-def gemm_roofline(stack, peaks):
+def layer_alg_bytes(stack, l):
+    """Bytes the method itself must move for layer l: X bf16, packed W, s_w + bias, Y bf16."""
+    _, M, K, N = stack.table[l]
+    return 2 * M * K + stack.layers[l].packed_bytes() + 6 * N + 2 * M * N
+
+
+def gemm_roofline(stack, peaks, mma_peak):
     """The dominant kernel family (the tcgen05 GEMMs) timed without the rest of the path: the 112
     GEMM launches of one timestep, each with the kernel variant the plan chose for its layer, on
     pre-quantized activations (so no DAQ launch in between), captured in one CUDA graph and timed
@@ -260,7 +269,8 @@ def gemm_roofline(stack, peaks):
             keep.append(w8)
             weights[l] = B.make_weight(w8, stack.layers[l].s_w, stack.layers[l].bias, N, K, 8)
             flags[l] &= ~B.DP_FLAG_UNPACK_FIRST
-        variants[("ws" if v["weight_stationary"] else "pair" if v["cta_group"] == 2 else "single") + str(v["tile_n"])
+        variants[("as" if v["weight_stationary"] == 2 else "ws" if v["weight_stationary"] else
+                  "pair" if v["cta_group"] == 2 else "single") + str(v["tile_n"])
                  + ("+unpack_first" if v["unpack_first"] else "")] += 1
 
     def run():
@@ -287,14 +297,25 @@ def gemm_roofline(stack, peaks):
     ms = statistics.median(times[1:])
     ops = sum(2.0 * stack.table[l][1] * stack.table[l][2] * stack.table[l][3] for l in idx)
     achieved = ops / (ms * 1e-3) / 1e12
-    peak = 2.0 * peaks["bf16"]
-    return {"kernel": "gemm_i8_kernel / gemm_ws_kernel (tcgen05 kind::i8), the 112 launches of one timestep",
+    # Denominator: the larger of (measured bf16 burst x the nominal int8:bf16 ratio of 2) and this
+    # library's own operand-resident kind::i8 instruction ceiling measured in the same run.
+    bf16x2 = 2.0 * peaks["bf16"]
+    peak = max(bf16x2, mma_peak or 0.0)
+    alg = sum(layer_alg_bytes(stack, l) for l in idx) / len(idx)
+    traffic = None
+    if LAYER_DRAM_BYTES is not None:
+        traffic = sum(LAYER_DRAM_BYTES[(stack.table[l][0].split(".")[1], stack.bits[l])] for l in idx) / len(idx)
+    return {"kernel": "gemm_i8_kernel (tcgen05 kind::i8), the 112 launches of one timestep",
             "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TOPS", "frac": achieved / peak,
-            "peak_note": f"{peaks['source']} bf16 burst x2 (nominal int8:bf16 ratio; the file has no int8 row); "
-                         f"sustained x2 = {2.0 * peaks['bf16_sustained']:.0f}; nominal dense int8 {NOMINAL_INT8_TOPS:.0f}",
-            "frac_of_nominal": achieved / NOMINAL_INT8_TOPS, "launches": len(idx),
+            "peak_note": f"max of {peaks['source']} bf16 burst x2 = {bf16x2:.0f} (nominal int8:bf16 ratio; the file has "
+                         f"no int8 row) and the kind::i8 instruction ceiling measured in this run = "
+                         f"{mma_peak or 0.0:.0f}; sustained bf16 x2 = {2.0 * peaks['bf16_sustained']:.0f}; "
+                         f"nominal dense int8 {NOMINAL_INT8_TOPS:.0f}",
+            "frac_of_bf16x2": achieved / bf16x2, "frac_of_nominal": achieved / NOMINAL_INT8_TOPS, "launches": len(idx),
             "avg_launch_us": 1e3 * ms / len(idx), "variants": dict(variants),
-            "traffic": GEMM_DRAM_BYTES_PER_LAUNCH}
+            "traffic": traffic, "traffic_note": "DRAM bytes of a whole layer (DAQ + GEMM launches, reads + writes), "
+                                                "mean over the step's 112 layers; algorithmic bytes beside it",
+            "algorithmic_bytes_per_layer": alg}
 
 
 def hbm_kernel_rooflines(stack, peaks):
@@ -364,6 +385,25 @@ def hbm_kernel_rooflines(stack, peaks):
                                                  "frac": by / t / 1e9 / peaks["hbm_gbs"]}
         del x, x2, q, q2
     return out
+
+
+def large_m_rooflines(peaks, mma_peak):
+    """Config 5 (M = 32768 tokens): the four block shapes at 3, 4 and 8 weight bits, the whole layer
+    (DAQ + weight expansion + GEMM, default dispatch of dp_wq_linear) and the GEMM alone on
+    pre-quantized activations, graph-timed with operand sets rotated past L2. Fractions: against the
+    per-layer roofline max(ops / int8 peak, algorithmic bytes / measured HBM bandwidth) for the
+    layer, against the int8 peak for the GEMM alone (same denominator as `roofline`)."""
+    from paper_2511_11446_b200 import sweep
+    int8_peak = max(2.0 * peaks["bf16"], mma_peak or 0.0)
+    rows = []
+    for name, K, N in sweep.SHAPES:
+        for bits in (3, 4, 8):
+            r = sweep.time_shape(name, 32768, K, N, bits, dict(peaks, bf16=int8_peak / 2.0), iters=8)
+            rows.append({"layer": name, "bits": bits, "layer_us": r["layer_us"], "layer_tops": r["layer_tops"],
+                         "layer_frac_of_roofline": r["layer_frac"], "bound": r["bound"], "gemm_us": r["gemm_us"],
+                         "gemm_tops": r["gemm_tops"], "gemm_frac_of_int8_peak": r["gemm_frac_int8_peak"],
+                         "gemm_frac_of_nominal": r["gemm_tops"] / NOMINAL_INT8_TOPS})
+    return {"M": 32768, "int8_peak_tops_used": int8_peak, "hbm_gbs_used": peaks["hbm_gbs"], "shapes": rows}
 
 
 def measure_mma_peak():

@@ -318,6 +318,56 @@ int dp_plan_run_host(const dp_plan* plan, const int32_t* steps, int32_t n_steps,
                      dp_stream stream);
 
 /*
+ * Algorithm 2, Phase A: budgeted joint planning of the per-layer bit plan and the kept timesteps
+ * (host arithmetic only; the latency table it consumes can be measured with dp_layer_latency_us).
+ *   Tail  = the last floor(rho * n_steps) step indices, always kept.
+ *   Init  : every layer at its first (largest) bit option, every step kept;
+ *           C_lat = sum_t step_cost[t] + sum_l c_lat[l][0],  C_mem = sum_l c_mem[l][0].
+ *   While C_lat > B_lat or C_mem > B_mem:
+ *     step candidate = the prunable (non-tail, still kept) step of least drift,
+ *                      S_step = step_cost[t] / (eps + drift[t]);
+ *     bit candidate  = the best-scored move "layer l: option j -> j + 1" among the layers' next moves,
+ *                      S_bit = (c_lat[l][j] - c_lat[l][j+1]) / (eps + sens[l]), restricted to moves after
+ *                      which C_mem <= B_mem when such a move exists;
+ *     if S_step > S_bit the step is dropped (C_lat -= step_cost[t]); else the move is applied
+ *     (C_lat, C_mem updated, the layer's next move becomes available).
+ * Readings where the listing is silent: costs are used exactly as supplied (one additive C_lat: the
+ * caller decides whether c_lat is per step or summed over the schedule); when no move satisfies the
+ * memory clause the best-scored move is taken anyway, since otherwise an overrun larger than one move
+ * could never be repaired; ties go to the lower layer index / lower timestep, and S_step == S_bit
+ * applies the bit move; the loop also ends when neither candidate exists (*feasible = 0).
+ *   options     : n_options[l] entries per layer, flattened in layer order (offset = running sum):
+ *                 opt_bits (descending), opt_c_lat, opt_c_mem
+ *   bitplan_out : [n_layers] chosen bits;  kept_out : [n_steps] 1 = kept
+ *   totals_out  : [2] final C_lat, C_mem (may be NULL);  feasible : may be NULL
+ * All pointers are HOST pointers. DP_ERR_INVALID_ARG on NULL / non-positive sizes / rho outside [0, 1].
+ */
+typedef struct dp_phase_a_problem {
+  int32_t n_steps;
+  const double* drift;      /* D_e(t) */
+  const double* step_cost;  /* c_step(t) */
+  int32_t n_layers;
+  const int32_t* n_options;
+  const int32_t* opt_bits;
+  const double* opt_c_lat;
+  const double* opt_c_mem;
+  const double* sens;       /* s_M(l) */
+  double B_lat, B_mem, rho, eps;
+} dp_phase_a_problem;
+int dp_plan_phase_a(const dp_phase_a_problem* problem, int32_t* bitplan_out, uint8_t* kept_out, double* totals_out,
+                    int32_t* feasible);
+
+/*
+ * One entry c_lat(l, b) of Phase A's latency table, measured with this library's kernels: the time of
+ * one whole quantized linear (DAQ + weight expansion + GEMM, as dp_wq_linear runs it with `flags`) for
+ * weight `w` (device pointers) at M tokens, in microseconds, averaged over `reps` back-to-back calls
+ * after two warm-up calls. Allocates and frees its own device buffers and synchronises: a plan-time
+ * call like dp_plan_create, not part of the hot path. (Algorithm 2's inputs c_lat(l, b); the paper
+ * measures them with its own integer kernels.)
+ */
+int dp_layer_latency_us(const dp_weight* w, int64_t M, uint32_t flags, int32_t reps, float* us_out);
+
+/*
  * Host helper: pack int8 weights w[N][K] (values in [-2^(b-1), 2^(b-1)-1]) into the layout
  * dp_weight documents. `out` is a host buffer of N*K*bits/8 bytes. Values out of range give
  * DP_ERR_INVALID_ARG.

@@ -209,3 +209,26 @@ def plan_run(layers, kept, xs):
 def bf16_to_f32(bits: np.ndarray) -> np.ndarray:
     """Exact widening of bf16 bit patterns (uint16) to float32."""
     return (bits.astype(np.uint32) << 16).view(np.float32)
+
+
+def phase_a(drift, step_cost, options, sens, B_lat, B_mem, rho, eps):
+    """Algorithm 2, Phase A. options[l] = list of (bits, c_lat, c_mem), largest bits first.
+    Returns (bitplan list, kept list of 0/1, (C_lat, C_mem), feasible)."""
+    T, L = len(drift), len(options)
+    d = np.ascontiguousarray(drift, np.float64)
+    c = np.ascontiguousarray(step_cost, np.float64)
+    n_opt = np.array([len(o) for o in options], np.int32)
+    bits = np.array([b for o in options for (b, _, _) in o], np.int32)
+    lat = np.array([x for o in options for (_, x, _) in o], np.float64)
+    mem = np.array([x for o in options for (_, _, x) in o], np.float64)
+    s = np.ascontiguousarray(sens, np.float64)
+    plan = np.empty(L, np.int32)
+    kept = np.empty(T, np.uint8)
+    tot = np.empty(2, np.float64)
+    f = lib().orc_phase_a
+    f.restype = C.c_int
+    f.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                  C.c_void_p, C.c_double, C.c_double, C.c_double, C.c_double, C.c_void_p, C.c_void_p, C.c_void_p]
+    ok = f(T, _p(d), _p(c), L, _p(n_opt), _p(bits), _p(lat), _p(mem), _p(s), B_lat, B_mem, rho, eps, _p(plan),
+           _p(kept), _p(tot))
+    return plan.tolist(), kept.tolist(), (float(tot[0]), float(tot[1])), bool(ok)

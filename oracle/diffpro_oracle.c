@@ -26,6 +26,9 @@
  *                  the int32 accumulator; bias add; bf16 output.
  *   orc_wq_linear  the four above in order.
  *   orc_plan_run   Algorithm 2, Phase B: for t in reverse(K*): forward every wrapped linear.
+ *   orc_phase_a    Algorithm 2, Phase A: the greedy budgeted joint planning of bits and kept steps,
+ *                  step by step in the listing's order; the "heap" and the sorted list are plain
+ *                  searches for the best-scored move and the least-drift step.
  *
  * Parity status: every function here is pinned by tests/test_oracle_*.py (brute force in exact
  * rational arithmetic, closed forms, invariants, library cross-checks). End-to-end image quality
@@ -311,4 +314,84 @@ void orc_plan_run(const orc_layer* layers, int32_t n_layers, const int32_t* kept
                     L->s_w, L->bias, y_ptrs[(int64_t)i * n_layers + l], L->N, scratch_w, scratch_q,
                     scratch_sa, scratch_acc);
     }
+}
+
+/* ---- joint planning (Algorithm 2, Phase A) ---------------------------------------------------- */
+
+/*
+ * Inputs as in the algorithm: drift D_e(t) and step latency c_step(t) for t < n_steps; for layer l
+ * its n_options[l] bit options (largest first) with c_lat, c_mem (flattened in layer order) and its
+ * sensitivity s_M(l); budgets B_lat, B_mem; protected-tail fraction rho; epsilon.
+ * Outputs: bitplan[l] = chosen bits, kept[t] = 1 if t is in K*, totals = {C_lat, C_mem}.
+ * Returns 1 if both budgets are met at exit, 0 if the moves ran out first.
+ * Readings (the listing is silent): one additive C_lat = sum of kept c_step + sum of current c_lat;
+ * the bit candidate is the best-scored next move among those after which C_mem <= B_mem, or, when
+ * there is none, the best-scored next move; ties: lower layer index, lower timestep; S_step must be
+ * strictly larger than S_bit for the step to be dropped.
+ */
+int orc_phase_a(int32_t n_steps, const double* drift, const double* step_cost, int32_t n_layers,
+                const int32_t* n_options, const int32_t* opt_bits, const double* opt_c_lat,
+                const double* opt_c_mem, const double* sens, double B_lat, double B_mem, double rho,
+                double eps, int32_t* bitplan, uint8_t* kept, double* totals) {
+  int64_t* off = (int64_t*)malloc((size_t)(n_layers + 1) * sizeof(int64_t));
+  int32_t* cur = (int32_t*)calloc((size_t)n_layers, sizeof(int32_t));
+  off[0] = 0;
+  for (int32_t l = 0; l < n_layers; ++l) off[l + 1] = off[l] + n_options[l];
+  const int32_t n_tail = (int32_t)floor(rho * (double)n_steps); /* Tail = last floor(rho |T|) indices */
+  double C_lat = 0.0, C_mem = 0.0;
+  for (int32_t t = 0; t < n_steps; ++t) { /* K <- T */
+    kept[t] = 1;
+    C_lat += step_cost[t];
+  }
+  for (int32_t l = 0; l < n_layers; ++l) { /* Pi(l) <- max B_l */
+    C_lat += opt_c_lat[off[l]];
+    C_mem += opt_c_mem[off[l]];
+  }
+  int feasible = 1;
+  while (C_lat > B_lat || C_mem > B_mem) {
+    /* step candidate: first of R = prunable kept steps by ascending drift */
+    int32_t ts = -1;
+    for (int32_t t = 0; t < n_steps - n_tail; ++t)
+      if (kept[t] && (ts < 0 || drift[t] < drift[ts])) ts = t;
+    /* bit candidate: top of H_bit subject to the memory clause */
+    int32_t lb = -1, lb_any = -1;
+    double sb = 0.0, sb_any = 0.0;
+    for (int32_t l = 0; l < n_layers; ++l) {
+      if (cur[l] + 1 >= n_options[l]) continue; /* no cheaper option left */
+      const int64_t i = off[l] + cur[l];
+      const double score = (opt_c_lat[i] - opt_c_lat[i + 1]) / (eps + sens[l]);
+      if (lb_any < 0 || score > sb_any) {
+        lb_any = l;
+        sb_any = score;
+      }
+      if (C_mem - (opt_c_mem[i] - opt_c_mem[i + 1]) <= B_mem && (lb < 0 || score > sb)) {
+        lb = l;
+        sb = score;
+      }
+    }
+    if (lb < 0) {
+      lb = lb_any;
+      sb = sb_any;
+    }
+    if (ts < 0 && lb < 0) {
+      feasible = 0;
+      break;
+    }
+    const double s_step = ts >= 0 ? step_cost[ts] / (eps + drift[ts]) : 0.0;
+    if (ts >= 0 && (lb < 0 || s_step > sb)) {
+      kept[ts] = 0; /* K <- K \ {t*} */
+      C_lat -= step_cost[ts];
+    } else {
+      const int64_t i = off[lb] + cur[lb];
+      C_lat -= opt_c_lat[i] - opt_c_lat[i + 1];
+      C_mem -= opt_c_mem[i] - opt_c_mem[i + 1];
+      cur[lb] += 1; /* Pi(l*) <- b' */
+    }
+  }
+  for (int32_t l = 0; l < n_layers; ++l) bitplan[l] = opt_bits[off[l] + cur[l]];
+  totals[0] = C_lat;
+  totals[1] = C_mem;
+  free(off);
+  free(cur);
+  return feasible;
 }

@@ -35,7 +35,7 @@ DP_STATIC_SCRATCH_BYTES = 10 << 20
 
 EXPORTS = ["dp_daq_quantize", "dp_daq_quantize_robust", "dp_wq_linear_workspace", "dp_wq_linear", "dp_wq_linear_static", "dp_plan_create",
            "dp_plan_workspace", "dp_plan_layer_variant", "dp_plan_layer_unpack_first", "dp_plan_set_layer_flags", "dp_plan_set_daq", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
-           "dp_plan_run_host", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_clip_rank", "dp_debug_skip_stage_load",
+           "dp_plan_run_host", "dp_plan_phase_a", "dp_layer_latency_us", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_clip_rank", "dp_debug_skip_stage_load",
            "dp_status_string",
            "dp_last_error", "dp_version"]
 
@@ -48,6 +48,13 @@ class dp_weight(C.Structure):
 class dp_debug(C.Structure):
     _fields_ = [("q", C.c_void_p), ("ldq", C.c_int64), ("s_a", C.c_void_p), ("acc", C.c_void_p),
                 ("ldacc", C.c_int64)]
+
+
+class dp_phase_a_problem(C.Structure):
+    _fields_ = [("n_steps", C.c_int32), ("drift", C.c_void_p), ("step_cost", C.c_void_p), ("n_layers", C.c_int32),
+                ("n_options", C.c_void_p), ("opt_bits", C.c_void_p), ("opt_c_lat", C.c_void_p),
+                ("opt_c_mem", C.c_void_p), ("sens", C.c_void_p), ("B_lat", C.c_double), ("B_mem", C.c_double),
+                ("rho", C.c_double), ("eps", C.c_double)]
 
 
 class DiffproError(RuntimeError):
@@ -101,6 +108,8 @@ def lib():
                                        C.c_void_p, C.c_size_t, C.c_void_p, C.c_uint32, C.c_void_p]
         L.dp_pack_weights_host.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         L.dp_bench_mma_i8.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.dp_plan_phase_a.argtypes = [C.POINTER(dp_phase_a_problem), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.dp_layer_latency_us.argtypes = [C.POINTER(dp_weight), C.c_int64, C.c_uint32, C.c_int32, C.c_void_p]
         L.dp_clip_rank.restype = C.c_int32
         L.dp_clip_rank.argtypes = [C.c_int32, C.c_int32]
         L.dp_debug_skip_stage_load.restype = None
@@ -239,6 +248,31 @@ def dp_plan_run_host(plan, steps, x_host, x_stage, y_dev, d2h_layer, y_host, wor
                                   x_stage.numel() * x_stage.element_size(), y_dev, d2h_layer, y_host,
                                   _ptr(workspace), workspace.numel() * workspace.element_size(),
                                   _ptr(device_status), flags, _stream(stream)), "dp_plan_run_host")
+
+
+def dp_plan_phase_a(drift, step_cost, options, sens, B_lat, B_mem, rho, eps):
+    """options[l] = list of (bits, c_lat, c_mem), largest bits first; the arrays are host data.
+    Returns (bitplan list, kept list of 0/1, (C_lat, C_mem), feasible)."""
+    import numpy as np
+    T, nl = len(drift), len(options)
+    d = np.ascontiguousarray(drift, np.float64)
+    c = np.ascontiguousarray(step_cost, np.float64)
+    n_opt = np.array([len(o) for o in options], np.int32)
+    bits = np.array([b for o in options for (b, _, _) in o], np.int32)
+    lat = np.array([x for o in options for (_, x, _) in o], np.float64)
+    mem = np.array([x for o in options for (_, _, x) in o], np.float64)
+    s = np.ascontiguousarray(sens, np.float64)
+    p = lambda a: a.ctypes.data_as(C.c_void_p)
+    prob = dp_phase_a_problem(T, p(d), p(c), nl, p(n_opt), p(bits), p(lat), p(mem), p(s), B_lat, B_mem, rho, eps)
+    plan, kept, tot, ok = np.empty(nl, np.int32), np.empty(T, np.uint8), np.empty(2, np.float64), C.c_int32(0)
+    _check(lib().dp_plan_phase_a(C.byref(prob), p(plan), p(kept), p(tot), C.byref(ok)), "dp_plan_phase_a")
+    return plan.tolist(), kept.tolist(), (float(tot[0]), float(tot[1])), bool(ok.value)
+
+
+def dp_layer_latency_us(w: dp_weight, M: int, flags=0, reps=20) -> float:
+    us = C.c_float(0.0)
+    _check(lib().dp_layer_latency_us(C.byref(w), M, flags, reps, C.byref(us)), "dp_layer_latency_us")
+    return float(us.value)
 
 
 def dp_pack_weights_host(w, bits: int):

@@ -2,9 +2,11 @@
 #include <stdarg.h>
 #include <string.h>
 
+#include <algorithm>
 #include <atomic>
 #include <mutex>
 #include <new>
+#include <queue>
 #include <vector>
 
 #include "dp_common.cuh"
@@ -955,6 +957,150 @@ extern "C" int dp_plan_run_host(const dp_plan* plan_c, const int32_t* steps, int
     }
   }
   return DP_OK;
+}
+
+// ---- Algorithm 2, Phase A --------------------------------------------------------------------------
+namespace {
+struct BitMove {
+  double score;
+  int32_t layer;
+  bool operator<(const BitMove& o) const {  // max-heap on score, ties to the lower layer index
+    return score < o.score || (score == o.score && layer > o.layer);
+  }
+};
+}  // namespace
+
+extern "C" int dp_plan_phase_a(const dp_phase_a_problem* q, int32_t* bitplan_out, uint8_t* kept_out,
+                               double* totals_out, int32_t* feasible) {
+  if (!q || !bitplan_out || !kept_out) return fail(DP_ERR_INVALID_ARG, "dp_plan_phase_a: NULL argument");
+  if (q->n_steps <= 0 || q->n_layers <= 0 || !q->drift || !q->step_cost || !q->n_options || !q->opt_bits ||
+      !q->opt_c_lat || !q->opt_c_mem || !q->sens || !(q->rho >= 0.0 && q->rho <= 1.0))
+    return fail(DP_ERR_INVALID_ARG, "dp_plan_phase_a: bad problem description");
+  const int32_t T = q->n_steps, L = q->n_layers;
+  std::vector<int64_t> off(L + 1, 0);
+  for (int32_t l = 0; l < L; ++l) {
+    if (q->n_options[l] <= 0) return fail(DP_ERR_INVALID_ARG, "dp_plan_phase_a: layer %d has no bit option", l);
+    off[l + 1] = off[l] + q->n_options[l];
+  }
+  const int32_t tail0 = T - static_cast<int32_t>(q->rho * T);  // steps tail0 .. T-1 are protected
+  // prunable steps by ascending drift (ties: lower timestep first)
+  std::vector<int32_t> order;
+  for (int32_t t = 0; t < tail0; ++t) order.push_back(t);
+  std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return q->drift[a] < q->drift[b]; });
+  size_t next_step = 0;
+  std::vector<int32_t> cur(L, 0);  // option index per layer
+  double C_lat = 0.0, C_mem = 0.0;
+  for (int32_t t = 0; t < T; ++t) {
+    kept_out[t] = 1;
+    C_lat += q->step_cost[t];
+  }
+  auto score_of = [&](int32_t l) {
+    const int64_t i = off[l] + cur[l];
+    return (q->opt_c_lat[i] - q->opt_c_lat[i + 1]) / (q->eps + q->sens[l]);
+  };
+  std::priority_queue<BitMove> heap;
+  for (int32_t l = 0; l < L; ++l) {
+    C_lat += q->opt_c_lat[off[l]];
+    C_mem += q->opt_c_mem[off[l]];
+    if (q->n_options[l] > 1) heap.push({score_of(l), l});
+  }
+  int ok = 1;
+  while (C_lat > q->B_lat || C_mem > q->B_mem) {
+    const bool has_step = next_step < order.size();
+    // bit candidate: the best-scored move that leaves the memory within budget, else the best-scored
+    // move; moves skipped while looking go back on the heap
+    bool has_bit = !heap.empty();
+    BitMove pick{0.0, -1};
+    if (has_bit) {
+      std::vector<BitMove> skipped;
+      while (!heap.empty()) {
+        const BitMove m = heap.top();
+        const int64_t i = off[m.layer] + cur[m.layer];
+        if (C_mem - (q->opt_c_mem[i] - q->opt_c_mem[i + 1]) <= q->B_mem) {
+          pick = m;
+          break;
+        }
+        skipped.push_back(m);
+        heap.pop();
+      }
+      if (pick.layer < 0) pick = skipped.front();  // none satisfies the clause: the top move
+      else heap.pop();
+      for (const BitMove& m : skipped)
+        if (m.layer != pick.layer) heap.push(m);
+    }
+    if (!has_step && !has_bit) {
+      ok = 0;
+      break;
+    }
+    const int32_t t = has_step ? order[next_step] : -1;
+    const double s_step = has_step ? q->step_cost[t] / (q->eps + q->drift[t]) : 0.0;
+    if (has_step && (!has_bit || s_step > pick.score)) {
+      kept_out[t] = 0;
+      C_lat -= q->step_cost[t];
+      ++next_step;
+      if (has_bit) heap.push(pick);
+    } else {
+      const int32_t l = pick.layer;
+      const int64_t i = off[l] + cur[l];
+      C_lat -= q->opt_c_lat[i] - q->opt_c_lat[i + 1];
+      C_mem -= q->opt_c_mem[i] - q->opt_c_mem[i + 1];
+      ++cur[l];
+      if (cur[l] + 1 < q->n_options[l]) heap.push({score_of(l), l});
+    }
+  }
+  for (int32_t l = 0; l < L; ++l) bitplan_out[l] = q->opt_bits[off[l] + cur[l]];
+  if (totals_out) {
+    totals_out[0] = C_lat;
+    totals_out[1] = C_mem;
+  }
+  if (feasible) *feasible = ok;
+  return DP_OK;
+}
+
+extern "C" int dp_layer_latency_us(const dp_weight* w, int64_t M, uint32_t flags, int32_t reps, float* us_out) {
+  if (!us_out || reps <= 0 || reps > 10000) return fail(DP_ERR_INVALID_ARG, "dp_layer_latency_us: bad reps / us_out");
+  int st = check_weight(w);
+  if (st != DP_OK) return st;
+  if (M <= 0) return fail(DP_ERR_SHAPE, "dp_layer_latency_us: M must be positive");
+  if (flags & ~kLinearFlags) return fail(DP_ERR_INVALID_ARG, "unknown flag bits 0x%x", flags);
+  if (int tst = check_tile_flags(flags, w->N)) return tst;
+  st = check_device();
+  if (st != DP_OK) return st;
+  void *x = nullptr, *y = nullptr, *ws = nullptr;
+  cudaStream_t stream = nullptr;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  const size_t xb = static_cast<size_t>(M) * w->K * 2, yb = static_cast<size_t>(M) * w->N * 2;
+  const size_t wb = dp_wq_linear_workspace(M, w->N, w->K, w->bits, flags);
+  cudaError_t e = cudaMalloc(&x, xb);
+  if (e == cudaSuccess) e = cudaMalloc(&y, yb);
+  if (e == cudaSuccess) e = cudaMalloc(&ws, wb);
+  if (e == cudaSuccess) e = cudaMemset(x, 0x3c, xb);  // bf16 0x3c3c = 0.0115: finite, non-zero
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreate(&e0);
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  st = e == cudaSuccess ? DP_OK : fail(DP_ERR_CUDA, "dp_layer_latency_us set-up: %s", cudaGetErrorString(e));
+  for (int it = 0; it < 2 + reps && st == DP_OK; ++it) {
+    if (it == 2) cudaEventRecord(e0, stream);
+    st = check_linear_args(w, x, w->K, nullptr, M, y, w->N, ws, wb, nullptr, flags);
+    if (st == DP_OK)
+      st = run_linear(w, x, w->K, nullptr, M, y, w->N, ws, nullptr, nullptr, flags, stream, nullptr, 0, 0, 0, nullptr,
+                      it > 0);
+  }
+  if (st == DP_OK) {
+    cudaEventRecord(e1, stream);
+    e = cudaEventSynchronize(e1);
+    float ms = 0.0f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    if (e != cudaSuccess) st = fail(DP_ERR_CUDA, "dp_layer_latency_us timing: %s", cudaGetErrorString(e));
+    else *us_out = ms * 1000.0f / static_cast<float>(reps);
+  }
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  if (stream) cudaStreamDestroy(stream);
+  cudaFree(x);
+  cudaFree(y);
+  cudaFree(ws);
+  return st;
 }
 
 // ---- host helpers ----------------------------------------------------------------------------------

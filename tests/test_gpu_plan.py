@@ -301,3 +301,49 @@ def test_plan_errors():
         assert e.value.status == B.DP_ERR_WORKSPACE
     finally:
         B.dp_plan_destroy(plan)
+
+
+def test_phase_a_on_measured_latencies_matches_oracle_and_runs():
+    """Algorithm 2 end to end on a small stack: c_lat(l, b) measured with the library's kernels, Phase A
+    (library) equal to the oracle's on the same table, and the resulting bit plan and kept steps run by
+    dp_plan_run against the oracle's layer outputs."""
+    from paper_2511_11446_b200 import planner
+    seed = synth.BASE_SEED + 21
+    table = [("a", 256, 256, 128), ("b", 256, 128, 256), ("c", 16, 256, 128), ("a2", 256, 256, 128)]
+    lat = planner.latency_table(table, reps=5)
+    assert all(v > 0.5 and v < 5e4 for v in lat.values()), lat
+    T = 10
+    drift = [float(np.exp(-t / 3.0)) + 0.01 * ((t * 7) % 3) for t in range(T)]
+    sens = [0.5, 2.0, 1.0, 0.1]
+    full = T * sum(lat[(M, K, N, 8)] for (_, M, K, N) in table) + T * 5.0
+    mem8 = sum(N * K + 6 * N for (_, M, K, N) in table)
+    bits, kept, totals, ok = planner.joint_plan(table, lat, sens, drift, 5.0, 0.8 * full, 0.7 * mem8)
+    options = [[(b, T * lat[(M, K, N, b)], N * K * b / 8 + 6 * N) for b in (8, 4, 3)] for (_, M, K, N) in table]
+    o_bits, o_kept, o_tot, o_ok = oracle.phase_a(drift, [5.0] * T, options, sens, 0.8 * full, 0.7 * mem8, 0.2, 1e-6)
+    assert bits == o_bits and kept == [t for t in range(T) if o_kept[t]] and ok == o_ok and ok
+    assert totals[1] <= 0.7 * mem8 and set(kept) >= {8, 9}
+    # deploy (Phase B) under the plan
+    Ls, Ws = [], []
+    for l, (name, M, K, N) in enumerate(table):
+        w, s_w = synth.weights(seed, l, N, K, bits[l])
+        b = synth.bias(seed, l, N)
+        Ls.append(DevLayer(w, s_w, b, bits[l]))
+        Ws.append((w, s_w, b))
+    plan = B.dp_plan_create([L.w for L in Ls], [M for (_, M, K, N) in table], 0)
+    try:
+        xs = [[synth.activations(seed, l, t, M, K, synth.sigma_t(t, T), n_out=2) for l, (_, M, K, N) in enumerate(table)]
+              for t in kept]
+        xd = [[to_dev_bf16(x) for x in row] for row in xs]
+        ys = [[torch.empty((M, N), dtype=torch.bfloat16, device="cuda") for (_, M, K, N) in table] for _ in kept]
+        ws = torch.empty(B.dp_plan_workspace(plan), dtype=torch.uint8, device="cuda")
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        B.dp_plan_run(plan, kept, 0, B.ptr_array([t.data_ptr() for row in xd for t in row]),
+                      B.ptr_array([t.data_ptr() for row in ys for t in row]), ws, st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        for i in range(len(kept)):
+            for l, (w, s_w, b) in enumerate(Ws):
+                ref = oracle.wq_linear(xs[i][l], oracle.pack(w, bits[l]), s_w, b, bits[l])
+                assert bf16_ulp_dist(bf16_to_np(ys[i][l]), ref).max() <= 1
+    finally:
+        B.dp_plan_destroy(plan)
