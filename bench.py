@@ -30,7 +30,10 @@ NOMINAL_INT8_TOPS = 4500.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one whole layer at M = 2048 (its DAQ launch, which for
 # packed layers also expands the weights, plus its GEMM launch), per (shape, weight bits), from the ncu
 # capture summarised in profiles/layer_dram_traffic_M2048.txt. None = no capture of the current kernels.
-LAYER_DRAM_BYTES = None
+LAYER_DRAM_BYTES = {("qkv", 8): 22796480, ("qkv", 4): 21250107, ("qkv", 3): 20888222,
+                    ("proj", 8): 10673745, ("proj", 4): 10187587, ("proj", 3): 10219431,
+                    ("fc1", 8): 28953344, ("fc1", 4): 27161833, ("fc1", 3): 26080140,
+                    ("fc2", 8): 29405184, ("fc2", 4): 25559239, ("fc2", 3): 24797924}
 
 
 def measured_peaks():
