@@ -40,7 +40,7 @@ typedef enum dp_status {
   DP_ERR_INVALID_ARG = 1, /* NULL where a pointer is required, negative size, bad flag        */
   DP_ERR_SHAPE = 2,       /* K not a multiple of 128, N not a multiple of 16, ld < row length  */
   DP_ERR_ALIGN = 3,       /* pointer or row pitch not 16-byte aligned                          */
-  DP_ERR_BITS = 4,        /* weight bit-width not in {3,4,8}                                   */
+  DP_ERR_BITS = 4,        /* weight bit-width not in {3,4,8,16}                                */
   DP_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than dp_*_workspace() says              */
   DP_ERR_ARCH = 6,        /* current device is not sm_100                                      */
   DP_ERR_CUDA = 7,        /* a CUDA runtime/driver call failed (see dp_last_error)             */
@@ -58,6 +58,10 @@ typedef void* dp_stream;
  *               little-endian bit stream (8 values per 32-bit word), code u = w + 8.
  *   bits == 3 : qweight is uint32 [N][3K/32]; field k = bits [3k, 3k+3) of the row's bit stream
  *               (32 values per 3 words; fields 10 and 21 of each group straddle words), u = w + 4.
+ *   bits == 16: a layer the plan keeps in 16-bit precision (Step 1's tiering sends the most sensitive
+ *               layers there; the paper's best plans freeze about a fifth of them): qweight is bf16
+ *               [N][K] row-major, s_w is ignored (may be NULL), the layer is y = x . W^T + bias with
+ *               fp32 accumulation and no DAQ; N % 64 == 0.
  * s_w  : fp32 [N], one scale per output channel (Step 5).
  * bias : bf16 [N] or NULL.
  * Requirements: K % 128 == 0, N % 16 == 0, N,K >= 128.
@@ -203,7 +207,9 @@ size_t dp_wq_linear_workspace(int64_t M, int32_t N, int32_t K, int32_t bits, uin
  *   dbg      : NULL or taps (slower path when dbg->acc is set)
  *   device_status : int32 device word or NULL; set to DP_ERR_TIMEOUT by a kernel whose wait expired
  * M == 0 is a no-op. Calls on the same stream are ordered; the workspace may be reused by the
- * next call on that stream.
+ * next call on that stream. For w->bits == 16 (pass-through layer) x is bf16, s_a_in and dbg must be
+ * NULL, no workspace is used, and the output is bf16_rne(fp32 sum + bias) with the sum accumulated in
+ * fp32 on the tensor cores (order unspecified: compare with a tolerance, not bit for bit).
  */
 int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_a_in, int64_t M,
                  void* y_bf16, int64_t ldy, void* workspace, size_t workspace_bytes,

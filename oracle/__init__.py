@@ -232,3 +232,19 @@ def phase_a(drift, step_cost, options, sens, B_lat, B_mem, rho, eps):
     ok = f(T, _p(d), _p(c), L, _p(n_opt), _p(bits), _p(lat), _p(mem), _p(s), B_lat, B_mem, rho, eps, _p(plan),
            _p(kept), _p(tot))
     return plan.tolist(), kept.tolist(), (float(tot[0]), float(tot[1])), bool(ok)
+
+
+def linear_bf16(x, w, bias=None):
+    """Pass-through linear of a 16-bit layer: x uint16 (bf16 bits) [M,K], w uint16 [N,K], bias uint16 [N]
+    or None. Returns (y uint16 [M,N], exact float64 [M,N], mag float64 [M,N] = sum_k |x w|)."""
+    _chk(x, np.uint16, "x")
+    _chk(w, np.uint16, "w")
+    M, K = x.shape
+    N = w.shape[0]
+    assert w.shape[1] == K
+    y = np.empty((M, N), np.uint16)
+    exact = np.empty((M, N), np.float64)
+    mag = np.empty((M, N), np.float64)
+    lib().orc_linear_bf16(_p(x), _i64(K), _p(w), _p(bias), _i64(M), _i64(N), _i64(K), _p(y), _i64(N), _p(exact),
+                          _p(mag))
+    return y, exact, mag

@@ -26,6 +26,9 @@
  *                  the int32 accumulator; bias add; bf16 output.
  *   orc_wq_linear  the four above in order.
  *   orc_plan_run   Algorithm 2, Phase B: for t in reverse(K*): forward every wrapped linear.
+ *   orc_linear_bf16  the layers a plan keeps in 16-bit precision (Step 1 tiering; Step 2 results): the
+ *                  plain linear y = x . W^T + bias on bf16 inputs, summed in double (every product of
+ *                  two bf16 values is exact in double), rounded once to bf16.
  *   orc_phase_a    Algorithm 2, Phase A: the greedy budgeted joint planning of bits and kept steps,
  *                  step by step in the listing's order; the "heap" and the sorted list are plain
  *                  searches for the best-scored move and the least-drift step.
@@ -313,6 +316,55 @@ void orc_plan_run(const orc_layer* layers, int32_t n_layers, const int32_t* kept
       orc_wq_linear(x_ptrs[(int64_t)i * n_layers + l], L->K, L->M, L->N, L->K, L->bits, L->qweight,
                     L->s_w, L->bias, y_ptrs[(int64_t)i * n_layers + l], L->N, scratch_w, scratch_q,
                     scratch_sa, scratch_acc);
+    }
+}
+
+/* ---- pass-through linear of 16-bit layers ------------------------------------------------------ */
+
+/* Round-to-nearest-even narrowing of a double to bf16 (one rounding: via the exactly representable
+   neighbours, not through float). */
+static uint16_t f64_to_bf16(double v) {
+  float f = (float)v; /* may double-round: repaired below by comparing the two candidates in double */
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  uint32_t lo = u & 0xFFFF0000u; /* candidate toward zero */
+  uint32_t hi = lo + 0x10000u;   /* candidate away from zero */
+  float flo, fhi;
+  memcpy(&flo, &lo, 4);
+  memcpy(&fhi, &hi, 4);
+  /* (float)v can land one bf16 step beyond the bracket only when v rounds up to hi exactly: then
+     lo == hi's pattern and the loop below still picks the nearer of the two neighbours of v */
+  if (fabs((double)flo) > fabs(v)) { /* v's magnitude is below lo: step the bracket down */
+    hi = lo;
+    lo = lo - 0x10000u;
+    memcpy(&flo, &lo, 4);
+    memcpy(&fhi, &hi, 4);
+  }
+  const double dl = fabs(v - (double)flo), dh = fabs((double)fhi - v);
+  if (dl < dh || (dl == dh && ((lo >> 16) & 1u) == 0)) return (uint16_t)(lo >> 16);
+  return (uint16_t)(hi >> 16);
+}
+
+/*
+ * x bf16 [M][ldx], w bf16 [N][K], bias bf16 [N] or NULL -> y bf16 [M][ldy]; optional exact[M][N]
+ * (the double-precision value before the final rounding) and mag[M][N] = sum_k |x w| (for error
+ * bounds of implementations that accumulate in lower precision).
+ */
+void orc_linear_bf16(const uint16_t* x, int64_t ldx, const uint16_t* w, const uint16_t* bias, int64_t M,
+                     int64_t N, int64_t K, uint16_t* y, int64_t ldy, double* exact, double* mag) {
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t n = 0; n < N; ++n) {
+      double s = 0.0, a = 0.0;
+      for (int64_t k = 0; k < K; ++k) {
+        const double p = (double)bf16_to_f32(x[m * ldx + k]) * (double)bf16_to_f32(w[n * K + k]);
+        s += p;
+        a += fabs(p);
+      }
+      if (bias) s += (double)bf16_to_f32(bias[n]);
+      y[m * ldy + n] = f64_to_bf16(s);
+      if (exact) exact[m * N + n] = s;
+      if (mag) mag[m * N + n] = a;
     }
 }
 

@@ -189,12 +189,14 @@ static bool as_pointers_ok(const dp_weight*) { return true; }
 
 static int check_weight(const dp_weight* w) {
   if (!w) return fail(DP_ERR_INVALID_ARG, "dp_weight is NULL");
-  if (w->bits != 3 && w->bits != 4 && w->bits != 8)
-    return fail(DP_ERR_BITS, "bits=%d not in {3,4,8}", w->bits);
+  if (w->bits != 3 && w->bits != 4 && w->bits != 8 && w->bits != 16)
+    return fail(DP_ERR_BITS, "bits=%d not in {3,4,8,16}", w->bits);
   if (w->N < 16 || w->K < 128 || (w->K % 128) || (w->N % 16))
     return fail(DP_ERR_SHAPE, "N=%d K=%d: need K %% 128 == 0, N %% 16 == 0", w->N, w->K);
+  if (w->bits == 16 && (w->N % 64))
+    return fail(DP_ERR_SHAPE, "N=%d: a 16-bit pass-through layer needs N %% 64 == 0", w->N);
   if (w->reserved != 0) return fail(DP_ERR_INVALID_ARG, "dp_weight.reserved must be 0");
-  if (!w->qweight || !w->s_w) return fail(DP_ERR_INVALID_ARG, "dp_weight has a NULL member");
+  if (!w->qweight || (!w->s_w && w->bits != 16)) return fail(DP_ERR_INVALID_ARG, "dp_weight has a NULL member");
   if (!aligned16(w->qweight) || (reinterpret_cast<uintptr_t>(w->s_w) & 3u) ||
       (w->bias && (reinterpret_cast<uintptr_t>(w->bias) & 1u)))
     return fail(DP_ERR_ALIGN, "dp_weight pointers misaligned");
@@ -211,6 +213,9 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
                       const CUtensorMap* tmap_a_cached, bool chained, int32_t* daq_sync = nullptr,
                       int pre = -1, int daq_rank = 1, int daq_bits = 8) {
   const bool pdl = !(flags & DP_FLAG_NO_PDL);
+  if (w->bits == 16)  // a layer the plan keeps in 16-bit precision: no DAQ, no scales (checked by the caller)
+    return launch_gemm_bf16(x, ldx, w->qweight, static_cast<const uint16_t*>(w->bias), M, w->N, w->K,
+                            static_cast<uint16_t*>(y), ldy, status, stream, pdl);
   // DAQ policy of a plan (dp_plan_set_daq): clip threshold below the maximum and/or fewer activation bits
   const bool robust = s_a_in == nullptr && (daq_rank > 1 || daq_bits < 8);
   if (use_simt(M, w->N, w->K, flags)) {
@@ -379,6 +384,8 @@ static int check_linear_args(const dp_weight* w, const void* x, int64_t ldx, con
     return fail(DP_ERR_INVALID_ARG, "FORCE_SIMT and FORCE_MMA are exclusive");
   if ((flags & DP_FLAG_UNPACK_FIRST) && (flags & DP_FLAG_NO_UNPACK_FIRST))
     return fail(DP_ERR_INVALID_ARG, "UNPACK_FIRST and NO_UNPACK_FIRST are exclusive");
+  if (w->bits == 16 && (s_a_in != nullptr || dbg != nullptr))
+    return fail(DP_ERR_INVALID_ARG, "a 16-bit pass-through layer takes bf16 activations and has no taps");
   if (M == 0) return DP_OK;
   if (!x || !y) return fail(DP_ERR_INVALID_ARG, "x or y is NULL");
   if (ldx < w->K || ldy < w->N) return fail(DP_ERR_SHAPE, "leading dimension smaller than the row");
@@ -392,7 +399,7 @@ static int check_linear_args(const dp_weight* w, const void* x, int64_t ldx, con
       return fail(DP_ERR_ALIGN, "dbg.acc misaligned or too narrow");
   }
   // scratch users: the library's own DAQ, and the int8 copy of the weights of the unpack-first form
-  if (!use_simt(M, w->N, w->K, flags) &&
+  if (w->bits != 16 && !use_simt(M, w->N, w->K, flags) &&
       (s_a_in == nullptr || want_unpack_first(flags, w->bits, false))) {
     const size_t need = dp_wq_linear_workspace(M, w->N, w->K, w->bits, flags);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))
@@ -408,7 +415,7 @@ static int check_linear_args(const dp_weight* w, const void* x, int64_t ldx, con
 using namespace dp;
 
 extern "C" size_t dp_wq_linear_workspace(int64_t M, int32_t N, int32_t K, int32_t bits, uint32_t flags) {
-  if (M <= 0 || K <= 0) return 256;
+  if (M <= 0 || K <= 0 || bits == 16) return 256;
   if (use_simt(M, N, K, flags)) return 256;
   size_t need = align256(scratch_q_bytes(M, K)) + align256(sizeof(float) * static_cast<size_t>(M));
   if (want_unpack_first(flags, bits, true)) need += align256(static_cast<size_t>(N) * K);
@@ -619,7 +626,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
     PlanLayer L;
     L.w = layers[l];
     L.M = M_per_layer[l];
-    L.simt = use_simt(L.M, L.w.N, L.w.K, flags);
+    L.simt = L.w.bits != 16 && use_simt(L.M, L.w.N, L.w.K, flags);
     L.bn = 0;
     L.cg = 1;
     L.ws = 0;
@@ -629,7 +636,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
       delete p;
       return fail(DP_ERR_SHAPE, "layer %d: K too large for the small-M kernel", l);
     }
-    if (!L.simt && L.M > 0) {
+    if (!L.simt && L.M > 0 && L.w.bits != 16) {
       uint32_t lf = flags;  // a pair request that this layer's N cannot honour falls back to the default
       // DAQ inside the GEMM kernel and a DAQ launch that also expands the weights exclude each other
       if ((lf & DP_FLAG_FUSED_DAQ) && !(lf & DP_FLAG_UNPACK_FIRST)) lf |= DP_FLAG_NO_UNPACK_FIRST;
@@ -666,6 +673,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
                                              (flags & ~(DP_FLAG_UNPACK_FIRST | DP_FLAG_NO_UNPACK_FIRST)) |
                                                  (L.pre ? DP_FLAG_UNPACK_FIRST : DP_FLAG_NO_UNPACK_FIRST));
     if (ws > p->workspace_bytes) p->workspace_bytes = ws;
+
     L.x_offset = p->x_bytes;
     p->x_bytes += align256(static_cast<size_t>(L.M) * L.w.K * 2);
     p->layers.push_back(L);
@@ -730,7 +738,7 @@ extern "C" int dp_plan_set_daq(dp_plan* plan, int32_t clip_percentile_e3, int32_
       return fail(DP_ERR_BITS, "dp_plan_set_daq: activation bits %d not in [2, 8]", act_bits_by_bin[b]);
   size_t need = plan->workspace_bytes;
   for (const PlanLayer& L : plan->layers) {
-    if (L.M == 0) continue;
+    if (L.M == 0 || L.w.bits == 16) continue;  // (16-bit pass-through layers have no DAQ)
     const int rank = clip_rank_of(clip_percentile_e3, L.w.K);
     if (rank > 64 || L.w.K > 4608)
       return fail(DP_ERR_SHAPE, "dp_plan_set_daq: a layer with K=%d would need clip rank %d (limits: K <= 4608, rank <= 64)",
@@ -754,7 +762,8 @@ extern "C" int dp_plan_set_layer_flags(dp_plan* plan, int32_t layer, uint32_t fl
                                      DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_UNPACK_FIRST |
                                      DP_FLAG_NO_UNPACK_FIRST | DP_FLAG_ACT_STATIONARY | DP_FLAG_NO_ACT_STATIONARY;
   if (flags & ~kVariantFlags) return fail(DP_ERR_INVALID_ARG, "dp_plan_set_layer_flags: flag bits 0x%x do not name a variant", flags);
-  if (L.simt || L.M == 0) return fail(DP_ERR_INVALID_ARG, "layer %d runs the small-M kernel: it has no variants", layer);
+  if (L.simt || L.M == 0 || L.w.bits == 16)
+    return fail(DP_ERR_INVALID_ARG, "layer %d runs the small-M or the 16-bit kernel: it has no variants", layer);
   if (int st = check_tile_flags(flags, L.w.N)) return st;
   if ((flags & DP_FLAG_WEIGHT_STATIONARY) && !gemm_ws_supported(L.w.N, L.w.K))
     return fail(DP_ERR_SHAPE, "layer %d: the weight-stationary kernel does not take N=%d K=%d", layer, L.w.N, L.w.K);
@@ -867,7 +876,7 @@ static int plan_run_step(dp_plan* plan, int32_t t, const void* const* xs, void* 
     if (!xs[l] || !ys[l]) return fail(DP_ERR_INVALID_ARG, "layer %d: NULL x or y", l);
     if (!aligned16(xs[l]) || !aligned16(ys[l])) return fail(DP_ERR_ALIGN, "layer %d: x/y misaligned", l);
     const CUtensorMap* ta = nullptr;
-    if (!L.simt) {
+    if (!L.simt && L.w.bits != 16) {
       int st = DP_OK;
       ta = cached_tmap_a(plan, workspace, L.M, L.w.K, &st);
       if (st != DP_OK) return st;

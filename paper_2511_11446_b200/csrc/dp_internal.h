@@ -137,6 +137,13 @@ int launch_gemm_ws(const GemmProblem& p, cudaStream_t stream, bool pdl);
 int gemm_init_device(int dev, int* num_sms_out, int* max_pairs_out);
 int gemm_ws_init_device();
 int gemm_as_init_device();
+int gemm_bf16_init_device();
+
+// gemm_bf16.cu -- pass-through linear of 16-bit layers (bf16 x bf16 -> fp32 -> bf16, tcgen05 kind::f16).
+int launch_gemm_bf16(const void* x, int64_t ldx, const void* w, const uint16_t* bias, int64_t M, int32_t N, int32_t K,
+                     uint16_t* y, int64_t ldy, int32_t* status, cudaStream_t stream, bool pdl);
+int gemm_encode_bytes_2d(CUtensorMap* out, const void* base, uint64_t inner_bytes, uint64_t rows, uint64_t pitch_bytes,
+                         uint32_t box_inner, uint32_t box_rows);
 
 // gemm_as.cu -- activation-stationary CTA-pair kernel (K <= 1152, 8-bit weights, tiled activations).
 bool gemm_as_supported(int32_t N, int32_t K);

@@ -380,6 +380,8 @@ int gemm_init_device(int dev, int* num_sms_out, int* max_pairs_out) {
   if (st != DP_OK) return st;
   st = gemm_as_init_device();
   if (st != DP_OK) return st;
+  st = gemm_bf16_init_device();
+  if (st != DP_OK) return st;
   *num_sms_out = sms;
   *max_pairs_out = pairs;
   return DP_OK;
@@ -397,6 +399,13 @@ static int encode_2d(CUtensorMap* out, const void* base, uint64_t inner_bytes, u
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(DP_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
   return DP_OK;
+}
+
+// Any row-major matrix seen as bytes: rows of inner_bytes at pitch_bytes, boxes of box_inner x box_rows
+// bytes, 128-byte swizzle.
+int gemm_encode_bytes_2d(CUtensorMap* out, const void* base, uint64_t inner_bytes, uint64_t rows, uint64_t pitch_bytes,
+                         uint32_t box_inner, uint32_t box_rows) {
+  return encode_2d(out, base, inner_bytes, rows, pitch_bytes, box_inner, box_rows, true);
 }
 
 int gemm_encode_a(CUtensorMap* out, const int8_t* q, int64_t M, int64_t K, int64_t ldq) {

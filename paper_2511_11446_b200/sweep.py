@@ -74,7 +74,7 @@ def time_shape(name, M, K, N, bits, peaks, seed=synth.BASE_SEED + 5, iters=None,
         t = _time(lambda s: B.dp_wq_linear(Ws[s].w, xs[s], K, None, M, ys[s], N, ws, None, status, flags),
                   n_sets, iters)
         out.update(layer_us=t, layer_tops=ops / t / 1e6, layer_gbs=by / t / 1e3, layer_frac=t_ideal / t)
-    if only in (None, "gemm"):
+    if only in (None, "gemm") and bits != 16:
         t = _time(lambda s: B.dp_wq_linear(Ws[s].w, qs[s], K, sas[s], M, ys[s], N, ws, None, status, flags),
                   n_sets, iters)
         out.update(gemm_us=t, gemm_tops=ops / t / 1e6, gemm_frac_int8_peak=ops / t / 1e6 / int8_peak)

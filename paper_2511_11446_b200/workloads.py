@@ -21,8 +21,10 @@ class DevWeights:
 
     def __init__(self, seed, layer, N, K, bits, with_bias=True):
         self.N, self.K, self.bits = N, K, bits
-        w, s_w = synth_cuda.weights(seed, layer, N, K, bits)
-        if bits == 8:
+        w, s_w = synth_cuda.weights(seed, layer, N, K, 8 if bits == 16 else bits)
+        if bits == 16:  # a pass-through layer: the dequantized 8-bit weights, rounded to bf16
+            self.qweight = (w.float() * s_w[:, None]).to(torch.bfloat16)
+        elif bits == 8:
             self.qweight = w
         else:
             packed = B.dp_pack_weights_host(w.cpu().numpy(), bits)
