@@ -54,7 +54,7 @@ gemm_as_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint8_t* sA = smem;                        // [KB][128 tokens][128] int8, 128-byte swizzled: the strip
   uint8_t* sB = sA + kAsMaxKB * A_BYTES;     // weight ring
   float* s_scale = reinterpret_cast<float*>(sB + kAsRingBytes);  // per-warp fp32 copies of weight scales and biases
-  uint64_t* a_full = reinterpret_cast<uint64_t*>(sB + kAsRingBytes + kAsEpiWarps * RowEpilogue::kScaleBytes);  // leader: both CTAs' k-block landed
+  uint64_t* a_full = reinterpret_cast<uint64_t*>(sB + kAsRingBytes + kAsEpiWarps * RowEpilogue<0>::kScaleBytes);  // leader: both CTAs' k-block landed
   uint64_t* w_full = a_full + kAsMaxKB;                                      // leader: both CTAs' stage landed
   uint64_t* w_empty = w_full + kAsMaxStages;                                 // every MMA reading the stage completed
   uint64_t* acc_full = w_empty + kAsMaxStages;
@@ -203,8 +203,8 @@ gemm_as_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   } else {
     // ================= epilogue =================
     const int ew = warp - kEpiWarp0;
-    RowEpilogue epi;
-    epi.init(warp, lane, s_scale + ew * (RowEpilogue::kScaleBytes / 4), map_to_cta(&acc_empty[0], 0),
+    RowEpilogue<0> epi;
+    epi.init(warp, lane, s_scale + ew * (RowEpilogue<0>::kScaleBytes / 4), map_to_cta(&acc_empty[0], 0),
              map_to_cta(&acc_empty[1], 0));
     const int ncols = ap.bns >> 1, col0 = (ew >> 2) * ncols;  // this warp's half of a sub-block's columns
     bool ok = true;
@@ -235,7 +235,7 @@ gemm_as_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 // ---- host side -------------------------------------------------------------------------------------
 constexpr size_t as_smem_bytes() {
   return 1024 + static_cast<size_t>(kAsMaxKB) * BM * BK + kAsRingBytes +
-         kAsEpiWarps * RowEpilogue::kScaleBytes +
+         kAsEpiWarps * RowEpilogue<0>::kScaleBytes +
          (kAsMaxKB + 2 * kAsMaxStages + 5) * 8 + 64;
 }
 

@@ -1,6 +1,6 @@
 // Device-side pieces shared by the tensor-core GEMM kernels of libdiffpro: tile constants, kernel
 // parameters, the in-shared-memory expansion of packed 3/4-bit weight tiles, and the dequant
-// epilogue of one warp (tcgen05.ld -> fp32 sequence -> bf16 -> staged, row-coalesced stores).
+// epilogue of one warp (tcgen05.ld -> fp32 sequence -> bf16 -> 32-byte stores, one token per thread).
 #pragma once
 
 #include <cuda_bf16.h>
@@ -16,9 +16,6 @@ constexpr int kUnpackThreads = kUnpackWarps * 32;
 __host__ __device__ constexpr int gemm_threads(int bits) {
   return (kUnpackWarp0 + (bits == 8 ? 0 : kUnpackWarps)) * 32;
 }
-// Output staging per epilogue warp: 32 tokens x CW bf16 (CW = columns handled per round: 32, or 16
-// where shared memory is short).
-__host__ __device__ constexpr int y_stage_bytes(int cw) { return 32 * cw * 2; }
 constexpr int kSmemBudget = 200 * 1024;
 constexpr int kPStages = 3;
 
@@ -201,185 +198,6 @@ __device__ __forceinline__ void unpack3_tile(const uint8_t* P, uint8_t* B, int t
   }
 }
 
-// ---- epilogue arithmetic -----------------------------------------------------------------------------
-// One output, in this order: t = (float)(acc / 2^SHIFT) (exact scaling), sc = s_a * s_w[n],
-// y = fma(t, sc, bias[n]); the caller rounds pairs to bf16 (nearest even).
-template <int SHIFT>
-__device__ __forceinline__ float dequant_one(uint32_t acc, float sa, float sw, float bias) {
-  float t = __int2float_rn(static_cast<int>(acc));
-  if constexpr (SHIFT != 0) t = __fmul_rn(t, 1.0f / (1 << SHIFT));  // exact: acc is a multiple of 2^SHIFT
-  return __fmaf_rn(t, __fmul_rn(sa, sw), bias);
-}
-
-// ---- the epilogue of one warp ---------------------------------------------------------------------------
-// Eight epilogue warps serve a CTA's 128 x BN accumulator: warp w may read TMEM lanes
-// 32 * (w % 4) .. +31 (its quadrant = 32 tokens); the two warps of a quadrant split the tile's
-// 64-column slabs. Each warp keeps a private copy of the scales and biases of its columns in shared
-// memory (no CTA-wide synchronisation) and a private 32 x 32 bf16 staging tile.
-template <int BN>
-struct EpiLayout {
-  static constexpr int SLABS = BN / 64;             // 64-column slabs per tile
-  static constexpr int SLABS_LO = (SLABS + 1) / 2;  // slabs of the first warp of a quadrant; the rest go to the second
-  static constexpr int ACTIVE = SLABS > 1 ? kEpiWarps : kEpiWarps / 2;  // BN = 64: one warp per quadrant
-  static constexpr int SCALE_FLOATS = kEpiWarps * 64 * SLABS_LO;         // per array (scales, biases)
-};
-
-template <int BN, int SHIFT, int CW = 32>
-struct EpilogueWarp {
-  using L = EpiLayout<BN>;
-  int qd, slab0, slab1, lane, staged_n;
-  float *ts, *tb;
-  const uint4* stage4;
-  uint32_t acc_empty_addr[2];  // (cluster) address of the barrier that collects drained buffers
-
-  __device__ __forceinline__ void init(int warp, int lane_, float* s_scale, float* s_bias, uint8_t* sY,
-                                       uint32_t acc_empty0, uint32_t acc_empty1) {
-    const int ew = warp - kEpiWarp0;
-    lane = lane_;
-    qd = warp & 3;
-    slab0 = ew < 4 ? 0 : L::SLABS_LO;
-    slab1 = ew < 4 ? L::SLABS_LO : L::SLABS;
-    ts = s_scale + ew * 64 * L::SLABS_LO;
-    tb = s_bias + ew * 64 * L::SLABS_LO;
-    uint8_t* stage = sY + ew * y_stage_bytes(CW);
-    stage4 = reinterpret_cast<const uint4*>(stage);
-    acc_empty_addr[0] = acc_empty0;
-    acc_empty_addr[1] = acc_empty1;
-    staged_n = -1;
-  }
-  __device__ __forceinline__ bool active() const { return slab0 < slab1; }
-
-  // One tile: columns n_blk * BN .., this CTA's token rows cta_row0 .. +127; the accumulator sits
-  // at TMEM column t_cols (buffer `buf`), published through acc_full (phase aph). Returns false if
-  // the wait was aborted.
-  __device__ __forceinline__ bool tile(const GemmParams& p, int n_blk, int cta_row0, uint32_t tmem_base,
-                                       uint32_t t_cols, uint64_t* acc_full, uint32_t aph, int buf,
-                                       volatile int* abort_flag) {
-    const int n0 = n_blk * BN;
-    const int row0 = cta_row0 + qd * 32;
-    // Accumulators are read in the fragment layout: this thread owns tokens row0 + r8 + 8 i
-    // (i = 0..3) and, per 32-column chunk, columns 8 j + 2 t4, + 1 (j = 0..3). Owning columns lets
-    // it fetch its scales and biases with plain (non-broadcast) 8-byte shared loads.
-    const int t4 = lane & 3, r8 = lane >> 2;
-    float sa[4];
-    if (p.x == nullptr) {  // scales from an earlier kernel: fetch them while waiting for the accumulator
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int64_t row = static_cast<int64_t>(row0) + r8 + 8 * i;
-        sa[i] = row < p.M ? __ldg(p.s_a + row) : 0.0f;
-      }
-    }
-    if (n_blk != staged_n) {
-      constexpr int NV = 2 * L::SLABS_LO;  // 32-column groups this warp may need
-      float sv[NV], bv[NV];
-#pragma unroll
-      for (int j = 0; j < NV; ++j) {
-        const int col = slab0 * 64 + lane + 32 * j;
-        sv[j] = col < slab1 * 64 ? __ldg(p.s_w + n0 + col) : 0.0f;
-        bv[j] = (col < slab1 * 64 && p.bias != nullptr)
-                    ? __uint_as_float(static_cast<uint32_t>(__ldg(p.bias + n0 + col)) << 16)
-                    : 0.0f;
-      }
-      __syncwarp();
-#pragma unroll
-      for (int j = 0; j < NV; ++j) {
-        ts[lane + 32 * j] = sv[j];
-        tb[lane + 32 * j] = bv[j];
-      }
-      __syncwarp();
-      staged_n = n_blk;
-    }
-    bool ok = mbar_wait(acc_full, aph, abort_flag);
-    ok = __all_sync(0xFFFFFFFFu, ok);
-    if (!ok) return false;
-    tc_fence_after();
-    if (p.x != nullptr) {  // scales written by other CTAs of this kernel: their tile is complete by now
-      (void)ld_acquire_gpu(p.sync + (cta_row0 >> 7));
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int64_t row = static_cast<int64_t>(row0) + r8 + 8 * i;
-        sa[i] = row < p.M ? *reinterpret_cast<const volatile float*>(p.s_a + row) : 0.0f;
-      }
-    }
-    const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + t_cols;
-    uint32_t* stage32 = reinterpret_cast<uint32_t*>(const_cast<uint4*>(stage4));
-    // Rounds of CW columns. Per round the warp reads its two 16-token halves from tensor memory (the
-    // next read is in flight while the current one is converted), writes bf16 pairs into its staging
-    // tile [32 tokens][CW * 2 bytes] and copies the tile out row-wise. The staging tile's 16-byte
-    // chunks are XOR-swizzled by the token index so that both the 4-byte writes and the 16-byte
-    // row-wise read-back are free of bank conflicts.
-    constexpr int G = CW / 8;  // 8-column groups per round = 16-byte chunks per staged row
-    auto swz = [](int rr) { return CW == 32 ? ((rr >> 1) & 3) : ((rr >> 2) & 1); };
-    auto tload = [&](int c, int h, uint32_t (&r)[4 * G]) {
-      const uint32_t addr = t_addr + (static_cast<uint32_t>(16 * h) << 16) + c * CW;
-      if constexpr (G == 4) tmem_ld_16x256b_x4(addr, r);
-      else tmem_ld_16x256b_x2(addr, r);
-    };
-    auto convert = [&](const uint32_t (&r)[4 * G], int c, int h, int lc) {  // tokens r8 + 16 h, r8 + 16 h + 8
-#pragma unroll
-      for (int j = 0; j < G; ++j) {
-        const float2 sw = *reinterpret_cast<const float2*>(ts + lc + 8 * j);
-        const float2 bb = *reinterpret_cast<const float2*>(tb + lc + 8 * j);
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const int rr = r8 + 16 * h + 8 * i;
-          const float s = sa[2 * h + i];
-          const __nv_bfloat162 v = __floats2bfloat162_rn(dequant_one<SHIFT>(r[4 * j + 2 * i], s, sw.x, bb.x),
-                                                         dequant_one<SHIFT>(r[4 * j + 2 * i + 1], s, sw.y, bb.y));
-          stage32[rr * (4 * G) + ((j ^ swz(rr)) << 2) + t4] = *reinterpret_cast<const uint32_t*>(&v);
-        }
-      }
-      if (p.dbg_acc != nullptr) {
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const int64_t row = static_cast<int64_t>(row0) + r8 + 16 * h + 8 * i;
-          if (row < p.M) {
-            int32_t* arow = p.dbg_acc + row * p.dbg_ldacc + n0 + c * CW + 2 * t4;
-#pragma unroll
-            for (int j = 0; j < G; ++j) {
-              arow[8 * j] = static_cast<int>(r[4 * j + 2 * i]) >> SHIFT;
-              arow[8 * j + 1] = static_cast<int>(r[4 * j + 2 * i + 1]) >> SHIFT;
-            }
-          }
-        }
-      }
-    };
-    const int c_begin = (64 / CW) * slab0, c_end = (64 / CW) * slab1;
-    uint32_t ra[4 * G], rb[4 * G];
-    tload(c_begin, 0, ra);
-    for (int c = c_begin; c < c_end; ++c) {
-      const int lc = (c - c_begin) * CW + 2 * t4;  // this thread's first column inside the staged scales
-      tmem_ld_wait();
-      tload(c, 1, rb);
-      convert(ra, c, 0, lc);
-      tmem_ld_wait();
-      if (c + 1 < c_end) {
-        tload(c + 1, 0, ra);
-      } else {  // this warp's last accumulators are in registers: hand the buffer back
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(acc_empty_addr[buf]);
-      }
-      convert(rb, c, 1, lc);
-      __syncwarp();
-      {  // staged round -> global: every store instruction covers whole row segments of CW * 2 bytes
-        const int ch = lane % G;
-        uint16_t* ycol = p.y + n0 + c * CW + ch * 8;
-#pragma unroll
-        for (int it = 0; it < G; ++it) {
-          const int rr = it * (32 / G) + lane / G;
-          const uint4 v = stage4[rr * G + (ch ^ swz(rr))];
-          const int64_t grow = static_cast<int64_t>(row0) + rr;
-          if (grow < p.M) *reinterpret_cast<uint4*>(ycol + grow * p.ldy) = v;
-        }
-      }
-      __syncwarp();  // the staging tile is rewritten by the next round
-    }
-    return true;
-  }
-};
-
-
 // ---- epilogue with one token per thread ---------------------------------------------------------------
 // A warp serves its tensor-memory quadrant (32 tokens, one per thread) over a range of accumulator
 // columns in rounds of 16: tcgen05.ld.32x32b.x16 (the next round's read is in flight while this one
@@ -392,6 +210,7 @@ struct EpilogueWarp {
 // a trip to L2 per round with only ten warps on the SM to hide it. What bounds an epilogue on B200
 // is the chip's store throughput (4.4 TB/s measured: about 15 bytes per clock and SM), then
 // instruction issue; arithmetic does not.
+template <int SHIFT>
 struct RowEpilogue {
   static constexpr int CW = 16;         // columns per round
   static constexpr int kMaxCols = 128;  // columns a warp may own (its private copy of scales and biases)
@@ -418,8 +237,8 @@ struct RowEpilogue {
                                        uint32_t t_col, uint64_t* acc_full, uint32_t aph, int buf,
                                        volatile int* abort_flag) {
     const int64_t row = static_cast<int64_t>(cta_row0) + qd * 32 + lane;
-    const float sa = row < p.M ? __ldg(p.s_a + row) : 0.0f;
-    const uint64_t sa2 = f32x2_pack(sa, sa);
+    float sa = 0.0f;
+    if (p.x == nullptr && row < p.M) sa = __ldg(p.s_a + row);  // from an earlier kernel: fetched while waiting
     if (col != staged_col) {
       float sv[4], bv[4];
 #pragma unroll
@@ -443,6 +262,11 @@ struct RowEpilogue {
     ok = __all_sync(0xFFFFFFFFu, ok);
     if (!ok) return false;
     tc_fence_after();
+    if (p.x != nullptr) {  // scales written by other CTAs of this kernel: their tile is complete by now
+      (void)ld_acquire_gpu(p.sync + (cta_row0 >> 7));
+      if (row < p.M) sa = *reinterpret_cast<const volatile float*>(p.s_a + row);
+    }
+    const uint64_t sa2 = f32x2_pack(sa, sa);
     const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + t_col;
     const float4* sw4 = reinterpret_cast<const float4*>(tsw);
     const float4* tb4 = reinterpret_cast<const float4*>(tbias);
@@ -469,10 +293,15 @@ struct RowEpilogue {
       for (int q = 0; q < 4; ++q) {  // four columns at a time
         const float4 sw = sw4[c * 4 + q];
         const float4 bb = tb4[c * 4 + q];
-        const uint64_t t01 = f32x2_pack(__int2float_rn(static_cast<int>(a[4 * q])),
-                                        __int2float_rn(static_cast<int>(a[4 * q + 1])));
-        const uint64_t t23 = f32x2_pack(__int2float_rn(static_cast<int>(a[4 * q + 2])),
-                                        __int2float_rn(static_cast<int>(a[4 * q + 3])));
+        uint64_t t01 = f32x2_pack(__int2float_rn(static_cast<int>(a[4 * q])),
+                                  __int2float_rn(static_cast<int>(a[4 * q + 1])));
+        uint64_t t23 = f32x2_pack(__int2float_rn(static_cast<int>(a[4 * q + 2])),
+                                  __int2float_rn(static_cast<int>(a[4 * q + 3])));
+        if constexpr (SHIFT != 0) {  // exact: the accumulator is a multiple of 2^SHIFT
+          const uint64_t down = f32x2_pack(1.0f / (1 << SHIFT), 1.0f / (1 << SHIFT));
+          t01 = f32x2_mul(t01, down);
+          t23 = f32x2_mul(t23, down);
+        }
         const uint64_t y01 = f32x2_fma(t01, f32x2_mul(sa2, f32x2_pack(sw.x, sw.y)), f32x2_pack(bb.x, bb.y));
         const uint64_t y23 = f32x2_fma(t23, f32x2_mul(sa2, f32x2_pack(sw.z, sw.w)), f32x2_pack(bb.z, bb.w));
         float y0, y1, y2, y3;
@@ -486,7 +315,7 @@ struct RowEpilogue {
         if (p.dbg_acc != nullptr) {
           int32_t* arow = p.dbg_acc + row * p.dbg_ldacc + col + c * CW;
 #pragma unroll
-          for (int i = 0; i < 16; ++i) arow[i] = static_cast<int>(a[i]);
+          for (int i = 0; i < 16; ++i) arow[i] = static_cast<int>(a[i]) >> SHIFT;
         }
         if (wide) {
           st_global_v8(yrow + c * CW, w);

@@ -14,8 +14,8 @@
 //   warp 1      MMA issuer: tcgen05.mma kind::i8, int32 accumulators in tensor memory (two
 //               accumulator buffers, so a tile's epilogue overlaps the next tile's mainloop)
 //   warps 2-9   epilogue: tcgen05.ld -> (float)acc * s_a[m]*s_w[n] + bias -> bf16 -> global; two warps
-//               per 32-token TMEM quadrant, each taking half of the tile's 64-column slabs, so one
-//               warp's conversion burst overlaps the other's shared-memory and store phases
+//               per 32-token TMEM quadrant, each taking half of the tile's columns, one token per
+//               thread and one 32-byte store per 16 columns
 //   warps 10-17 unpack (3/4-bit only): packed tile in smem -> int8 operand tile in smem, written in
 //               the swizzled layout the MMA descriptor expects, then fence.proxy.async
 //
@@ -50,9 +50,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint8_t* sA = smem;
   uint8_t* sB = sA + NS * A_BYTES;
   uint8_t* sP = sB + NS * B_BYTES;
-  uint8_t* sY = sP + NP * P_BYTES;  // [epilogue warps][32 tokens][64 bytes] output staging
-  uint8_t* tail = sY + kEpiWarps * y_stage_bytes(32);
-  uint64_t* full_a = reinterpret_cast<uint64_t*>(tail);
+  float* s_scale = reinterpret_cast<float*>(sP + NP * P_BYTES);  // per epilogue warp: fp32 copies of its columns' scales, biases
+  uint64_t* full_a = reinterpret_cast<uint64_t*>(s_scale + kEpiWarps * (RowEpilogue<SHIFT>::kScaleBytes / 4));
   uint64_t* bready = full_a + NS;
   uint64_t* empty = bready + NS;
   uint64_t* peer_ready = empty + NS;  // pair leader only: the other CTA's stage is loaded (and expanded)
@@ -62,10 +61,6 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint64_t* acc_empty = acc_full + 2;  // CG = 2: the leader's copy collects both CTAs' epilogue warps
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  using EL = EpiLayout<BN>;
-  float* s_scale = reinterpret_cast<float*>(  // per-warp copies of the tile's weight scales, then biases
-      (reinterpret_cast<uintptr_t>(tmem_slot + 4) + 15) & ~uintptr_t(15));
-  float* s_bias = s_scale + EL::SCALE_FLOATS;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int KB = p.K / BK;
@@ -95,7 +90,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&acc_full[i], 1);
-      mbar_init(&acc_empty[i], CG * EL::ACTIVE);  // one arrival per epilogue warp
+      mbar_init(&acc_empty[i], CG * kEpiWarps);  // one arrival per epilogue warp
     }
     *abort_flag = 0;
     fence_barrier_init();
@@ -262,22 +257,26 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       }
     }
   } else if (warp < kUnpackWarp0) {
-    // ================= epilogue =================
-    EpilogueWarp<BN, SHIFT> epi;
-    epi.init(warp, lane, s_scale, s_bias, sY,
+    // ================= epilogue: quadrant (warp & 3), column half (ew >> 2) =================
+    const int ew = warp - kEpiWarp0;
+    RowEpilogue<SHIFT> epi;
+    epi.init(warp, lane, s_scale + ew * (RowEpilogue<SHIFT>::kScaleBytes / 4),
              CG == 2 ? map_to_cta(&acc_empty[0], 0) : smem_u32(&acc_empty[0]),
              CG == 2 ? map_to_cta(&acc_empty[1], 0) : smem_u32(&acc_empty[1]));
+    constexpr int NCOLS = BN / 2;
+    const int col0 = (ew >> 2) * NCOLS;
     if (p.x != nullptr) {  // quantize this CTA's share of the tokens first (all eight warps)
       if (p.early_w) pdl_wait();  // x comes from the preceding kernel, whose GEMM may still read the scratch
-      daq_phase<PERM>(p, warp - kEpiWarp0, lane);
+      daq_phase<PERM>(p, ew, lane);
     }
-    bool ok = epi.active();
+    bool ok = true;
     int tcount = 0;
-    if (ok && p.early_w && p.x == nullptr) pdl_wait();  // s_a is written by the preceding kernel
+    if (p.early_w && p.x == nullptr) pdl_wait();  // s_a is written by the preceding kernel
     for (int tile = first_tile; tile < total_tiles && ok; tile += tile_stride, ++tcount) {
       const int buf = tcount & 1;
-      ok = epi.tile(p, tile % p.n_tiles, (tile / p.n_tiles) * (BM * CG) + static_cast<int>(rank) * BM,
-                    tmem_base, buf * (TCOLS / 2), &acc_full[buf], (tcount >> 1) & 1, buf, abort_flag);
+      ok = epi.tile(p, (tile % p.n_tiles) * BN + col0, NCOLS,
+                    (tile / p.n_tiles) * (BM * CG) + static_cast<int>(rank) * BM, tmem_base,
+                    buf * (TCOLS / 2) + col0, &acc_full[buf], (tcount >> 1) & 1, buf, abort_flag);
     }
   } else {
     // ================= unpack (3/4-bit weights) =================
@@ -320,8 +319,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 template <int BN, int BITS, int CG>
 constexpr size_t gemm_smem_bytes() {
   return 1024 + static_cast<size_t>(num_stages(BN / CG, BITS)) * ab_stage_bytes(BN / CG) +
-         kPStages * p_stage_bytes(BN / CG, BITS) + kEpiWarps * y_stage_bytes(32) +
-         (4 * 8 + 2 * kPStages + 4) * 8 + 32 + 2 * kEpiWarps * 64 * ((BN / 64 + 1) / 2) * 4 + 64;
+         kPStages * p_stage_bytes(BN / CG, BITS) + kEpiWarps * RowEpilogue<0>::kScaleBytes +
+         (4 * 8 + 2 * kPStages + 4) * 8 + 32 + 64;
 }
 
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

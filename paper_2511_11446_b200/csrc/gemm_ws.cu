@@ -21,10 +21,7 @@ namespace dp {
 
 constexpr int kWsMaxKB = 9;   // k-blocks of 128 a resident strip may have (K <= 1152)
 // Activation ring depth: what is left of shared memory beside the resident strip.
-// At BN = 256 the epilogue works in 16-column rounds (half the staging memory) to make room for a
-// fourth stage.
-__host__ __device__ constexpr int ws_epi_cols(int bn) { return bn >= 256 ? 16 : 32; }
-__host__ __device__ constexpr int ws_stages(int bn) { return bn >= 256 ? 4 : 5; }
+__host__ __device__ constexpr int ws_stages(int bn) { return bn >= 256 ? 4 : 6; }
 
 template <int BN, int BITS, bool PERM>
 __global__ void __launch_bounds__(gemm_threads(BITS), 1)
@@ -42,9 +39,8 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sW = smem;                            // [KB][BNL][128] int8, 128-byte swizzled: the strip
   uint8_t* sA = sW + kWsMaxKB * B_BYTES;         // activation ring (and packed-tile staging)
-  uint8_t* sY = sA + NS * A_BYTES;
-  uint8_t* tail = sY + kEpiWarps * y_stage_bytes(ws_epi_cols(BN));
-  uint64_t* full_a = reinterpret_cast<uint64_t*>(tail);
+  float* s_scale = reinterpret_cast<float*>(sA + NS * A_BYTES);  // per epilogue warp: fp32 copies of scales, biases
+  uint64_t* full_a = reinterpret_cast<uint64_t*>(s_scale + kEpiWarps * (RowEpilogue<SHIFT>::kScaleBytes / 4));
   uint64_t* empty = full_a + NS;
   uint64_t* peer_ready = empty + NS;  // leader only
   uint64_t* pfull = peer_ready + NS;
@@ -56,9 +52,6 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint64_t* w_free = w_peer + 1;       // every MMA that reads the current strip has completed
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(w_free + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  using EL = EpiLayout<BN>;
-  float* s_scale = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(tmem_slot + 4) + 15) & ~uintptr_t(15));
-  float* s_bias = s_scale + EL::SCALE_FLOATS;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int KB = p.K / BK;
@@ -80,7 +73,7 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&acc_full[i], 1);
-      mbar_init(&acc_empty[i], CG * EL::ACTIVE);
+      mbar_init(&acc_empty[i], CG * kEpiWarps);
     }
     mbar_init(w_full, BITS == 8 ? 1 : kUnpackThreads);
     mbar_init(w_peer, 1);
@@ -216,20 +209,24 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       }
     }
   } else if (warp < kUnpackWarp0) {
-    // ================= epilogue =================
-    EpilogueWarp<BN, SHIFT, ws_epi_cols(BN)> epi;
-    epi.init(warp, lane, s_scale, s_bias, sY, map_to_cta(&acc_empty[0], 0), map_to_cta(&acc_empty[1], 0));
+    // ================= epilogue: quadrant (warp & 3), column half (ew >> 2) =================
+    const int ew = warp - kEpiWarp0;
+    RowEpilogue<SHIFT> epi;
+    epi.init(warp, lane, s_scale + ew * (RowEpilogue<SHIFT>::kScaleBytes / 4), map_to_cta(&acc_empty[0], 0),
+             map_to_cta(&acc_empty[1], 0));
+    constexpr int NCOLS = BN / 2;
+    const int col0 = (ew >> 2) * NCOLS;
     if (p.x != nullptr) {  // quantize this CTA's share of the tokens first (all eight warps)
       if (p.early_w) pdl_wait();
-      daq_phase<PERM>(p, warp - kEpiWarp0, lane);
+      daq_phase<PERM>(p, ew, lane);
     }
-    bool ok = epi.active();
+    bool ok = true;
     int tcount = 0;
-    if (ok && p.early_w && p.x == nullptr) pdl_wait();  // s_a is written by the preceding kernel
+    if (p.early_w && p.x == nullptr) pdl_wait();  // s_a is written by the preceding kernel
     for (int item = item0; item < item1 && ok; ++item, ++tcount) {
       const int buf = tcount & 1;
-      ok = epi.tile(p, strip_of(item), mtile_of(item) * (BM * CG) + static_cast<int>(rank) * BM, tmem_base,
-                    buf * (TCOLS / 2), &acc_full[buf], (tcount >> 1) & 1, buf, abort_flag);
+      ok = epi.tile(p, strip_of(item) * BN + col0, NCOLS, mtile_of(item) * (BM * CG) + static_cast<int>(rank) * BM,
+                    tmem_base, buf * (TCOLS / 2) + col0, &acc_full[buf], (tcount >> 1) & 1, buf, abort_flag);
     }
   } else {
     // ================= weight expansion (3/4-bit): once per strip =================
@@ -278,8 +275,8 @@ gemm_ws_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 // ---- host side -------------------------------------------------------------------------------------
 template <int BN>
 constexpr size_t ws_smem_bytes() {
-  return 1024 + static_cast<size_t>(kWsMaxKB) * (BN / 2) * BK + ws_stages(BN) * BM * BK + kEpiWarps * y_stage_bytes(ws_epi_cols(BN)) +
-         (5 * ws_stages(BN) + 4 + 3) * 8 + 32 + 2 * EpiLayout<BN>::SCALE_FLOATS * 4 + 64;
+  return 1024 + static_cast<size_t>(kWsMaxKB) * (BN / 2) * BK + ws_stages(BN) * BM * BK +
+         kEpiWarps * RowEpilogue<0>::kScaleBytes + (5 * ws_stages(BN) + 4 + 3) * 8 + 32 + 64;
 }
 
 template <int BN, int BITS, bool PERM>
