@@ -248,3 +248,23 @@ def linear_bf16(x, w, bias=None):
     lib().orc_linear_bf16(_p(x), _i64(K), _p(w), _p(bias), _i64(M), _i64(N), _i64(K), _p(y), _i64(N), _p(exact),
                           _p(mag))
     return y, exact, mag
+
+
+def wq_linear_grouped(x, qweight, s_w, bias, bits: int, g: int, zeros=None):
+    """Layer with group-wise weight scales: s_w fp32 [N, K/g], zeros uint8 [N, K/g] or None (symmetric).
+    Returns y uint16 [M, N]."""
+    _chk(x, np.uint16, "x")
+    _chk(s_w, np.float32, "s_w")
+    M, K = x.shape
+    N = qweight.shape[0]
+    assert K % g == 0 and s_w.shape == (N, K // g)
+    if zeros is not None:
+        _chk(zeros, np.uint8, "zeros")
+        assert zeros.shape == (N, K // g)
+    y = np.empty((M, N), np.uint16)
+    sw_ = np.empty((N, K), np.int8)
+    sq = np.empty((M, K), np.int8)
+    ssa = np.empty(M, np.float32)
+    lib().orc_wq_linear_grouped(_p(x), _i64(K), _i64(M), _i64(N), _i64(K), C.c_int(bits), _i64(g), _p(qweight),
+                                _p(s_w), _p(zeros), _p(bias), _p(y), _i64(N), _p(sw_), _p(sq), _p(ssa))
+    return y

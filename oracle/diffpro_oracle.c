@@ -26,6 +26,11 @@
  *                  the int32 accumulator; bias add; bf16 output.
  *   orc_wq_linear  the four above in order.
  *   orc_plan_run   Algorithm 2, Phase B: for t in reverse(K*): forward every wrapped linear.
+ *   orc_wq_linear_grouped  Step 2's storage format: group-wise weight scales (one scale, and optionally one
+ *                  zero-point, per output channel and group of g consecutive input channels) in place
+ *                  of one scale per output channel. Reading taken (the paper gives no arithmetic):
+ *                  acc_G = sum over the group of q * (u - z) exactly in int32; t = 0, then for the
+ *                  groups in order t = fma((float)acc_G, s_w[n][G], t); y = bf16(fma(t, s_a[m], bias)).
  *   orc_linear_bf16  the layers a plan keeps in 16-bit precision (Step 1 tiering; Step 2 results): the
  *                  plain linear y = x . W^T + bias on bf16 inputs, summed in double (every product of
  *                  two bf16 values is exact in double), rounded once to bf16.
@@ -316,6 +321,38 @@ void orc_plan_run(const orc_layer* layers, int32_t n_layers, const int32_t* kept
       orc_wq_linear(x_ptrs[(int64_t)i * n_layers + l], L->K, L->M, L->N, L->K, L->bits, L->qweight,
                     L->s_w, L->bias, y_ptrs[(int64_t)i * n_layers + l], L->N, scratch_w, scratch_q,
                     scratch_sa, scratch_acc);
+    }
+}
+
+/* ---- group-wise weight scales (Step 2: "row/group-wise quantization with scale + zero-point") ---- */
+
+/*
+ * x bf16 [M][ldx]; qweight packed per `bits` (offset-binary codes u, as everywhere); group size g
+ * (K % g == 0); s_w fp32 [N][K/g]; zeros uint8 [N][K/g] or NULL (NULL = the symmetric code
+ * z = 2^(bits-1), i.e. w = u - z is the two's-complement value the per-channel path uses);
+ * bias bf16 [N] or NULL -> y bf16 [M][ldy]. Scratch as orc_wq_linear.
+ */
+void orc_wq_linear_grouped(const uint16_t* x, int64_t ldx, int64_t M, int64_t N, int64_t K, int bits, int64_t g,
+                           const void* qweight, const float* s_w, const uint8_t* zeros, const uint16_t* bias,
+                           uint16_t* y, int64_t ldy, int8_t* scratch_w, int8_t* scratch_q, float* scratch_sa) {
+  const int64_t ng = K / g;
+  const int half = 1 << (bits - 1);
+  orc_daq(x, M, K, ldx, scratch_q, K, scratch_sa, 0);
+  orc_unpack(qweight, N, K, bits, scratch_w); /* w = u - 2^(bits-1) */
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t n = 0; n < N; ++n) {
+      float t = 0.0f;
+      for (int64_t G = 0; G < ng; ++G) {
+        int32_t acc = 0;
+        const int z = zeros ? (int)zeros[n * ng + G] : half;
+        for (int64_t k = G * g; k < (G + 1) * g; ++k) {
+          const int u = (int)scratch_w[n * K + k] + half; /* the stored code */
+          acc += (int32_t)scratch_q[m * K + k] * (int32_t)(u - z);
+        }
+        t = fmaf((float)acc, s_w[n * ng + G], t);
+      }
+      y[m * ldy + n] = f32_to_bf16(fmaf(t, scratch_sa[m], bias ? bf16_to_f32(bias[n]) : 0.0f));
     }
 }
 
