@@ -64,16 +64,26 @@ typedef void* dp_stream;
  *               fp32 accumulation and no DAQ; N % 64 == 0.
  * s_w  : fp32 [N], one scale per output channel (Step 5).
  * bias : bf16 [N] or NULL.
+ * Group-wise scales (Step 2: the GPTQ storage format of the paper's plans, groups of 32..288 input
+ * channels with a scale and a zero-point each): group_size = g > 0 (g % 32 == 0, K % g == 0, bits in
+ * {3, 4, 8}, N % 128 == 0) makes s_w fp32 [N][K/g], one scale per output channel and group of g
+ * consecutive k, and `zeros` uint8 [N][K/g] or NULL the zero-points in code units (NULL = 2^(bits-1),
+ * the symmetric code): the weight is s_w[n][k/g] * (u[n][k] - zeros[n][k/g]). The layer is then
+ *     acc_G = sum_{k in group G} q[m,k] * (u[n,k] - z[n,G])            (exact int32)
+ *     t = 0;  for G = 0 .. K/g - 1:  t = fma((float)acc_G, s_w[n][G], t)   (fp32, in this order)
+ *     y = bf16_rne(fma(t, s_a[m], bias[n]))
+ * group_size = 0: one scale per output channel, `zeros` must be NULL.
  * Requirements: K % 128 == 0, N % 16 == 0, N,K >= 128.
  */
 typedef struct dp_weight {
   int32_t N;
   int32_t K;
   int32_t bits;
-  int32_t reserved; /* must be 0 */
+  int32_t group_size; /* 0 = one scale per output channel */
   const void* qweight;
   const float* s_w;
   const void* bias;
+  const void* zeros;  /* group-wise layers only: uint8 [N][K/g] or NULL */
 } dp_weight;
 
 /* Optional taps for tests: any member may be NULL. */
@@ -195,6 +205,11 @@ int32_t dp_clip_rank(int32_t clip_percentile_e3, int32_t K);
  * their scales between the two kernels of the large-M path). Never 0; multiple of 256. */
 size_t dp_wq_linear_workspace(int64_t M, int32_t N, int32_t K, int32_t bits, uint32_t flags);
 
+/* The same for a layer with group-wise scales (w->group_size > 0): such a layer always runs on the
+ * tensor cores, whatever M is, on an int8 copy of its weights, and with zero-points also needs the
+ * tokens' per-group code sums: the bytes for all of that. */
+size_t dp_wq_linear_workspace_grouped(int64_t M, const dp_weight* w);
+
 /*
  * One quantized linear: y[M][N] = dequant( DAQ(x)[M][K] . unpack(w)[N][K]^T ) + bias.
  *   Step 5 / Implementation: INT8 x INT8 -> INT32, per-output-channel weight scale; epilogue
@@ -207,7 +222,8 @@ size_t dp_wq_linear_workspace(int64_t M, int32_t N, int32_t K, int32_t bits, uin
  *   dbg      : NULL or taps (slower path when dbg->acc is set)
  *   device_status : int32 device word or NULL; set to DP_ERR_TIMEOUT by a kernel whose wait expired
  * M == 0 is a no-op. Calls on the same stream are ordered; the workspace may be reused by the
- * next call on that stream. For w->bits == 16 (pass-through layer) x is bf16, s_a_in and dbg must be
+ * next call on that stream. A layer with w->group_size > 0 needs dp_wq_linear_workspace_grouped bytes,
+ * takes bf16 activations only (s_a_in NULL) and has no taps. For w->bits == 16 (pass-through layer) x is bf16, s_a_in and dbg must be
  * NULL, no workspace is used, and the output is bf16_rne(fp32 sum + bias) with the sum accumulated in
  * fp32 on the tensor cores (order unspecified: compare with a tolerance, not bit for bit).
  */

@@ -33,7 +33,7 @@ def DP_FLAG_TILE_N(bn: int) -> int:
 
 DP_STATIC_SCRATCH_BYTES = 10 << 20
 
-EXPORTS = ["dp_daq_quantize", "dp_daq_quantize_robust", "dp_wq_linear_workspace", "dp_wq_linear", "dp_wq_linear_static", "dp_plan_create",
+EXPORTS = ["dp_daq_quantize", "dp_daq_quantize_robust", "dp_wq_linear_workspace", "dp_wq_linear_workspace_grouped", "dp_wq_linear", "dp_wq_linear_static", "dp_plan_create",
            "dp_plan_workspace", "dp_plan_layer_variant", "dp_plan_layer_unpack_first", "dp_plan_set_layer_flags", "dp_plan_set_daq", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
            "dp_plan_run_host", "dp_plan_phase_a", "dp_layer_latency_us", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_clip_rank", "dp_debug_skip_stage_load",
            "dp_status_string",
@@ -41,8 +41,8 @@ EXPORTS = ["dp_daq_quantize", "dp_daq_quantize_robust", "dp_wq_linear_workspace"
 
 
 class dp_weight(C.Structure):
-    _fields_ = [("N", C.c_int32), ("K", C.c_int32), ("bits", C.c_int32), ("reserved", C.c_int32),
-                ("qweight", C.c_void_p), ("s_w", C.c_void_p), ("bias", C.c_void_p)]
+    _fields_ = [("N", C.c_int32), ("K", C.c_int32), ("bits", C.c_int32), ("group_size", C.c_int32),
+                ("qweight", C.c_void_p), ("s_w", C.c_void_p), ("bias", C.c_void_p), ("zeros", C.c_void_p)]
 
 
 class dp_debug(C.Structure):
@@ -76,6 +76,8 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.dp_wq_linear_workspace.restype = C.c_size_t
         L.dp_wq_linear_workspace.argtypes = [C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_uint32]
+        L.dp_wq_linear_workspace_grouped.restype = C.c_size_t
+        L.dp_wq_linear_workspace_grouped.argtypes = [C.c_int64, C.POINTER(dp_weight)]
         L.dp_plan_workspace.restype = C.c_size_t
         L.dp_plan_workspace.argtypes = [C.c_void_p]
         L.dp_plan_layer_variant.argtypes = [C.c_void_p, C.c_int32] + [C.POINTER(C.c_int32)] * 4
@@ -132,9 +134,10 @@ def _check(st, where):
         raise DiffproError(st, where)
 
 
-def make_weight(qweight: torch.Tensor, s_w: torch.Tensor, bias, N: int, K: int, bits: int) -> dp_weight:
-    return dp_weight(N, K, bits, 0, qweight.data_ptr(), s_w.data_ptr(),
-                     None if bias is None else bias.data_ptr())
+def make_weight(qweight: torch.Tensor, s_w: torch.Tensor, bias, N: int, K: int, bits: int, group_size: int = 0,
+                zeros=None) -> dp_weight:
+    return dp_weight(N, K, bits, group_size, qweight.data_ptr(), s_w.data_ptr(),
+                     None if bias is None else bias.data_ptr(), None if zeros is None else zeros.data_ptr())
 
 
 def dp_daq_quantize(x, M, K, ldx, q, ldq, s_a, rowsum=None, stream=None):
@@ -144,6 +147,10 @@ def dp_daq_quantize(x, M, K, ldx, q, ldq, s_a, rowsum=None, stream=None):
 
 def dp_wq_linear_workspace(M, N, K, bits, flags=0) -> int:
     return int(lib().dp_wq_linear_workspace(M, N, K, bits, flags))
+
+
+def dp_wq_linear_workspace_grouped(M, w: dp_weight) -> int:
+    return int(lib().dp_wq_linear_workspace_grouped(M, C.byref(w)))
 
 
 def dp_clip_rank(clip_percentile_e3: int, K: int) -> int:

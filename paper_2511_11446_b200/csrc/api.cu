@@ -195,7 +195,14 @@ static int check_weight(const dp_weight* w) {
     return fail(DP_ERR_SHAPE, "N=%d K=%d: need K %% 128 == 0, N %% 16 == 0", w->N, w->K);
   if (w->bits == 16 && (w->N % 64))
     return fail(DP_ERR_SHAPE, "N=%d: a 16-bit pass-through layer needs N %% 64 == 0", w->N);
-  if (w->reserved != 0) return fail(DP_ERR_INVALID_ARG, "dp_weight.reserved must be 0");
+  if (w->group_size < 0 || (w->group_size == 0 && w->zeros != nullptr))
+    return fail(DP_ERR_INVALID_ARG, "dp_weight: negative group_size, or zero-points without groups");
+  if (w->group_size > 0) {
+    if (w->bits == 16) return fail(DP_ERR_BITS, "a 16-bit pass-through layer has no weight scales, hence no groups");
+    if ((w->group_size % 32) || (w->K % w->group_size) || (w->N % 128))
+      return fail(DP_ERR_SHAPE, "group-wise scales: need g %% 32 == 0, K %% g == 0, N %% 128 == 0 (g=%d K=%d N=%d)",
+                  w->group_size, w->K, w->N);
+  }
   if (!w->qweight || (!w->s_w && w->bits != 16)) return fail(DP_ERR_INVALID_ARG, "dp_weight has a NULL member");
   if (!aligned16(w->qweight) || (reinterpret_cast<uintptr_t>(w->s_w) & 3u) ||
       (w->bias && (reinterpret_cast<uintptr_t>(w->bias) & 1u)))
@@ -218,6 +225,31 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
                             static_cast<uint16_t*>(y), ldy, status, stream, pdl);
   // DAQ policy of a plan (dp_plan_set_daq): clip threshold below the maximum and/or fewer activation bits
   const bool robust = s_a_in == nullptr && (daq_rank > 1 || daq_bits < 8);
+  if (w->group_size > 0) {
+    // Group-wise scales: DAQ into the tiled scratch (packed weights expanded to int8 by the same
+    // launch), the per-group code sums when there are zero-points, then the folding GEMM.
+    uint8_t* ws8 = static_cast<uint8_t*>(workspace);
+    int8_t* wq = static_cast<int8_t*>(workspace);
+    float* wsa = reinterpret_cast<float*>(ws8 + align256(scratch_q_bytes(M, w->K)));
+    size_t off = align256(scratch_q_bytes(M, w->K)) + align256(sizeof(float) * static_cast<size_t>(M));
+    const int8_t* w8 = static_cast<const int8_t*>(w->qweight);
+    UnpackJob job{nullptr, nullptr, 0, 0, 0};
+    if (w->bits < 8) {
+      int8_t* dst = reinterpret_cast<int8_t*>(ws8 + off);
+      off += align256(static_cast<size_t>(w->N) * w->K);
+      job = UnpackJob{static_cast<const uint32_t*>(w->qweight), dst, static_cast<int64_t>(w->N) * w->K / 32, w->bits, 0};
+      w8 = dst;
+    }
+    int32_t* rowsum = w->zeros != nullptr ? reinterpret_cast<int32_t*>(ws8 + off) : nullptr;
+    int st = robust ? launch_daq_robust(x, M, w->K, ldx, wq, w->K, wsa, nullptr, daq_rank, daq_bits, true, stream, pdl,
+                                        w->bits < 8 ? &job : nullptr)
+                    : launch_daq(x, M, w->K, ldx, wq, w->K, wsa, nullptr, KORDER_NATURAL, true, stream, pdl,
+                                 w->bits < 8 ? &job : nullptr);
+    if (st != DP_OK) return st;
+    return launch_gemm_grp(wq, w->K, true, wsa, w8, w->bits, w->group_size, w->s_w, static_cast<const uint8_t*>(w->zeros),
+                           static_cast<const uint16_t*>(w->bias), rowsum, M, w->N, w->K, static_cast<uint16_t*>(y), ldy,
+                           status, stream, pdl);
+  }
   if (use_simt(M, w->N, w->K, flags)) {
     if (static_cast<size_t>(w->K) > simt_max_k())
       return fail(DP_ERR_SHAPE, "K=%d too large for the small-M kernel", w->K);
@@ -386,6 +418,8 @@ static int check_linear_args(const dp_weight* w, const void* x, int64_t ldx, con
     return fail(DP_ERR_INVALID_ARG, "UNPACK_FIRST and NO_UNPACK_FIRST are exclusive");
   if (w->bits == 16 && (s_a_in != nullptr || dbg != nullptr))
     return fail(DP_ERR_INVALID_ARG, "a 16-bit pass-through layer takes bf16 activations and has no taps");
+  if (w->group_size > 0 && (s_a_in != nullptr || dbg != nullptr))
+    return fail(DP_ERR_INVALID_ARG, "a layer with group-wise scales takes bf16 activations and has no taps");
   if (M == 0) return DP_OK;
   if (!x || !y) return fail(DP_ERR_INVALID_ARG, "x or y is NULL");
   if (ldx < w->K || ldy < w->N) return fail(DP_ERR_SHAPE, "leading dimension smaller than the row");
@@ -397,6 +431,12 @@ static int check_linear_args(const dp_weight* w, const void* x, int64_t ldx, con
       return fail(DP_ERR_ALIGN, "dbg.q misaligned or too narrow");
     if (dbg->acc && (dbg->ldacc < w->N || (reinterpret_cast<uintptr_t>(dbg->acc) & 3u)))
       return fail(DP_ERR_ALIGN, "dbg.acc misaligned or too narrow");
+  }
+  if (w->group_size > 0) {
+    const size_t need = dp_wq_linear_workspace_grouped(M, w);
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+      return fail(DP_ERR_WORKSPACE, "workspace needs %zu bytes, 256-byte aligned (got %zu)", need, workspace_bytes);
+    return DP_OK;
   }
   // scratch users: the library's own DAQ, and the int8 copy of the weights of the unpack-first form
   if (w->bits != 16 && !use_simt(M, w->N, w->K, flags) &&
@@ -419,6 +459,14 @@ extern "C" size_t dp_wq_linear_workspace(int64_t M, int32_t N, int32_t K, int32_
   if (use_simt(M, N, K, flags)) return 256;
   size_t need = align256(scratch_q_bytes(M, K)) + align256(sizeof(float) * static_cast<size_t>(M));
   if (want_unpack_first(flags, bits, true)) need += align256(static_cast<size_t>(N) * K);
+  return need;
+}
+
+extern "C" size_t dp_wq_linear_workspace_grouped(int64_t M, const dp_weight* w) {
+  if (!w || M <= 0 || w->K <= 0 || w->group_size <= 0) return 256;
+  size_t need = align256(scratch_q_bytes(M, w->K)) + align256(sizeof(float) * static_cast<size_t>(M));
+  if (w->bits < 8) need += align256(static_cast<size_t>(w->N) * w->K);
+  if (w->zeros != nullptr) need += align256(sizeof(int32_t) * static_cast<size_t>(M) * (w->K / w->group_size));
   return need;
 }
 
@@ -468,7 +516,8 @@ extern "C" int dp_wq_linear_static(const dp_weight* w, const void* x_bf16, int64
   if (!(flags & DP_FLAG_UNPACK_FIRST)) flags |= DP_FLAG_NO_UNPACK_FIRST;
   int st = check_weight(w);
   if (st != DP_OK) return st;
-  const size_t need = dp_wq_linear_workspace(M, w->N, w->K, w->bits, flags);
+  const size_t need = w->group_size > 0 ? dp_wq_linear_workspace_grouped(M, w)
+                                        : dp_wq_linear_workspace(M, w->N, w->K, w->bits, flags);
   if (need > DP_STATIC_SCRATCH_BYTES)
     return fail(DP_ERR_WORKSPACE,
                 "dp_wq_linear_static: M=%lld K=%d needs %zu bytes of scratch, the built-in array holds %u; "
@@ -626,7 +675,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
     PlanLayer L;
     L.w = layers[l];
     L.M = M_per_layer[l];
-    L.simt = L.w.bits != 16 && use_simt(L.M, L.w.N, L.w.K, flags);
+    L.simt = L.w.bits != 16 && L.w.group_size == 0 && use_simt(L.M, L.w.N, L.w.K, flags);
     L.bn = 0;
     L.cg = 1;
     L.ws = 0;
@@ -636,7 +685,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
       delete p;
       return fail(DP_ERR_SHAPE, "layer %d: K too large for the small-M kernel", l);
     }
-    if (!L.simt && L.M > 0 && L.w.bits != 16) {
+    if (!L.simt && L.M > 0 && L.w.bits != 16 && L.w.group_size == 0) {
       uint32_t lf = flags;  // a pair request that this layer's N cannot honour falls back to the default
       // DAQ inside the GEMM kernel and a DAQ launch that also expands the weights exclude each other
       if ((lf & DP_FLAG_FUSED_DAQ) && !(lf & DP_FLAG_UNPACK_FIRST)) lf |= DP_FLAG_NO_UNPACK_FIRST;
@@ -669,9 +718,11 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
         return st;
       }
     }
-    const size_t ws = dp_wq_linear_workspace(L.M, L.w.N, L.w.K, L.w.bits,
-                                             (flags & ~(DP_FLAG_UNPACK_FIRST | DP_FLAG_NO_UNPACK_FIRST)) |
-                                                 (L.pre ? DP_FLAG_UNPACK_FIRST : DP_FLAG_NO_UNPACK_FIRST));
+    const size_t ws = L.w.group_size > 0
+                          ? dp_wq_linear_workspace_grouped(L.M, &L.w)
+                          : dp_wq_linear_workspace(L.M, L.w.N, L.w.K, L.w.bits,
+                                                   (flags & ~(DP_FLAG_UNPACK_FIRST | DP_FLAG_NO_UNPACK_FIRST)) |
+                                                       (L.pre ? DP_FLAG_UNPACK_FIRST : DP_FLAG_NO_UNPACK_FIRST));
     if (ws > p->workspace_bytes) p->workspace_bytes = ws;
 
     L.x_offset = p->x_bytes;
@@ -738,7 +789,7 @@ extern "C" int dp_plan_set_daq(dp_plan* plan, int32_t clip_percentile_e3, int32_
       return fail(DP_ERR_BITS, "dp_plan_set_daq: activation bits %d not in [2, 8]", act_bits_by_bin[b]);
   size_t need = plan->workspace_bytes;
   for (const PlanLayer& L : plan->layers) {
-    if (L.M == 0 || L.w.bits == 16) continue;  // (16-bit pass-through layers have no DAQ)
+    if (L.M == 0 || L.w.bits == 16 || L.w.group_size > 0) continue;  // no DAQ / scratch already sized for any rule
     const int rank = clip_rank_of(clip_percentile_e3, L.w.K);
     if (rank > 64 || L.w.K > 4608)
       return fail(DP_ERR_SHAPE, "dp_plan_set_daq: a layer with K=%d would need clip rank %d (limits: K <= 4608, rank <= 64)",
@@ -762,8 +813,9 @@ extern "C" int dp_plan_set_layer_flags(dp_plan* plan, int32_t layer, uint32_t fl
                                      DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_NO_WEIGHT_STATIONARY | DP_FLAG_UNPACK_FIRST |
                                      DP_FLAG_NO_UNPACK_FIRST | DP_FLAG_ACT_STATIONARY | DP_FLAG_NO_ACT_STATIONARY;
   if (flags & ~kVariantFlags) return fail(DP_ERR_INVALID_ARG, "dp_plan_set_layer_flags: flag bits 0x%x do not name a variant", flags);
-  if (L.simt || L.M == 0 || L.w.bits == 16)
-    return fail(DP_ERR_INVALID_ARG, "layer %d runs the small-M or the 16-bit kernel: it has no variants", layer);
+  if (L.simt || L.M == 0 || L.w.bits == 16 || L.w.group_size > 0)
+    return fail(DP_ERR_INVALID_ARG, "layer %d runs the small-M, the 16-bit or the group-wise kernel: it has no variants",
+                layer);
   if (int st = check_tile_flags(flags, L.w.N)) return st;
   if ((flags & DP_FLAG_WEIGHT_STATIONARY) && !gemm_ws_supported(L.w.N, L.w.K))
     return fail(DP_ERR_SHAPE, "layer %d: the weight-stationary kernel does not take N=%d K=%d", layer, L.w.N, L.w.K);
@@ -876,7 +928,7 @@ static int plan_run_step(dp_plan* plan, int32_t t, const void* const* xs, void* 
     if (!xs[l] || !ys[l]) return fail(DP_ERR_INVALID_ARG, "layer %d: NULL x or y", l);
     if (!aligned16(xs[l]) || !aligned16(ys[l])) return fail(DP_ERR_ALIGN, "layer %d: x/y misaligned", l);
     const CUtensorMap* ta = nullptr;
-    if (!L.simt && L.w.bits != 16) {
+    if (!L.simt && L.w.bits != 16 && L.w.group_size == 0) {
       int st = DP_OK;
       ta = cached_tmap_a(plan, workspace, L.M, L.w.K, &st);
       if (st != DP_OK) return st;
@@ -1079,7 +1131,8 @@ extern "C" int dp_layer_latency_us(const dp_weight* w, int64_t M, uint32_t flags
   cudaStream_t stream = nullptr;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   const size_t xb = static_cast<size_t>(M) * w->K * 2, yb = static_cast<size_t>(M) * w->N * 2;
-  const size_t wb = dp_wq_linear_workspace(M, w->N, w->K, w->bits, flags);
+  const size_t wb = w->group_size > 0 ? dp_wq_linear_workspace_grouped(M, w)
+                                      : dp_wq_linear_workspace(M, w->N, w->K, w->bits, flags);
   cudaError_t e = cudaMalloc(&x, xb);
   if (e == cudaSuccess) e = cudaMalloc(&y, yb);
   if (e == cudaSuccess) e = cudaMalloc(&ws, wb);

@@ -138,6 +138,12 @@ int gemm_init_device(int dev, int* num_sms_out, int* max_pairs_out);
 int gemm_ws_init_device();
 int gemm_as_init_device();
 int gemm_bf16_init_device();
+int gemm_grp_init_device();
+
+// gemm_grp.cu -- layers with group-wise weight scales (and zero-points): folding tensor-core kernel.
+int launch_gemm_grp(const int8_t* q, int64_t ldq, bool a_tiled, const float* s_a, const int8_t* w8, int32_t bits,
+                    int32_t g, const float* s_w, const uint8_t* zeros, const uint16_t* bias, int32_t* rowsum, int64_t M,
+                    int32_t N, int32_t K, uint16_t* y, int64_t ldy, int32_t* status, cudaStream_t stream, bool pdl);
 
 // gemm_bf16.cu -- pass-through linear of 16-bit layers (bf16 x bf16 -> fp32 -> bf16, tcgen05 kind::f16).
 int launch_gemm_bf16(const void* x, int64_t ldx, const void* w, const uint16_t* bias, int64_t M, int32_t N, int32_t K,

@@ -381,6 +381,8 @@ int gemm_init_device(int dev, int* num_sms_out, int* max_pairs_out) {
   if (st != DP_OK) return st;
   st = gemm_bf16_init_device();
   if (st != DP_OK) return st;
+  st = gemm_grp_init_device();
+  if (st != DP_OK) return st;
   *num_sms_out = sms;
   *max_pairs_out = pairs;
   return DP_OK;
