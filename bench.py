@@ -478,6 +478,8 @@ def main():
     ap.add_argument("--only", default=None, choices=["layer", "gemm", "daq"])
     ap.add_argument("--iters", type=int, default=None)
     ap.add_argument("--flags", type=lambda v: int(v, 0), default=0, help="dp_wq_linear tuning flags for --sweep")
+    ap.add_argument("--group", type=int, default=0, help="--sweep with group-wise weight scales of this group size")
+    ap.add_argument("--zero-points", action="store_true", help="--sweep --group with zero-points")
     ap.add_argument("--save-variants", default=None,
                     help="write the per-layer kernel variants the autotuner chose to this JSON file")
     ap.add_argument("--load-variants", default=None,
@@ -503,7 +505,8 @@ def main():
         from paper_2511_11446_b200 import sweep
         torch.cuda.set_device(0)
         sweep.run(args.sweep, [int(b) for b in args.bits.split(",")], measured_peaks(), only=args.only,
-                  layers=args.layers.split(",") if args.layers else None, iters=args.iters, flags=args.flags)
+                  layers=args.layers.split(",") if args.layers else None, iters=args.iters, flags=args.flags,
+                  group=args.group, zeros=args.zero_points)
         return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -274,22 +274,32 @@ gemm_grp_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 
 // Per-group sums of a token's int8 codes, rowsum[m][G] = sum_{k in G} q[m,k] (the zero-point term of the
 // fold), from the tiled scratch the DAQ launch wrote ([row tile][k block][128][128]) or a row-major q.
-__global__ void __launch_bounds__(256)
+// One warp per token: a lane sums 16 consecutive codes per load (a group is a multiple of 32 codes,
+// so the 16 belong to one group) and adds the partial sum to the group's counter in shared memory.
+constexpr int kRowsumWarps = 8, kRowsumMaxGroups = 160;  // K <= 5120 at g = 32
+__global__ void __launch_bounds__(kRowsumWarps * 32)
 group_rowsum_kernel(const int8_t* __restrict__ q, int64_t M, int K, int64_t ldq, int tiled, int g, int ng,
                     int32_t* __restrict__ rowsum) {
+  __shared__ int sums[kRowsumWarps][kRowsumMaxGroups];
   pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t m = static_cast<int64_t>(blockIdx.x) * kRowsumWarps + warp;
+  for (int G = lane; G < ng; G += 32) sums[warp][G] = 0;
+  __syncwarp();
   pdl_wait();
-  const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (idx >= M * ng) return;
-  const int64_t m = idx / ng;
-  const int G = static_cast<int>(idx - m * ng);
-  int sum = 0;
-  for (int k = G * g; k < (G + 1) * g; k += 4) {
+  if (m >= M) return;
+  for (int k = lane * 16; k < K; k += 32 * 16) {
     const int8_t* src = tiled ? q + ((m >> 7) * (K >> 7) + (k >> 7)) * 16384 + (m & 127) * 128 + (k & 127)
                               : q + m * ldq + k;
-    sum = __dp4a(*reinterpret_cast<const int*>(src), 0x01010101, sum);
+    const uint4 v = *reinterpret_cast<const uint4*>(src);
+    int s = __dp4a(static_cast<int>(v.x), 0x01010101, 0);
+    s = __dp4a(static_cast<int>(v.y), 0x01010101, s);
+    s = __dp4a(static_cast<int>(v.z), 0x01010101, s);
+    s = __dp4a(static_cast<int>(v.w), 0x01010101, s);
+    atomicAdd(&sums[warp][k / g], s);
   }
-  rowsum[idx] = sum;
+  __syncwarp();
+  for (int G = lane; G < ng; G += 32) rowsum[m * ng + G] = sums[warp][G];
 }
 
 // ---- host side -------------------------------------------------------------------------------------
@@ -314,9 +324,10 @@ int launch_gemm_grp(const int8_t* q, int64_t ldq, bool a_tiled, const float* s_a
     return fail(DP_ERR_SHAPE, "group-wise layer: need N %% 128 == 0, g %% 32 == 0, K %% g == 0 (N=%d K=%d g=%d)", N, K, g);
   const int ng = K / g;
   if (zeros != nullptr) {
-    const int64_t n = M * ng;
-    const cudaError_t e = launch(group_rowsum_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, stream,
-                                 pdl, q, M, static_cast<int>(K), ldq, a_tiled ? 1 : 0, static_cast<int>(g), ng, rowsum);
+    if (ng > kRowsumMaxGroups) return fail(DP_ERR_SHAPE, "group-wise zero-points: more than %d groups per row", kRowsumMaxGroups);
+    const cudaError_t e = launch(group_rowsum_kernel, dim3(static_cast<unsigned>((M + kRowsumWarps - 1) / kRowsumWarps)),
+                                 dim3(kRowsumWarps * 32), 0, stream, pdl, q, M, static_cast<int>(K), ldq,
+                                 a_tiled ? 1 : 0, static_cast<int>(g), ng, rowsum);
     if (e != cudaSuccess) return fail(DP_ERR_CUDA, "group row-sum launch failed: %s", cudaGetErrorString(e));
   }
   CUtensorMap ta, tw;

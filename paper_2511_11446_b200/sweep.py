@@ -50,6 +50,32 @@ def _time(fn, n_sets, iters, warmup=3):
     return e0.elapsed_time(e1) * 1e3 / iters
 
 
+def time_grouped(name, M, K, N, bits, g, zeros, peaks, seed=synth.BASE_SEED + 5, iters=None):
+    """Whole layer with group-wise weight scales (group size g, optional zero-points), graph-timed like
+    time_shape; the scales are seeded positive numbers (their values do not change the work)."""
+    per_set = 2 * M * K + M * K + 2 * M * N + N * K * bits // 8
+    n_sets = max(2, min(24, -(-2 * L2_BYTES // per_set)))
+    iters = iters or max(10, min(200, int(2e9 // per_set)))
+    iters = -(-iters // n_sets) * n_sets
+    Ws = [DevWeights(seed, s, N, K, bits) for s in range(n_sets)]
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+    sc = [torch.rand((N, K // g), generator=gen, device="cuda") * 1e-2 + 1e-4 for _ in range(n_sets)]
+    zs = [torch.randint(0, 1 << bits, (N, K // g), generator=gen, device="cuda", dtype=torch.uint8) if zeros else None
+          for _ in range(n_sets)]
+    ws_ = [B.make_weight(Ws[s].qweight, sc[s], Ws[s].bias, N, K, bits, g, zs[s]) for s in range(n_sets)]
+    xs = [synth_cuda.activations(seed, s, 0, M, K, 1.0, n_out=max(1, K // 100)) for s in range(n_sets)]
+    ys = [torch.empty((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(n_sets)]
+    ws = torch.empty(B.dp_wq_linear_workspace_grouped(M, ws_[0]), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    t = _time(lambda s: B.dp_wq_linear(ws_[s], xs[s], K, None, M, ys[s], N, ws, None, status, 0), n_sets, iters)
+    assert int(status.item()) == 0, "a kernel reported DP_ERR_TIMEOUT"
+    ops = 2.0 * M * N * K
+    by = alg_bytes(M, K, N, bits) + (4 + (1 if zeros else 0)) * N * (K // g) - 4 * N
+    t_ideal = max(ops / (2.0 * peaks["bf16"] * 1e12), by / (peaks["hbm_gbs"] * 1e9)) * 1e6
+    return {"layer": name, "M": M, "K": K, "N": N, "bits": bits, "group_size": g, "zero_points": bool(zeros),
+            "layer_us": t, "layer_tops": ops / t / 1e6, "ideal_us": t_ideal, "layer_frac": t_ideal / t}
+
+
 def time_shape(name, M, K, N, bits, peaks, seed=synth.BASE_SEED + 5, iters=None, only=None, flags=0):
     per_set = 2 * M * K + M * K + 2 * M * N + N * K * bits // 8
     n_sets = max(2, min(24, -(-2 * L2_BYTES // per_set)))
@@ -86,18 +112,27 @@ def time_shape(name, M, K, N, bits, peaks, seed=synth.BASE_SEED + 5, iters=None,
     return out
 
 
-def run(workload, bits_list, peaks, only=None, layers=None, iters=None, flags=0, emit=print):
+def run(workload, bits_list, peaks, only=None, layers=None, iters=None, flags=0, emit=print, group=0, zeros=False):
     M, batch = WORKLOADS[workload]
     rows = []
     for name, K, N in SHAPES:
         if layers and name not in layers:
             continue
         for bits in bits_list:
+            if group:
+                r = time_grouped(name, M, K, N, bits, group, zeros, peaks, iters=iters)
+                r["workload"] = workload
+                rows.append(r)
+                emit(json.dumps(r))
+                torch.cuda.empty_cache()
+                continue
             r = time_shape(name, M, K, N, bits, peaks, iters=iters, only=only, flags=flags)
             r["workload"] = workload
             rows.append(r)
             emit(json.dumps(r))
             torch.cuda.empty_cache()
+    if group:
+        return rows
     if not layers or "adaln" in layers:
         for bits in bits_list:
             r = time_shape("adaln", batch, synth.HIDDEN, synth.ADALN, bits, peaks, iters=iters, only="layer",
