@@ -230,6 +230,7 @@ def run_ours(args):
         out["mma_i8_peak_tops_measured"] = mma_peak
         out["roofline_hbm_kernels"] = hbm_kernel_rooflines(stack, peaks)
         out["roofline_large_m"] = large_m_rooflines(peaks, mma_peak)
+        out["next_rows"] = next_row_timings(peaks)
         out["e2e"] = e2e(stack, ops_step, world)
         tops, dt, desc, cores = oracle_sample()
         out["cpu_baseline"] = {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
@@ -407,6 +408,23 @@ def large_m_rooflines(peaks, mma_peak):
                          "gemm_tops": r["gemm_tops"], "gemm_frac_of_int8_peak": r["gemm_frac_int8_peak"],
                          "gemm_frac_of_nominal": r["gemm_tops"] / NOMINAL_INT8_TOPS})
     return {"M": 32768, "int8_peak_tops_used": int8_peak, "hbm_gbs_used": peaks["hbm_gbs"], "shapes": rows}
+
+
+def next_row_timings(peaks):
+    """The rows beyond the per-channel W{3,4,8}A8 path, whole layers at M = 2048, graph-timed with
+    operands rotated past L2: group-wise weight scales (Step 2's storage format; g = 128 and 32, 4-bit,
+    with and without zero-points) and 16-bit pass-through layers (bf16, fp32 accumulation; fraction
+    against the measured bf16 tensor rate)."""
+    from paper_2511_11446_b200 import sweep
+    out = {"M": 2048, "grouped": [], "passthrough_bf16": []}
+    for name, K, N in sweep.SHAPES:
+        for g, zp in ((128, False), (128, True), (32, False)):
+            r = sweep.time_grouped(name, 2048, K, N, 4, g, zp, peaks)
+            out["grouped"].append({k: r[k] for k in ("layer", "bits", "group_size", "zero_points", "layer_us", "layer_tops")})
+        r = sweep.time_shape(name, 2048, K, N, 16, peaks, only="layer")
+        out["passthrough_bf16"].append({"layer": name, "layer_us": r["layer_us"], "tflops": r["layer_tops"],
+                                        "frac_of_measured_bf16": r["layer_tops"] / peaks["bf16"]})
+    return out
 
 
 def measure_mma_peak():

@@ -268,3 +268,25 @@ def wq_linear_grouped(x, qweight, s_w, bias, bits: int, g: int, zeros=None):
     lib().orc_wq_linear_grouped(_p(x), _i64(K), _i64(M), _i64(N), _i64(K), C.c_int(bits), _i64(g), _p(qweight),
                                 _p(s_w), _p(zeros), _p(bias), _p(y), _i64(N), _p(sw_), _p(sq), _p(ssa))
     return y
+
+
+def wq_linear_residual(x, qweight, s_w, bias, bits: int, res, gate=None, rows_per_gate: int = 1):
+    """Layer with the residual (and optional per-sample gate) taken into the epilogue. res uint16 [M, N];
+    gate uint16 [ceil(M / rows_per_gate), N] or None. Returns y uint16 [M, N]."""
+    _chk(x, np.uint16, "x")
+    _chk(res, np.uint16, "res")
+    M, K = x.shape
+    N = qweight.shape[0]
+    assert res.shape == (M, N)
+    if gate is not None:
+        _chk(gate, np.uint16, "gate")
+        assert gate.shape == (-(-M // rows_per_gate), N)
+    y = np.empty((M, N), np.uint16)
+    sw_ = np.empty((N, K), np.int8)
+    sq = np.empty((M, K), np.int8)
+    ssa = np.empty(M, np.float32)
+    sacc = np.empty((M, N), np.int32)
+    lib().orc_wq_linear_residual(_p(x), _i64(K), _i64(M), _i64(N), _i64(K), C.c_int(bits), _p(qweight), _p(s_w),
+                                 _p(bias), _p(res), _i64(N), _p(gate), _i64(rows_per_gate), _p(y), _i64(N), _p(sw_),
+                                 _p(sq), _p(ssa), _p(sacc))
+    return y

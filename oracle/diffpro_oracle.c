@@ -31,6 +31,11 @@
  *                  of one scale per output channel. Reading taken (the paper gives no arithmetic):
  *                  acc_G = sum over the group of q * (u - z) exactly in int32; t = 0, then for the
  *                  groups in order t = fma((float)acc_G, s_w[n][G], t); y = bf16(fma(t, s_a[m], bias)).
+ *   orc_wq_linear_residual  the residual connection around a wrapped linear taken into its epilogue
+ *                  (Step 3: residual adds stay in higher precision; a DiT block adds the projection
+ *                  and MLP outputs to its stream scaled by an adaLN gate per sample and channel).
+ *                  Reading: lin = fma((float)acc, s_a*s_w, bias) as in orc_epilogue, then in fp32
+ *                  v = fma(gate, lin, res) (gate given) or v = lin + res, y = bf16(v).
  *   orc_linear_bf16  the layers a plan keeps in 16-bit precision (Step 1 tiering; Step 2 results): the
  *                  plain linear y = x . W^T + bias on bf16 inputs, summed in double (every product of
  *                  two bf16 values is exact in double), rounded once to bf16.
@@ -321,6 +326,32 @@ void orc_plan_run(const orc_layer* layers, int32_t n_layers, const int32_t* kept
       orc_wq_linear(x_ptrs[(int64_t)i * n_layers + l], L->K, L->M, L->N, L->K, L->bits, L->qweight,
                     L->s_w, L->bias, y_ptrs[(int64_t)i * n_layers + l], L->N, scratch_w, scratch_q,
                     scratch_sa, scratch_acc);
+    }
+}
+
+/* ---- residual (and gate) in the epilogue -------------------------------------------------------- */
+
+/*
+ * As orc_wq_linear, then y[m][n] = bf16( gate ? fma(gate[m / rows_per_gate][n], lin, res[m][n]) : lin + res[m][n] )
+ * with lin the fp32 value orc_epilogue rounds to bf16. res bf16 [M][ldr]; gate bf16
+ * [ceil(M / rows_per_gate)][N] or NULL.
+ */
+void orc_wq_linear_residual(const uint16_t* x, int64_t ldx, int64_t M, int64_t N, int64_t K, int bits,
+                            const void* qweight, const float* s_w, const uint16_t* bias, const uint16_t* res,
+                            int64_t ldr, const uint16_t* gate, int64_t rows_per_gate, uint16_t* y, int64_t ldy,
+                            int8_t* scratch_w, int8_t* scratch_q, float* scratch_sa, int32_t* scratch_acc) {
+  orc_daq(x, M, K, ldx, scratch_q, K, scratch_sa, 0);
+  orc_unpack(qweight, N, K, bits, scratch_w);
+  orc_gemm_i32(scratch_q, K, scratch_w, M, N, K, scratch_acc, N);
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t n = 0; n < N; ++n) {
+      const float t = (float)scratch_acc[m * N + n];
+      const float sc = scratch_sa[m] * s_w[n];
+      const float lin = fmaf(t, sc, bias ? bf16_to_f32(bias[n]) : 0.0f);
+      const float r = bf16_to_f32(res[m * ldr + n]);
+      const float v = gate ? fmaf(bf16_to_f32(gate[(m / rows_per_gate) * N + n]), lin, r) : lin + r;
+      y[m * ldy + n] = f32_to_bf16(v);
     }
 }
 
