@@ -414,10 +414,16 @@ def next_row_timings(peaks):
     """The rows beyond the per-channel W{3,4,8}A8 path, whole layers at M = 2048, graph-timed with
     operands rotated past L2: group-wise weight scales (Step 2's storage format; g = 128 and 32, 4-bit,
     with and without zero-points) and 16-bit pass-through layers (bf16, fp32 accumulation; fraction
-    against the measured bf16 tensor rate)."""
+    against the measured bf16 tensor rate), and the gated residual add taken into the epilogue of the two
+    layers that feed the token stream, beside the same layer without it."""
     from paper_2511_11446_b200 import sweep
-    out = {"M": 2048, "grouped": [], "passthrough_bf16": []}
+    out = {"M": 2048, "grouped": [], "passthrough_bf16": [], "gated_residual": []}
     for name, K, N in sweep.SHAPES:
+        if N == 1152:  # the two layers of a DiT block that feed the token stream: proj and fc2
+            r = sweep.time_residual(name, 2048, K, N, 4, peaks)
+            plain = sweep.time_shape(name, 2048, K, N, 4, peaks, only="layer")
+            out["gated_residual"].append({"layer": name, "bits": 4, "layer_us": r["layer_us"],
+                                          "plain_layer_us": plain["layer_us"]})
         for g, zp in ((128, False), (128, True), (32, False)):
             r = sweep.time_grouped(name, 2048, K, N, 4, g, zp, peaks)
             out["grouped"].append({k: r[k] for k in ("layer", "bits", "group_size", "zero_points", "layer_us", "layer_tops")})

@@ -232,6 +232,36 @@ int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_
                  const dp_debug* dbg, int32_t* device_status, uint32_t flags, dp_stream stream);
 
 /*
+ * The residual connection around a wrapped linear, taken into its epilogue (Step 3 keeps residual
+ * adds in higher precision; a DiT block adds its attention projection and MLP output to the token
+ * stream scaled by an adaLN gate per sample and channel). With lin[m][n] the fp32 value that
+ * dp_wq_linear rounds to bf16 (Eq. 3's dequantized output plus bias):
+ *
+ *     y[m][n] = bf16( gate ? fma(gate[m / rows_per_gate][n], lin, residual[m][n]) : lin + residual[m][n] )
+ *
+ * evaluated in fp32 with one rounding to bf16 at the end, so the layer's output never passes through
+ * bf16 before the add and the stream is read and written once instead of three times.
+ */
+typedef struct dp_residual {
+  const void* residual;  /* device: bf16 [M][ldr]; may be the output buffer itself (ldr == ldy): each
+                            element is read before it is overwritten, by the same thread          */
+  int64_t ldr;           /* elements between rows, >= N, multiple of 8; residual 16-byte aligned  */
+  const void* gate;      /* device: bf16 [ceil(M / rows_per_gate)][N], 16-byte aligned, or NULL   */
+  int64_t rows_per_gate; /* tokens that share a gate row (tokens per sample), >= 1; ignored without gate */
+} dp_residual;
+
+/*
+ * dp_wq_linear(w, x_bf16, ldx, NULL, M, ...) with the epilogue above. Per-channel weight scales at
+ * 3, 4 or 8 bits only (DP_ERR_INVALID_ARG for a 16-bit or group-wise layer); always runs a tensor-core
+ * kernel (DP_FLAG_FORCE_SIMT is refused) on int8 operands: packed weights are expanded into the
+ * workspace first (DP_FLAG_UNPACK_FIRST is implied, DP_FLAG_NO_UNPACK_FIRST ignored). Workspace:
+ * dp_wq_linear_workspace(M, N, K, bits, flags | DP_FLAG_FORCE_MMA | DP_FLAG_UNPACK_FIRST). Other arguments, flags and errors as dp_wq_linear.
+ */
+int dp_wq_linear_residual(const dp_weight* w, const void* x_bf16, int64_t ldx, int64_t M, const dp_residual* r,
+                          void* y_bf16, int64_t ldy, void* workspace, size_t workspace_bytes,
+                          int32_t* device_status, uint32_t flags, dp_stream stream);
+
+/*
  * dp_wq_linear for callers that cannot allocate device memory. (The paper has no counterpart: this
  * is a deployment convenience of the library, not a step of the method.)
  *

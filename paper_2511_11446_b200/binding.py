@@ -33,7 +33,7 @@ def DP_FLAG_TILE_N(bn: int) -> int:
 
 DP_STATIC_SCRATCH_BYTES = 10 << 20
 
-EXPORTS = ["dp_daq_quantize", "dp_daq_quantize_robust", "dp_wq_linear_workspace", "dp_wq_linear_workspace_grouped", "dp_wq_linear", "dp_wq_linear_static", "dp_plan_create",
+EXPORTS = ["dp_daq_quantize", "dp_daq_quantize_robust", "dp_wq_linear_workspace", "dp_wq_linear_workspace_grouped", "dp_wq_linear", "dp_wq_linear_static", "dp_wq_linear_residual", "dp_plan_create",
            "dp_plan_workspace", "dp_plan_layer_variant", "dp_plan_layer_unpack_first", "dp_plan_set_layer_flags", "dp_plan_set_daq", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
            "dp_plan_run_host", "dp_plan_phase_a", "dp_layer_latency_us", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_clip_rank", "dp_debug_skip_stage_load",
            "dp_status_string",
@@ -97,6 +97,9 @@ def lib():
         L.dp_wq_linear.argtypes = [C.POINTER(dp_weight), C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                    C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t,
                                    C.POINTER(dp_debug), C.c_void_p, C.c_uint32, C.c_void_p]
+        L.dp_wq_linear_residual.argtypes = [C.POINTER(dp_weight), C.c_void_p, C.c_int64, C.c_int64, C.POINTER(dp_residual),
+                                            C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p, C.c_uint32,
+                                            C.c_void_p]
         L.dp_wq_linear_static.argtypes = [C.POINTER(dp_weight), C.c_void_p, C.c_int64, C.c_int64, C.c_void_p,
                                           C.c_int64, C.c_void_p, C.c_uint32, C.c_void_p]
         L.dp_plan_create.argtypes = [C.POINTER(dp_weight), C.c_int32, C.POINTER(C.c_int64), C.c_uint32,
@@ -173,6 +176,19 @@ def dp_wq_linear(w: dp_weight, x, ldx, s_a_in, M, y, ldy, workspace, dbg: dp_deb
     _check(lib().dp_wq_linear(C.byref(w), _ptr(x), ldx, _ptr(s_a_in), M, _ptr(y), ldy, _ptr(workspace),
                               ws_bytes, None if dbg is None else C.byref(dbg), _ptr(device_status),
                               flags, _stream(stream)), "dp_wq_linear")
+
+
+class dp_residual(C.Structure):
+    _fields_ = [("residual", C.c_void_p), ("ldr", C.c_int64), ("gate", C.c_void_p), ("rows_per_gate", C.c_int64)]
+
+
+def dp_wq_linear_residual(w: dp_weight, x, ldx, M, residual, ldr, gate, rows_per_gate, y, ldy, workspace, ws_bytes,
+                          device_status=None, flags=0, stream=None):
+    """dp_wq_linear on bf16 activations with y = bf16(gate * lin + residual) (gate None: lin + residual)
+    in the epilogue; residual may be y."""
+    r = dp_residual(residual.data_ptr(), ldr, None if gate is None else gate.data_ptr(), rows_per_gate)
+    _check(lib().dp_wq_linear_residual(C.byref(w), _ptr(x), ldx, M, C.byref(r), _ptr(y), ldy, _ptr(workspace),
+                                       ws_bytes, _ptr(device_status), flags, _stream(stream)), "dp_wq_linear_residual")
 
 
 def dp_wq_linear_static(w: dp_weight, x, ldx, M, y, ldy, device_status=None, flags=0, stream=None):

@@ -218,7 +218,7 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
                       void* y, int64_t ldy, void* workspace, const dp_debug* dbg, int32_t* status,
                       uint32_t flags, cudaStream_t stream, const CUtensorMap* tmap_w, int bn, int cg, int ws,
                       const CUtensorMap* tmap_a_cached, bool chained, int32_t* daq_sync = nullptr,
-                      int pre = -1, int daq_rank = 1, int daq_bits = 8) {
+                      int pre = -1, int daq_rank = 1, int daq_bits = 8, const dp_residual* res = nullptr) {
   const bool pdl = !(flags & DP_FLAG_NO_PDL);
   if (w->bits == 16)  // a layer the plan keeps in 16-bit precision: no DAQ, no scales (checked by the caller)
     return launch_gemm_bf16(x, ldx, w->qweight, static_cast<const uint16_t*>(w->bias), M, w->N, w->K,
@@ -293,6 +293,7 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
   // extra CTAs of the DAQ launch) and the 8-bit kernel runs on that copy, instead of every CTA
   // expanding the weight tiles it needs in shared memory.
   if (pre < 0) pre = want_unpack_first(flags, w->bits, s_a_in == nullptr) ? 1 : 0;
+  if (res != nullptr) pre = 1;  // its epilogue is built into the 8-bit streaming kernels
   if (robust) {  // that kernel writes codes in natural k order only: packed layers run on the int8 copy
     pre = 1;
     daq_sync = nullptr;
@@ -380,6 +381,12 @@ static int run_linear(const dp_weight* w, const void* x, int64_t ldx, const floa
   g.ldy = ldy;
   g.dbg_acc = dbg ? dbg->acc : nullptr;
   g.dbg_ldacc = dbg ? dbg->ldacc : 0;
+  if (res != nullptr) {
+    g.res = static_cast<const uint16_t*>(res->residual);
+    g.ldr = res->ldr;
+    g.gate = static_cast<const uint16_t*>(res->gate);
+    g.rows_per_gate = res->gate ? res->rows_per_gate : 1;
+  }
   g.M = M;
   g.N = w->N;
   g.K = w->K;
@@ -480,6 +487,33 @@ extern "C" int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, cons
   if (st != DP_OK) return st;
   return run_linear(w, x, ldx, s_a_in, M, y_bf16, ldy, workspace, dbg, device_status, flags,
                     static_cast<cudaStream_t>(stream), nullptr, 0, 0, 0, nullptr, false);
+}
+
+extern "C" int dp_wq_linear_residual(const dp_weight* w, const void* x_bf16, int64_t ldx, int64_t M,
+                                     const dp_residual* r, void* y_bf16, int64_t ldy, void* workspace,
+                                     size_t workspace_bytes, int32_t* device_status, uint32_t flags,
+                                     dp_stream stream) {
+  if (flags & DP_FLAG_FORCE_SIMT)
+    return fail(DP_ERR_INVALID_ARG, "dp_wq_linear_residual runs tensor-core kernels only");
+  if (flags & (DP_FLAG_WEIGHT_STATIONARY | DP_FLAG_ACT_STATIONARY))
+    return fail(DP_ERR_INVALID_ARG, "dp_wq_linear_residual runs the streaming kernels only");
+  flags = (flags & ~DP_FLAG_NO_UNPACK_FIRST) | DP_FLAG_FORCE_MMA | DP_FLAG_UNPACK_FIRST | DP_FLAG_NO_WEIGHT_STATIONARY |
+          DP_FLAG_NO_ACT_STATIONARY;
+  int st = check_linear_args(w, x_bf16, ldx, nullptr, M, y_bf16, ldy, workspace, workspace_bytes, nullptr, flags);
+  if (st != DP_OK) return st;
+  if (w->bits == 16 || w->group_size > 0)
+    return fail(DP_ERR_INVALID_ARG, "dp_wq_linear_residual takes per-channel layers of 3, 4 or 8 bits");
+  if (!r) return fail(DP_ERR_INVALID_ARG, "dp_residual is NULL");
+  if (M == 0) return DP_OK;
+  if (!r->residual) return fail(DP_ERR_INVALID_ARG, "dp_residual.residual is NULL");
+  if (r->ldr < w->N) return fail(DP_ERR_SHAPE, "dp_residual.ldr smaller than the row");
+  if (!aligned16(r->residual) || (r->ldr % 8) || (r->gate && !aligned16(r->gate)))
+    return fail(DP_ERR_ALIGN, "residual / gate pointers and pitch must be 16-byte aligned");
+  if (r->gate && r->rows_per_gate < 1) return fail(DP_ERR_SHAPE, "rows_per_gate=%lld", (long long)r->rows_per_gate);
+  st = check_device();
+  if (st != DP_OK) return st;
+  return run_linear(w, x_bf16, ldx, nullptr, M, y_bf16, ldy, workspace, nullptr, device_status, flags,
+                    static_cast<cudaStream_t>(stream), nullptr, 0, 0, 0, nullptr, false, nullptr, -1, 1, 8, r);
 }
 
 // ---- the linear for callers that cannot allocate ---------------------------------------------------

@@ -99,6 +99,10 @@ struct GemmProblem {
   int64_t ldy;
   int32_t* dbg_acc;
   int64_t dbg_ldacc;
+  const uint16_t* res = nullptr;  // residual (and gate) taken into the epilogue, see dp_wq_linear_residual
+  int64_t ldr = 0;
+  const uint16_t* gate = nullptr;
+  int64_t rows_per_gate = 1;
   int64_t M;
   int32_t N, K, bits, bn;
   int32_t cg;       // 1: one CTA per 128-row tile; 2: a CTA pair per 256-row tile

@@ -38,6 +38,13 @@ struct GemmParams {
   int64_t ldy;
   int32_t* dbg_acc;
   int64_t dbg_ldacc;
+  // Residual taken into the epilogue (res != nullptr): y = bf16(gate ? fma(gate, lin, res) : lin + res)
+  // in fp32, lin the value otherwise rounded to bf16. res [M][ldr] bf16 (may be y itself); gate
+  // [ceil(M / rows_per_gate)][N] bf16 or nullptr.
+  const uint16_t* res;
+  int64_t ldr;
+  const uint16_t* gate;
+  int64_t rows_per_gate;
   int64_t M;
   int32_t N, K;
   int32_t m_tiles, n_tiles;  // m_tiles counts row tiles of 128 * CG tokens
@@ -233,6 +240,9 @@ struct RowEpilogue {
   // Output columns col .. col + ncols - 1 (col and ncols multiples of 16, ncols at most 128), this
   // CTA's tokens cta_row0 .. +127; their accumulators start at tensor-memory column t_col (buffer
   // `buf`, published on acc_full with phase aph). False if the wait was aborted.
+  // RES: the kernel takes the residual (and gate) of GemmParams into the output; without it those
+  // members are ignored.
+  template <bool RES = false>
   __device__ __forceinline__ bool tile(const GemmParams& p, int col, int ncols, int cta_row0, uint32_t tmem_base,
                                        uint32_t t_col, uint64_t* acc_full, uint32_t aph, int buf,
                                        volatile int* abort_flag) {
@@ -258,6 +268,22 @@ struct RowEpilogue {
       __syncwarp();
       staged_col = col;
     }
+    // Residual and gate of this thread's token, fetched one round ahead of their use (plain loads: the
+    // residual may be the output buffer, whose 32 bytes this thread reads before it overwrites them).
+    const bool has_res = RES && p.res != nullptr && row < p.M;
+    const bool has_gate = has_res && p.gate != nullptr;
+    const uint16_t* rrow = has_res ? p.res + row * p.ldr + col : nullptr;
+    const uint16_t* grow = has_gate ? p.gate + (row / p.rows_per_gate) * p.N + col : nullptr;
+    uint4 rn0 = make_uint4(0, 0, 0, 0), rn1 = rn0, gn0 = rn0, gn1 = rn0;
+    if (has_res) {  // the later rounds' lines on their way into L2 while the accumulators are still being summed
+      for (int b = 128; b < ncols * 2; b += 128) prefetch_l2(reinterpret_cast<const uint8_t*>(rrow) + b);
+      rn0 = ld_global_v4(rrow);
+      rn1 = ld_global_v4(rrow + 8);
+    }
+    if (has_gate) {
+      gn0 = ld_global_v4(grow);
+      gn1 = ld_global_v4(grow + 8);
+    }
     bool ok = mbar_wait(acc_full, aph, abort_flag);
     ok = __all_sync(0xFFFFFFFFu, ok);
     if (!ok) return false;
@@ -277,6 +303,18 @@ struct RowEpilogue {
     uint32_t ra[16];
     tmem_ld_32x16(t_addr, ra);
     for (int c = 0; c < rounds; ++c) {
+      const uint32_t rr[8] = {rn0.x, rn0.y, rn0.z, rn0.w, rn1.x, rn1.y, rn1.z, rn1.w};
+      const uint32_t gg[8] = {gn0.x, gn0.y, gn0.z, gn0.w, gn1.x, gn1.y, gn1.z, gn1.w};
+      if (RES && c + 1 < rounds) {
+        if (has_res) {
+          rn0 = ld_global_v4(rrow + (c + 1) * CW);
+          rn1 = ld_global_v4(rrow + (c + 1) * CW + 8);
+        }
+        if (has_gate) {
+          gn0 = ld_global_v4(grow + (c + 1) * CW);
+          gn1 = ld_global_v4(grow + (c + 1) * CW + 8);
+        }
+      }
       tmem_ld_wait();
       uint32_t a[16];
 #pragma unroll
@@ -307,6 +345,21 @@ struct RowEpilogue {
         float y0, y1, y2, y3;
         f32x2_unpack(y01, y0, y1);
         f32x2_unpack(y23, y2, y3);
+        if (RES && p.res != nullptr) {  // uniform over the grid
+          const float r0 = __uint_as_float(rr[2 * q] << 16), r1 = __uint_as_float(rr[2 * q] & 0xFFFF0000u);
+          const float r2 = __uint_as_float(rr[2 * q + 1] << 16), r3 = __uint_as_float(rr[2 * q + 1] & 0xFFFF0000u);
+          if (p.gate != nullptr) {
+            y0 = fmaf(__uint_as_float(gg[2 * q] << 16), y0, r0);
+            y1 = fmaf(__uint_as_float(gg[2 * q] & 0xFFFF0000u), y1, r1);
+            y2 = fmaf(__uint_as_float(gg[2 * q + 1] << 16), y2, r2);
+            y3 = fmaf(__uint_as_float(gg[2 * q + 1] & 0xFFFF0000u), y3, r3);
+          } else {
+            y0 = __fadd_rn(y0, r0);
+            y1 = __fadd_rn(y1, r1);
+            y2 = __fadd_rn(y2, r2);
+            y3 = __fadd_rn(y3, r3);
+          }
+        }
         const __nv_bfloat162 v01 = __floats2bfloat162_rn(y0, y1), v23 = __floats2bfloat162_rn(y2, y3);
         w[2 * q] = *reinterpret_cast<const uint32_t*>(&v01);
         w[2 * q + 1] = *reinterpret_cast<const uint32_t*>(&v23);

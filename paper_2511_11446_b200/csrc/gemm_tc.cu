@@ -34,7 +34,7 @@
 namespace dp {
 
 // ---- the kernel ----------------------------------------------------------------------------------
-template <int BN, int BITS, bool PERM, int CG>
+template <int BN, int BITS, bool PERM, int CG, bool RES = false>
 __global__ void __launch_bounds__(gemm_threads(BITS), 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                const GemmParams p) {
@@ -274,7 +274,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (p.early_w && p.x == nullptr) pdl_wait();  // s_a is written by the preceding kernel
     for (int tile = first_tile; tile < total_tiles && ok; tile += tile_stride, ++tcount) {
       const int buf = tcount & 1;
-      ok = epi.tile(p, (tile % p.n_tiles) * BN + col0, NCOLS,
+      ok = epi.template tile<RES>(p, (tile % p.n_tiles) * BN + col0, NCOLS,
                     (tile / p.n_tiles) * (BM * CG) + static_cast<int>(rank) * BM, tmem_base,
                     buf * (TCOLS / 2) + col0, &acc_full[buf], (tcount >> 1) & 1, buf, abort_flag);
     }
@@ -331,6 +331,11 @@ static EncodeFn g_encode = nullptr;  // the driver's tensor-map encoder (one per
 
 template <int BN, int BITS, bool PERM, int CG>
 static cudaError_t set_attr() {
+  if constexpr (BITS == 8) {  // the form with a residual in the epilogue exists for 8-bit operands only
+    cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<BN, 8, false, CG, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(gemm_smem_bytes<BN, 8, CG>()));
+    if (e != cudaSuccess) return e;
+  }
   return cudaFuncSetAttribute(gemm_i8_kernel<BN, BITS, PERM, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               static_cast<int>(gemm_smem_bytes<BN, BITS, CG>()));
 }
@@ -461,6 +466,9 @@ static cudaError_t launch_bn(const GemmProblem& g, const GemmParams& p, dim3 gri
   const dim3 block(gemm_threads(g.bits));
   switch (g.bits) {
     case 8:
+      if (g.res != nullptr)
+        return launch_cluster(gemm_i8_kernel<BN, 8, false, CG, true>, grid, block, gemm_smem_bytes<BN, 8, CG>(), stream,
+                              pdl, CG, g.tmap_a, g.tmap_w, p);
       return launch_cluster(gemm_i8_kernel<BN, 8, false, CG>, grid, block, gemm_smem_bytes<BN, 8, CG>(), stream,
                             pdl, CG, g.tmap_a, g.tmap_w, p);
     case 4:
@@ -481,6 +489,7 @@ void gemm_debug_skip_stage_load(int32_t kb) { g_skip_kb = kb < 0 ? -1 : kb; }
 
 int launch_gemm(const GemmProblem& g, cudaStream_t stream, bool pdl) {
   if (g.M == 0) return DP_OK;
+  if (g.res != nullptr && g.bits != 8) return fail(DP_ERR_INVALID_ARG, "residual epilogue: 8-bit operands only");
   const int cg = g.cg == 2 ? 2 : 1;
   GemmParams p;
   if (cg == 1 && g.bits == 8) {
@@ -494,6 +503,10 @@ int launch_gemm(const GemmProblem& g, cudaStream_t stream, bool pdl) {
   p.ldy = g.ldy;
   p.dbg_acc = g.dbg_acc;
   p.dbg_ldacc = g.dbg_ldacc;
+  p.res = g.res;
+  p.ldr = g.ldr;
+  p.gate = g.gate;
+  p.rows_per_gate = g.rows_per_gate;
   p.M = g.M;
   p.N = g.N;
   p.K = g.K;

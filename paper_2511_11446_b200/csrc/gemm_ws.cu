@@ -333,6 +333,10 @@ int launch_gemm_ws(const GemmProblem& g, cudaStream_t stream, bool pdl) {
   p.ldy = g.ldy;
   p.dbg_acc = g.dbg_acc;
   p.dbg_ldacc = g.dbg_ldacc;
+  p.res = nullptr;  // the residual epilogue is built for the streaming kernels only
+  p.ldr = 0;
+  p.gate = nullptr;
+  p.rows_per_gate = 1;
   p.M = g.M;
   p.N = g.N;
   p.K = g.K;

@@ -76,6 +76,31 @@ def time_grouped(name, M, K, N, bits, g, zeros, peaks, seed=synth.BASE_SEED + 5,
             "layer_us": t, "layer_tops": ops / t / 1e6, "ideal_us": t_ideal, "layer_frac": t_ideal / t}
 
 
+def time_residual(name, M, K, N, bits, peaks, rows_per_gate=1024, seed=synth.BASE_SEED + 5, iters=None):
+    """Whole layer with the gated residual in its epilogue (x <- x + gate * layer(h), written over x),
+    graph-timed like time_shape; the stream adds 2*M*N bytes of reads to the layer's algorithmic bytes."""
+    per_set = 2 * M * K + M * K + 4 * M * N + N * K * bits // 8
+    n_sets = max(2, min(24, -(-2 * L2_BYTES // per_set)))
+    iters = iters or max(10, min(200, int(2e9 // per_set)))
+    iters = -(-iters // n_sets) * n_sets
+    Ws = [DevWeights(seed, s, N, K, bits) for s in range(n_sets)]
+    xs = [synth_cuda.activations(seed, s, 0, M, K, 1.0, n_out=max(1, K // 100)) for s in range(n_sets)]
+    rs = [torch.zeros((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(n_sets)]
+    gates = [torch.full((-(-M // rows_per_gate), N), 0.5, dtype=torch.bfloat16, device="cuda") for _ in range(n_sets)]
+    fl = B.DP_FLAG_FORCE_MMA | B.DP_FLAG_UNPACK_FIRST
+    nws = B.dp_wq_linear_workspace(M, N, K, bits, fl)
+    ws = torch.empty(nws, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    t = _time(lambda s: B.dp_wq_linear_residual(Ws[s].w, xs[s], K, M, rs[s], N, gates[s], rows_per_gate, rs[s], N, ws,
+                                                nws, status, 0), n_sets, iters)
+    assert int(status.item()) == 0, "a kernel reported DP_ERR_TIMEOUT"
+    ops = 2.0 * M * N * K
+    by = alg_bytes(M, K, N, bits) + 2 * M * N
+    t_ideal = max(ops / (2.0 * peaks["bf16"] * 1e12), by / (peaks["hbm_gbs"] * 1e9)) * 1e6
+    return {"layer": name, "M": M, "K": K, "N": N, "bits": bits, "layer_us": t, "layer_tops": ops / t / 1e6,
+            "ideal_us": t_ideal, "layer_frac": t_ideal / t}
+
+
 def time_shape(name, M, K, N, bits, peaks, seed=synth.BASE_SEED + 5, iters=None, only=None, flags=0):
     per_set = 2 * M * K + M * K + 2 * M * N + N * K * bits // 8
     n_sets = max(2, min(24, -(-2 * L2_BYTES // per_set)))
