@@ -71,22 +71,59 @@ __device__ __forceinline__ void fetch_unit(const uint32_t* __restrict__ row, int
   }
 }
 
-// Token `warp` of this CTA -> int8 in shared memory, by one warp (rows `pitch` bytes apart), and
-// its scale: DAQ here (Step 3, Eq. "daq"), or a copy when the caller passes quantized tokens.
+// Order in which a token's codes are laid out in shared memory for the matrix-instruction form. The
+// contraction may visit k in any order as long as both operands agree, so the activations take the
+// order in which cheap mask operations leave the weight codes of a packed unit:
+//   ORDER_NATURAL  k ascending (8-bit weights, and the CUDA-core form);
+//   ORDER_NIBBLE   within every 8 codes the even positions first, then the odd ones (4-bit: the low
+//                  and the high nibbles of a packed word);
+//   ORDER_PERIOD   within every 32 codes, word c (c = 0..7) holds positions c, 8 + c, 16 + c, 24 + c
+//                  (3-bit: the fields at the same place of the four 3-byte periods of a packed unit).
+enum { ORDER_NATURAL = 0, ORDER_NIBBLE = 1, ORDER_PERIOD = 2 };
+
+template <int ORDER>
+__device__ __forceinline__ void store_codes(int8_t* row, const int i, const uint2 v) {
+  if constexpr (ORDER == ORDER_NATURAL) {
+    reinterpret_cast<uint2*>(row)[i] = v;
+  } else if constexpr (ORDER == ORDER_NIBBLE) {
+    reinterpret_cast<uint2*>(row)[i] = make_uint2(__byte_perm(v.x, v.y, 0x6420), __byte_perm(v.x, v.y, 0x7531));
+  } else {  // codes 8p .. 8p + 7 of a unit go to byte p of its eight words
+    uint8_t* unit = reinterpret_cast<uint8_t*>(row) + (i >> 2) * 32 + (i & 3);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      unit[4 * c] = static_cast<uint8_t>(v.x >> (8 * c));
+      unit[4 * (c + 4)] = static_cast<uint8_t>(v.y >> (8 * c));
+    }
+  }
+}
+
+// Token `warp` of this CTA -> int8 in shared memory, by one warp (rows `pitch` bytes apart), its
+// scale and (srs != nullptr) the sum of its codes: DAQ here (Step 3, Eq. "daq"), or a copy when the
+// caller passes quantized tokens.
+template <int ORDER = ORDER_NATURAL>
 __device__ __forceinline__ void stage_tokens(const SimtArgs& a, const int64_t m0, const int block_x,
-                                             int8_t* sq, const int pitch, float* ssa, const int warp) {
+                                             int8_t* sq, const int pitch, float* ssa, const int warp,
+                                             int* srs = nullptr) {
   const int lane = threadIdx.x & 31;
   const int K = a.K;
   {
     const int64_t row = m0 + warp;
-    uint2* dst = reinterpret_cast<uint2*>(sq + warp * pitch);
+    int8_t* dst = sq + warp * pitch;
     const int nvec = K >> 3;
+    const bool tap_q = block_x == 0 && row < a.M && a.dbg_q != nullptr;  // optional taps, written once per token
+    uint2* dq = tap_q ? reinterpret_cast<uint2*>(a.dbg_q + row * a.dbg_ldq) : nullptr;
+    int sum = 0;
     if (row >= a.M) {
-      for (int i = lane; i < nvec; i += 32) dst[i] = make_uint2(0, 0);
+      for (int i = lane; i < nvec; i += 32) reinterpret_cast<uint2*>(dst)[i] = make_uint2(0, 0);
       if (lane == 0) ssa[warp] = 0.0f;
     } else if (a.s_a_in != nullptr) {
       const uint2* src = reinterpret_cast<const uint2*>(static_cast<const int8_t*>(a.x) + row * a.ldx);
-      for (int i = lane; i < nvec; i += 32) dst[i] = src[i];
+      for (int i = lane; i < nvec; i += 32) {
+        const uint2 v = src[i];
+        sum = __dp4a(static_cast<int>(v.x), 0x01010101, __dp4a(static_cast<int>(v.y), 0x01010101, sum));
+        store_codes<ORDER>(dst, i, v);
+        if (tap_q) dq[i] = v;
+      }
       if (lane == 0) ssa[warp] = a.s_a_in[row];
     } else {
       const uint4* xr = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(a.x) + row * a.ldx);
@@ -120,19 +157,20 @@ __device__ __forceinline__ void stage_tokens(const SimtArgs& a, const int64_t m0
           b[2 * j + 1] =
               __float_as_uint(__fmaf_rn(__uint_as_float(in[j] & 0xFFFF0000u), inv, magic)) & 0xFFu;
         }
-        dst[i] = make_uint2(b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24),
-                            b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24));
+        const uint2 w = make_uint2(b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24),
+                                   b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24));
+        sum = __dp4a(static_cast<int>(w.x), 0x01010101, __dp4a(static_cast<int>(w.y), 0x01010101, sum));
+        store_codes<ORDER>(dst, i, w);
+        if (tap_q) dq[i] = w;
       }
       if (lane == 0) ssa[warp] = sc;
     }
-    if (block_x == 0 && row < a.M) {  // optional taps, written once per token
-      if (a.dbg_sa != nullptr && lane == 0) a.dbg_sa[row] = ssa[warp];
-      if (a.dbg_q != nullptr) {
-        __syncwarp();
-        uint2* dq = reinterpret_cast<uint2*>(a.dbg_q + row * a.dbg_ldq);
-        for (int i = lane; i < nvec; i += 32) dq[i] = dst[i];
-      }
+    if (srs != nullptr) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+      if (lane == 0) srs[warp] = sum;
     }
+    if (block_x == 0 && row < a.M && a.dbg_sa != nullptr && lane == 0) a.dbg_sa[row] = ssa[warp];
   }
 }
 
@@ -243,41 +281,13 @@ __device__ __forceinline__ void mma_m16n8k32_s8(int (&c)[4], uint32_t a0, uint32
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Packed unit -> 8 words of 4 int8 holding w * 2^(8 - BITS) (the code, sign bit flipped, in the top
-// bits of its byte), k ascending: cheaper than true values, and the int32 sums come out as exact
-// multiples of 2^(8 - BITS) that the epilogue shifts back.
-template <int BITS>
-__device__ __forceinline__ void expand_unit_top(const uint32_t (&pk)[BITS], uint32_t (&w)[8]) {
-  if constexpr (BITS == 8) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) w[i] = pk[i];
-  } else if constexpr (BITS == 4) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint32_t v = pk[i] ^ 0x88888888u;
-      const uint32_t lo = (v << 4) & 0xF0F0F0F0u, hi = v & 0xF0F0F0F0u;
-      w[2 * i] = __byte_perm(lo, hi, 0x5140);
-      w[2 * i + 1] = __byte_perm(lo, hi, 0x7362);
-    }
-  } else {
-    // sign bits (bit 2 of every 3-bit field of the 96-bit unit) flipped first
-    const uint32_t p0 = pk[0] ^ 0x24924924u, p1 = pk[1] ^ 0x49249249u, p2 = pk[2] ^ 0x92492492u;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int bit = 12 * j;  // the word's four fields start here
-      uint32_t x;
-      if (bit == 0) x = p0;
-      else if (bit < 24) x = p0 >> bit;
-      else if (bit < 32) x = __funnelshift_r(p0, p1, bit);
-      else if (bit < 56) x = p1 >> (bit - 32);
-      else if (bit < 64) x = __funnelshift_r(p1, p2, bit - 32);
-      else x = p2 >> (bit - 64);
-      // fields 0, 2 and fields 1, 3 move to the tops of their bytes by one multiplication each
-      // (the two shifted copies inside a product do not overlap, so nothing carries)
-      const uint32_t e = (x & 0x1C7u) * 0x8020u, o = (x & 0xE38u) * 0x100400u;
-      w[j] = (e & 0x00E000E0u) | (o & 0xE000E000u);
-    }
-  }
+// The same with unsigned 8-bit B (weight) operands.
+__device__ __forceinline__ void mma_m16n8k32_s8u8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                  uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.u8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+               "{%0, %1, %2, %3};"
+               : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 // Packed unit `unit` of a staged weight row.
@@ -318,7 +328,8 @@ __device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block
   int8_t* sq = reinterpret_cast<int8_t*>(smem);                             // [kMmaRows][qpitch]
   float* ssa = reinterpret_cast<float*>(smem + kMmaRows * qpitch);          // [kMmaRows]
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ssa + kMmaRows);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ssa + kMmaRows + 4);         // [kMmaWarps][kMmaMaxStages]
+  int* srs = reinterpret_cast<int*>(ssa + kMmaRows + 4);                    // [kMmaRows] sums of the tokens' codes
+  uint64_t* bars = reinterpret_cast<uint64_t*>(srs + kMmaRows);             // [kMmaWarps][kMmaMaxStages]
   uint8_t* ring = reinterpret_cast<uint8_t*>(bars + kMmaWarps * kMmaMaxStages);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -354,21 +365,22 @@ __device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block
   int f_it = 0, f_c = 0, f_blk = blk0, f_s = 0;
   auto issue = [&]() {
     if (f_it < total) {
-      if (lane == 0) {
-        const uint8_t* src = wbase + static_cast<int64_t>(f_blk) * kMmaCh * rowbytes;
-        uint8_t* dst = myring + f_s * stage;
-
-        if constexpr (BITS < 8) {
+      const uint8_t* src = wbase + static_cast<int64_t>(f_blk) * kMmaCh * rowbytes;
+      uint8_t* dst = myring + f_s * stage;
+      if constexpr (BITS < 8) {
+        if (lane == 0) {
           const uint32_t bytes = static_cast<uint32_t>(kMmaCh * rowbytes);
           mbar_arrive_expect_tx(&bar[f_s], bytes);
           bulk_load_1d(dst, src, bytes, &bar[f_s]);
-        } else {
-          const uint32_t bytes = static_cast<uint32_t>(min(CJ, kj - f_c * CJ) * 128);
-          mbar_arrive_expect_tx(&bar[f_s], kMmaCh * bytes);
-          src += f_c * (CJ * 128);
-#pragma unroll
-          for (int r = 0; r < kMmaCh; ++r) bulk_load_1d(dst + r * kMmaPitch8, src + r * rowbytes, bytes, &bar[f_s]);
         }
+      } else {
+        // one copy per row: issued by eight lanes at once (a bulk copy costs its issuing thread
+        // 115-280 cycles; in sequence that was the longest phase of an 8-bit stage)
+        const uint32_t bytes = static_cast<uint32_t>(min(CJ, kj - f_c * CJ) * 128);
+        if (lane == 0) mbar_arrive_expect_tx(&bar[f_s], kMmaCh * bytes);
+        __syncwarp();
+        if (lane < kMmaCh)
+          bulk_load_1d(dst + lane * kMmaPitch8, src + f_c * (CJ * 128) + lane * rowbytes, bytes, &bar[f_s]);
       }
       ++f_it;
       if (++f_s == S) f_s = 0;
@@ -378,15 +390,18 @@ __device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block
 #pragma unroll 1
   for (int s = 0; s < S; ++s) issue();  // in flight across the prologue
   if (a.early_w) pdl_wait();
+  constexpr int ORDER = BITS == 4 ? ORDER_NIBBLE : BITS == 3 ? ORDER_PERIOD : ORDER_NATURAL;
   for (int r = warp; r < (two ? kMmaRows : kMmaRows / 2); r += kMmaWarps)
-    stage_tokens(a, m0, block_x, sq, qpitch, ssa, r);
+    stage_tokens<ORDER>(a, m0, block_x, sq, qpitch, ssa, r, srs);
   __syncthreads();
 
-  // Four accumulator sets, one per matrix instruction of a unit: consecutive instructions never
-  // wait on each other's results.
-  int c[4][4];
+  // One accumulator set per matrix instruction of a unit: consecutive instructions never wait on each
+  // other's results. For packed weights the sets also differ in the power of two their operands
+  // carry (see unit_step).
+  constexpr int NC = BITS == 3 ? 5 : 4;
+  int c[NC][4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) c[i][0] = c[i][1] = c[i][2] = c[i][3] = 0;
+  for (int i = 0; i < NC; ++i) c[i][0] = c[i][1] = c[i][2] = c[i][3] = 0;
   int c_c = 0, c_blk = blk0, st = 0;
   uint32_t ph = 0;
   const int8_t* qrow = sq + g * qpitch + t * 32;
@@ -400,8 +415,13 @@ __device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block
         const int tok = g + 8 * h;
         const int64_t row = m0 + tok;
         if (row < a.M) {
-          const int i = 2 * h + e;  // exact shift: the sum is a multiple of 2^(8 - BITS)
-          const int mine = (c[0][i] + c[1][i] + c[2][i] + c[3][i]) >> (8 - BITS);
+          const int i = 2 * h + e;
+          // Packed weights enter as unsigned fields u = w + 2^(BITS-1), each set carrying its power of
+          // two (the shifts are exact), so the sum of the tokens' codes comes off at the end.
+          int mine;
+          if constexpr (BITS == 8) mine = c[0][i] + c[1][i] + c[2][i] + c[3][i];
+          else if constexpr (BITS == 4) mine = c[0][i] + c[1][i] + ((c[2][i] + c[3][i]) >> 4) - 8 * srs[tok];
+          else mine = c[0][i] + c[1][i] + (c[2][i] >> 2) + (c[3][i] >> 4) + (c[4][i] >> 5) - 4 * srs[tok];
           const float y = __fmaf_rn(static_cast<float>(mine), __fmul_rn(ssa[tok], sw[e]), bs[e]);
           a.y[row * a.ldy + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
           if (a.dbg_acc != nullptr) a.dbg_acc[row * a.dbg_ldacc + n] = mine;
@@ -409,19 +429,54 @@ __device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block
       }
     }
   };
-  // One unit of the staged chunk against tokens g (and g + 8 when TWO).
+  // One unit (32 codes of this lane's channel) of the staged chunk against tokens g (and g + 8 when
+  // TWO). qu: the unit's 32 activation codes of token g in the k order of this bit width.
   auto unit_step = [&](const uint8_t* srow, const int8_t* qu, const int u, auto two_tag) {
     constexpr bool TWO = decltype(two_tag)::value;
-    uint32_t pk[BITS], w[8];
+    const uint4 l0 = *reinterpret_cast<const uint4*>(qu), l1 = *reinterpret_cast<const uint4*>(qu + 16);
+    uint4 h0 = make_uint4(0u, 0u, 0u, 0u), h1 = h0;
+    if constexpr (TWO) {
+      h0 = *reinterpret_cast<const uint4*>(qu + 8 * qpitch);
+      h1 = *reinterpret_cast<const uint4*>(qu + 8 * qpitch + 16);
+    }
+    uint32_t pk[BITS];
     stage_unit<BITS>(srow, u, pk);
-    expand_unit_top<BITS>(pk, w);
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const uint4 lo = *reinterpret_cast<const uint4*>(qu + 16 * h);
-      uint4 hi = make_uint4(0u, 0u, 0u, 0u);
-      if constexpr (TWO) hi = *reinterpret_cast<const uint4*>(qu + 8 * qpitch + 16 * h);
-      mma_m16n8k32_s8(c[2 * h], lo.x, hi.x, lo.y, hi.y, w[4 * h], w[4 * h + 1]);
-      mma_m16n8k32_s8(c[2 * h + 1], lo.z, hi.z, lo.w, hi.w, w[4 * h + 2], w[4 * h + 3]);
+    if constexpr (BITS == 8) {
+      mma_m16n8k32_s8(c[0], l0.x, h0.x, l0.y, h0.y, pk[0], pk[1]);
+      mma_m16n8k32_s8(c[1], l0.z, h0.z, l0.w, h0.w, pk[2], pk[3]);
+      mma_m16n8k32_s8(c[2], l1.x, h1.x, l1.y, h1.y, pk[4], pk[5]);
+      mma_m16n8k32_s8(c[3], l1.z, h1.z, l1.w, h1.w, pk[6], pk[7]);
+    } else if constexpr (BITS == 4) {
+      // A packed word's low nibbles are its even codes, its high nibbles its odd codes times 16: one
+      // mask each, no shifts. Activation words (ORDER_NIBBLE): even, odd codes of word 0, of word 1, ...
+      constexpr uint32_t LO = 0x0F0F0F0Fu, HI = 0xF0F0F0F0u;
+      mma_m16n8k32_s8u8(c[0], l0.x, h0.x, l0.z, h0.z, pk[0] & LO, pk[1] & LO);
+      mma_m16n8k32_s8u8(c[1], l1.x, h1.x, l1.z, h1.z, pk[2] & LO, pk[3] & LO);
+      mma_m16n8k32_s8u8(c[2], l0.y, h0.y, l0.w, h0.w, pk[0] & HI, pk[1] & HI);
+      mma_m16n8k32_s8u8(c[3], l1.y, h1.y, l1.w, h1.w, pk[2] & HI, pk[3] & HI);
+    } else {
+      // The 96-bit unit is four periods of three bytes, eight codes each. r0, r1, r2 collect the
+      // periods' first, second, third bytes; then the field of code class j (codes j, 8 + j, 16 + j,
+      // 24 + j: activation word j under ORDER_PERIOD) sits at the same bits of every byte:
+      //   r0: class 0 bits 0-2, class 1 bits 3-5, class 2 (low two bits) bits 6-7
+      //   r1: class 2 (high bit) bit 0, class 3 bits 1-3, class 4 bits 4-6, class 5 (low bit) bit 7
+      //   r2: class 5 (high two bits) bits 0-1, class 6 bits 2-4, class 7 bits 5-7
+      // Masked (and moved by a bit or two where that makes two fields carry the same power of two),
+      // each field is an unsigned operand byte worth its true value times 1, 4, 16 or 32; the two
+      // parts of the straddling classes 2 and 5 are separate operands against the same activations.
+      const uint32_t x0 = __byte_perm(pk[0], pk[1], 0x0630), x1 = __byte_perm(pk[0], pk[1], 0x0741),
+                     x2 = __byte_perm(pk[0], pk[1], 0x0052);
+      const uint32_t r0 = __byte_perm(x0, pk[2], 0x5210), r1 = __byte_perm(x1, pk[2], 0x6210),
+                     r2 = __byte_perm(x2, pk[2], 0x7410);
+      // times 1: class 0 | high bit of class 2 (worth 4);  low bit of class 5 | its high bits (worth 2)
+      mma_m16n8k32_s8u8(c[0], l0.x, h0.x, l0.z, h0.z, r0 & 0x07070707u, (r1 & 0x01010101u) << 2);
+      mma_m16n8k32_s8u8(c[1], l1.y, h1.y, l1.y, h1.y, (r1 >> 7) & 0x01010101u, (r2 & 0x03030303u) << 1);
+      // times 4: class 3 (moved up one bit) | class 6
+      mma_m16n8k32_s8u8(c[2], l0.w, h0.w, l1.z, h1.z, (r1 & 0x0E0E0E0Eu) << 1, r2 & 0x1C1C1C1Cu);
+      // times 16: class 1 (moved up one bit) | class 4
+      mma_m16n8k32_s8u8(c[3], l0.y, h0.y, l1.x, h1.x, (r0 & 0x38383838u) << 1, r1 & 0x70707070u);
+      // times 32: class 7 | low bits of class 2 (moved down one bit)
+      mma_m16n8k32_s8u8(c[4], l1.w, h1.w, l0.z, h0.z, r2 & 0xE0E0E0E0u, (r0 & 0xC0C0C0C0u) >> 1);
     }
   };
   int it = 0;
@@ -455,7 +510,7 @@ __device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block
     if (++c_c == nc) {
       epilogue();
 #pragma unroll
-      for (int i = 0; i < 4; ++i) c[i][0] = c[i][1] = c[i][2] = c[i][3] = 0;
+      for (int i = 0; i < NC; ++i) c[i][0] = c[i][1] = c[i][2] = c[i][3] = 0;
       c_c = 0;
       c_blk += stride;
     }
@@ -561,7 +616,7 @@ simt_group_kernel(SimtGroupArgs g) {
 static bool simt_use_mma(int32_t K) { return K <= kMmaMaxK; }
 static size_t simt_smem_bytes(int32_t K) {
   if (!simt_use_mma(K)) return static_cast<size_t>(kSimtRows) * K + kSimtRows * sizeof(float);
-  return static_cast<size_t>(kMmaRows) * (K + 16) + kMmaRows * sizeof(float) + 16 +
+  return static_cast<size_t>(kMmaRows) * (K + 16) + kMmaRows * sizeof(float) + 16 + kMmaRows * sizeof(int) +
          sizeof(uint64_t) * kMmaWarps * kMmaMaxStages + static_cast<size_t>(kMmaWarps) * kMmaRingBytes;
 }
 
