@@ -941,9 +941,14 @@ static int plan_run_step(dp_plan* plan, int32_t t, const void* const* xs, void* 
     ga.status = status;
     ga.daq_rank = robust ? clip_rank_of(plan->daq_p_e3, G.w.K) : 1;
     ga.daq_bits = act_bits;
-    ga.q_scratch = static_cast<int8_t*>(workspace);
-    ga.sa_scratch = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) +
-                                             align256(static_cast<size_t>(ga.n_layers) * ga.M * ga.K));
+    // Plain DAQ runs inside the grouped kernel: every CTA quantizes its layer's few tokens while its
+    // first weight copies are in flight (a separate quantization launch in front cost a kernel
+    // boundary and a DRAM round trip, 6-8 us of a 35 us group). The percentile / a-bit form keeps
+    // its own launch into the workspace.
+    ga.q_scratch = robust ? static_cast<int8_t*>(workspace) : nullptr;
+    ga.sa_scratch = robust ? reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) +
+                                                      align256(static_cast<size_t>(ga.n_layers) * ga.M * ga.K))
+                           : nullptr;
     for (size_t i = 0; i < grp.size(); ++i) {
       const int l = grp[i];
       const PlanLayer& L = plan->layers[l];

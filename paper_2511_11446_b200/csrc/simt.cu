@@ -390,7 +390,31 @@ __device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block
 #pragma unroll 1
   for (int s = 0; s < S; ++s) issue();  // in flight across the prologue
   if (a.early_w) pdl_wait();
+  // Scale and bias of channels 2t, 2t + 1: of the current block, and fetched one block ahead for the
+  // next (a load issued at the top of the block it is needed in came back, under a saturated memory
+  // system, a couple of thousand cycles later, and its first use stalled the warp for that long).
+  float sw[2] = {0.0f, 0.0f}, bs[2] = {0.0f, 0.0f};
+  float nsw[2] = {0.0f, 0.0f};
+  uint32_t nbs[2] = {0u, 0u};
+  auto fetch_scales = [&](const int blk) {
+    if (blk < nblocks) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int n = blk * kMmaCh + 2 * t + e;
+        nsw[e] = a.s_w[n];
+        nbs[e] = a.bias != nullptr ? static_cast<uint32_t>(a.bias[n]) : 0u;
+      }
+    }
+  };
+  auto take_scales = [&]() {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      sw[e] = nsw[e];
+      bs[e] = __uint_as_float(nbs[e] << 16);
+    }
+  };
   constexpr int ORDER = BITS == 4 ? ORDER_NIBBLE : BITS == 3 ? ORDER_PERIOD : ORDER_NATURAL;
+  fetch_scales(blk0);  // of the first block: back by the time the tokens are staged
   for (int r = warp; r < (two ? kMmaRows : kMmaRows / 2); r += kMmaWarps)
     stage_tokens<ORDER>(a, m0, block_x, sq, qpitch, ssa, r, srs);
   __syncthreads();
@@ -405,7 +429,6 @@ __device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block
   int c_c = 0, c_blk = blk0, st = 0;
   uint32_t ph = 0;
   const int8_t* qrow = sq + g * qpitch + t * 32;
-  float sw[2] = {0.0f, 0.0f}, bs[2] = {0.0f, 0.0f};  // of channels 2t, 2t + 1 of the current block
   auto epilogue = [&]() {
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
@@ -481,13 +504,9 @@ __device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block
   };
   int it = 0;
   for (; it < total; ++it) {
-    if (c_c == 0) {  // the block's scales and biases: in flight while its chunks are contracted
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int n = c_blk * kMmaCh + 2 * t + e;
-        sw[e] = a.s_w[n];
-        bs[e] = a.bias != nullptr ? __uint_as_float(static_cast<uint32_t>(a.bias[n]) << 16) : 0.0f;
-      }
+    if (c_c == 0) {
+      take_scales();
+      fetch_scales(c_blk + stride);
     }
     if (!mbar_wait(&bar[st], ph, abort_flag)) break;
     const int nj = min(CJ, kj - c_c * CJ);
