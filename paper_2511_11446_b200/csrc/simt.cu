@@ -422,7 +422,7 @@ __device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block
   // One accumulator set per matrix instruction of a unit: consecutive instructions never wait on each
   // other's results. For packed weights the sets also differ in the power of two their operands
   // carry (see unit_step).
-  constexpr int NC = BITS == 3 ? 5 : 4;
+  constexpr int NC = 4;
   int c[NC][4];
 #pragma unroll
   for (int i = 0; i < NC; ++i) c[i][0] = c[i][1] = c[i][2] = c[i][3] = 0;
@@ -444,7 +444,7 @@ __device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block
           int mine;
           if constexpr (BITS == 8) mine = c[0][i] + c[1][i] + c[2][i] + c[3][i];
           else if constexpr (BITS == 4) mine = c[0][i] + c[1][i] + ((c[2][i] + c[3][i]) >> 4) - 8 * srs[tok];
-          else mine = c[0][i] + c[1][i] + (c[2][i] >> 2) + (c[3][i] >> 4) + (c[4][i] >> 5) - 4 * srs[tok];
+          else mine = c[0][i] + c[1][i] + (c[2][i] >> 2) + (c[3][i] >> 4) - 4 * srs[tok];
           const float y = __fmaf_rn(static_cast<float>(mine), __fmul_rn(ssa[tok], sw[e]), bs[e]);
           a.y[row * a.ldy + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
           if (a.dbg_acc != nullptr) a.dbg_acc[row * a.dbg_ldacc + n] = mine;
@@ -484,22 +484,23 @@ __device__ __forceinline__ void simt_mma_body(const SimtArgs& a, const int block
       //   r0: class 0 bits 0-2, class 1 bits 3-5, class 2 (low two bits) bits 6-7
       //   r1: class 2 (high bit) bit 0, class 3 bits 1-3, class 4 bits 4-6, class 5 (low bit) bit 7
       //   r2: class 5 (high two bits) bits 0-1, class 6 bits 2-4, class 7 bits 5-7
-      // Masked (and moved by a bit or two where that makes two fields carry the same power of two),
-      // each field is an unsigned operand byte worth its true value times 1, 4, 16 or 32; the two
-      // parts of the straddling classes 2 and 5 are separate operands against the same activations.
+      // Masked (and moved by a few bits where that makes two fields carry the same power of two),
+      // each field is an unsigned operand byte worth its true value times 1, 4 or 16; the two parts of
+      // the straddling classes 2 and 5 are put together first. The contraction is bound by the rate of
+      // the matrix instructions, so the few extra logic operations that save a fifth instruction pay.
       const uint32_t x0 = __byte_perm(pk[0], pk[1], 0x0630), x1 = __byte_perm(pk[0], pk[1], 0x0741),
                      x2 = __byte_perm(pk[0], pk[1], 0x0052);
       const uint32_t r0 = __byte_perm(x0, pk[2], 0x5210), r1 = __byte_perm(x1, pk[2], 0x6210),
                      r2 = __byte_perm(x2, pk[2], 0x7410);
-      // times 1: class 0 | high bit of class 2 (worth 4);  low bit of class 5 | its high bits (worth 2)
-      mma_m16n8k32_s8u8(c[0], l0.x, h0.x, l0.z, h0.z, r0 & 0x07070707u, (r1 & 0x01010101u) << 2);
-      mma_m16n8k32_s8u8(c[1], l1.y, h1.y, l1.y, h1.y, (r1 >> 7) & 0x01010101u, (r2 & 0x03030303u) << 1);
+      const uint32_t f2 = ((r0 >> 6) & 0x03030303u) | ((r1 & 0x01010101u) << 2);
+      const uint32_t f5 = ((r1 >> 7) & 0x01010101u) | ((r2 & 0x03030303u) << 1);
+      // times 1: class 0 | class 2;  class 5 | class 7 (moved down)
+      mma_m16n8k32_s8u8(c[0], l0.x, h0.x, l0.z, h0.z, r0 & 0x07070707u, f2);
+      mma_m16n8k32_s8u8(c[1], l1.y, h1.y, l1.w, h1.w, f5, (r2 >> 5) & 0x07070707u);
       // times 4: class 3 (moved up one bit) | class 6
       mma_m16n8k32_s8u8(c[2], l0.w, h0.w, l1.z, h1.z, (r1 & 0x0E0E0E0Eu) << 1, r2 & 0x1C1C1C1Cu);
       // times 16: class 1 (moved up one bit) | class 4
       mma_m16n8k32_s8u8(c[3], l0.y, h0.y, l1.x, h1.x, (r0 & 0x38383838u) << 1, r1 & 0x70707070u);
-      // times 32: class 7 | low bits of class 2 (moved down one bit)
-      mma_m16n8k32_s8u8(c[4], l1.w, h1.w, l0.z, h0.z, r2 & 0xE0E0E0E0u, (r0 & 0xC0C0C0C0u) >> 1);
     }
   };
   int it = 0;
@@ -695,7 +696,7 @@ int launch_simt_group(const SimtGroupArgs& g, cudaStream_t stream, bool pdl) {
     const int full = (g.N / kMmaCh + kMmaWarps - 1) / kMmaWarps;
     double cost[kSimtGroupMax], total = 0.0;
     for (int l = 0; l < g.n_layers; ++l) {
-      cost[l] = g.layer[l].bits == 8 ? 1.6 : g.layer[l].bits == 4 ? 1.0 : 1.2;
+      cost[l] = g.layer[l].bits == 8 ? 1.75 : g.layer[l].bits == 4 ? 1.0 : 1.1;
       total += cost[l];
     }
     int begin = 0;
