@@ -435,17 +435,17 @@ def next_row_timings(peaks):
 
 def measure_mma_peak():
     import torch
-    from paper_2511_11446_b200 import binding as B
+    from paper_2511_11446_b200 import probe
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
     iters = 20000
-    B.dp_bench_mma_i8(sms, 2000, 256, st)
+    probe.dp_probe_mma_i8(sms, 2000, 256, st)
     torch.cuda.synchronize()
     best = 0.0
     for _ in range(3):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        B.dp_bench_mma_i8(sms, iters, 256, st)
+        probe.dp_probe_mma_i8(sms, iters, 256, st)
         e1.record()
         torch.cuda.synchronize()
         best = max(best, 2.0 * 128 * 256 * 128 * iters * sms / (e0.elapsed_time(e1) * 1e-3) / 1e12)

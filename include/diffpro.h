@@ -360,7 +360,9 @@ int dp_plan_run(const dp_plan* plan, const int32_t* steps, int32_t n_steps, int3
  *   x_stage : device buffer of 2 * dp_plan_x_bytes(plan) bytes
  *   y_dev   : host array [n_layers] of device output buffers (overwritten every step)
  *   y_host  : host array [n_steps] of host pointers receiving layer `d2h_layer`'s output per step
- * Returns after enqueueing; the caller synchronises `stream`.
+ * Returns after enqueueing; the caller synchronises `stream`. The internal copy stream starts behind
+ * everything already enqueued on `stream` when the call is made, so consecutive calls (or a
+ * dp_plan_run on the same workspace) need no synchronisation in between.
  */
 size_t dp_plan_x_bytes(const dp_plan* plan);
 int dp_plan_run_host(const dp_plan* plan, const int32_t* steps, int32_t n_steps,
@@ -425,15 +427,6 @@ int dp_layer_latency_us(const dp_weight* w, int64_t M, uint32_t flags, int32_t r
  * DP_ERR_INVALID_ARG.
  */
 int dp_pack_weights_host(const int8_t* w, int32_t N, int32_t K, int32_t bits, void* out);
-
-/*
- * Measurement helper: each of `ctas` CTAs issues `iters` groups of four back-to-back tcgen05
- * kind::i8 MMAs (128 x tile_n x 32 each; tile_n a multiple of 16 up to 256) on operands resident in
- * shared memory, no global loads; used to establish the measured INT8 tensor ceiling of the device.
- * Enqueues one kernel on `stream`; ops = 2*128*tile_n*128*iters*ctas.
- */
-int dp_bench_mma_i8(int32_t ctas, int32_t iters, int32_t tile_n, int32_t* device_status,
-                    dp_stream stream);
 
 /*
  * Test hook for the bounded device waits (no counterpart in the paper). The next launch of the

@@ -35,7 +35,7 @@ DP_STATIC_SCRATCH_BYTES = 10 << 20
 
 EXPORTS = ["dp_daq_quantize", "dp_daq_quantize_robust", "dp_wq_linear_workspace", "dp_wq_linear_workspace_grouped", "dp_wq_linear", "dp_wq_linear_static", "dp_wq_linear_residual", "dp_plan_create",
            "dp_plan_workspace", "dp_plan_layer_variant", "dp_plan_layer_unpack_first", "dp_plan_set_layer_flags", "dp_plan_set_daq", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
-           "dp_plan_run_host", "dp_plan_phase_a", "dp_layer_latency_us", "dp_pack_weights_host", "dp_bench_mma_i8", "dp_clip_rank", "dp_debug_skip_stage_load",
+           "dp_plan_run_host", "dp_plan_phase_a", "dp_layer_latency_us", "dp_pack_weights_host", "dp_clip_rank", "dp_debug_skip_stage_load",
            "dp_status_string",
            "dp_last_error", "dp_version"]
 
@@ -112,7 +112,6 @@ def lib():
                                        C.POINTER(C.c_void_p), C.c_int32, C.POINTER(C.c_void_p),
                                        C.c_void_p, C.c_size_t, C.c_void_p, C.c_uint32, C.c_void_p]
         L.dp_pack_weights_host.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
-        L.dp_bench_mma_i8.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         L.dp_plan_phase_a.argtypes = [C.POINTER(dp_phase_a_problem), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.dp_layer_latency_us.argtypes = [C.POINTER(dp_weight), C.c_int64, C.c_uint32, C.c_int32, C.c_void_p]
         L.dp_clip_rank.restype = C.c_int32
@@ -307,11 +306,6 @@ def dp_pack_weights_host(w, bits: int):
     _check(lib().dp_pack_weights_host(w.ctypes.data_as(C.c_void_p), N, K, bits,
                                       out.ctypes.data_as(C.c_void_p)), "dp_pack_weights_host")
     return out
-
-
-def dp_bench_mma_i8(ctas, iters, tile_n=256, device_status=None, stream=None):
-    _check(lib().dp_bench_mma_i8(ctas, iters, tile_n, _ptr(device_status), _stream(stream)),
-           "dp_bench_mma_i8")
 
 
 def dp_version() -> int:

@@ -1,4 +1,4 @@
-"""Builds libdiffpro.so (and the input-generator library) in-tree with nvcc for sm_100a.
+"""Builds libdiffpro.so (and the input-generator and measurement-probe libraries) in-tree with nvcc for sm_100a.
 
     python -m paper_2511_11446_b200.build [--force] [--verbose]
 
@@ -19,13 +19,16 @@ SYNTH_LIB = os.path.join(HERE, "libdpsynth.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
-SOURCES = ["api.cu", "daq.cu", "simt.cu", "gemm_tc.cu", "gemm_ws.cu", "gemm_as.cu", "gemm_bf16.cu", "gemm_grp.cu", "peak.cu"]
+SOURCES = ["api.cu", "daq.cu", "simt.cu", "gemm_tc.cu", "gemm_ws.cu", "gemm_as.cu", "gemm_bf16.cu", "gemm_grp.cu"]
 SYNTH_SOURCES = ["synth_cuda.cu"]
+PROBE_LIB = os.path.join(HERE, "libdpprobe.so")
+PROBE_SOURCES = ["peak.cu"]
 
 
 def _deps():
     hdrs = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
     hdrs.append(os.path.join(os.path.dirname(HERE), "include", "diffpro.h"))
+    hdrs.append(os.path.join(os.path.dirname(HERE), "include", "diffpro_probe.h"))
     return hdrs
 
 
@@ -65,7 +68,8 @@ def build(force: bool = False, verbose: bool = False):
     if force:
         for f in os.listdir(OBJ):
             os.remove(os.path.join(OBJ, f))
-    return _link(LIB, SOURCES, verbose), _link(SYNTH_LIB, SYNTH_SOURCES, verbose)
+    return (_link(LIB, SOURCES, verbose), _link(SYNTH_LIB, SYNTH_SOURCES, verbose),
+            _link(PROBE_LIB, PROBE_SOURCES, verbose))
 
 
 if __name__ == "__main__":

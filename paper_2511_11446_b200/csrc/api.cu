@@ -596,7 +596,7 @@ struct dp_plan {
   // of the three time bins of [0, daq_timesteps)
   int32_t daq_p_e3, daq_timesteps, daq_bits[3];
   cudaStream_t copy_stream;
-  cudaEvent_t ev_copied[2], ev_consumed[2];
+  cudaEvent_t ev_copied[2], ev_consumed[2], ev_entry;
 };
 
 // Times every kernel variant that can run this layer shape (the whole layer: DAQ + GEMM, as the
@@ -699,6 +699,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
   p->daq_timesteps = 0;
   p->daq_bits[0] = p->daq_bits[1] = p->daq_bits[2] = 8;
   for (int i = 0; i < 2; ++i) p->ev_copied[i] = p->ev_consumed[i] = nullptr;
+  p->ev_entry = nullptr;
   for (int32_t l = 0; l < n_layers; ++l) {
     st = check_weight(&layers[l]);
     if (st == DP_OK && M_per_layer[l] < 0) st = fail(DP_ERR_SHAPE, "layer %d: negative M", l);
@@ -798,6 +799,7 @@ extern "C" int dp_plan_create(const dp_weight* layers, int32_t n_layers, const i
     }
   }
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_entry, cudaEventDisableTiming);
   for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
     e = cudaEventCreateWithFlags(&p->ev_copied[i], cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_consumed[i], cudaEventDisableTiming);
@@ -895,6 +897,7 @@ extern "C" void dp_plan_destroy(dp_plan* plan) {
   for (int i = 0; i < 2; ++i) {
     if (plan->ev_copied[i]) cudaEventDestroy(plan->ev_copied[i]);
     if (plan->ev_consumed[i]) cudaEventDestroy(plan->ev_consumed[i]);
+    if (i == 0 && plan->ev_entry) cudaEventDestroy(plan->ev_entry);
   }
   if (plan->copy_stream) cudaStreamDestroy(plan->copy_stream);
   if (plan->daq_sync) cudaFree(plan->daq_sync);
@@ -1030,6 +1033,10 @@ extern "C" int dp_plan_run_host(const dp_plan* plan_c, const int32_t* steps, int
     return fail(DP_ERR_INVALID_ARG, "bad d2h_layer / y_host");
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   std::vector<const void*> xs(n);
+  // The copy stream starts behind everything already enqueued on `stream`: an earlier call's last
+  // steps (or any other work of the caller) may still be reading the staging halves.
+  DP_CUDA_OK(cudaEventRecord(plan->ev_entry, stream));
+  DP_CUDA_OK(cudaStreamWaitEvent(plan->copy_stream, plan->ev_entry, 0));
   int j = 0;
   for (int32_t i = n_steps - 1; i >= 0; --i, ++j) {
     const int h = j & 1;

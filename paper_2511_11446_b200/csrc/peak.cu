@@ -1,9 +1,9 @@
-// Measurement helper: the INT8 tensor-core ceiling of the device as seen by this library's own
-// instruction stream. Each CTA fills one 128 x 128 (A) and one 256 x 128 (B) int8 operand tile in
+// Measurement probe (its own shared object, libdpprobe.so; not part of the product library): the
+// INT8 tensor-core ceiling of the device as seen by this library's own instruction stream. Each CTA fills one 128 x 128 (A) and one 256 x 128 (B) int8 operand tile in
 // shared memory with pseudo-random bytes and issues `iters` k-blocks of four tcgen05.mma kind::i8
 // (128 x tile_n x 32) each, alternating between two accumulator buffers; no global traffic.
 #include "dp_common.cuh"
-#include "dp_internal.h"
+#include "../../include/diffpro_probe.h"
 
 namespace dp {
 
@@ -67,18 +67,19 @@ __global__ void __launch_bounds__(128, 1) mma_i8_peak_kernel(int iters, int tile
 
 }  // namespace dp
 
-extern "C" int dp_bench_mma_i8(int32_t ctas, int32_t iters, int32_t tile_n, int32_t* device_status,
-                               dp_stream stream) {
+extern "C" int dp_probe_mma_i8(int32_t ctas, int32_t iters, int32_t tile_n, int32_t* device_status, void* stream) {
   using namespace dp;
-  if (ctas <= 0 || iters <= 0 || iters > (1 << 22) || tile_n < 16 || tile_n > 256 || (tile_n % 16))
-    return fail(DP_ERR_INVALID_ARG, "dp_bench_mma_i8: bad ctas/iters/tile_n");
-  int st = check_device();
-  if (st != DP_OK) return st;
+  if (ctas <= 0 || iters <= 0 || iters > (1 << 22) || tile_n < 16 || tile_n > 256 || (tile_n % 16)) return DP_PROBE_BAD_ARG;
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+    return DP_PROBE_CUDA;
+  if (major != 10) return DP_PROBE_ARCH;
   const size_t smem = 128 * 1024;  // more than half an SM: one CTA (and one TMEM allocation) per SM
-  DP_CUDA_OK(cudaFuncSetAttribute(mma_i8_peak_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  static_cast<int>(smem)));
-  cudaError_t e = launch(mma_i8_peak_kernel, dim3(ctas), dim3(128), smem,
-                         static_cast<cudaStream_t>(stream), false, iters, tile_n, device_status);
-  if (e != cudaSuccess) return fail(DP_ERR_CUDA, "peak kernel launch: %s", cudaGetErrorString(e));
-  return DP_OK;
+  if (cudaFuncSetAttribute(mma_i8_peak_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) !=
+      cudaSuccess)
+    return DP_PROBE_CUDA;
+  cudaError_t e = launch(mma_i8_peak_kernel, dim3(ctas), dim3(128), smem, static_cast<cudaStream_t>(stream), false,
+                         iters, tile_n, device_status);
+  return e == cudaSuccess ? DP_PROBE_OK : DP_PROBE_CUDA;
 }

@@ -24,6 +24,18 @@ def test_exports_match_header():
     assert L.dp_status_string(B.DP_ERR_TIMEOUT).decode() == "DP_ERR_TIMEOUT"
 
 
+def test_probe_library_exports_its_header():
+    """The measurement probes live in a library of their own, outside the product ABI."""
+    from paper_2511_11446_b200 import probe
+    hdr = open(os.path.join(ROOT, "include", "diffpro_probe.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(dp_[a-z0-9_]+)\s*\(", hdr))
+    assert declared == {"dp_probe_mma_i8"}
+    for name in declared:
+        assert getattr(probe.lib(), name) is not None
+        assert not hasattr(B.lib(), name)
+
+
 @pytest.mark.parametrize("bits", [3, 4, 8])
 def test_host_packer_agrees_with_oracle_codec(bits):
     rng = np.random.default_rng(bits)
