@@ -213,7 +213,9 @@ def run_ours(args):
         "clocks": clocks,
     }
 
-    if rank == 0:
+    if rank == 0 and args.timed_only:
+        print(json.dumps(out))
+    elif rank == 0:
         # ---- roofline of the dominant kernel (tcgen05 GEMM), timed alone with CUDA events ----
         mma_peak = measure_mma_peak()
         out["roofline"] = gemm_roofline(stack, peaks, mma_peak)
@@ -512,6 +514,9 @@ def main():
     ap.add_argument("--daq-policy", default=None,
                     help="P:a,b,c = run the plan under dp_plan_set_daq(P/1000 percent clip, activation bits of the "
                          "three time bins); default: the absmax, 8-bit rule the headline metric is defined on")
+    ap.add_argument("--timed-only", action="store_true",
+                    help="only the timed plan run (no roofline, side measurements, end-to-end or CPU legs): for runs "
+                         "under a profiler; its line is not a benchmark result")
     ap.add_argument("--hbm-kernels", action="store_true",
                     help="time only the HBM-bound kernels (grouped adaLN launch, DAQ at M=32768) and print their rooflines")
     args = ap.parse_args()
