@@ -290,3 +290,22 @@ def wq_linear_residual(x, qweight, s_w, bias, bits: int, res, gate=None, rows_pe
                                  _p(bias), _p(res), _i64(N), _p(gate), _i64(rows_per_gate), _p(y), _i64(N), _p(sw_),
                                  _p(sq), _p(ssa), _p(sacc))
     return y
+
+
+def ln_modulate_daq(x, shift=None, scale=None, rows_per_sample: int = 1, eps: float = 1e-6, tap=False):
+    """LayerNorm (no affine) + adaLN modulation + DAQ of bf16 tokens x uint16 [M, K]; shift, scale uint16
+    [ceil(M / rows_per_sample), K] or both None. Returns (q int8 [M,K], s_a fp32 [M]) and, with tap,
+    the fp32 activations that were quantized."""
+    _chk(x, np.uint16, "x")
+    M, K = x.shape
+    assert (shift is None) == (scale is None)
+    if shift is not None:
+        _chk(shift, np.uint16, "shift")
+        _chk(scale, np.uint16, "scale")
+        assert shift.shape == scale.shape == (-(-M // rows_per_sample), K)
+    q = np.empty((M, K), np.int8)
+    s_a = np.empty(M, np.float32)
+    h = np.empty((M, K), np.float32) if tap else None
+    lib().orc_ln_modulate_daq(_p(x), _i64(M), _i64(K), _i64(K), _p(shift), _p(scale), _i64(rows_per_sample),
+                              C.c_float(eps), _p(q), _i64(K), _p(s_a), _p(h))
+    return (q, s_a, h) if tap else (q, s_a)

@@ -36,6 +36,14 @@
  *                  and MLP outputs to its stream scaled by an adaLN gate per sample and channel).
  *                  Reading: lin = fma((float)acc, s_a*s_w, bias) as in orc_epilogue, then in fp32
  *                  v = fma(gate, lin, res) (gate given) or v = lin + res, y = bf16(v).
+ *   orc_ln_modulate_daq  the operator in front of a block's qkv and fc1 linears taken into their DAQ
+ *                  (Step 3: LayerNorms stay in higher precision; a DiT block feeds those linears
+ *                  LayerNorm(x) * (1 + scale) + shift with a per-sample adaLN scale and shift), so the
+ *                  normalized activations are quantized without ever being rounded to bf16. Reading:
+ *                  mean and variance (biased, E[x^2] - mean^2) of a token in double from the exact
+ *                  sums of its bf16 values, rstd = 1 / sqrt(var + eps) in double, both rounded to
+ *                  fp32; then in fp32 n = (x - mean) * rstd, h = fma(n, 1 + scale, shift); then Eq.
+ *                  "daq" on h exactly as orc_daq does on bf16 values.
  *   orc_linear_bf16  the layers a plan keeps in 16-bit precision (Step 1 tiering; Step 2 results): the
  *                  plain linear y = x . W^T + bias on bf16 inputs, summed in double (every product of
  *                  two bf16 values is exact in double), rounded once to bf16.
@@ -125,6 +133,65 @@ void orc_daq(const uint16_t* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, in
 #pragma omp parallel for schedule(static)
   for (int64_t m = 0; m < M; ++m)
     daq_row(x + m * ldx, K, q + m * ldq, s_a + m, rowsum ? rowsum + m : 0);
+}
+
+/* ---- LayerNorm + adaLN modulation in front of DAQ ----------------------------------------------- */
+
+/*
+ * x bf16 [M][ldx]; shift, scale bf16 [ceil(M / rows_per_sample)][K] (both NULL: no modulation); eps as
+ * in torch's layer_norm. q int8 [M][ldq], s_a fp32 [M]; h (optional) fp32 [M][K]: the modulated
+ * normalized activations that were quantized.
+ */
+void orc_ln_modulate_daq(const uint16_t* x, int64_t M, int64_t K, int64_t ldx, const uint16_t* shift,
+                         const uint16_t* scale, int64_t rows_per_sample, float eps, int8_t* q, int64_t ldq,
+                         float* s_a, float* h_out) {
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m) {
+    const uint16_t* xr = x + m * ldx;
+    double s1 = 0.0, s2 = 0.0; /* exact: bf16 values and their squares, K of them, fit a double's significand */
+    for (int64_t k = 0; k < K; ++k) {
+      const double v = (double)bf16_to_f32(xr[k]);
+      s1 += v;
+      s2 += v * v;
+    }
+    const double mean_d = s1 / (double)K;
+    double var_d = s2 / (double)K - mean_d * mean_d;
+    if (var_d < 0.0) var_d = 0.0;
+    const float mean = (float)mean_d;
+    const float rstd = (float)(1.0 / sqrt(var_d + (double)eps));
+    float* h = (float*)malloc((size_t)K * sizeof(float));
+    const int64_t sample = m / rows_per_sample;
+    float a = 0.0f;
+    for (int64_t k = 0; k < K; ++k) {
+      const float d = bf16_to_f32(xr[k]) - mean;
+      const float n = d * rstd;
+      float v = n;
+      if (scale) {
+        const float g = 1.0f + bf16_to_f32(scale[sample * K + k]);
+        v = fmaf(n, g, bf16_to_f32(shift[sample * K + k]));
+      }
+      h[k] = v;
+      if (fabsf(v) > a) a = fabsf(v);
+      if (h_out) h_out[m * K + k] = v;
+    }
+    int8_t* qr = q + m * ldq;
+    if (a < 0x1p-100f) {
+      s_a[m] = 0.0f;
+      for (int64_t k = 0; k < K; ++k) qr[k] = 0;
+    } else {
+      const float alpha = a / 127.0f;
+      const float inv_alpha = 127.0f / a;
+      s_a[m] = alpha;
+      for (int64_t k = 0; k < K; ++k) {
+        /* two fp32 values: the product is exact in double */
+        double r = nearbyint((double)h[k] * (double)inv_alpha);
+        if (r > 127.0) r = 127.0;
+        if (r < -127.0) r = -127.0;
+        qr[k] = (int8_t)r;
+      }
+    }
+    free(h);
+  }
 }
 
 /* ---- DAQ with percentile clip and a-bit codes (Eq. "daq", p < 100; Step 6) ------------------- */
