@@ -417,9 +417,11 @@ def next_row_timings(peaks):
     operands rotated past L2: group-wise weight scales (Step 2's storage format; g = 128 and 32, 4-bit,
     with and without zero-points) and 16-bit pass-through layers (bf16, fp32 accumulation; fraction
     against the measured bf16 tensor rate), and the gated residual add taken into the epilogue of the two
-    layers that feed the token stream, beside the same layer without it."""
+    layers that feed the token stream, beside the same layer without it; LayerNorm + adaLN modulation
+    taken into DAQ beside plain DAQ of the same tokens (M = 2048 and 32768)."""
     from paper_2511_11446_b200 import sweep
-    out = {"M": 2048, "grouped": [], "passthrough_bf16": [], "gated_residual": []}
+    out = {"M": 2048, "grouped": [], "passthrough_bf16": [], "gated_residual": [],
+           "ln_modulate_daq": [sweep.time_ln_daq(2048, 1152, peaks), sweep.time_ln_daq(32768, 1152, peaks)]}
     for name, K, N in sweep.SHAPES:
         if N == 1152:  # the two layers of a DiT block that feed the token stream: proj and fc2
             r = sweep.time_residual(name, 2048, K, N, 4, peaks)

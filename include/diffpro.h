@@ -232,6 +232,28 @@ int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, const float* s_
                  const dp_debug* dbg, int32_t* device_status, uint32_t flags, dp_stream stream);
 
 /*
+ * LayerNorm + adaLN modulation taken into DAQ (Step 3 keeps LayerNorms in higher precision and
+ * quantizes the wrapped linears' activations on the fly, Eq. "daq"; in a DiT block the qkv and fc1
+ * linears are fed LayerNorm(x) * (1 + scale) + shift with one scale and shift vector per sample).
+ * One pass over the bf16 stream x [M][ldx] writes int8 codes q [M][ldq] and token scales s_a [M],
+ * ready for dp_wq_linear(w, q, ldq, s_a, ...); the normalized values exist only in fp32:
+ *
+ *     mean, var   of the token's K values (var = E[x^2] - mean^2), in double, rounded to fp32
+ *     rstd        = 1 / sqrt(var + eps), in double, rounded to fp32
+ *     n[k]        = (x[k] - mean) * rstd                              fp32, two roundings
+ *     h[k]        = fma(n[k], 1 + scale[s][k], shift[s][k])           fp32, s = m / rows_per_sample
+ *     q, s_a      = Eq. "daq" on h (absmax / 127, round half to even), as dp_daq_quantize on bf16
+ *
+ * shift, scale: device bf16 [ceil(M / rows_per_sample)][K], 16-byte aligned, or both NULL (plain
+ * LayerNorm without affine parameters). K a multiple of 8, at most 4608; x, q 16-byte aligned, ldx a
+ * multiple of 8, ldq of 16. Enqueues one kernel. Errors: DP_ERR_INVALID_ARG, DP_ERR_SHAPE,
+ * DP_ERR_ALIGN, DP_ERR_ARCH.
+ */
+int dp_ln_modulate_daq(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, const void* shift_bf16,
+                       const void* scale_bf16, int64_t rows_per_sample, float eps, int8_t* q, int64_t ldq,
+                       float* s_a, dp_stream stream);
+
+/*
  * The residual connection around a wrapped linear, taken into its epilogue (Step 3 keeps residual
  * adds in higher precision; a DiT block adds its attention projection and MLP output to the token
  * stream scaled by an adaLN gate per sample and channel). With lin[m][n] the fp32 value that

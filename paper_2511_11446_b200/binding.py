@@ -33,7 +33,7 @@ def DP_FLAG_TILE_N(bn: int) -> int:
 
 DP_STATIC_SCRATCH_BYTES = 10 << 20
 
-EXPORTS = ["dp_daq_quantize", "dp_daq_quantize_robust", "dp_wq_linear_workspace", "dp_wq_linear_workspace_grouped", "dp_wq_linear", "dp_wq_linear_static", "dp_wq_linear_residual", "dp_plan_create",
+EXPORTS = ["dp_daq_quantize", "dp_daq_quantize_robust", "dp_wq_linear_workspace", "dp_wq_linear_workspace_grouped", "dp_wq_linear", "dp_wq_linear_static", "dp_wq_linear_residual", "dp_ln_modulate_daq", "dp_plan_create",
            "dp_plan_workspace", "dp_plan_layer_variant", "dp_plan_layer_unpack_first", "dp_plan_set_layer_flags", "dp_plan_set_daq", "dp_plan_destroy", "dp_plan_run", "dp_plan_x_bytes",
            "dp_plan_run_host", "dp_plan_phase_a", "dp_layer_latency_us", "dp_pack_weights_host", "dp_clip_rank", "dp_debug_skip_stage_load",
            "dp_status_string",
@@ -97,6 +97,8 @@ def lib():
         L.dp_wq_linear.argtypes = [C.POINTER(dp_weight), C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                    C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t,
                                    C.POINTER(dp_debug), C.c_void_p, C.c_uint32, C.c_void_p]
+        L.dp_ln_modulate_daq.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64,
+                                         C.c_float, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
         L.dp_wq_linear_residual.argtypes = [C.POINTER(dp_weight), C.c_void_p, C.c_int64, C.c_int64, C.POINTER(dp_residual),
                                             C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p, C.c_uint32,
                                             C.c_void_p]
@@ -175,6 +177,12 @@ def dp_wq_linear(w: dp_weight, x, ldx, s_a_in, M, y, ldy, workspace, dbg: dp_deb
     _check(lib().dp_wq_linear(C.byref(w), _ptr(x), ldx, _ptr(s_a_in), M, _ptr(y), ldy, _ptr(workspace),
                               ws_bytes, None if dbg is None else C.byref(dbg), _ptr(device_status),
                               flags, _stream(stream)), "dp_wq_linear")
+
+
+def dp_ln_modulate_daq(x, M, K, ldx, shift, scale, rows_per_sample, eps, q, ldq, s_a, stream=None):
+    """LayerNorm + adaLN modulation + DAQ of bf16 tokens in one pass (shift, scale may both be None)."""
+    _check(lib().dp_ln_modulate_daq(_ptr(x), M, K, ldx, _ptr(shift), _ptr(scale), rows_per_sample, eps, _ptr(q), ldq,
+                                    _ptr(s_a), _stream(stream)), "dp_ln_modulate_daq")
 
 
 class dp_residual(C.Structure):

@@ -19,7 +19,7 @@ SYNTH_LIB = os.path.join(HERE, "libdpsynth.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
-SOURCES = ["api.cu", "daq.cu", "simt.cu", "gemm_tc.cu", "gemm_ws.cu", "gemm_as.cu", "gemm_bf16.cu", "gemm_grp.cu"]
+SOURCES = ["api.cu", "daq.cu", "simt.cu", "gemm_tc.cu", "gemm_ws.cu", "gemm_as.cu", "gemm_bf16.cu", "gemm_grp.cu", "ln.cu"]
 SYNTH_SOURCES = ["synth_cuda.cu"]
 PROBE_LIB = os.path.join(HERE, "libdpprobe.so")
 PROBE_SOURCES = ["peak.cu"]

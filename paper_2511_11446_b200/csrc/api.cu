@@ -489,6 +489,26 @@ extern "C" int dp_wq_linear(const dp_weight* w, const void* x, int64_t ldx, cons
                     static_cast<cudaStream_t>(stream), nullptr, 0, 0, 0, nullptr, false);
 }
 
+extern "C" int dp_ln_modulate_daq(const void* x, int64_t M, int64_t K, int64_t ldx, const void* shift,
+                                  const void* scale, int64_t rows_per_sample, float eps, int8_t* q, int64_t ldq,
+                                  float* s_a, dp_stream stream) {
+  if (M < 0 || K <= 0 || (K % 8) || K > 4608) return fail(DP_ERR_SHAPE, "dp_ln_modulate_daq: M=%lld K=%lld", (long long)M, (long long)K);
+  if ((shift == nullptr) != (scale == nullptr))
+    return fail(DP_ERR_INVALID_ARG, "dp_ln_modulate_daq: shift and scale come together");
+  if (shift != nullptr && rows_per_sample < 1) return fail(DP_ERR_SHAPE, "rows_per_sample=%lld", (long long)rows_per_sample);
+  if (!(eps >= 0.0f)) return fail(DP_ERR_INVALID_ARG, "dp_ln_modulate_daq: eps must be >= 0");
+  if (M == 0) return DP_OK;
+  if (!x || !q || !s_a) return fail(DP_ERR_INVALID_ARG, "dp_ln_modulate_daq: NULL argument");
+  if (ldx < K || ldq < K) return fail(DP_ERR_SHAPE, "leading dimension smaller than the row");
+  if (!aligned16(x) || !aligned16(q) || (ldx % 8) || (ldq % 16) || (reinterpret_cast<uintptr_t>(s_a) & 3u) ||
+      (shift && (!aligned16(shift) || !aligned16(scale))))
+    return fail(DP_ERR_ALIGN, "dp_ln_modulate_daq: pointers and pitches must be 16-byte aligned");
+  int st = check_device();
+  if (st != DP_OK) return st;
+  return launch_ln_modulate_daq(x, M, K, ldx, shift, scale, shift ? rows_per_sample : 1, eps, q, ldq, s_a,
+                                static_cast<cudaStream_t>(stream), false);
+}
+
 extern "C" int dp_wq_linear_residual(const dp_weight* w, const void* x_bf16, int64_t ldx, int64_t M,
                                      const dp_residual* r, void* y_bf16, int64_t ldy, void* workspace,
                                      size_t workspace_bytes, int32_t* device_status, uint32_t flags,

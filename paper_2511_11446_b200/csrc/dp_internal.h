@@ -31,6 +31,10 @@ int launch_daq(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int6
                float* s_a, int32_t* rowsum, int korder, bool tiled, cudaStream_t stream, bool pdl,
                const UnpackJob* unpack = nullptr);
 int launch_unpack(const UnpackJob& job, cudaStream_t stream, bool pdl);
+// ln.cu -- LayerNorm + adaLN modulation + DAQ in one pass (K a multiple of 8, at most 4608)
+int launch_ln_modulate_daq(const void* x, int64_t M, int64_t K, int64_t ldx, const void* shift, const void* scale,
+                           int64_t rows_per_sample, float eps, int8_t* q, int64_t ldq, float* s_a,
+                           cudaStream_t stream, bool pdl);
 int launch_daq_robust(const void* x, int64_t M, int64_t K, int64_t ldx, int8_t* q, int64_t ldq, float* s_a,
                       int32_t* rowsum, int clip_rank, int act_bits, bool tiled, cudaStream_t stream, bool pdl,
                       const UnpackJob* unpack);

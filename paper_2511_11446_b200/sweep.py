@@ -76,6 +76,28 @@ def time_grouped(name, M, K, N, bits, g, zeros, peaks, seed=synth.BASE_SEED + 5,
             "layer_us": t, "layer_tops": ops / t / 1e6, "ideal_us": t_ideal, "layer_frac": t_ideal / t}
 
 
+def time_ln_daq(M, K, peaks, rows_per_sample=256, seed=synth.BASE_SEED + 5, iters=None):
+    """LayerNorm + adaLN modulation + DAQ in one pass against plain DAQ of the same tokens (both read
+    2 bytes and write 1 byte per element), graph-timed with buffers rotated past L2."""
+    per_set = 3 * M * K
+    n_sets = max(2, min(24, -(-2 * L2_BYTES // per_set)))
+    iters = iters or max(10, min(200, int(2e9 // per_set)))
+    iters = -(-iters // n_sets) * n_sets
+    xs = [synth_cuda.activations(seed, s, 0, M, K, 1.0, n_out=max(1, K // 100)) for s in range(n_sets)]
+    qs = [torch.empty((M, K), dtype=torch.int8, device="cuda") for _ in range(n_sets)]
+    sas = [torch.empty(M, dtype=torch.float32, device="cuda") for _ in range(n_sets)]
+    S = -(-M // rows_per_sample)
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+    shift = (torch.randn((S, K), generator=gen, device="cuda") * 0.3).to(torch.bfloat16)
+    scale = (torch.randn((S, K), generator=gen, device="cuda") * 0.3).to(torch.bfloat16)
+    t_ln = _time(lambda s: B.dp_ln_modulate_daq(xs[s], M, K, K, shift, scale, rows_per_sample, 1e-6, qs[s], K, sas[s]),
+                 n_sets, iters)
+    t_daq = _time(lambda s: B.dp_daq_quantize(xs[s], M, K, K, qs[s], K, sas[s]), n_sets, iters)
+    by = 3 * M * K + 4 * M
+    return {"M": M, "K": K, "ln_modulate_daq_us": t_ln, "daq_us": t_daq, "bytes": by,
+            "frac_of_hbm": by / (t_ln * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+
+
 def time_residual(name, M, K, N, bits, peaks, rows_per_gate=1024, seed=synth.BASE_SEED + 5, iters=None):
     """Whole layer with the gated residual in its epilogue (x <- x + gate * layer(h), written over x),
     graph-timed like time_shape; the stream adds 2*M*N bytes of reads to the layer's algorithmic bytes."""
