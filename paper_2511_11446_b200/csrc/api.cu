@@ -128,7 +128,9 @@ static void choose_tile(uint32_t flags, int64_t M, int32_t N, int32_t K, int32_t
   // By default only with 256-channel strips: with 192-channel ones the resident strip leaves the
   // activation ring too shallow for the rate the tensor core then asks of it, and the streaming pair
   // kernel is 3-6 % faster (measured at M = 32768: qkv 139 -> 133 us, proj 67 -> 63).
-  if (ws_ok && ((flags & DP_FLAG_WEIGHT_STATIONARY) || (M >= kWsMinRows && gemm_ws_pick_bn(N) == 256))) {
+  // (Packed weights expanded inside the GEMM keep it at either width: expanding a strip once instead
+  // of once per tile is worth far more: qkv at 3 bits 121 us against 182.)
+  if (ws_ok && ((flags & DP_FLAG_WEIGHT_STATIONARY) || (M >= kWsMinRows && (bits < 8 || gemm_ws_pick_bn(N) == 256)))) {
     const int fb = forced_bn(flags);
     *bn = ((fb == 192 || fb == 256) && N % fb == 0) ? fb : gemm_ws_pick_bn(N);
     *cg = 2;
