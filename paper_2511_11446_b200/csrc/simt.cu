@@ -16,10 +16,14 @@
 // shared-memory stages (3- and 4-bit: one copy of eight whole rows per stage; 8-bit: one copy per
 // row and third of K; completion counted in bytes on the stage's mbarrier), so
 // HBM sees a few thousand long sequential streams and the bytes in flight do not depend on
-// registers. Lane (g, t) = (lane / 4, lane % 4) reads the units 4j + t of row g from the stage,
-// expands them to int8 and feeds them as B fragments; because a dot product may visit k in any
-// order as long as both operands agree, the A fragments are simply the same units of tokens g and
-// g + 8 from shared memory (row pitch K + 16 keeps those 128-bit reads conflict-free).
+// registers. Lane (g, t) = (lane / 4, lane % 4) reads the units 4j + t of row g from the stage and
+// feeds them as B fragments: 8-bit codes as they are; packed 3- and 4-bit codes as UNSIGNED bytes
+// that one mask (and at most a short shift) isolates where the field already sits, the power of two
+// such a byte carries being common to an accumulator set and shifted out exactly at the end, the
+// offset 2^(b-1) leaving as 2^(b-1) times the sum of the token's codes. Because a dot product may
+// visit k in any order as long as both operands agree, the A fragments are the same units of tokens
+// g and g + 8 from shared memory, staged in the k order the masks produce (row pitch K + 16 keeps
+// those 128-bit reads conflict-free).
 #include <cuda_bf16.h>
 
 #include <algorithm>
