@@ -79,8 +79,9 @@ struct QRow {
                     : reinterpret_cast<uint2*>(q + row * ldq);
   }
   __device__ __forceinline__ void store(int idx, uint2 v) const {
-    if (tiled) base[(idx >> 4) * 2048 + (idx & 15)] = v;  // next k block: + 16384 bytes
-    else base[idx] = v;
+    uint2* p = tiled ? base + (idx >> 4) * 2048 + (idx & 15) : base + idx;  // next k block: + 16384 bytes
+    // read next by another kernel, through L2: no L1 allocation
+    asm volatile("st.global.L1::no_allocate.v2.b32 [%0], {%1, %2};" ::"l"(p), "r"(v.x), "r"(v.y) : "memory");
   }
 };
 

@@ -402,10 +402,12 @@ __device__ __forceinline__ uint4 ld_global_v4(const void* p) {
   return v;
 }
 
-// 32-byte global store (sm_100): `p` 32-byte aligned.
+// 32-byte global store (sm_100): `p` 32-byte aligned. Output rows are written once and not read back
+// by the kernel, so they bypass L1 allocation (measured: 2-8 % shorter layers at M = 2048, 3 % at
+// M = 32768 for the widest outputs; an L2 evict-first policy on top changed nothing).
 __device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&w)[8]) {
-  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]),
-               "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+  asm volatile("st.global.L1::no_allocate.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(w[0]),
+               "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
                : "memory");
 }
 
