@@ -301,9 +301,7 @@ __device__ __forceinline__ void unpack_units(const UnpackJob& job, const int blo
     const uint32_t pk[3] = {p[0], p[1], p[2]};
     expand_unit<3>(pk, w);
   }
-  uint4* o = reinterpret_cast<uint4*>(job.out) + u * 2;
-  o[0] = make_uint4(w[0], w[1], w[2], w[3]);
-  o[1] = make_uint4(w[4], w[5], w[6], w[7]);
+  st_global_v8(reinterpret_cast<uint4*>(job.out) + u * 2, w);  // 32 bytes, read next by the GEMM through L2
 }
 
 }  // namespace dp
