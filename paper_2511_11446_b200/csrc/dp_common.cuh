@@ -394,6 +394,10 @@ __device__ __forceinline__ void tmem_ld_wait() {
 }
 
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+// `bytes` (a multiple of 16, from a 16-byte aligned address) on their way into L2; nothing waits on it
+__device__ __forceinline__ void bulk_prefetch_l2(const void* p, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
 
 // 16-byte load through the coherent path (never ld.global.nc): for data the same kernel also writes.
 __device__ __forceinline__ uint4 ld_global_v4(const void* p) {
