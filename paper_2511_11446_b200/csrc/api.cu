@@ -1000,19 +1000,23 @@ static int plan_run_step(dp_plan* plan, int32_t t, const void* const* xs, void* 
       ta = cached_tmap_a(plan, workspace, L.M, L.w.K, &st);
       if (st != DP_OK) return st;
     }
-    // the next tensor-core layer's packed weights start towards L2 while this layer's GEMM runs
-    gemm_set_next_weights(nullptr, 0);
+    // The next tensor-core layer's packed weights and its input start towards L2 while this layer's
+    // GEMM runs. A hint, not a reordering: if that input is still to be written (by this layer, say),
+    // the hint fetches bytes that the write then replaces in L2, and nothing is read before its turn.
+    gemm_set_next_reads(nullptr, 0, nullptr, 0);
     for (int j = l + 1; j < n; ++j) {
       const PlanLayer& Nx = plan->layers[j];
       if (Nx.M == 0 || (plan->grouped[j] && !group_splits(j))) continue;
-      if (!Nx.simt) gemm_set_next_weights(Nx.w.qweight, static_cast<size_t>(Nx.w.N) * Nx.w.K * Nx.w.bits / 8);
+      if (!Nx.simt && xs[j] != nullptr)
+        gemm_set_next_reads(Nx.w.qweight, static_cast<size_t>(Nx.w.N) * Nx.w.K * Nx.w.bits / 8, xs[j],
+                            static_cast<size_t>(Nx.M) * Nx.w.K * 2);
       break;
     }
     int st = run_linear(&L.w, xs[l], L.w.K, nullptr, L.M, ys[l], L.w.N, workspace, nullptr, status,
                         plan->flags, stream, L.simt ? nullptr : &L.tmap_w, L.bn, L.cg, L.ws, ta, *chained,
                         L.simt ? nullptr : plan->daq_sync, L.simt ? 0 : L.pre,
                         robust ? clip_rank_of(plan->daq_p_e3, L.w.K) : 1, act_bits);
-    gemm_set_next_weights(nullptr, 0);
+    gemm_set_next_reads(nullptr, 0, nullptr, 0);
     if (st != DP_OK) return st;
     *chained = true;
   }

@@ -135,9 +135,10 @@ int gemm_encode_w(CUtensorMap* out, const void* qweight, int32_t N, int32_t K, i
                   int32_t bn, int32_t cg);
 int launch_gemm(const GemmProblem& p, cudaStream_t stream, bool pdl);
 void gemm_debug_skip_stage_load(int32_t kb);  // see dp_debug_skip_stage_load
-// Constants (a plan's next layer's weights) that the calling thread's next launch_gemm sends on their
-// way into L2 while it runs; cleared by that launch. A hint: any valid device range of the caller's.
-void gemm_set_next_weights(const void* p, size_t bytes);
+// Two ranges (a plan's next layer's packed weights and its bf16 input) that the calling thread's next
+// launch_gemm sends on their way into L2 while it runs; cleared by that launch. Hints: any valid
+// device ranges of the caller's, or nullptr.
+void gemm_set_next_reads(const void* w, size_t w_bytes, const void* x, size_t x_bytes);
 
 // gemm_ws.cu -- weight-stationary CTA-pair kernel (K <= 1152, N a multiple of 192 or 256).
 bool gemm_ws_supported(int32_t N, int32_t K);

@@ -61,11 +61,12 @@ struct GemmParams {
   int32_t a_tiled;  // activations are stored as contiguous 128 x 128 tiles
   int32_t early_w;  // weights may be fetched before the preceding kernel on the stream has finished
   int32_t* status;
-  // Constants another launch will read soon (a plan's next layer's packed weights): each CTA sends its
-  // slice on the way into L2 while this kernel, which leaves HBM mostly idle at a few thousand tokens,
-  // runs. A hint only; nullptr: none.
-  const uint8_t* pf = nullptr;
-  uint32_t pf_bytes = 0, pf_slice = 0;
+  // Two ranges a later launch will read soon (a plan's next layer's packed weights and its bf16 input):
+  // each CTA sends its slices on the way into L2 while this kernel, which leaves HBM mostly idle at a
+  // few thousand tokens, runs. Hints only (L2 is the point of coherence: a range rewritten after the
+  // hint is simply current when it is read); nullptr: none.
+  const uint8_t* pf[2] = {nullptr, nullptr};
+  uint32_t pf_bytes[2] = {0, 0}, pf_slice[2] = {0, 0};
   int32_t dbg_skip_kb = -1;  // test hook (dp_debug_skip_stage_load): k-block whose loads are left out, or -1
 };
 

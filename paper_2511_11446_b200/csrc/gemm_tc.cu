@@ -113,11 +113,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   const uint32_t tmem_base = *tmem_slot;
 
   pdl_launch_dependents();
-  if (threadIdx.x == kEpiWarp0 * 32 && p.pf != nullptr) {  // an epilogue thread: idle until the first accumulators
-    const uint32_t off = blockIdx.x * p.pf_slice;
-    if (off < p.pf_bytes) {
-      uint32_t n = min(p.pf_slice, p.pf_bytes - off);
-      for (uint32_t o = 0; o < n; o += 32768u) bulk_prefetch_l2(p.pf + off + o, min(32768u, n - o));
+  if (threadIdx.x == kEpiWarp0 * 32) {  // an epilogue thread: idle until the first accumulators
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const uint32_t off = blockIdx.x * p.pf_slice[r];
+      if (p.pf[r] != nullptr && off < p.pf_bytes[r]) {
+        const uint32_t n = min(p.pf_slice[r], p.pf_bytes[r] - off);
+        for (uint32_t o = 0; o < n; o += 32768u) bulk_prefetch_l2(p.pf[r] + off + o, min(32768u, n - o));
+      }
     }
   }
   // Activations and their scales come from the preceding kernel on the stream: the roles that read
@@ -490,12 +493,14 @@ static cudaError_t launch_bn(const GemmProblem& g, const GemmParams& p, dim3 gri
   }
 }
 
-// Next weights a plan wants on their way into L2 (consumed by the calling thread's next launch_gemm).
-static thread_local const void* g_pf_ptr = nullptr;
-static thread_local size_t g_pf_bytes = 0;
-void gemm_set_next_weights(const void* p, size_t bytes) {
-  g_pf_ptr = p;
-  g_pf_bytes = bytes;
+// Ranges a plan wants on their way into L2 (consumed by the calling thread's next launch_gemm).
+static thread_local const void* g_pf_ptr[2] = {nullptr, nullptr};
+static thread_local size_t g_pf_bytes[2] = {0, 0};
+void gemm_set_next_reads(const void* w, size_t w_bytes, const void* x, size_t x_bytes) {
+  g_pf_ptr[0] = w;
+  g_pf_bytes[0] = w_bytes;
+  g_pf_ptr[1] = x;
+  g_pf_bytes[1] = x_bytes;
 }
 
 // dp_debug_skip_stage_load: consumed by the calling thread's next single-CTA 8-bit launch.
@@ -539,13 +544,15 @@ int launch_gemm(const GemmProblem& g, cudaStream_t stream, bool pdl) {
   const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
   const int64_t slots = cg == 2 ? (gemm_max_pairs() > 0 ? gemm_max_pairs() : num_sms() / 2) : num_sms();
   const dim3 grid(static_cast<unsigned>((tiles < slots ? tiles : slots) * cg));
-  if (g_pf_ptr != nullptr && g_pf_bytes >= 16 && g_pf_bytes < (1ull << 31) &&
-      (reinterpret_cast<uintptr_t>(g_pf_ptr) & 15u) == 0) {
-    p.pf = static_cast<const uint8_t*>(g_pf_ptr);
-    p.pf_bytes = static_cast<uint32_t>(g_pf_bytes & ~static_cast<size_t>(15));
-    p.pf_slice = ((p.pf_bytes + grid.x - 1) / grid.x + 15u) & ~15u;
+  for (int r = 0; r < 2; ++r) {
+    if (g_pf_ptr[r] != nullptr && g_pf_bytes[r] >= 16 && g_pf_bytes[r] < (1ull << 31) &&
+        (reinterpret_cast<uintptr_t>(g_pf_ptr[r]) & 15u) == 0) {
+      p.pf[r] = static_cast<const uint8_t*>(g_pf_ptr[r]);
+      p.pf_bytes[r] = static_cast<uint32_t>(g_pf_bytes[r] & ~static_cast<size_t>(15));
+      p.pf_slice[r] = ((p.pf_bytes[r] + grid.x - 1) / grid.x + 15u) & ~15u;
+    }
+    g_pf_ptr[r] = nullptr;
   }
-  g_pf_ptr = nullptr;
   cudaError_t e;
   if (cg == 2) {
     switch (g.bn) {
