@@ -1007,9 +1007,11 @@ static int plan_run_step(dp_plan* plan, int32_t t, const void* const* xs, void* 
     for (int j = l + 1; j < n; ++j) {
       const PlanLayer& Nx = plan->layers[j];
       if (Nx.M == 0 || (plan->grouped[j] && !group_splits(j))) continue;
-      if (!Nx.simt && xs[j] != nullptr)
-        gemm_set_next_reads(Nx.w.qweight, static_cast<size_t>(Nx.w.N) * Nx.w.K * Nx.w.bits / 8, xs[j],
-                            static_cast<size_t>(Nx.M) * Nx.w.K * 2);
+      const size_t wb = static_cast<size_t>(Nx.w.N) * Nx.w.K * Nx.w.bits / 8;
+      const size_t xb = static_cast<size_t>(Nx.M) * Nx.w.K * 2;
+      // (only what fits L2 beside this layer's own operands: at tens of thousands of tokens an input
+      // is larger than that and the hint would only evict)
+      if (!Nx.simt && xs[j] != nullptr) gemm_set_next_reads(Nx.w.qweight, wb, xb <= (32u << 20) ? xs[j] : nullptr, xb);
       break;
     }
     int st = run_linear(&L.w, xs[l], L.w.K, nullptr, L.M, ys[l], L.w.N, workspace, nullptr, status,
