@@ -176,12 +176,14 @@ def run_ours(args):
     torch.cuda.synchronize()
 
     # ---- device-resident timing: K plan runs (graph replays), CUDA events on the launch stream ----
+    # the clock sampler starts with the warm-up replays (the same work): nvidia-smi needs a few tenths
+    # of a second to come up, more than a short timed region lasts
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for _ in range(args.warmup):
         graph.replay()
     torch.cuda.synchronize()
     D.barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.cudart().cudaProfilerStart()  # lets `ncu --profile-from-start off` see only the timed region
