@@ -257,7 +257,7 @@ int dp_ln_modulate_daq(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, co
  * The residual connection around a wrapped linear, taken into its epilogue (Step 3 keeps residual
  * adds in higher precision; a DiT block adds its attention projection and MLP output to the token
  * stream scaled by an adaLN gate per sample and channel). With lin[m][n] the fp32 value that
- * dp_wq_linear rounds to bf16 (Eq. 3's dequantized output plus bias):
+ * dp_wq_linear rounds to bf16 (Step 5's dequantized output plus bias):
  *
  *     y[m][n] = bf16( gate ? fma(gate[m / rows_per_gate][n], lin, residual[m][n]) : lin + residual[m][n] )
  *
@@ -368,6 +368,11 @@ void dp_plan_destroy(dp_plan* plan);
  * and length matter to the linears). Visits i = n_steps-1-start_index, ..., 0, so a caller can
  * resume an interrupted schedule by passing the number of steps already done as start_index.
  * x_ptrs / y_ptrs are HOST arrays of device pointers. Enqueues only; capturable in a CUDA graph.
+ * While a layer's GEMM runs, its kernel issues L2 prefetch hints for the next layer's packed weights
+ * and (up to 32 MB) for the next layer's input buffer. These are hints on memory the call is going to
+ * read anyway: no layer is computed before its turn, and an input that an earlier layer of the same
+ * step still writes (x of one layer aliasing y of another) is read only after that write, as the
+ * stream order says.
  */
 int dp_plan_run(const dp_plan* plan, const int32_t* steps, int32_t n_steps, int32_t start_index,
                 const void* const* x_ptrs, void* const* y_ptrs, void* workspace,
