@@ -348,3 +348,44 @@ def test_phase_a_on_measured_latencies_matches_oracle_and_runs():
                 assert bf16_ulp_dist(bf16_to_np(ys[i][l]), ref).max() <= 1
     finally:
         B.dp_plan_destroy(plan)
+
+
+def test_chained_layers_whose_input_is_an_earlier_output():
+    """A plan whose layer l + 1 reads the buffer layer l writes (x of one aliasing y of the other): the
+    L2 hints a GEMM gives for the next layer's input must not let anything be read before its turn.
+    Three chained linears over two steps, against the oracle's chain, several times in a row."""
+    M, dims, bits = 1024, (384, 512, 256, 384), (8, 4, 3)
+    ws_, dev, lay = [], [], []
+    for l in range(3):
+        K, N = dims[l], dims[l + 1]
+        w, s_w = synth.weights(SEED + 50, l, N, K, bits[l])
+        b = synth.bias(SEED + 50, l, N)
+        dev.append(DevLayer(w, s_w, b, bits[l]))
+        lay.append((oracle.pack(w, bits[l]), s_w, b, bits[l]))
+    steps = [3, 7]
+    x0 = [synth.activations(SEED + 50, 0, t, M, dims[0], 1.0, n_out=4) for t in steps]
+    want = []
+    for i in range(len(steps)):
+        h, outs = x0[i], []
+        for pw, s_w, b, bt in lay:
+            h = oracle.wq_linear(h, pw, s_w, b, bt)
+            outs.append(h)
+        want.append(outs)
+    plan = B.dp_plan_create([d.w for d in dev], [M] * 3)
+    try:
+        ws = torch.empty(B.dp_plan_workspace(plan), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for rep in range(3):
+            xd = [to_dev_bf16(x0[i]) for i in range(len(steps))]
+            yd = [[torch.full((M, dims[l + 1]), float("nan"), dtype=torch.bfloat16, device="cuda") for l in range(3)]
+                  for _ in steps]
+            xp = B.ptr_array([(xd[i] if l == 0 else yd[i][l - 1]).data_ptr() for i in range(len(steps)) for l in range(3)])
+            yp = B.ptr_array([yd[i][l].data_ptr() for i in range(len(steps)) for l in range(3)])
+            B.dp_plan_run(plan, steps, 0, xp, yp, ws, status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            for i in range(len(steps)):
+                for l in range(3):
+                    assert np.array_equal(bf16_to_np(yd[i][l]), want[i][l]), (rep, i, l)
+    finally:
+        B.dp_plan_destroy(plan)
