@@ -97,12 +97,13 @@ class DitStack:
 
     def launches_per_timestep(self):
         """Kernel launches of this library per timestep: DAQ + GEMM per token linear; the small-M
-        (adaLN) linears of a step share, per 32 of them, one grouped DAQ launch and one grouped
-        linear launch when the plan groups them."""
+        (adaLN) linears of a step share, per 32 of them, one grouped launch that also quantizes their
+        tokens when the plan groups them (under a percentile / a-bit DAQ policy a second, small
+        quantization launch goes in front of it)."""
         small = sum(1 for (_, M, K, N) in self.table if M <= 32)
         big = len(self.table) - small
         grouped = bool(self.flags & B.DP_FLAG_GROUP_SMALL_M)
-        return 2 * big + (2 * -(-small // 32) if grouped else small)
+        return 2 * big + (-(-small // 32) if grouped else small)
 
     # ---- execution ----
     def ptrs(self, n_steps=None):
